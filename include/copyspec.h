@@ -1,0 +1,209 @@
+/*
+ * copyspec.h - C ABI of the B200 (sm_100a) copy-and-verify decode step of CopySpec
+ * (arXiv 2502.08923, "Accelerating LLMs with Speculative Copy-and-Paste").
+ *
+ * One decode step is: search the token history for an earlier occurrence of the last
+ * gamma tokens and copy the k tokens that followed it as a draft (Sec. 3.1, 3.2); run
+ * ONE forward of the target model over [last token, draft] against the KV cache
+ * (Sec. 3.2); take the greedy token per row and accept the longest agreeing prefix plus
+ * one extra token (Sec. 3.2, App. B.2); drop the KV entries of the rejected tokens
+ * (App. B.2, App. B.3 step 2(b)).
+ *
+ * General conventions
+ *   - All pointers are DEVICE pointers unless a parameter says "host".
+ *   - Ownership: the caller allocates and frees every buffer (history, lengths, drafts,
+ *     KV cache, weights, workspace, outputs).  The library allocates no device memory.
+ *     A context keeps the weight and workspace pointers given to cs_create; they must
+ *     outlive it.  Other pointers are used only during the call (and by the work the
+ *     call enqueued on `stream`).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls
+ *     marked "async" only enqueue work.  Work of one context must stay on one stream at
+ *     a time (its workspace is shared by consecutive calls).
+ *   - Errors: every call returns a cs_status.  Argument errors are found on the host
+ *     before anything is launched.  Conditions only the device can see (capacity, a
+ *     bounded wait that ran out) are recorded in a device status word that
+ *     cs_sync_status returns; the offending sequence is left unmodified.  Nothing traps.
+ *   - Integer outputs are bit-reproducible from run to run.
+ *
+ * Layouts
+ *   history    int32 [B][stride]; sequence b holds hist_len[b] accepted tokens: prompt,
+ *              earlier turns and everything generated so far (Sec. 3.1).
+ *   KV cache   bf16 [n_layers][2 (K then V)][max_batch][n_kv_heads][max_seq][head_dim],
+ *              contiguous; K is stored rotated (RoPE applied).  Only positions
+ *              [0, kv_len[b]) of sequence b are meaningful (App. B.2).
+ *   weights    bf16 row-major [out][in]:  embed [V][d], lm_head [V][d], final_norm [d];
+ *              per layer attn_norm [d], wqkv [(H + 2 Hkv) Dh][d] (q rows, k rows, v
+ *              rows), wo [d][H Dh], ffn_norm [d], w_gate_up [2 F][d] (gate rows then up
+ *              rows), w_down [d][F].  All base pointers 16-byte aligned; d, H*Dh and F
+ *              multiples of 8.
+ *   blocks     a verification block of sequence b has rows r = 0..draft_len[b]:
+ *              row 0 is the last accepted token (whose K/V are not cached yet), row r>0
+ *              is draft token r-1; row r sits at absolute position kv_len[b] + r.
+ *
+ * State kept between steps of the loop: hist_len[b] = n counts every accepted token
+ * including the last one; kv_len[b] = n - 1.
+ *
+ * Precision: weights, GEMM activation operands and the KV cache are bf16; accumulation,
+ * the residual stream, norms, RoPE and softmax are fp32.
+ */
+#ifndef COPYSPEC_H
+#define COPYSPEC_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct cs_ctx cs_ctx; /* opaque; host memory owned by the library */
+
+typedef enum {
+  CS_OK = 0,
+  CS_ERR_ARG = -1,         /* NULL pointer, negative size, gamma < 1, k > k_max, ...      */
+  CS_ERR_SHAPE = -2,       /* model shape the kernels do not support                      */
+  CS_ERR_CAPACITY = -3,    /* KV cache, history row or workspace too small                */
+  CS_ERR_CUDA = -4,        /* a CUDA runtime/driver call failed (see cs_last_error)       */
+  CS_ERR_TIMEOUT = -5,     /* a bounded device-side wait ran out                          */
+  CS_ERR_UNSUPPORTED = -6  /* valid request outside what is built                         */
+} cs_status;
+
+/* Which occurrence is used when the last gamma tokens recur more than once.  The paper
+ * takes the first one (Sec. 3.2 footnote; App. B.3 step 1(c)); the latest one is the
+ * default here. */
+typedef enum { CS_MATCH_LATEST = 0, CS_MATCH_FIRST = 1 } cs_match_policy;
+
+typedef struct {
+  int32_t n_layers, d_model, n_heads, n_kv_heads, head_dim, d_ffn, vocab;
+  int32_t max_seq;   /* KV positions per sequence                                        */
+  int32_t max_batch; /* sequences per call                                               */
+  int32_t k_max;     /* largest draft length; max_batch * (k_max + 1) <= 256             */
+  float rope_theta, rms_eps;
+} cs_model_config;
+
+typedef struct {
+  const void* embed;
+  const void* lm_head;
+  const void* final_norm;
+  /* host arrays of n_layers device pointers each */
+  const void* const* attn_norm;
+  const void* const* wqkv;
+  const void* const* wo;
+  const void* const* ffn_norm;
+  const void* const* w_gate_up;
+  const void* const* w_down;
+} cs_weights;
+
+#define CS_TAU_HIST 65
+typedef struct {
+  uint64_t steps;     /* verification forwards, summed over sequences                    */
+  uint64_t attempts;  /* steps that had a match, i.e. a copy attempt                     */
+  uint64_t accepted;  /* draft tokens accepted (sum of tau)                              */
+  uint64_t emitted;   /* tokens appended to the histories                                */
+  uint64_t no_match;  /* steps without a match (plain one-token decode)                  */
+  uint64_t tau_hist[CS_TAU_HIST]; /* attempts by accepted length                         */
+} cs_stats;
+
+/* Bytes of device workspace cs_create needs for this configuration (0 on a bad config).
+ * Host-only arithmetic; needs no GPU. */
+size_t cs_workspace_bytes(const cs_model_config* cfg);
+
+/* Builds a context.  `cfg` and `weights` are host structs (copied); `workspace` is a
+ * 1024-byte aligned device buffer of at least cs_workspace_bytes(cfg) bytes.  Clears the
+ * workspace.  Synchronous.  Errors: CS_ERR_ARG, CS_ERR_SHAPE (head_dim not 32, 64 or
+ * 128; n_heads not a multiple of n_kv_heads; max_batch*(k_max+1) > 256; dims not
+ * multiples of 8), CS_ERR_CAPACITY, CS_ERR_CUDA. */
+cs_status cs_create(cs_ctx** out, const cs_model_config* cfg, const cs_weights* weights,
+                    void* workspace, size_t workspace_bytes);
+void cs_destroy(cs_ctx* ctx);
+
+/* Text of the last host-side error of this context (static string if ctx is NULL). */
+const char* cs_last_error(const cs_ctx* ctx);
+
+/* Waits for `stream`, then returns and clears the device status word of the context:
+ * CS_OK, CS_ERR_CAPACITY, CS_ERR_ARG (cs_kv_truncate asked to grow) or CS_ERR_TIMEOUT. */
+cs_status cs_sync_status(cs_ctx* ctx, void* stream);
+
+/* Suffix-match search and draft gather (Sec. 3.1; Sec. 3.2; App. B.3 step 1).  Async.
+ * For each sequence b with n = hist_len[b]: among all p0 in [0, n - 2 gamma] with
+ * hist[b][p0 + j] == hist[b][n - gamma + j] for every j < gamma (exact token equality;
+ * the match may not overlap the key, App. B.3 step 1(c)), match_pos[b] is the largest
+ * (LATEST) or smallest (FIRST), or -1 if there is none or n < 2 gamma.  The draft is
+ * the draft_len[b] = min(k, n - (p0 + gamma)) tokens that follow the match (0 without a
+ * match); draft entries past draft_len[b] are set to -1.
+ *   hist [B][stride] int32, hist_len [B] int32, match_pos [B], draft [B][k],
+ *   draft_len [B].  1 <= gamma <= 8, 0 <= k, B >= 0 (B == 0 is a no-op).
+ *   Needs no context and no scratch memory.  Errors: CS_ERR_ARG, CS_ERR_CUDA. */
+cs_status cs_find_match(const int32_t* hist, const int32_t* hist_len, int B, int stride,
+                        int gamma, int k, cs_match_policy policy, int32_t* match_pos,
+                        int32_t* draft, int32_t* draft_len, void* stream);
+
+/* One verification forward plus acceptance (Sec. 3.2; App. B.2; App. B.3 step 2). Async.
+ * Evaluates the block [last_tok[b], draft[b][0 .. draft_len[b])] of every sequence at
+ * positions kv_len[b].. in one forward, appends the block's K/V rows to the cache,
+ * takes argmax_ids[b][r] = the lowest id with the largest logit of row r (never
+ * writing logits to memory unless logits_dbg is given), and accepts
+ *   tau = the largest j <= draft_len[b] with draft[b][i] == target[i] for all i < j,
+ * where target[r] = argmax_ids[b][r], or target_script[b][r] when target_script is not
+ * NULL (scripted-target mode: the forward and argmax are still computed in full, but
+ * acceptance follows the given stream).  Outputs: accept_len[b] = tau, out_tokens[b][0..
+ * tau] = target[0..tau] (tau accepted tokens and one extra token, Sec. 3.2; the rest of
+ * the row is -1), and kv_len[b] += tau + 1, which is the truncation of App. B.2: the
+ * cached rows of rejected tokens lie beyond kv_len and are dead.
+ *   last_tok [B], draft [B][k], draft_len [B] (0..k), kv_len [B] in/out,
+ *   target_script [B][k+1] or NULL, accept_len [B], out_tokens [B][k+1],
+ *   argmax_ids [B][k+1] (rows past draft_len[b] are -1),
+ *   logits_dbg fp32 [B][k+1][vocab] or NULL.
+ * A sequence with kv_len[b] + draft_len[b] + 1 > max_seq is skipped (accept_len -1,
+ * nothing modified) and CS_ERR_CAPACITY is recorded in the status word.
+ * Errors on the host: CS_ERR_ARG (NULL, B > max_batch, k > k_max). */
+cs_status cs_verify_step(cs_ctx* ctx, const int32_t* last_tok, const int32_t* draft,
+                         const int32_t* draft_len, int B, int k, void* kv_cache,
+                         int32_t* kv_len, const int32_t* target_script, int32_t* accept_len,
+                         int32_t* out_tokens, int32_t* argmax_ids, float* logits_dbg,
+                         void* stream);
+
+/* KV truncation to an accepted length (App. B.2; App. B.3 step 2(b)).  Async.
+ * kv_len[b] = new_len[b] where 0 <= new_len[b] <= kv_len[b]; otherwise kv_len[b] is
+ * left as is and CS_ERR_ARG is recorded in the status word.  The cache is contiguous
+ * and indexed by length, so no K/V bytes move. */
+cs_status cs_kv_truncate(cs_ctx* ctx, int32_t* kv_len, const int32_t* new_len, int B,
+                         void* stream);
+
+/* The generation loop (App. B.3 steps 1, 2 and 4; Sec. 3.2).  Synchronous.
+ * Repeats {search, gather, verify, accept, truncate, append} for all B sequences until
+ * each has emitted max_new tokens (the last block is clipped) or, in real mode, has
+ * emitted eos_id (tokens after it are dropped; eos_id < 0 = none).  On entry the cache
+ * must hold positions [0, hist_len[b] - 1) and kv_len[b] = hist_len[b] - 1.  Accepted
+ * tokens are appended to hist and hist_len/kv_len advance.  `script` [B][max_new]
+ * switches to scripted-target mode: row r of a step is checked against
+ * script[b][emitted_b + r]; the emitted stream then equals the script.  k = 0 gives
+ * plain one-token decoding from the same kernels.
+ *   stats_out: host pointer or NULL.  stride >= hist_len[b] + max_new and
+ *   max_seq >= hist_len[b] + max_new + k are required (checked on the device:
+ *   CS_ERR_CAPACITY, that sequence stops).
+ * Returns the first error among the host checks, CUDA and the device status word. */
+cs_status cs_decode_loop(cs_ctx* ctx, int32_t* hist, int32_t* hist_len, int B, int stride,
+                         void* kv_cache, int32_t* kv_len, int gamma, int k,
+                         cs_match_policy policy, int max_new, int eos_id,
+                         const int32_t* script, cs_stats* stats_out, void* stream);
+
+/* Helper off the hot path: computes the KV cache of positions [0, hist_len[b] - 1) by
+ * running the forward over the history in blocks with every row forced (no LM head, no
+ * acceptance), and sets kv_len[b] = hist_len[b] - 1.  `max_len` (host) is an upper bound
+ * of hist_len.  Async. */
+cs_status cs_prefill(cs_ctx* ctx, const int32_t* hist, const int32_t* hist_len, int B,
+                     int stride, int max_len, void* kv_cache, int32_t* kv_len, void* stream);
+
+/* Building block of the forward of Sec. 3.2, exposed for testing the tensor-core path in
+ * isolation: Y[rows][N] (fp32) = X[rows][K] (bf16) times W[N][K]^T (bf16), fp32
+ * accumulation.  rows <= 256; K a multiple of 8; X must be readable for
+ * ceil(rows/16)*16 rows.  Uses the context's workspace (so it must not overlap other
+ * work of the context).  Async. */
+cs_status cs_linear(cs_ctx* ctx, const void* X, const void* W, int rows, int N, int K,
+                    float* Y, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* COPYSPEC_H */

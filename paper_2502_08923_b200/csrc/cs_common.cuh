@@ -1,0 +1,155 @@
+// Shared declarations of the copy-and-verify library: context layout, launch helpers,
+// the device status word.  Every .cu file of the library includes this.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <string.h>
+
+#include "copyspec.h"
+
+// ---------------------------------------------------------------- device status word
+// Bits OR-ed into the context's status word by kernels; cs_sync_status maps them.
+enum : int {
+  CS_DEV_CAPACITY = 1,  // KV cache / history row too small for this step
+  CS_DEV_BADARG = 2,    // cs_kv_truncate asked to grow
+  CS_DEV_TIMEOUT = 4    // a bounded wait ran out
+};
+
+static constexpr int CS_MAX_ROWS = 256;   // rows of one verification block (UMMA N limit)
+static constexpr int CS_GEMM_BM = 128;    // out-features per CTA tile (UMMA M)
+static constexpr int CS_GEMM_BK = 64;     // K elements per stage (one 128-byte swizzle row)
+static constexpr int CS_MAX_GAMMA = 8;
+static constexpr int CS_MAX_SPLITS = 16;  // split-K factor limit
+static constexpr int CS_SPLIT_TILE_CAP = 640;  // tiles * splits never exceeds this (unless splits == 1)
+
+struct GemmPlan {
+  CUtensorMap tmW;      // weights [N][K], box 128 x 64, 128-byte swizzle
+  const __nv_bfloat16* W;
+  int N, K;
+  int splits;           // split-K factor
+  int kb_per_split;     // 64-wide K blocks per split
+};
+
+struct LayerPlan {
+  GemmPlan qkv, o, gate_up, down;
+  const __nv_bfloat16 *attn_norm, *ffn_norm;
+};
+
+struct cs_ctx {
+  cs_model_config cfg;
+  int max_rows;      // max_batch * (k_max + 1)
+  int rows_pad;      // rounded up to 16
+  int attn_splits;   // split-KV factor
+  bool gemm_simt;    // bring-up path: plain CUDA-core GEMM instead of tcgen05
+  int num_sms;
+
+  const __nv_bfloat16 *embed, *final_norm;
+  LayerPlan* layers;  // host array
+  GemmPlan lm;
+
+  // workspace partition (device)
+  char* ws;
+  size_t ws_bytes;
+  float* x;                  // residual stream fp32 [rows_pad][d]
+  __nv_bfloat16* xn;         // normed activations bf16 [rows_pad][d]
+  __nv_bfloat16* attn_out;   // attention output bf16 [rows_pad][H*Dh]
+  __nv_bfloat16* act;        // SwiGLU output bf16 [rows_pad][F]
+  __nv_bfloat16* qbuf;       // rotated queries bf16 [rows_pad][H*Dh]
+  float* partial;            // split-K partial sums fp32 [splits][rows][N]
+  size_t partial_elems;
+  float* attn_o;             // split-KV partial outputs [splits][rows][H][Dh]
+  float* attn_ml;            // split-KV (max, sum) [splits][rows][H][2]
+  float* rope_cs;            // cos/sin of this block [rows][Dh/2][2]
+  double* inv_freq;          // theta^(-2i/Dh) [Dh/2]
+  float* tile_max;           // LM-head tile maxima [tiles][rows_pad]
+  int* tile_idx;             // and their token ids
+  int* row_tok;              // token id per row [rows_pad]
+  int* row_pos;              // absolute position per row
+  int* row_lim;              // number of keys a row attends to (0 = dead row)
+  int* row_write;            // 1 = this row's K/V go into the cache
+  int* seq_ok;               // per sequence: 1 = takes part in this step
+  int* d_status;             // device status word
+  // loop state, all [max_batch] unless noted
+  int* loop_last;
+  int* loop_draft;           // [max_batch][k_max]
+  int* loop_dlen;
+  int* loop_mpos;
+  int* loop_emitted;
+  int* loop_done;            // [max_batch] + 1 (last = number of finished sequences)
+  int* loop_accept;
+  int* loop_out;             // [max_batch][k_max+1]
+  int* loop_argmax;          // [max_batch][k_max+1]
+  unsigned long long* loop_stats;  // image of cs_stats
+
+  // activation operand maps, rebuilt when the block height changes
+  int act_ntok;
+  CUtensorMap tmXn, tmAttn, tmAct;
+
+  char err[256];
+};
+
+#define CS_CUDA_OK(ctx, call)                                                          \
+  do {                                                                                 \
+    cudaError_t e__ = (call);                                                          \
+    if (e__ != cudaSuccess) {                                                          \
+      if (ctx) snprintf((ctx)->err, sizeof((ctx)->err), "%s: %s", #call,               \
+                        cudaGetErrorString(e__));                                      \
+      return CS_ERR_CUDA;                                                              \
+    }                                                                                  \
+  } while (0)
+
+static inline int cs_ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// split-K factor limit for a GEMM of `tiles` 128-row tiles and `kb` 64-wide K blocks
+static inline int cs_max_splits(int tiles, int kb) {
+  int s = CS_SPLIT_TILE_CAP / tiles;
+  if (s > CS_MAX_SPLITS) s = CS_MAX_SPLITS;
+  if (s > kb / 4) s = kb / 4;
+  return s < 1 ? 1 : s;
+}
+
+// ------------------------------------------------------------------ kernel launchers
+// cs_match.cu
+cs_status cs_launch_find_match(const int32_t* hist, const int32_t* hist_len, int B, int stride,
+                               int gamma, int k, int policy, int32_t* match_pos, int32_t* draft,
+                               int32_t* draft_len, int32_t* last_tok, const int32_t* skip,
+                               cudaStream_t st);
+// cs_gemm.cu
+cs_status cs_gemm_plan(cs_ctx* ctx, GemmPlan* g, const void* w, int N, int K, bool allow_split);
+cs_status cs_make_act_map(cs_ctx* ctx, CUtensorMap* tm, const void* base, int rows_total, int K,
+                          int box_rows);
+// mode 0: partial[s][row][n] fp32; mode 1: per-tile argmax (tile_max/tile_idx) + optional logits
+cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX,
+                         const __nv_bfloat16* X, int rows, int mode, float* out, float* logits,
+                         cudaStream_t st);
+// cs_layers.cu
+void cs_launch_block_setup(cs_ctx* ctx, const int32_t* last_tok, const int32_t* draft,
+                           const int32_t* draft_len, const int32_t* kv_len, int B, int k,
+                           cudaStream_t st);
+void cs_launch_prefill_setup(cs_ctx* ctx, const int32_t* hist, const int32_t* hist_len, int B,
+                             int stride, int start, int R, cudaStream_t st);
+void cs_launch_embed(cs_ctx* ctx, int rows, cudaStream_t st);
+void cs_launch_rmsnorm(cs_ctx* ctx, const float* partial, int splits, const __nv_bfloat16* gain,
+                       int rows, cudaStream_t st);
+void cs_launch_qkv_post(cs_ctx* ctx, int splits, void* kv_cache, int layer, int B, int R,
+                        cudaStream_t st);
+void cs_launch_attention(cs_ctx* ctx, const void* kv_cache, int layer, int B, int R,
+                         cudaStream_t st);
+void cs_launch_swiglu(cs_ctx* ctx, int splits, int rows, cudaStream_t st);
+void cs_launch_accept(cs_ctx* ctx, int B, int k, const int32_t* draft, const int32_t* draft_len,
+                      const int32_t* script, int script_stride, const int32_t* script_off,
+                      int script_limit, int32_t* accept_len, int32_t* out_tokens,
+                      int32_t* argmax_ids, int32_t* kv_len, int update_kv, cudaStream_t st);
+void cs_launch_truncate(cs_ctx* ctx, int32_t* kv_len, const int32_t* new_len, int B,
+                        cudaStream_t st);
+void cs_launch_prefill_finish(cs_ctx* ctx, const int32_t* hist_len, int32_t* kv_len, int B,
+                              cudaStream_t st);
+void cs_launch_loop_init(cs_ctx* ctx, const int32_t* hist_len, const int32_t* kv_len, int B,
+                         int stride, int max_new, int k, cudaStream_t st);
+void cs_launch_loop_commit(cs_ctx* ctx, int32_t* hist, int32_t* hist_len, int B, int stride,
+                           int32_t* kv_len, int k, int max_new, int eos_id, int scripted,
+                           cudaStream_t st);
