@@ -1,0 +1,468 @@
+// C ABI of the copy-and-verify library: argument checks, workspace layout, the chain of
+// kernels of one verification step and the device-resident generation loop.
+#include <math.h>
+#include <stdlib.h>
+
+#include <new>
+
+#include "cs_common.cuh"
+
+namespace {
+
+struct WsLayout {
+  size_t x, xn, attn_out, act, qbuf, partial, attn_o, attn_ml, rope_cs, inv_freq, tile_max, tile_idx,
+      row_tok, row_pos, row_lim, row_write, seq_ok, status, loop_last, loop_draft, loop_dlen, loop_mpos,
+      loop_emitted, loop_done, loop_accept, loop_out, loop_argmax, loop_stats, total;
+  size_t partial_elems;
+  int attn_splits;
+};
+
+bool config_ok(const cs_model_config* c) {
+  if (c == nullptr) return false;
+  if (c->n_layers < 1 || c->d_model < 8 || c->n_heads < 1 || c->n_kv_heads < 1 || c->d_ffn < 8 ||
+      c->vocab < 1 || c->max_seq < 1 || c->max_batch < 1 || c->k_max < 0)
+    return false;
+  if (c->head_dim != 32 && c->head_dim != 64 && c->head_dim != 128) return false;
+  if (c->n_heads % c->n_kv_heads) return false;
+  if ((long)c->max_batch * (c->k_max + 1) > CS_MAX_ROWS) return false;
+  if (c->d_model % 8 || c->d_ffn % 8 || (c->n_heads * c->head_dim) % 8) return false;
+  return true;
+}
+
+size_t take(size_t* off, size_t bytes) {
+  const size_t at = *off;
+  *off = (at + bytes + 1023) & ~(size_t)1023;
+  return at;
+}
+
+WsLayout ws_layout(const cs_model_config* c) {
+  WsLayout L;
+  const size_t rows = CS_MAX_ROWS;
+  const size_t d = c->d_model, qd = (size_t)c->n_heads * c->head_dim, F = c->d_ffn;
+  const size_t qkv = qd + 2 * (size_t)c->n_kv_heads * c->head_dim;
+  // largest splits * N over the four projections of a layer
+  size_t pe = 0;
+  const size_t shapes[4][2] = {{qkv, d}, {d, qd}, {2 * F, d}, {d, F}};
+  for (int i = 0; i < 4; ++i) {
+    const int tiles = cs_ceil_div((int)shapes[i][0], CS_GEMM_BM), kb = cs_ceil_div((int)shapes[i][1], CS_GEMM_BK);
+    const size_t e = (size_t)cs_max_splits(tiles, kb) * shapes[i][0];
+    if (e > pe) pe = e;
+  }
+  L.partial_elems = pe * rows;
+  int as = cs_ceil_div(c->max_seq, 256);
+  L.attn_splits = as < 1 ? 1 : (as > 32 ? 32 : as);
+  const size_t lm_tiles = cs_ceil_div(c->vocab, CS_GEMM_BM);
+  size_t off = 0;
+  L.x = take(&off, rows * d * 4);
+  L.xn = take(&off, rows * d * 2);
+  L.attn_out = take(&off, rows * qd * 2);
+  L.act = take(&off, rows * F * 2);
+  L.qbuf = take(&off, rows * qd * 2);
+  L.partial = take(&off, L.partial_elems * 4);
+  L.attn_o = take(&off, (size_t)L.attn_splits * rows * qd * 4);
+  L.attn_ml = take(&off, (size_t)L.attn_splits * rows * c->n_heads * 2 * 4);
+  L.rope_cs = take(&off, rows * c->head_dim * 4);
+  L.inv_freq = take(&off, (size_t)c->head_dim / 2 * 8);
+  L.tile_max = take(&off, lm_tiles * rows * 4);
+  L.tile_idx = take(&off, lm_tiles * rows * 4);
+  L.row_tok = take(&off, rows * 4);
+  L.row_pos = take(&off, rows * 4);
+  L.row_lim = take(&off, rows * 4);
+  L.row_write = take(&off, rows * 4);
+  L.seq_ok = take(&off, rows * 4);
+  L.status = take(&off, 256);
+  L.loop_last = take(&off, rows * 4);
+  L.loop_draft = take(&off, rows * 4);
+  L.loop_dlen = take(&off, rows * 4);
+  L.loop_mpos = take(&off, rows * 4);
+  L.loop_emitted = take(&off, rows * 4);
+  L.loop_done = take(&off, (rows + 1) * 4);
+  L.loop_accept = take(&off, rows * 4);
+  L.loop_out = take(&off, rows * 4);
+  L.loop_argmax = take(&off, rows * 4);
+  L.loop_stats = take(&off, sizeof(cs_stats));
+  L.total = off;
+  return L;
+}
+
+cs_status fail(cs_ctx* ctx, cs_status s, const char* msg) {
+  if (ctx) snprintf(ctx->err, sizeof(ctx->err), "%s", msg);
+  return s;
+}
+
+cs_status ensure_act_maps(cs_ctx* ctx, int n_tok) {
+  if (ctx->act_ntok == n_tok) return CS_OK;
+  const cs_model_config& c = ctx->cfg;
+  cs_status s;
+  if ((s = cs_make_act_map(ctx, &ctx->tmXn, ctx->xn, CS_MAX_ROWS, c.d_model, n_tok)) != CS_OK) return s;
+  if ((s = cs_make_act_map(ctx, &ctx->tmAttn, ctx->attn_out, CS_MAX_ROWS, c.n_heads * c.head_dim, n_tok)) != CS_OK)
+    return s;
+  if ((s = cs_make_act_map(ctx, &ctx->tmAct, ctx->act, CS_MAX_ROWS, c.d_ffn, n_tok)) != CS_OK) return s;
+  ctx->act_ntok = n_tok;
+  return CS_OK;
+}
+
+// The forward of Sec. 3.2 over the rows prepared by a *_setup kernel: B sequences of R
+// rows each.  With `with_lm` the LM head leaves per-tile (max, id) pairs for k_accept.
+cs_status enqueue_forward(cs_ctx* ctx, int B, int R, void* kv_cache, bool with_lm, float* logits,
+                          cudaStream_t st) {
+  const cs_model_config& c = ctx->cfg;
+  const int rows = B * R;
+  cs_status s = ensure_act_maps(ctx, cs_ceil_div(rows, 16) * 16);
+  if (s != CS_OK) return s;
+  cs_launch_embed(ctx, rows, st);
+  int prev_splits = 0;
+  for (int l = 0; l < c.n_layers; ++l) {
+    const LayerPlan& L = ctx->layers[l];
+    cs_launch_rmsnorm(ctx, l == 0 ? nullptr : ctx->partial, prev_splits, L.attn_norm, rows, st);
+    if ((s = cs_launch_gemm(ctx, &L.qkv, &ctx->tmXn, ctx->xn, rows, 0, ctx->partial, nullptr, st)) != CS_OK) return s;
+    cs_launch_qkv_post(ctx, L.qkv.splits, kv_cache, l, B, R, st);
+    cs_launch_attention(ctx, kv_cache, l, B, R, st);
+    if ((s = cs_launch_gemm(ctx, &L.o, &ctx->tmAttn, ctx->attn_out, rows, 0, ctx->partial, nullptr, st)) != CS_OK) return s;
+    cs_launch_rmsnorm(ctx, ctx->partial, L.o.splits, L.ffn_norm, rows, st);
+    if ((s = cs_launch_gemm(ctx, &L.gate_up, &ctx->tmXn, ctx->xn, rows, 0, ctx->partial, nullptr, st)) != CS_OK) return s;
+    cs_launch_swiglu(ctx, L.gate_up.splits, rows, st);
+    if ((s = cs_launch_gemm(ctx, &L.down, &ctx->tmAct, ctx->act, rows, 0, ctx->partial, nullptr, st)) != CS_OK) return s;
+    prev_splits = L.down.splits;
+  }
+  if (with_lm) {
+    cs_launch_rmsnorm(ctx, ctx->partial, prev_splits, ctx->final_norm, rows, st);
+    if ((s = cs_launch_gemm(ctx, &ctx->lm, &ctx->tmXn, ctx->xn, rows, 1, nullptr, logits, st)) != CS_OK) return s;
+  }
+  CS_CUDA_OK(ctx, cudaGetLastError());
+  return CS_OK;
+}
+
+__global__ void k_reduce_partial(const float* __restrict__ partial, int splits, int rows, int N,
+                                 float* __restrict__ y) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= (size_t)rows * N) return;
+  float v = 0.f;
+  for (int s = 0; s < splits; ++s) v += partial[(size_t)s * rows * N + i];
+  y[i] = v;
+}
+
+cs_status status_from_bits(cs_ctx* ctx, int bits) {
+  if (bits & CS_DEV_TIMEOUT) return fail(ctx, CS_ERR_TIMEOUT, "a bounded device-side wait ran out");
+  if (bits & CS_DEV_CAPACITY) return fail(ctx, CS_ERR_CAPACITY, "KV cache or history row too small for a sequence");
+  if (bits & CS_DEV_BADARG) return fail(ctx, CS_ERR_ARG, "device-side argument check failed (lengths inconsistent)");
+  return CS_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t cs_workspace_bytes(const cs_model_config* cfg) {
+  if (!config_ok(cfg)) return 0;
+  return ws_layout(cfg).total;
+}
+
+const char* cs_last_error(const cs_ctx* ctx) { return ctx ? ctx->err : "no context"; }
+
+cs_status cs_create(cs_ctx** out, const cs_model_config* cfg, const cs_weights* w, void* workspace,
+                    size_t workspace_bytes) {
+  if (out == nullptr) return CS_ERR_ARG;
+  *out = nullptr;
+  if (cfg == nullptr || w == nullptr || workspace == nullptr) return CS_ERR_ARG;
+  if (!config_ok(cfg)) return CS_ERR_SHAPE;
+  if (w->embed == nullptr || w->lm_head == nullptr || w->final_norm == nullptr || w->attn_norm == nullptr ||
+      w->wqkv == nullptr || w->wo == nullptr || w->ffn_norm == nullptr || w->w_gate_up == nullptr ||
+      w->w_down == nullptr)
+    return CS_ERR_ARG;
+  const WsLayout L = ws_layout(cfg);
+  if (workspace_bytes < L.total) return CS_ERR_CAPACITY;
+  if (reinterpret_cast<uintptr_t>(workspace) & 1023) return CS_ERR_ARG;
+
+  cs_ctx* ctx = new (std::nothrow) cs_ctx();
+  if (ctx == nullptr) return CS_ERR_ARG;
+  memset(static_cast<void*>(ctx), 0, sizeof(*ctx));
+  ctx->cfg = *cfg;
+  ctx->max_rows = cfg->max_batch * (cfg->k_max + 1);
+  ctx->rows_pad = CS_MAX_ROWS;
+  ctx->attn_splits = L.attn_splits;
+  ctx->partial_elems = L.partial_elems;
+  const char* env = getenv("CS_GEMM_SIMT");
+  ctx->gemm_simt = (env != nullptr && env[0] == '1');
+  ctx->layers = new (std::nothrow) LayerPlan[cfg->n_layers];
+  cs_status s = CS_OK;
+  int dev = 0;
+  cudaDeviceProp prop;
+#define CREATE_OK(call)                                                                        \
+  do {                                                                                         \
+    cudaError_t e__ = (call);                                                                  \
+    if (e__ != cudaSuccess) {                                                                  \
+      fprintf(stderr, "cs_create: %s: %s\n", #call, cudaGetErrorString(e__));                  \
+      cs_destroy(ctx);                                                                         \
+      return CS_ERR_CUDA;                                                                      \
+    }                                                                                          \
+  } while (0)
+  if (ctx->layers == nullptr) { cs_destroy(ctx); return CS_ERR_ARG; }
+  CREATE_OK(cudaGetDevice(&dev));
+  CREATE_OK(cudaGetDeviceProperties(&prop, dev));
+  if (prop.major != 10) {
+    fprintf(stderr, "cs_create: this library is built for sm_100a only (device is sm_%d%d)\n", prop.major, prop.minor);
+    cs_destroy(ctx);
+    return CS_ERR_UNSUPPORTED;
+  }
+  ctx->num_sms = prop.multiProcessorCount;
+  char* base = static_cast<char*>(workspace);
+  ctx->ws = base;
+  ctx->ws_bytes = L.total;
+  CREATE_OK(cudaMemset(base, 0, L.total));
+  ctx->x = reinterpret_cast<float*>(base + L.x);
+  ctx->xn = reinterpret_cast<__nv_bfloat16*>(base + L.xn);
+  ctx->attn_out = reinterpret_cast<__nv_bfloat16*>(base + L.attn_out);
+  ctx->act = reinterpret_cast<__nv_bfloat16*>(base + L.act);
+  ctx->qbuf = reinterpret_cast<__nv_bfloat16*>(base + L.qbuf);
+  ctx->partial = reinterpret_cast<float*>(base + L.partial);
+  ctx->attn_o = reinterpret_cast<float*>(base + L.attn_o);
+  ctx->attn_ml = reinterpret_cast<float*>(base + L.attn_ml);
+  ctx->rope_cs = reinterpret_cast<float*>(base + L.rope_cs);
+  ctx->inv_freq = reinterpret_cast<double*>(base + L.inv_freq);
+  ctx->tile_max = reinterpret_cast<float*>(base + L.tile_max);
+  ctx->tile_idx = reinterpret_cast<int*>(base + L.tile_idx);
+  ctx->row_tok = reinterpret_cast<int*>(base + L.row_tok);
+  ctx->row_pos = reinterpret_cast<int*>(base + L.row_pos);
+  ctx->row_lim = reinterpret_cast<int*>(base + L.row_lim);
+  ctx->row_write = reinterpret_cast<int*>(base + L.row_write);
+  ctx->seq_ok = reinterpret_cast<int*>(base + L.seq_ok);
+  ctx->d_status = reinterpret_cast<int*>(base + L.status);
+  ctx->loop_last = reinterpret_cast<int*>(base + L.loop_last);
+  ctx->loop_draft = reinterpret_cast<int*>(base + L.loop_draft);
+  ctx->loop_dlen = reinterpret_cast<int*>(base + L.loop_dlen);
+  ctx->loop_mpos = reinterpret_cast<int*>(base + L.loop_mpos);
+  ctx->loop_emitted = reinterpret_cast<int*>(base + L.loop_emitted);
+  ctx->loop_done = reinterpret_cast<int*>(base + L.loop_done);
+  ctx->loop_accept = reinterpret_cast<int*>(base + L.loop_accept);
+  ctx->loop_out = reinterpret_cast<int*>(base + L.loop_out);
+  ctx->loop_argmax = reinterpret_cast<int*>(base + L.loop_argmax);
+  ctx->loop_stats = reinterpret_cast<unsigned long long*>(base + L.loop_stats);
+
+  // rotary frequencies theta^(-2i/Dh), in double
+  {
+    const int half = cfg->head_dim / 2;
+    double f[64];
+    for (int i = 0; i < half; ++i) f[i] = pow((double)cfg->rope_theta, -2.0 * i / cfg->head_dim);
+    CREATE_OK(cudaMemcpy(ctx->inv_freq, f, sizeof(double) * half, cudaMemcpyHostToDevice));
+  }
+  ctx->embed = static_cast<const __nv_bfloat16*>(w->embed);
+  ctx->final_norm = static_cast<const __nv_bfloat16*>(w->final_norm);
+  const int d = cfg->d_model, qd = cfg->n_heads * cfg->head_dim, F = cfg->d_ffn;
+  const int qkv = qd + 2 * cfg->n_kv_heads * cfg->head_dim;
+  for (int l = 0; l < cfg->n_layers && s == CS_OK; ++l) {
+    LayerPlan& P = ctx->layers[l];
+    if (!w->attn_norm[l] || !w->wqkv[l] || !w->wo[l] || !w->ffn_norm[l] || !w->w_gate_up[l] || !w->w_down[l]) {
+      s = CS_ERR_ARG;
+      break;
+    }
+    P.attn_norm = static_cast<const __nv_bfloat16*>(w->attn_norm[l]);
+    P.ffn_norm = static_cast<const __nv_bfloat16*>(w->ffn_norm[l]);
+    if ((s = cs_gemm_plan(ctx, &P.qkv, w->wqkv[l], qkv, d, true)) != CS_OK) break;
+    if ((s = cs_gemm_plan(ctx, &P.o, w->wo[l], d, qd, true)) != CS_OK) break;
+    if ((s = cs_gemm_plan(ctx, &P.gate_up, w->w_gate_up[l], 2 * F, d, true)) != CS_OK) break;
+    if ((s = cs_gemm_plan(ctx, &P.down, w->w_down[l], d, F, true)) != CS_OK) break;
+  }
+  if (s == CS_OK) s = cs_gemm_plan(ctx, &ctx->lm, w->lm_head, cfg->vocab, d, false);
+  if (s != CS_OK) {
+    fprintf(stderr, "cs_create: %s\n", ctx->err);
+    cs_destroy(ctx);
+    return s;
+  }
+#undef CREATE_OK
+  *out = ctx;
+  return CS_OK;
+}
+
+void cs_destroy(cs_ctx* ctx) {
+  if (ctx == nullptr) return;
+  delete[] ctx->layers;
+  delete ctx;
+}
+
+cs_status cs_sync_status(cs_ctx* ctx, void* stream) {
+  if (ctx == nullptr) return CS_ERR_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int bits = 0;
+  CS_CUDA_OK(ctx, cudaMemcpyAsync(&bits, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost, st));
+  CS_CUDA_OK(ctx, cudaMemsetAsync(ctx->d_status, 0, sizeof(int), st));
+  CS_CUDA_OK(ctx, cudaStreamSynchronize(st));
+  return status_from_bits(ctx, bits);
+}
+
+cs_status cs_find_match(const int32_t* hist, const int32_t* hist_len, int B, int stride, int gamma, int k,
+                        cs_match_policy policy, int32_t* match_pos, int32_t* draft, int32_t* draft_len,
+                        void* stream) {
+  if (B < 0 || k < 0 || stride < 0) return CS_ERR_ARG;
+  if (gamma < 1 || gamma > CS_MAX_GAMMA) return CS_ERR_ARG;
+  if (policy != CS_MATCH_LATEST && policy != CS_MATCH_FIRST) return CS_ERR_ARG;
+  if (B == 0) return CS_OK;
+  if (B > 65535) return CS_ERR_ARG;
+  if (hist == nullptr || hist_len == nullptr || match_pos == nullptr || draft_len == nullptr ||
+      (draft == nullptr && k > 0))
+    return CS_ERR_ARG;
+  return cs_launch_find_match(hist, hist_len, B, stride, gamma, k, (int)policy, match_pos, draft, draft_len,
+                              nullptr, nullptr, static_cast<cudaStream_t>(stream));
+}
+
+cs_status cs_verify_step(cs_ctx* ctx, const int32_t* last_tok, const int32_t* draft, const int32_t* draft_len,
+                         int B, int k, void* kv_cache, int32_t* kv_len, const int32_t* target_script,
+                         int32_t* accept_len, int32_t* out_tokens, int32_t* argmax_ids, float* logits_dbg,
+                         void* stream) {
+  if (ctx == nullptr) return CS_ERR_ARG;
+  if (B < 1 || B > ctx->cfg.max_batch || k < 0 || k > ctx->cfg.k_max) return fail(ctx, CS_ERR_ARG, "B or k out of range");
+  if (last_tok == nullptr || draft_len == nullptr || (draft == nullptr && k > 0) || kv_cache == nullptr ||
+      kv_len == nullptr || accept_len == nullptr || out_tokens == nullptr || argmax_ids == nullptr)
+    return fail(ctx, CS_ERR_ARG, "NULL argument");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cs_launch_block_setup(ctx, last_tok, draft, draft_len, kv_len, nullptr, B, k, st);
+  cs_status s = enqueue_forward(ctx, B, k + 1, kv_cache, true, logits_dbg, st);
+  if (s != CS_OK) return s;
+  cs_launch_accept(ctx, B, k, draft, draft_len, target_script, k + 1, nullptr, k + 1, accept_len, out_tokens,
+                   argmax_ids, kv_len, 1, st);
+  CS_CUDA_OK(ctx, cudaGetLastError());
+  return CS_OK;
+}
+
+cs_status cs_kv_truncate(cs_ctx* ctx, int32_t* kv_len, const int32_t* new_len, int B, void* stream) {
+  if (ctx == nullptr) return CS_ERR_ARG;
+  if (B < 0 || kv_len == nullptr || new_len == nullptr) return fail(ctx, CS_ERR_ARG, "bad argument");
+  if (B == 0) return CS_OK;
+  cs_launch_truncate(ctx, kv_len, new_len, B, static_cast<cudaStream_t>(stream));
+  CS_CUDA_OK(ctx, cudaGetLastError());
+  return CS_OK;
+}
+
+cs_status cs_prefill(cs_ctx* ctx, const int32_t* hist, const int32_t* hist_len, int B, int stride, int max_len,
+                     void* kv_cache, int32_t* kv_len, void* stream) {
+  if (ctx == nullptr) return CS_ERR_ARG;
+  if (B < 1 || B > ctx->cfg.max_batch || hist == nullptr || hist_len == nullptr || kv_cache == nullptr ||
+      kv_len == nullptr || max_len < 0 || stride < max_len)
+    return fail(ctx, CS_ERR_ARG, "bad argument");
+  if (max_len - 1 > ctx->cfg.max_seq) return fail(ctx, CS_ERR_CAPACITY, "history longer than the KV cache");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int R = CS_MAX_ROWS / B;
+  const int total = max_len - 1;   // positions whose K/V are cached
+  for (int start = 0; start < total; start += R) {
+    const int r = (total - start < R) ? total - start : R;
+    cs_launch_prefill_setup(ctx, hist, hist_len, B, stride, start, r, st);
+    cs_status s = enqueue_forward(ctx, B, r, kv_cache, false, nullptr, st);
+    if (s != CS_OK) return s;
+  }
+  if (total <= 0) cs_launch_prefill_setup(ctx, hist, hist_len, B, stride, 0, 1, st);   // sets seq_ok
+  cs_launch_prefill_finish(ctx, hist_len, kv_len, B, st);
+  CS_CUDA_OK(ctx, cudaGetLastError());
+  return CS_OK;
+}
+
+cs_status cs_decode_loop(cs_ctx* ctx, int32_t* hist, int32_t* hist_len, int B, int stride, void* kv_cache,
+                         int32_t* kv_len, int gamma, int k, cs_match_policy policy, int max_new, int eos_id,
+                         const int32_t* script, cs_stats* stats_out, void* stream) {
+  if (ctx == nullptr) return CS_ERR_ARG;
+  if (B < 1 || B > ctx->cfg.max_batch || k < 0 || k > ctx->cfg.k_max || gamma < 1 || gamma > CS_MAX_GAMMA ||
+      max_new < 0 || stride < 1)
+    return fail(ctx, CS_ERR_ARG, "B, k, gamma, max_new or stride out of range");
+  if (policy != CS_MATCH_LATEST && policy != CS_MATCH_FIRST) return fail(ctx, CS_ERR_ARG, "bad policy");
+  if (hist == nullptr || hist_len == nullptr || kv_cache == nullptr || kv_len == nullptr)
+    return fail(ctx, CS_ERR_ARG, "NULL argument");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const char* env = getenv("CS_NO_GRAPH");
+  const bool use_graph = !(env != nullptr && env[0] == '1');
+
+  cs_launch_loop_init(ctx, hist_len, kv_len, B, stride, max_new, k, st);
+  CS_CUDA_OK(ctx, cudaGetLastError());
+  // the activation maps must exist before capture (encoding is host work)
+  cs_status s = ensure_act_maps(ctx, cs_ceil_div(B * (k + 1), 16) * 16);
+  if (s != CS_OK) return s;
+
+  auto enqueue_step = [&]() -> cs_status {
+    cs_status r = cs_launch_find_match(hist, hist_len, B, stride, gamma, k, (int)policy, ctx->loop_mpos,
+                                       ctx->loop_draft, ctx->loop_dlen, ctx->loop_last, ctx->loop_done, st);
+    if (r != CS_OK) return fail(ctx, r, "match kernel launch failed");
+    cs_launch_block_setup(ctx, ctx->loop_last, ctx->loop_draft, ctx->loop_dlen, kv_len, ctx->loop_done, B, k, st);
+    r = enqueue_forward(ctx, B, k + 1, kv_cache, true, nullptr, st);
+    if (r != CS_OK) return r;
+    cs_launch_accept(ctx, B, k, ctx->loop_draft, ctx->loop_dlen, script, max_new, ctx->loop_emitted, max_new,
+                     ctx->loop_accept, ctx->loop_out, ctx->loop_argmax, kv_len, 0, st);
+    cs_launch_loop_commit(ctx, hist, hist_len, B, stride, kv_len, k, max_new, eos_id, script != nullptr, st);
+    return CS_OK;
+  };
+
+  cudaGraph_t graph = nullptr;
+  cudaGraphExec_t exec = nullptr;
+  if (use_graph) {
+    CS_CUDA_OK(ctx, cudaStreamBeginCapture(st, cudaStreamCaptureModeRelaxed));
+    s = enqueue_step();
+    cudaError_t e = cudaStreamEndCapture(st, &graph);
+    if (s != CS_OK) { if (graph) cudaGraphDestroy(graph); return s; }
+    CS_CUDA_OK(ctx, e);
+    e = cudaGraphInstantiate(&exec, graph, 0);
+    if (e != cudaSuccess) { cudaGraphDestroy(graph); CS_CUDA_OK(ctx, e); }
+  }
+  int* h_done = nullptr;
+  cudaError_t e = cudaMallocHost(&h_done, sizeof(int));
+  if (e != cudaSuccess) {
+    if (exec) cudaGraphExecDestroy(exec);
+    if (graph) cudaGraphDestroy(graph);
+    CS_CUDA_OK(ctx, e);
+  }
+  *h_done = 0;
+  const int poll = 4;
+  int steps = 0;
+  s = CS_OK;
+  while (steps < max_new && s == CS_OK) {
+    const int nrun = (max_new - steps < poll) ? max_new - steps : poll;
+    for (int i = 0; i < nrun && s == CS_OK; ++i) {
+      if (use_graph) {
+        if (cudaGraphLaunch(exec, st) != cudaSuccess) s = fail(ctx, CS_ERR_CUDA, "cudaGraphLaunch failed");
+      } else {
+        s = enqueue_step();
+      }
+    }
+    steps += nrun;
+    if (s != CS_OK) break;
+    if (cudaMemcpyAsync(h_done, ctx->loop_done + ctx->cfg.max_batch, sizeof(int), cudaMemcpyDeviceToHost, st) !=
+            cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) {
+      s = fail(ctx, CS_ERR_CUDA, cudaGetErrorString(cudaGetLastError()));
+      break;
+    }
+    if (*h_done >= B) break;
+  }
+  if (s == CS_OK && stats_out != nullptr) {
+    if (cudaMemcpyAsync(stats_out, ctx->loop_stats, sizeof(cs_stats), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+      s = fail(ctx, CS_ERR_CUDA, "copying the statistics failed");
+  }
+  if (cudaStreamSynchronize(st) != cudaSuccess && s == CS_OK) s = fail(ctx, CS_ERR_CUDA, "stream synchronize failed");
+  cudaFreeHost(h_done);
+  if (exec) cudaGraphExecDestroy(exec);
+  if (graph) cudaGraphDestroy(graph);
+  if (s != CS_OK) return s;
+  return cs_sync_status(ctx, stream);
+}
+
+cs_status cs_linear(cs_ctx* ctx, const void* X, const void* W, int rows, int N, int K, float* Y, void* stream) {
+  if (ctx == nullptr) return CS_ERR_ARG;
+  if (X == nullptr || W == nullptr || Y == nullptr || rows < 1 || rows > CS_MAX_ROWS || N < 1 || K < 8 || (K % 8))
+    return fail(ctx, CS_ERR_ARG, "bad argument");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  GemmPlan g;
+  cs_status s = cs_gemm_plan(ctx, &g, W, N, K, true);
+  if (s != CS_OK) return s;
+  while (g.splits > 1 && (size_t)g.splits * rows * N > ctx->partial_elems) {   // fit the workspace
+    g.kb_per_split *= 2;
+    g.splits = cs_ceil_div(cs_ceil_div(K, CS_GEMM_BK), g.kb_per_split);
+  }
+  if ((size_t)g.splits * rows * N > ctx->partial_elems) return fail(ctx, CS_ERR_CAPACITY, "workspace too small for this GEMM");
+  const int n_tok = cs_ceil_div(rows, 16) * 16;
+  CUtensorMap tmX;
+  if ((s = cs_make_act_map(ctx, &tmX, X, n_tok, K, n_tok)) != CS_OK) return s;
+  if ((s = cs_launch_gemm(ctx, &g, &tmX, static_cast<const __nv_bfloat16*>(X), rows, 0, ctx->partial, nullptr, st)) != CS_OK)
+    return s;
+  const size_t total = (size_t)rows * N;
+  k_reduce_partial<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(ctx->partial, g.splits, rows, N, Y);
+  CS_CUDA_OK(ctx, cudaGetLastError());
+  return CS_OK;
+}
+
+}  // extern "C"

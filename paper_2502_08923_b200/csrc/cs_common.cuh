@@ -128,8 +128,8 @@ cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX,
                          cudaStream_t st);
 // cs_layers.cu
 void cs_launch_block_setup(cs_ctx* ctx, const int32_t* last_tok, const int32_t* draft,
-                           const int32_t* draft_len, const int32_t* kv_len, int B, int k,
-                           cudaStream_t st);
+                           const int32_t* draft_len, const int32_t* kv_len, const int32_t* skip,
+                           int B, int k, cudaStream_t st);
 void cs_launch_prefill_setup(cs_ctx* ctx, const int32_t* hist, const int32_t* hist_len, int B,
                              int stride, int start, int R, cudaStream_t st);
 void cs_launch_embed(cs_ctx* ctx, int rows, cudaStream_t st);

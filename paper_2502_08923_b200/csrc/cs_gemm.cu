@@ -1,0 +1,473 @@
+// Skinny bf16 projections of the verification forward (Sec. 3.2): Y = X W^T with at most
+// 256 token rows and a large weight matrix that is streamed from HBM exactly once.
+//
+// The weight matrix is the M operand of the tensor-core instruction ("swap A/B"): one CTA
+// owns 128 output features (UMMA M = 128) and all token rows (UMMA N = rows rounded up to
+// 16), so even an 11-row block fills the 128 TMEM lanes.  Weights and activations arrive
+// as TMA tiles of 64 K-elements (one 128-byte swizzled row per feature / token) through an
+// mbarrier ring; one thread issues tcgen05.mma into a TMEM accumulator; four warps read
+// it back with tcgen05.ld.  K is split across CTAs (grid.y) so that every GEMM puts about
+// two CTAs on each SM; each split writes its fp32 partial sums, which the consumer kernel
+// adds in a fixed order (deterministic, no atomics).  In LM-head mode the epilogue reduces
+// each tile to (max logit, token id) per row instead of writing logits.
+//
+// Every wait is bounded: when it runs out the CTA records CS_DEV_TIMEOUT, drains its
+// copies, frees its TMEM and returns.
+#include "cs_common.cuh"
+
+namespace {
+
+constexpr int kThreads = 192;          // warps 0-3 epilogue, warp 4 TMA producer, warp 5 MMA
+constexpr int kTileABytes = CS_GEMM_BM * CS_GEMM_BK * 2;   // 16 KB
+constexpr unsigned long long kWaitLimitNs = 2000000000ull; // 2 s
+
+struct GemmArgs {
+  int rows, n_tok, N, K;
+  int num_kb, kb_per_split, stages, mode;
+  float* out;        // mode 0: partial sums [splits][rows][N]
+  float* tile_max;   // mode 1: [tiles][tile_stride]
+  int* tile_idx;
+  int tile_stride;
+  float* logits;     // mode 1, optional: [rows][N]
+  int* status;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false when another role of this CTA gave up or 2 s passed.
+__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  unsigned long long t0 = 0;
+  for (uint32_t it = 0;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 1023u) == 1023u) {
+      if (*abort_flag) return false;
+      const unsigned long long now = globaltimer_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > kWaitLimitNs) return false;
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0,
+                                            int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1)
+      : "memory");
+}
+// K-major operand tile, 128-byte swizzle: rows of 128 bytes, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);   // start address / 16
+  d |= (uint64_t)1 << 16;                      // leading-dimension offset (unused here)
+  d |= (uint64_t)(1024 >> 4) << 32;            // stride between 8-row groups / 16
+  d |= (uint64_t)1 << 46;                      // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                      // 128-byte swizzle
+  return d;
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]),
+        "=r"(v[15])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, GemmArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  uint8_t* smem = smem_raw + (((raw + 1023u) & ~1023u) - raw);   // operand tiles need 1024-byte alignment
+  const int stage_bytes = kTileABytes + a.n_tok * 128;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)a.stages * stage_bytes);
+  // bars[0..stages) = tile landed, bars[stages..2*stages) = tile consumed, bars[2*stages] = accumulator done
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * a.stages + 1);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  volatile int* s_never = reinterpret_cast<volatile int*>(tmem_slot + 2);   // stays 0: drains wait on time only
+  float* red_val = reinterpret_cast<float*>(tmem_slot + 4);       // [4][n_tok] (mode 1)
+  int* red_idx = reinterpret_cast<int*>(red_val + 4 * a.n_tok);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tile = blockIdx.x, split = blockIdx.y;
+  const int n0 = tile * CS_GEMM_BM;
+  const int kb0 = split * a.kb_per_split;
+  const int kb1 = min(a.num_kb, kb0 + a.kb_per_split);
+  const int nkb = max(0, kb1 - kb0);
+  uint32_t tmem_cols = 32;
+  while ((int)tmem_cols < a.n_tok) tmem_cols <<= 1;
+
+  const uint32_t bar_full = smem_u32(bars), bar_empty = smem_u32(bars + a.stages),
+                 bar_acc = smem_u32(bars + 2 * a.stages);
+  if (threadIdx.x == 128) {
+    for (int s = 0; s < a.stages; ++s) {
+      mbar_init(bar_full + 8 * s, 1);
+      mbar_init(bar_empty + 8 * s, 1);
+    }
+    mbar_init(bar_acc, 1);
+    *s_abort = 0;
+    *s_never = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmW) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmX) : "memory");
+  }
+  if (warp == 5) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(tmem_cols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot;
+  bool ok = true;
+
+  if (warp == 4) {
+    // ------------------------------------------------------------- TMA producer
+    if (lane == 0) {
+      int i = 0;
+      for (; i < nkb; ++i) {
+        const int s = i % a.stages;
+        const uint32_t ph = (uint32_t)(i / a.stages) & 1u;
+        if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, s_abort)) { ok = false; break; }
+        const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
+        mbar_expect_tx(bar_full + 8 * s, (uint32_t)stage_bytes);
+        tma_load_2d(sa, &tmW, bar_full + 8 * s, (kb0 + i) * CS_GEMM_BK, n0);
+        tma_load_2d(sa + kTileABytes, &tmX, bar_full + 8 * s, (kb0 + i) * CS_GEMM_BK, 0);
+      }
+      if (!ok) {
+        *s_abort = 1;
+        atomicOr(a.status, CS_DEV_TIMEOUT);
+      }
+      if (*s_abort) {
+        // copies still in flight must land before this CTA's shared memory is released
+        for (int j = max(0, i - a.stages); j < i; ++j)
+          mbar_wait(bar_full + 8 * (j % a.stages), (uint32_t)(j / a.stages) & 1u, s_never);
+      }
+    }
+  } else if (warp == 5) {
+    // ------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      // bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n_tok
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(a.n_tok >> 3) << 17) |
+                             ((uint32_t)(CS_GEMM_BM >> 4) << 24);
+      for (int i = 0; i < nkb; ++i) {
+        const int s = i % a.stages;
+        const uint32_t ph = (uint32_t)(i / a.stages) & 1u;
+        if (!mbar_wait(bar_full + 8 * s, ph, s_abort)) { ok = false; break; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
+        const uint64_t da = umma_desc(sa), db = umma_desc(sa + kTileABytes);
+#pragma unroll
+        for (int kk = 0; kk < CS_GEMM_BK / 16; ++kk)   // 16 K-elements = 32 bytes per instruction
+          umma_bf16(tmem_base, da + 2 * kk, db + 2 * kk, idesc, (i > 0 || kk > 0) ? 1u : 0u);
+        umma_commit(bar_empty + 8 * s);
+      }
+      if (!ok) {
+        *s_abort = 1;
+        atomicOr(a.status, CS_DEV_TIMEOUT);
+      }
+      umma_commit(bar_acc);
+    }
+  } else {
+    // ------------------------------------------------------------- epilogue (warps 0-3)
+    const int feat = n0 + warp * 32 + lane;
+    if (nkb > 0) ok = mbar_wait(bar_acc, 0, s_abort);
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    ok = __all_sync(0xffffffffu, ok) && (*s_abort == 0);
+    if (!ok) {
+      if (lane == 0) atomicOr(a.status, CS_DEV_TIMEOUT);
+    } else {
+      for (int c0 = 0; c0 < a.n_tok && c0 < a.rows; c0 += 16) {
+        uint32_t v[16];
+        if (nkb > 0) {
+          tmem_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) v[j] = 0u;
+        }
+        if (a.mode == 0) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const int tok = c0 + j;
+            if (tok < a.rows && feat < a.N)
+              a.out[((size_t)split * a.rows + tok) * a.N + feat] = __uint_as_float(v[j]);
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const int tok = c0 + j;
+            float val = (feat < a.N) ? __uint_as_float(v[j]) : -INFINITY;
+            int idx = feat;
+            if (a.logits != nullptr && tok < a.rows && feat < a.N)
+              a.logits[(size_t)tok * a.N + feat] = val;
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) {
+              const float ov = __shfl_xor_sync(0xffffffffu, val, off);
+              const int oi = __shfl_xor_sync(0xffffffffu, idx, off);
+              if (ov > val || (ov == val && oi < idx)) { val = ov; idx = oi; }
+            }
+            if (lane == 0) { red_val[warp * a.n_tok + tok] = val; red_idx[warp * a.n_tok + tok] = idx; }
+          }
+        }
+      }
+    }
+    if (a.mode == 1) {
+      asm volatile("bar.sync 1, 128;" ::: "memory");   // the four epilogue warps only
+      if (ok) {
+        for (int tok = threadIdx.x; tok < a.rows; tok += 128) {
+          float val = red_val[tok];
+          int idx = red_idx[tok];
+#pragma unroll
+          for (int w = 1; w < 4; ++w) {
+            const float ov = red_val[w * a.n_tok + tok];
+            const int oi = red_idx[w * a.n_tok + tok];
+            if (ov > val || (ov == val && oi < idx)) { val = ov; idx = oi; }
+          }
+          a.tile_max[(size_t)tile * a.tile_stride + tok] = val;
+          a.tile_idx[(size_t)tile * a.tile_stride + tok] = idx;
+        }
+      }
+    }
+  }
+  // ---------------------------------------------------------------- teardown
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 5) {
+    if (*s_abort && lane == 0 && nkb > 0) mbar_wait(bar_acc, 0, s_never);  // MMAs retired
+    __syncwarp();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols)
+                 : "memory");
+  }
+}
+
+// ------------------------------------------------------------------ bring-up path
+// Plain CUDA-core GEMM with the same contract (one warp per output feature).  Selected
+// with CS_GEMM_SIMT=1; it exists to check the tensor-core kernel on the device.
+__global__ void __launch_bounds__(256)
+k_gemm_simt(const __nv_bfloat16* __restrict__ X, const __nv_bfloat16* __restrict__ W, int rows, int N,
+            int K, float* __restrict__ out) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int feat = blockIdx.x * 8 + warp;
+  if (feat >= N) return;
+  for (int r0 = 0; r0 < rows; r0 += 16) {
+    float acc[16];
+#pragma unroll
+    for (int r = 0; r < 16; ++r) acc[r] = 0.f;
+    for (int k = lane * 8; k < K; k += 256) {
+      const uint4 wv = *reinterpret_cast<const uint4*>(W + (size_t)feat * K + k);
+      const __nv_bfloat162* w2 = reinterpret_cast<const __nv_bfloat162*>(&wv);
+#pragma unroll
+      for (int r = 0; r < 16; ++r) {
+        if (r0 + r < rows) {
+          const uint4 xv = *reinterpret_cast<const uint4*>(X + (size_t)(r0 + r) * K + k);
+          const __nv_bfloat162* x2 = reinterpret_cast<const __nv_bfloat162*>(&xv);
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float2 wf = __bfloat1622float2(w2[e]), xf = __bfloat1622float2(x2[e]);
+            acc[r] = fmaf(wf.x, xf.x, acc[r]);
+            acc[r] = fmaf(wf.y, xf.y, acc[r]);
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int r = 0; r < 16; ++r) {
+      float v = acc[r];
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+      if (lane == 0 && r0 + r < rows) out[(size_t)(r0 + r) * N + feat] = v;
+    }
+  }
+}
+
+// per 128-feature tile (max, lowest id) of a logits matrix, for the bring-up path
+__global__ void k_tile_argmax(const float* __restrict__ logits, int rows, int N, float* tile_max,
+                              int* tile_idx, int tile_stride) {
+  const int tile = blockIdx.x, tok = blockIdx.y;
+  const int lane = threadIdx.x;   // 32 threads
+  float val = -INFINITY;
+  int idx = INT32_MAX;
+  for (int f = tile * CS_GEMM_BM + lane; f < min(N, (tile + 1) * CS_GEMM_BM); f += 32) {
+    const float v = logits[(size_t)tok * N + f];
+    if (v > val || (v == val && f < idx)) { val = v; idx = f; }
+  }
+  for (int off = 16; off > 0; off >>= 1) {
+    const float ov = __shfl_xor_sync(0xffffffffu, val, off);
+    const int oi = __shfl_xor_sync(0xffffffffu, idx, off);
+    if (ov > val || (ov == val && oi < idx)) { val = ov; idx = oi; }
+  }
+  if (lane == 0) {
+    tile_max[(size_t)tile * tile_stride + tok] = val;
+    tile_idx[(size_t)tile * tile_stride + tok] = idx;
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn == nullptr) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// [rows][K] bf16 row-major, tiles of box_rows x 64 elements, 128-byte swizzle, zero fill
+cs_status encode_2d(cs_ctx* ctx, CUtensorMap* tm, const void* base, int rows, int K, int box_rows,
+                    bool weights) {
+  EncodeTiledFn enc = get_encode();
+  if (enc == nullptr) {
+    snprintf(ctx->err, sizeof(ctx->err), "cuTensorMapEncodeTiled is not available");
+    return CS_ERR_CUDA;
+  }
+  if ((reinterpret_cast<uintptr_t>(base) & 15) != 0 || (K % 8) != 0) {
+    snprintf(ctx->err, sizeof(ctx->err), "operand needs a 16-byte aligned base and K %% 8 == 0");
+    return CS_ERR_SHAPE;
+  }
+  cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+  cuuint32_t box[2] = {(cuuint32_t)CS_GEMM_BK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box,
+                   estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                   weights ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    snprintf(ctx->err, sizeof(ctx->err), "cuTensorMapEncodeTiled failed with %d (rows %d, K %d, box %d)",
+             (int)r, rows, K, box_rows);
+    return CS_ERR_CUDA;
+  }
+  return CS_OK;
+}
+
+}  // namespace
+
+cs_status cs_gemm_plan(cs_ctx* ctx, GemmPlan* g, const void* w, int N, int K, bool allow_split) {
+  g->W = static_cast<const __nv_bfloat16*>(w);
+  g->N = N;
+  g->K = K;
+  const int tiles = cs_ceil_div(N, CS_GEMM_BM), kb = cs_ceil_div(K, CS_GEMM_BK);
+  const int slots = 2 * ctx->num_sms;
+  int best = 1;
+  long best_cost = -1;
+  const int smax = allow_split ? cs_max_splits(tiles, kb) : 1;
+  for (int s = 1; s <= smax; ++s) {
+    const long cost = (long)cs_ceil_div(tiles * s, slots) * (cs_ceil_div(kb, s) + 2);
+    if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = s; }
+  }
+  g->kb_per_split = cs_ceil_div(kb, best);
+  g->splits = cs_ceil_div(kb, g->kb_per_split);
+  if (ctx->gemm_simt) { g->splits = 1; g->kb_per_split = kb; return CS_OK; }
+  return encode_2d(ctx, &g->tmW, w, N, K, CS_GEMM_BM, true);
+}
+
+cs_status cs_make_act_map(cs_ctx* ctx, CUtensorMap* tm, const void* base, int rows_total, int K,
+                          int box_rows) {
+  if (ctx->gemm_simt) return CS_OK;
+  return encode_2d(ctx, tm, base, rows_total, K, box_rows, false);
+}
+
+cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX, const __nv_bfloat16* X,
+                         int rows, int mode, float* out, float* logits, cudaStream_t st) {
+  const int tiles = cs_ceil_div(g->N, CS_GEMM_BM);
+  if (ctx->gemm_simt) {
+    float* dst = out;
+    if (mode == 1) {
+      dst = logits;
+      if (dst == nullptr) {
+        if ((size_t)rows * g->N > ctx->partial_elems) {
+          snprintf(ctx->err, sizeof(ctx->err), "bring-up GEMM: logits do not fit the workspace");
+          return CS_ERR_UNSUPPORTED;
+        }
+        dst = ctx->partial;
+      }
+    }
+    k_gemm_simt<<<cs_ceil_div(g->N, 8), 256, 0, st>>>(X, g->W, rows, g->N, g->K, dst);
+    if (mode == 1)
+      k_tile_argmax<<<dim3(tiles, rows), 32, 0, st>>>(dst, rows, g->N, ctx->tile_max, ctx->tile_idx,
+                                                      ctx->rows_pad);
+    CS_CUDA_OK(ctx, cudaGetLastError());
+    return CS_OK;
+  }
+  GemmArgs a;
+  a.rows = rows;
+  a.n_tok = cs_ceil_div(rows, 16) * 16;
+  a.N = g->N;
+  a.K = g->K;
+  a.num_kb = cs_ceil_div(g->K, CS_GEMM_BK);
+  a.kb_per_split = g->kb_per_split;
+  a.mode = mode;
+  a.out = out;
+  a.tile_max = ctx->tile_max;
+  a.tile_idx = ctx->tile_idx;
+  a.tile_stride = ctx->rows_pad;
+  a.logits = logits;
+  a.status = ctx->d_status;
+  const int stage_bytes = kTileABytes + a.n_tok * 128;
+  const int fixed = 1024 /*alignment slack*/ + (2 * 8 + 1) * 8 + 16 + 8 * a.n_tok * 4;
+  // small blocks: two CTAs per SM (about 100 KB each); large blocks: one CTA with the whole SM
+  int stages = (100 * 1024 - fixed) / stage_bytes;
+  if (stages < 4) stages = (220 * 1024 - fixed) / stage_bytes;
+  if (stages > 8) stages = 8;
+  if (stages < 2) {
+    snprintf(ctx->err, sizeof(ctx->err), "GEMM stage of %d bytes does not fit shared memory", stage_bytes);
+    return CS_ERR_UNSUPPORTED;
+  }
+  a.stages = stages;
+  const size_t smem = (size_t)fixed + (size_t)stages * stage_bytes;
+  static size_t smem_set = 0;
+  if (smem > smem_set) {
+    CS_CUDA_OK(ctx, cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+    smem_set = 227 * 1024;
+  }
+  k_gemm_tc<<<dim3(tiles, g->splits), kThreads, smem, st>>>(g->tmW, *tmX, a);
+  CS_CUDA_OK(ctx, cudaGetLastError());
+  return CS_OK;
+}

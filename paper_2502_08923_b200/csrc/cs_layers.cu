@@ -1,0 +1,612 @@
+// Everything of the verification forward that is not a weight GEMM (Sec. 3.2; App. B.2):
+// block assembly, embedding, RMSNorm with the split-K reduction and residual add folded
+// in, RoPE + KV append, causal block attention over the KV cache, SwiGLU, the final
+// argmax / prefix acceptance, KV truncation and the loop's commit step.
+#include <math.h>
+
+#include "cs_common.cuh"
+
+namespace {
+
+// ----------------------------------------------------------------- block assembly
+// Rows of sequence b: r = 0 is the last accepted token, r = 1..draft_len[b] the draft
+// (Sec. 3.2: the speculative tokens are appended to the context).  Rows past the draft
+// are dead: they are computed but attend to nothing and write nothing.
+__global__ void k_block_setup(const int* __restrict__ last_tok, const int* __restrict__ draft,
+                              const int* __restrict__ draft_len, const int* __restrict__ kv_len,
+                              const int* __restrict__ skip, int B, int k, int max_seq, int vocab,
+                              int half, const double* __restrict__ inv_freq, int* row_tok, int* row_pos,
+                              int* row_lim, int* row_write, int* seq_ok, float* rope_cs, int* status) {
+  const int R = k + 1, rows = B * R;
+  for (int row = threadIdx.x; row < rows; row += blockDim.x) {
+    const int b = row / R, r = row % R;
+    int dl = draft_len[b];
+    dl = dl < 0 ? 0 : (dl > k ? k : dl);
+    const int kv = kv_len[b];
+    const bool skipped = (skip != nullptr && skip[b] != 0);
+    const bool fits = (kv >= 0 && kv + dl + 1 <= max_seq);
+    const bool ok = fits && !skipped;
+    if (r == 0) {
+      seq_ok[b] = ok ? 1 : 0;
+      if (!fits && !skipped) atomicOr(status, CS_DEV_CAPACITY);
+    }
+    const bool valid = ok && r <= dl;
+    int tok = (r == 0 || !valid) ? last_tok[b] : draft[(size_t)b * k + r - 1];
+    tok = tok < 0 ? 0 : (tok >= vocab ? vocab - 1 : tok);
+    row_tok[row] = tok;
+    row_pos[row] = (kv < 0 ? 0 : kv) + r;
+    row_lim[row] = valid ? kv + r + 1 : 0;
+    row_write[row] = valid ? 1 : 0;
+  }
+  for (int i = threadIdx.x; i < rows * half; i += blockDim.x) {
+    const int row = i / half, j = i % half;
+    const int b = row / R, r = row % R;
+    const int kv = kv_len[b];
+    const double ang = (double)((kv < 0 ? 0 : kv) + r) * inv_freq[j];
+    double s, c;
+    sincos(ang, &s, &c);
+    rope_cs[2 * i] = (float)c;
+    rope_cs[2 * i + 1] = (float)s;
+  }
+}
+
+// Forced rows for filling the cache from a history: row r of sequence b is token
+// hist[b][start + r]; only positions below hist_len[b] - 1 are computed.
+__global__ void k_prefill_setup(const int* __restrict__ hist, const int* __restrict__ hist_len, int B,
+                                int stride, int start, int R, int max_seq, int vocab, int half,
+                                const double* __restrict__ inv_freq, int* row_tok, int* row_pos,
+                                int* row_lim, int* row_write, int* seq_ok, float* rope_cs, int* status) {
+  const int rows = B * R;
+  for (int row = threadIdx.x; row < rows; row += blockDim.x) {
+    const int b = row / R, r = row % R;
+    const int p = start + r;
+    const int n = hist_len[b];
+    const bool fits = (n - 1 <= max_seq && n <= stride);
+    if (r == 0) {
+      seq_ok[b] = fits ? 1 : 0;
+      if (!fits) atomicOr(status, CS_DEV_CAPACITY);
+    }
+    const bool valid = fits && p < n - 1;
+    int tok = valid ? hist[(size_t)b * stride + p] : 0;
+    tok = tok < 0 ? 0 : (tok >= vocab ? vocab - 1 : tok);
+    row_tok[row] = tok;
+    row_pos[row] = p;
+    row_lim[row] = valid ? p + 1 : 0;
+    row_write[row] = valid ? 1 : 0;
+  }
+  for (int i = threadIdx.x; i < rows * half; i += blockDim.x) {
+    const int row = i / half, j = i % half;
+    const double ang = (double)(start + row % R) * inv_freq[j];
+    double s, c;
+    sincos(ang, &s, &c);
+    rope_cs[2 * i] = (float)c;
+    rope_cs[2 * i + 1] = (float)s;
+  }
+}
+
+__global__ void k_embed(const __nv_bfloat16* __restrict__ E, const int* __restrict__ row_tok, int d,
+                        float* __restrict__ x) {
+  const int row = blockIdx.x;
+  const __nv_bfloat16* e = E + (size_t)row_tok[row] * d;
+  for (int i = threadIdx.x * 2; i < d; i += blockDim.x * 2) {
+    const float2 v = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(e + i));
+    *reinterpret_cast<float2*>(x + (size_t)row * d + i) = v;
+  }
+}
+
+// x += sum_s partial[s] (the projection that closed the previous sub-layer), then
+// xn = bf16(x * rsqrt(mean(x^2) + eps) * g).  One CTA per row.
+__global__ void __launch_bounds__(256)
+k_rmsnorm(float* __restrict__ x, const float* __restrict__ partial, int splits, int rows, int d,
+          const __nv_bfloat16* __restrict__ gain, float eps, __nv_bfloat16* __restrict__ xn) {
+  const int row = blockIdx.x;
+  float* xr = x + (size_t)row * d;
+  float ss = 0.f;
+  for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
+    float4 v = *reinterpret_cast<const float4*>(xr + i);
+    for (int s = 0; s < splits; ++s) {
+      const float4 p = *reinterpret_cast<const float4*>(partial + ((size_t)s * rows + row) * d + i);
+      v.x += p.x; v.y += p.y; v.z += p.z; v.w += p.w;
+    }
+    if (splits > 0) *reinterpret_cast<float4*>(xr + i) = v;
+    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+  }
+  __shared__ float red[8];
+  __shared__ float s_scale;
+  for (int off = 16; off > 0; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float t = 0.f;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t += red[w];
+    s_scale = rsqrtf(t / (float)d + eps);
+  }
+  __syncthreads();
+  const float sc = s_scale;
+  for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
+    const float4 v = *reinterpret_cast<const float4*>(xr + i);
+    const float2 g0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(gain + i));
+    const float2 g1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(gain + i + 2));
+    __nv_bfloat162 o0 = __floats2bfloat162_rn(v.x * sc * g0.x, v.y * sc * g0.y);
+    __nv_bfloat162 o1 = __floats2bfloat162_rn(v.z * sc * g1.x, v.w * sc * g1.y);
+    *reinterpret_cast<__nv_bfloat162*>(xn + (size_t)row * d + i) = o0;
+    *reinterpret_cast<__nv_bfloat162*>(xn + (size_t)row * d + i + 2) = o1;
+  }
+}
+
+// Sum the QKV split-K partials, rotate q and k (rotate-half pairing) at the row's
+// absolute position, store q as the bf16 attention operand and append k, v to the cache.
+__global__ void k_qkv_post(const float* __restrict__ partial, int splits, int rows, int H, int Hkv, int Dh,
+                           const float* __restrict__ rope_cs, const int* __restrict__ row_pos,
+                           const int* __restrict__ row_write, int R, __nv_bfloat16* __restrict__ qbuf,
+                           __nv_bfloat16* __restrict__ kv, int layer, int max_batch, int max_seq) {
+  const int row = blockIdx.x, head = blockIdx.y, i = threadIdx.x;
+  const int half = Dh >> 1, N = (H + 2 * Hkv) * Dh;
+  float a = 0.f, b = 0.f;
+  for (int s = 0; s < splits; ++s) {
+    const float* p = partial + ((size_t)s * rows + row) * N + (size_t)head * Dh;
+    a += p[i];
+    b += p[i + half];
+  }
+  const float c = rope_cs[2 * (row * half + i)], sn = rope_cs[2 * (row * half + i) + 1];
+  if (head < H) {
+    __nv_bfloat16* q = qbuf + (size_t)row * H * Dh + (size_t)head * Dh;
+    q[i] = __float2bfloat16_rn(a * c - b * sn);
+    q[i + half] = __float2bfloat16_rn(b * c + a * sn);
+    return;
+  }
+  if (!row_write[row]) return;
+  const int bseq = row / R;
+  const bool is_k = head < H + Hkv;
+  const int kvh = is_k ? head - H : head - H - Hkv;
+  __nv_bfloat16* dst = kv + ((((size_t)layer * 2 + (is_k ? 0 : 1)) * max_batch + bseq) * Hkv + kvh) *
+                                (size_t)max_seq * Dh + (size_t)row_pos[row] * Dh;
+  if (is_k) {
+    dst[i] = __float2bfloat16_rn(a * c - b * sn);
+    dst[i + half] = __float2bfloat16_rn(b * c + a * sn);
+  } else {
+    dst[i] = __float2bfloat16_rn(a);
+    dst[i + half] = __float2bfloat16_rn(b);
+  }
+}
+
+// ------------------------------------------------------------------ attention
+// One CTA = one (sequence, KV head), one slice of the keys, up to 48 query rows (the
+// G query heads of the group times the block rows).  K/V tiles of 64 keys are staged in
+// shared memory once and reused by all rows; scores and the running softmax are fp32.
+constexpr int kAttnThreads = 256;
+constexpr int kAttnRowsPerWarp = 6;
+constexpr int kAttnRows = 8 * kAttnRowsPerWarp;   // 48
+constexpr int kAttnKeys = 64;
+
+template <int DH>
+__global__ void __launch_bounds__(kAttnThreads)
+k_attn_partial(const __nv_bfloat16* __restrict__ qbuf, const __nv_bfloat16* __restrict__ kv,
+               const int* __restrict__ row_lim, int layer, int R, int H, int Hkv, int max_batch,
+               int max_seq, int nsplit, float scale, float* __restrict__ out_o, float* __restrict__ out_ml,
+               int rows) {
+  constexpr int KSTRIDE = DH + 8;          // bf16 elements; 16 bytes of padding kill bank conflicts
+  constexpr int DPL = DH / 32;             // output dims per lane
+  extern __shared__ __align__(16) uint8_t smem[];
+  __nv_bfloat16* Ks = reinterpret_cast<__nv_bfloat16*>(smem);
+  __nv_bfloat16* Vs = Ks + kAttnKeys * KSTRIDE;
+  float* Qs = reinterpret_cast<float*>(Vs + kAttnKeys * KSTRIDE);      // [48][DH]
+  float* Ps = Qs + kAttnRows * DH;                                      // [8][6][64]
+  __shared__ int s_lim[kAttnRows];
+  __shared__ int s_grow[kAttnRows];   // global row
+  __shared__ int s_head[kAttnRows];
+
+  const int G = H / Hkv;
+  const int b = blockIdx.x / Hkv, kvh = blockIdx.x % Hkv;
+  const int split = blockIdx.y, rt = blockIdx.z;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nq = G * R;                       // query rows of this (sequence, KV head)
+  const int q0 = rt * kAttnRows;
+  const int nrows = min(kAttnRows, nq - q0);
+
+  // query row idx -> (head g, block row r)
+  for (int i = threadIdx.x; i < kAttnRows; i += kAttnThreads) {
+    if (i < nrows) {
+      const int g = (q0 + i) / R, r = (q0 + i) % R;
+      s_grow[i] = b * R + r;
+      s_head[i] = kvh * G + g;
+      s_lim[i] = row_lim[b * R + r];
+    } else {
+      s_grow[i] = 0; s_head[i] = 0; s_lim[i] = 0;
+    }
+  }
+  __syncthreads();
+  int lmax = 0;
+  for (int i = 0; i < nrows; ++i) lmax = max(lmax, s_lim[i]);
+  for (int i = threadIdx.x; i < kAttnRows * DH; i += kAttnThreads) {
+    const int qi = i / DH, dd = i % DH;
+    Qs[i] = (qi < nrows) ? __bfloat162float(qbuf[((size_t)s_grow[qi] * H + s_head[qi]) * DH + dd]) : 0.f;
+  }
+
+  const int ntiles = (lmax + kAttnKeys - 1) / kAttnKeys;
+  const int tps = (ntiles + nsplit - 1) / nsplit;
+  const int t0 = split * tps, t1 = min(ntiles, t0 + tps);
+  const __nv_bfloat16* Kg = kv + ((((size_t)layer * 2 + 0) * max_batch + b) * Hkv + kvh) * (size_t)max_seq * DH;
+  const __nv_bfloat16* Vg = kv + ((((size_t)layer * 2 + 1) * max_batch + b) * Hkv + kvh) * (size_t)max_seq * DH;
+
+  float m[kAttnRowsPerWarp], l[kAttnRowsPerWarp], o[kAttnRowsPerWarp][DPL];
+#pragma unroll
+  for (int i = 0; i < kAttnRowsPerWarp; ++i) {
+    m[i] = -INFINITY; l[i] = 0.f;
+#pragma unroll
+    for (int dd = 0; dd < DPL; ++dd) o[i][dd] = 0.f;
+  }
+
+  for (int t = t0; t < t1; ++t) {
+    const int key0 = t * kAttnKeys;
+    __syncthreads();   // previous tile fully consumed (also covers the Q staging)
+    // stage K and V: 16-byte chunks, keys past the longest row are zero-filled
+    constexpr int CPR = DH / 8;
+    for (int c = threadIdx.x; c < kAttnKeys * CPR; c += kAttnThreads) {
+      const int j = c / CPR, cc = c % CPR;
+      uint4 kq = make_uint4(0, 0, 0, 0), vq = make_uint4(0, 0, 0, 0);
+      if (key0 + j < lmax) {
+        kq = *reinterpret_cast<const uint4*>(Kg + (size_t)(key0 + j) * DH + cc * 8);
+        vq = *reinterpret_cast<const uint4*>(Vg + (size_t)(key0 + j) * DH + cc * 8);
+      }
+      *reinterpret_cast<uint4*>(Ks + j * KSTRIDE + cc * 8) = kq;
+      *reinterpret_cast<uint4*>(Vs + j * KSTRIDE + cc * 8) = vq;
+    }
+    __syncthreads();
+    // scores: lane owns keys lane and lane + 32
+    float sc[kAttnRowsPerWarp][2];
+#pragma unroll
+    for (int i = 0; i < kAttnRowsPerWarp; ++i) { sc[i][0] = 0.f; sc[i][1] = 0.f; }
+#pragma unroll 2
+    for (int c = 0; c < CPR; ++c) {
+      const uint4 k0 = *reinterpret_cast<const uint4*>(Ks + lane * KSTRIDE + c * 8);
+      const uint4 k1 = *reinterpret_cast<const uint4*>(Ks + (lane + 32) * KSTRIDE + c * 8);
+      float kf0[8], kf1[8];
+      const __nv_bfloat162* p0 = reinterpret_cast<const __nv_bfloat162*>(&k0);
+      const __nv_bfloat162* p1 = reinterpret_cast<const __nv_bfloat162*>(&k1);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float2 f0 = __bfloat1622float2(p0[e]), f1 = __bfloat1622float2(p1[e]);
+        kf0[2 * e] = f0.x; kf0[2 * e + 1] = f0.y; kf1[2 * e] = f1.x; kf1[2 * e + 1] = f1.y;
+      }
+#pragma unroll
+      for (int i = 0; i < kAttnRowsPerWarp; ++i) {
+        const float* q = Qs + (warp + 8 * i) * DH + c * 8;
+        const float4 qa = *reinterpret_cast<const float4*>(q), qb = *reinterpret_cast<const float4*>(q + 4);
+        const float qv[8] = {qa.x, qa.y, qa.z, qa.w, qb.x, qb.y, qb.z, qb.w};
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          sc[i][0] = fmaf(qv[e], kf0[e], sc[i][0]);
+          sc[i][1] = fmaf(qv[e], kf1[e], sc[i][1]);
+        }
+      }
+    }
+    // running softmax per row
+    float corr[kAttnRowsPerWarp];
+#pragma unroll
+    for (int i = 0; i < kAttnRowsPerWarp; ++i) {
+      const int lim = s_lim[warp + 8 * i];
+      float s0 = (key0 + lane < lim) ? sc[i][0] * scale : -INFINITY;
+      float s1 = (key0 + lane + 32 < lim) ? sc[i][1] * scale : -INFINITY;
+      float mx = fmaxf(s0, s1);
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+      const float mn = fmaxf(m[i], mx);
+      const float p0 = (s0 == -INFINITY) ? 0.f : expf(s0 - mn);
+      const float p1 = (s1 == -INFINITY) ? 0.f : expf(s1 - mn);
+      float ps = p0 + p1;
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) ps += __shfl_xor_sync(0xffffffffu, ps, off);
+      corr[i] = (m[i] == -INFINITY) ? 0.f : expf(m[i] - mn);
+      l[i] = l[i] * corr[i] + ps;
+      m[i] = mn;
+      Ps[(warp * kAttnRowsPerWarp + i) * kAttnKeys + lane] = p0;
+      Ps[(warp * kAttnRowsPerWarp + i) * kAttnKeys + lane + 32] = p1;
+    }
+    __syncwarp();
+#pragma unroll
+    for (int i = 0; i < kAttnRowsPerWarp; ++i)
+#pragma unroll
+      for (int dd = 0; dd < DPL; ++dd) o[i][dd] *= corr[i];
+    // o += P V : lane owns DPL consecutive output dims
+    for (int j = 0; j < kAttnKeys; ++j) {
+      float vf[DPL];
+#pragma unroll
+      for (int dd = 0; dd < DPL; ++dd) vf[dd] = __bfloat162float(Vs[j * KSTRIDE + lane * DPL + dd]);
+#pragma unroll
+      for (int i = 0; i < kAttnRowsPerWarp; ++i) {
+        const float p = Ps[(warp * kAttnRowsPerWarp + i) * kAttnKeys + j];
+#pragma unroll
+        for (int dd = 0; dd < DPL; ++dd) o[i][dd] = fmaf(p, vf[dd], o[i][dd]);
+      }
+    }
+    __syncwarp();
+  }
+  // unnormalised partial result of this key slice
+#pragma unroll
+  for (int i = 0; i < kAttnRowsPerWarp; ++i) {
+    const int qi = warp + 8 * i;
+    if (qi < nrows) {
+      const size_t base = ((size_t)split * rows + s_grow[qi]) * H + s_head[qi];
+#pragma unroll
+      for (int dd = 0; dd < DPL; ++dd) out_o[base * DH + lane * DPL + dd] = o[i][dd];
+      if (lane == 0) { out_ml[base * 2] = m[i]; out_ml[base * 2 + 1] = l[i]; }
+    }
+  }
+}
+
+// Combine the key slices: o = sum_s o_s e^(m_s - M) / sum_s l_s e^(m_s - M).
+__global__ void k_attn_merge(const float* __restrict__ in_o, const float* __restrict__ in_ml, int nsplit,
+                             int rows, int H, int Dh, __nv_bfloat16* __restrict__ attn_out) {
+  const int row = blockIdx.x, h = blockIdx.y, dd = threadIdx.x;
+  float M = -INFINITY;
+  for (int s = 0; s < nsplit; ++s) M = fmaxf(M, in_ml[(((size_t)s * rows + row) * H + h) * 2]);
+  float L = 0.f, acc = 0.f;
+  for (int s = 0; s < nsplit; ++s) {
+    const size_t base = ((size_t)s * rows + row) * H + h;
+    const float ms = in_ml[base * 2];
+    if (ms == -INFINITY) continue;
+    const float w = expf(ms - M);
+    L += in_ml[base * 2 + 1] * w;
+    acc += in_o[base * Dh + dd] * w;
+  }
+  attn_out[((size_t)row * H + h) * Dh + dd] = __float2bfloat16_rn(L > 0.f ? acc / L : 0.f);
+}
+
+// act = bf16( silu(gate) * up ), gate/up summed over the split-K partials
+__global__ void k_swiglu(const float* __restrict__ partial, int splits, int rows, int F,
+                         __nv_bfloat16* __restrict__ act) {
+  const int row = blockIdx.y;
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= F) return;
+  float g = 0.f, u = 0.f;
+  for (int s = 0; s < splits; ++s) {
+    const float* p = partial + ((size_t)s * rows + row) * (2 * (size_t)F);
+    g += p[j];
+    u += p[F + j];
+  }
+  act[(size_t)row * F + j] = __float2bfloat16_rn(g / (1.f + expf(-g)) * u);
+}
+
+// ------------------------------------------------------------------ acceptance
+// Reduce the LM-head tile maxima to the greedy token of each row (lowest id on ties),
+// then accept the longest prefix of the draft that agrees with the target tokens and
+// emit it plus one extra token (Sec. 3.2; App. B.2).  One CTA per sequence.
+__global__ void __launch_bounds__(128)
+k_accept(const float* __restrict__ tile_max, const int* __restrict__ tile_idx, int tiles, int tile_stride,
+         int k, const int* __restrict__ draft, const int* __restrict__ draft_len,
+         const int* __restrict__ seq_ok, const int* __restrict__ script, int script_stride,
+         const int* __restrict__ script_off, int script_limit, int* __restrict__ accept_len,
+         int* __restrict__ out_tokens, int* __restrict__ argmax_ids, int* __restrict__ kv_len,
+         int update_kv) {
+  const int b = blockIdx.x, R = k + 1;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  __shared__ int s_arg[CS_MAX_ROWS];
+  int dl = draft_len[b];
+  dl = dl < 0 ? 0 : (dl > k ? k : dl);
+  const bool ok = seq_ok[b] != 0;
+  for (int r = warp; r < R; r += 4) {
+    float val = -INFINITY;
+    int idx = INT32_MAX;
+    if (ok && r <= dl) {
+      const int row = b * R + r;
+      for (int t = lane; t < tiles; t += 32) {
+        const float v = tile_max[(size_t)t * tile_stride + row];
+        const int id = tile_idx[(size_t)t * tile_stride + row];
+        if (v > val || (v == val && id < idx)) { val = v; idx = id; }
+      }
+      for (int off = 16; off > 0; off >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, val, off);
+        const int oi = __shfl_xor_sync(0xffffffffu, idx, off);
+        if (ov > val || (ov == val && oi < idx)) { val = ov; idx = oi; }
+      }
+    }
+    if (lane == 0) s_arg[r] = (ok && r <= dl && idx != INT32_MAX) ? idx : -1;
+  }
+  __syncthreads();
+  for (int r = threadIdx.x; r < R; r += blockDim.x) argmax_ids[(size_t)b * R + r] = s_arg[r];
+  if (threadIdx.x == 0) {
+    if (!ok) {
+      accept_len[b] = -1;
+      for (int r = 0; r < R; ++r) out_tokens[(size_t)b * R + r] = -1;
+      return;
+    }
+    const int off = (script != nullptr && script_off != nullptr) ? script_off[b] : 0;
+    int tau = 0;
+    bool open = true;
+    for (int r = 0; r < R; ++r) {
+      int tgt = s_arg[r];
+      if (script != nullptr) tgt = (off + r < script_limit) ? script[(size_t)b * script_stride + off + r] : -1;
+      if (r > dl) tgt = -1;
+      // row r's target is emitted iff all earlier draft tokens were accepted
+      out_tokens[(size_t)b * R + r] = open ? tgt : -1;
+      if (open) {
+        if (r < dl && draft[(size_t)b * k + r] == tgt) tau = r + 1; else open = false;
+      }
+    }
+    accept_len[b] = tau;
+    if (update_kv) kv_len[b] += tau + 1;
+  }
+}
+
+__global__ void k_truncate(int* kv_len, const int* new_len, int B, int* status) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= B) return;
+  const int nl = new_len[b];
+  if (nl < 0 || nl > kv_len[b]) atomicOr(status, CS_DEV_BADARG);
+  else kv_len[b] = nl;
+}
+
+__global__ void k_prefill_finish(const int* hist_len, const int* seq_ok, int* kv_len, int B) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b < B && seq_ok[b]) kv_len[b] = max(0, hist_len[b] - 1);
+}
+
+// ------------------------------------------------------------------ loop bookkeeping
+__global__ void k_loop_init(const int* hist_len, const int* kv_len, int B, int stride, int max_new, int k,
+                            int max_seq, int max_batch, int* emitted, int* done,
+                            unsigned long long* stats, int* status) {
+  const int t = threadIdx.x;
+  for (int i = t; i < (int)(sizeof(cs_stats) / 8); i += blockDim.x) stats[i] = 0ull;
+  __shared__ int s_done;
+  if (t == 0) s_done = 0;
+  __syncthreads();
+  for (int b = t; b < B; b += blockDim.x) {
+    const int n = hist_len[b];
+    const bool fits = n >= 1 && n + max_new <= stride && n + max_new + k <= max_seq;
+    const bool consistent = kv_len[b] == n - 1;
+    emitted[b] = 0;
+    int d = 0;
+    if (!fits) { atomicOr(status, CS_DEV_CAPACITY); d = 1; }
+    else if (!consistent) { atomicOr(status, CS_DEV_BADARG); d = 1; }
+    else if (max_new <= 0) d = 1;
+    done[b] = d;
+    if (d) atomicAdd(&s_done, 1);
+  }
+  __syncthreads();
+  if (t == 0) done[max_batch] = s_done;
+}
+
+// Append the step's tokens to the history (App. B.3 step 4), clip at max_new, stop at
+// EOS in real mode, advance the lengths (the KV truncation of App. B.2) and count.
+__global__ void k_loop_commit(int* hist, int* hist_len, int B, int stride, int* kv_len, int k, int max_new,
+                              int eos_id, int scripted, const int* accept, const int* out, const int* mpos,
+                              int* emitted, int* done, int max_batch, unsigned long long* stats) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= B || done[b]) return;
+  cs_stats* st = reinterpret_cast<cs_stats*>(stats);
+  const int tau = accept[b];
+  if (tau < 0) {            // the step skipped this sequence (capacity): it stops here
+    done[b] = 1;
+    atomicAdd(&done[max_batch], 1);
+    return;
+  }
+  const int R = k + 1;
+  const int n = hist_len[b], e = emitted[b];
+  int c = min(tau + 1, max_new - e);
+  bool fin = false;
+  if (!scripted && eos_id >= 0) {
+    for (int i = 0; i < c; ++i)
+      if (out[(size_t)b * R + i] == eos_id) { c = i + 1; fin = true; break; }
+  }
+  for (int i = 0; i < c; ++i) hist[(size_t)b * stride + n + i] = out[(size_t)b * R + i];
+  hist_len[b] = n + c;
+  kv_len[b] = n + c - 1;
+  emitted[b] = e + c;
+  if (e + c >= max_new) fin = true;
+  atomicAdd((unsigned long long*)&st->steps, 1ull);
+  atomicAdd((unsigned long long*)&st->emitted, (unsigned long long)c);
+  if (mpos[b] >= 0) {
+    atomicAdd((unsigned long long*)&st->attempts, 1ull);
+    atomicAdd((unsigned long long*)&st->accepted, (unsigned long long)(c - 1));
+    atomicAdd((unsigned long long*)&st->tau_hist[min(c - 1, CS_TAU_HIST - 1)], 1ull);
+  } else {
+    atomicAdd((unsigned long long*)&st->no_match, 1ull);
+  }
+  if (fin) {
+    done[b] = 1;
+    atomicAdd(&done[max_batch], 1);
+  }
+}
+
+template <int DH>
+void launch_attn(cs_ctx* ctx, const void* kv_cache, int layer, int B, int R, cudaStream_t st) {
+  const cs_model_config& c = ctx->cfg;
+  const int G = c.n_heads / c.n_kv_heads;
+  const int rt = cs_ceil_div(G * R, kAttnRows);
+  const size_t smem = (size_t)2 * kAttnKeys * (DH + 8) * 2 + (size_t)kAttnRows * DH * 4 +
+                      (size_t)8 * kAttnRowsPerWarp * kAttnKeys * 4;
+  static bool set = false;
+  if (!set) {
+    cudaFuncSetAttribute(k_attn_partial<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    set = true;
+  }
+  k_attn_partial<DH><<<dim3(B * c.n_kv_heads, ctx->attn_splits, rt), kAttnThreads, smem, st>>>(
+      ctx->qbuf, static_cast<const __nv_bfloat16*>(kv_cache), ctx->row_lim, layer, R, c.n_heads,
+      c.n_kv_heads, c.max_batch, c.max_seq, ctx->attn_splits, 1.0f / sqrtf((float)DH), ctx->attn_o,
+      ctx->attn_ml, B * R);
+}
+
+}  // namespace
+
+void cs_launch_block_setup(cs_ctx* ctx, const int32_t* last_tok, const int32_t* draft,
+                           const int32_t* draft_len, const int32_t* kv_len, const int32_t* skip, int B,
+                           int k, cudaStream_t st) {
+  const cs_model_config& c = ctx->cfg;
+  k_block_setup<<<1, 256, 0, st>>>(last_tok, draft, draft_len, kv_len, skip, B, k, c.max_seq, c.vocab,
+                                   c.head_dim / 2, ctx->inv_freq, ctx->row_tok, ctx->row_pos, ctx->row_lim,
+                                   ctx->row_write, ctx->seq_ok, ctx->rope_cs, ctx->d_status);
+}
+
+void cs_launch_prefill_setup(cs_ctx* ctx, const int32_t* hist, const int32_t* hist_len, int B, int stride,
+                             int start, int R, cudaStream_t st) {
+  const cs_model_config& c = ctx->cfg;
+  k_prefill_setup<<<1, 256, 0, st>>>(hist, hist_len, B, stride, start, R, c.max_seq, c.vocab, c.head_dim / 2,
+                                     ctx->inv_freq, ctx->row_tok, ctx->row_pos, ctx->row_lim, ctx->row_write,
+                                     ctx->seq_ok, ctx->rope_cs, ctx->d_status);
+}
+
+void cs_launch_embed(cs_ctx* ctx, int rows, cudaStream_t st) {
+  k_embed<<<rows, 128, 0, st>>>(ctx->embed, ctx->row_tok, ctx->cfg.d_model, ctx->x);
+}
+
+void cs_launch_rmsnorm(cs_ctx* ctx, const float* partial, int splits, const __nv_bfloat16* gain, int rows,
+                       cudaStream_t st) {
+  k_rmsnorm<<<rows, 256, 0, st>>>(ctx->x, partial, partial ? splits : 0, rows, ctx->cfg.d_model, gain,
+                                  ctx->cfg.rms_eps, ctx->xn);
+}
+
+void cs_launch_qkv_post(cs_ctx* ctx, int splits, void* kv_cache, int layer, int B, int R, cudaStream_t st) {
+  const cs_model_config& c = ctx->cfg;
+  k_qkv_post<<<dim3(B * R, c.n_heads + 2 * c.n_kv_heads), c.head_dim / 2, 0, st>>>(
+      ctx->partial, splits, B * R, c.n_heads, c.n_kv_heads, c.head_dim, ctx->rope_cs, ctx->row_pos,
+      ctx->row_write, R, ctx->qbuf, static_cast<__nv_bfloat16*>(kv_cache), layer, c.max_batch, c.max_seq);
+}
+
+void cs_launch_attention(cs_ctx* ctx, const void* kv_cache, int layer, int B, int R, cudaStream_t st) {
+  const cs_model_config& c = ctx->cfg;
+  switch (c.head_dim) {
+    case 32: launch_attn<32>(ctx, kv_cache, layer, B, R, st); break;
+    case 64: launch_attn<64>(ctx, kv_cache, layer, B, R, st); break;
+    default: launch_attn<128>(ctx, kv_cache, layer, B, R, st); break;
+  }
+  k_attn_merge<<<dim3(B * R, c.n_heads), c.head_dim, 0, st>>>(ctx->attn_o, ctx->attn_ml, ctx->attn_splits,
+                                                              B * R, c.n_heads, c.head_dim, ctx->attn_out);
+}
+
+void cs_launch_swiglu(cs_ctx* ctx, int splits, int rows, cudaStream_t st) {
+  k_swiglu<<<dim3(cs_ceil_div(ctx->cfg.d_ffn, 256), rows), 256, 0, st>>>(ctx->partial, splits, rows,
+                                                                         ctx->cfg.d_ffn, ctx->act);
+}
+
+void cs_launch_accept(cs_ctx* ctx, int B, int k, const int32_t* draft, const int32_t* draft_len,
+                      const int32_t* script, int script_stride, const int32_t* script_off, int script_limit,
+                      int32_t* accept_len, int32_t* out_tokens, int32_t* argmax_ids, int32_t* kv_len,
+                      int update_kv, cudaStream_t st) {
+  k_accept<<<B, 128, 0, st>>>(ctx->tile_max, ctx->tile_idx, cs_ceil_div(ctx->cfg.vocab, CS_GEMM_BM),
+                              ctx->rows_pad, k, draft, draft_len, ctx->seq_ok, script, script_stride,
+                              script_off, script_limit, accept_len, out_tokens, argmax_ids, kv_len, update_kv);
+}
+
+void cs_launch_truncate(cs_ctx* ctx, int32_t* kv_len, const int32_t* new_len, int B, cudaStream_t st) {
+  k_truncate<<<cs_ceil_div(B, 128), 128, 0, st>>>(kv_len, new_len, B, ctx->d_status);
+}
+
+void cs_launch_prefill_finish(cs_ctx* ctx, const int32_t* hist_len, int32_t* kv_len, int B, cudaStream_t st) {
+  k_prefill_finish<<<cs_ceil_div(B, 128), 128, 0, st>>>(hist_len, ctx->seq_ok, kv_len, B);
+}
+
+void cs_launch_loop_init(cs_ctx* ctx, const int32_t* hist_len, const int32_t* kv_len, int B, int stride,
+                         int max_new, int k, cudaStream_t st) {
+  k_loop_init<<<1, 256, 0, st>>>(hist_len, kv_len, B, stride, max_new, k, ctx->cfg.max_seq,
+                                 ctx->cfg.max_batch, ctx->loop_emitted, ctx->loop_done, ctx->loop_stats,
+                                 ctx->d_status);
+}
+
+void cs_launch_loop_commit(cs_ctx* ctx, int32_t* hist, int32_t* hist_len, int B, int stride, int32_t* kv_len,
+                           int k, int max_new, int eos_id, int scripted, cudaStream_t st) {
+  k_loop_commit<<<cs_ceil_div(B, 128), 128, 0, st>>>(hist, hist_len, B, stride, kv_len, k, max_new, eos_id,
+                                                     scripted, ctx->loop_accept, ctx->loop_out, ctx->loop_mpos,
+                                                     ctx->loop_emitted, ctx->loop_done, ctx->cfg.max_batch,
+                                                     ctx->loop_stats);
+}
