@@ -1,0 +1,244 @@
+"""ctypes binding of libcopyspec.so: same names as the C ABI (include/copyspec.h),
+argument marshalling only.  PyTorch provides device memory and the current stream; every
+step of the path runs in the library's CUDA kernels.  There is no CPU fallback: if the
+library cannot be loaded, every call raises."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+from . import build as _build
+
+CS_OK = 0
+CS_ERR_ARG, CS_ERR_SHAPE, CS_ERR_CAPACITY, CS_ERR_CUDA, CS_ERR_TIMEOUT, CS_ERR_UNSUPPORTED = -1, -2, -3, -4, -5, -6
+LATEST, FIRST = 0, 1
+TAU_HIST = 65
+
+_STATUS = {0: "CS_OK", -1: "CS_ERR_ARG", -2: "CS_ERR_SHAPE", -3: "CS_ERR_CAPACITY", -4: "CS_ERR_CUDA",
+           -5: "CS_ERR_TIMEOUT", -6: "CS_ERR_UNSUPPORTED"}
+
+
+class CsError(RuntimeError):
+    def __init__(self, code, where, detail=""):
+        self.code = code
+        super().__init__(f"{where}: {_STATUS.get(code, code)} {detail}".strip())
+
+
+class CsModelConfig(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("n_layers", "d_model", "n_heads", "n_kv_heads", "head_dim",
+                                         "d_ffn", "vocab", "max_seq", "max_batch", "k_max")] + \
+               [("rope_theta", C.c_float), ("rms_eps", C.c_float)]
+
+
+class CsWeights(C.Structure):
+    _fields_ = [("embed", C.c_void_p), ("lm_head", C.c_void_p), ("final_norm", C.c_void_p)] + \
+               [(n, C.POINTER(C.c_void_p)) for n in ("attn_norm", "wqkv", "wo", "ffn_norm", "w_gate_up", "w_down")]
+
+
+class CsStats(C.Structure):
+    _fields_ = [(n, C.c_uint64) for n in ("steps", "attempts", "accepted", "emitted", "no_match")] + \
+               [("tau_hist", C.c_uint64 * TAU_HIST)]
+
+    def as_dict(self):
+        return {"steps": self.steps, "attempts": self.attempts, "accepted": self.accepted,
+                "emitted": self.emitted, "no_match": self.no_match, "tau_hist": list(self.tau_hist)}
+
+
+EXPORTS = ("cs_workspace_bytes", "cs_create", "cs_destroy", "cs_last_error", "cs_sync_status",
+           "cs_find_match", "cs_verify_step", "cs_kv_truncate", "cs_decode_loop", "cs_prefill", "cs_linear")
+
+_lib = None
+
+
+def lib_path() -> str:
+    return _build.LIB
+
+
+def load(build_if_missing: bool = True) -> C.CDLL:
+    """Load libcopyspec.so (building it with nvcc first when it is missing or stale)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if build_if_missing:
+        _build.build()
+    if not os.path.exists(_build.LIB):
+        raise RuntimeError("libcopyspec.so is not built: run `python -m paper_2502_08923_b200.build`")
+    lib = C.CDLL(_build.LIB)
+    vp, ip, i = C.c_void_p, C.c_void_p, C.c_int
+    lib.cs_workspace_bytes.restype = C.c_size_t
+    lib.cs_workspace_bytes.argtypes = [C.POINTER(CsModelConfig)]
+    lib.cs_create.restype = i
+    lib.cs_create.argtypes = [C.POINTER(C.c_void_p), C.POINTER(CsModelConfig), C.POINTER(CsWeights), vp, C.c_size_t]
+    lib.cs_destroy.restype = None
+    lib.cs_destroy.argtypes = [vp]
+    lib.cs_last_error.restype = C.c_char_p
+    lib.cs_last_error.argtypes = [vp]
+    lib.cs_sync_status.restype = i
+    lib.cs_sync_status.argtypes = [vp, vp]
+    lib.cs_find_match.restype = i
+    lib.cs_find_match.argtypes = [ip, ip, i, i, i, i, i, ip, ip, ip, vp]
+    lib.cs_verify_step.restype = i
+    lib.cs_verify_step.argtypes = [vp, ip, ip, ip, i, i, vp, ip, ip, ip, ip, ip, vp, vp]
+    lib.cs_kv_truncate.restype = i
+    lib.cs_kv_truncate.argtypes = [vp, ip, ip, i, vp]
+    lib.cs_decode_loop.restype = i
+    lib.cs_decode_loop.argtypes = [vp, ip, ip, i, i, vp, ip, i, i, i, i, i, ip, C.POINTER(CsStats), vp]
+    lib.cs_prefill.restype = i
+    lib.cs_prefill.argtypes = [vp, ip, ip, i, i, i, vp, ip, vp]
+    lib.cs_linear.restype = i
+    lib.cs_linear.argtypes = [vp, vp, vp, i, i, i, vp, vp]
+    _lib = lib
+    return lib
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("expected a contiguous CUDA tensor")
+    return C.c_void_p(t.data_ptr())
+
+
+def _i32(t, name):
+    if t is not None and t.dtype != torch.int32:
+        raise ValueError(f"{name} must be int32")
+    return _ptr(t)
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def cs_find_match(hist, hist_len, gamma, k, policy=LATEST, out=None):
+    """Suffix-match search and draft gather.  hist [B][stride] int32, hist_len [B] int32 (CUDA).
+    Returns (match_pos [B], draft [B][k], draft_len [B]); `out` may supply those tensors."""
+    lib = load()
+    B, stride = hist.shape
+    if out is None:
+        out = (torch.empty(B, dtype=torch.int32, device=hist.device),
+               torch.empty(B, max(k, 1), dtype=torch.int32, device=hist.device)[:, :k].contiguous(),
+               torch.empty(B, dtype=torch.int32, device=hist.device))
+    mp, dr, dl = out
+    rc = lib.cs_find_match(_i32(hist, "hist"), _i32(hist_len, "hist_len"), B, stride, gamma, k, policy,
+                           _i32(mp, "match_pos"), C.c_void_p(dr.data_ptr()) if k > 0 else None,
+                           _i32(dl, "draft_len"), _stream())
+    if rc != CS_OK:
+        raise CsError(rc, "cs_find_match")
+    return mp, dr, dl
+
+
+class Context:
+    """Owns the device workspace and the cs_ctx handle for one model."""
+
+    def __init__(self, cfg, weights, max_seq, max_batch, k_max):
+        lib = load()
+        self.lib = lib
+        self.cfg = cfg
+        self.max_seq, self.max_batch, self.k_max = max_seq, max_batch, k_max
+        self.c_cfg = CsModelConfig(cfg.n_layers, cfg.d_model, cfg.n_heads, cfg.n_kv_heads, cfg.head_dim,
+                                   cfg.d_ffn, cfg.vocab, max_seq, max_batch, k_max, cfg.rope_theta, cfg.rms_eps)
+        nbytes = lib.cs_workspace_bytes(C.byref(self.c_cfg))
+        if nbytes == 0:
+            raise CsError(CS_ERR_SHAPE, "cs_workspace_bytes", "unsupported configuration")
+        self.workspace_bytes = nbytes
+        raw = torch.empty(nbytes + 1024, dtype=torch.uint8, device="cuda")
+        off = (-raw.data_ptr()) % 1024
+        self._raw = raw
+        self.weights = weights          # keeps the tensors alive
+        L = cfg.n_layers
+        self._arrs = {}
+        cw = CsWeights()
+        for name in ("embed", "lm_head", "final_norm"):
+            t = weights[name]
+            assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()
+            setattr(cw, name, t.data_ptr())
+        for name in ("attn_norm", "wqkv", "wo", "ffn_norm", "w_gate_up", "w_down"):
+            arr = (C.c_void_p * L)()
+            for l in range(L):
+                t = weights["layers"][l][name]
+                assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()
+                arr[l] = t.data_ptr()
+            self._arrs[name] = arr
+            setattr(cw, name, C.cast(arr, C.POINTER(C.c_void_p)))
+        self.handle = C.c_void_p()
+        rc = lib.cs_create(C.byref(self.handle), C.byref(self.c_cfg), C.byref(cw),
+                           C.c_void_p(raw.data_ptr() + off), nbytes)
+        if rc != CS_OK:
+            raise CsError(rc, "cs_create")
+
+    def close(self):
+        if getattr(self, "handle", None):
+            self.lib.cs_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, rc, where):
+        if rc != CS_OK:
+            msg = self.lib.cs_last_error(self.handle)
+            raise CsError(rc, where, msg.decode() if msg else "")
+
+    def alloc_kv(self):
+        c = self.cfg
+        return torch.zeros(c.n_layers, 2, self.max_batch, c.n_kv_heads, self.max_seq, c.head_dim,
+                           dtype=torch.bfloat16, device="cuda")
+
+    def cs_sync_status(self):
+        return self.lib.cs_sync_status(self.handle, _stream())
+
+    def cs_verify_step(self, last_tok, draft, draft_len, kv_cache, kv_len, target_script=None, out=None,
+                       logits_dbg=None):
+        """One verification forward + acceptance.  Returns (accept_len [B], out_tokens [B][k+1],
+        argmax_ids [B][k+1]); kv_len is advanced in place."""
+        B = last_tok.shape[0]
+        k = draft.shape[1] if draft is not None and draft.dim() == 2 else 0
+        dev = last_tok.device
+        if out is None:
+            out = (torch.empty(B, dtype=torch.int32, device=dev),
+                   torch.empty(B, k + 1, dtype=torch.int32, device=dev),
+                   torch.empty(B, k + 1, dtype=torch.int32, device=dev))
+        al, ot, am = out
+        rc = self.lib.cs_verify_step(self.handle, _i32(last_tok, "last_tok"),
+                                     C.c_void_p(draft.data_ptr()) if k > 0 else None,
+                                     _i32(draft_len, "draft_len"), B, k, _ptr(kv_cache), _i32(kv_len, "kv_len"),
+                                     _i32(target_script, "target_script"), _i32(al, "accept_len"),
+                                     _i32(ot, "out_tokens"), _i32(am, "argmax_ids"), _ptr(logits_dbg), _stream())
+        self._check(rc, "cs_verify_step")
+        return al, ot, am
+
+    def cs_kv_truncate(self, kv_len, new_len):
+        rc = self.lib.cs_kv_truncate(self.handle, _i32(kv_len, "kv_len"), _i32(new_len, "new_len"),
+                                     kv_len.shape[0], _stream())
+        self._check(rc, "cs_kv_truncate")
+
+    def cs_prefill(self, hist, hist_len, max_len, kv_cache, kv_len):
+        B, stride = hist.shape
+        rc = self.lib.cs_prefill(self.handle, _i32(hist, "hist"), _i32(hist_len, "hist_len"), B, stride,
+                                 int(max_len), _ptr(kv_cache), _i32(kv_len, "kv_len"), _stream())
+        self._check(rc, "cs_prefill")
+
+    def cs_decode_loop(self, hist, hist_len, kv_cache, kv_len, gamma, k, max_new, policy=LATEST, eos_id=-1,
+                       script=None):
+        """The generation loop; returns the statistics as a dict.  hist/hist_len/kv_len advance in place."""
+        B, stride = hist.shape
+        st = CsStats()
+        rc = self.lib.cs_decode_loop(self.handle, _i32(hist, "hist"), _i32(hist_len, "hist_len"), B, stride,
+                                     _ptr(kv_cache), _i32(kv_len, "kv_len"), gamma, k, policy, max_new, eos_id,
+                                     _i32(script, "script"), C.byref(st), _stream())
+        self._check(rc, "cs_decode_loop")
+        return st.as_dict()
+
+    def cs_linear(self, X, W, rows=None):
+        """Y[rows][N] fp32 = X[rows][K] bf16 @ W[N][K]^T bf16 through the tensor-core GEMM."""
+        rows = X.shape[0] if rows is None else rows
+        N, K = W.shape
+        Y = torch.empty(rows, N, dtype=torch.float32, device=X.device)
+        rc = self.lib.cs_linear(self.handle, _ptr(X), _ptr(W), rows, N, K, _ptr(Y), _stream())
+        self._check(rc, "cs_linear")
+        return Y

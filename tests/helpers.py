@@ -1,0 +1,33 @@
+"""Shared set-up of the GPU parity tests: the same seeded weights go to the CUDA library
+(bf16 on the device) and to the CPU oracle."""
+import numpy as np
+import torch
+
+from oracle import copyspec_oracle as O
+from paper_2502_08923_b200 import binding as cs, inputs
+
+LOGIT_TOL = 2e-2     # max |logit difference| with bf16 operands and fp32 accumulation
+
+
+def make_pair(cfg, max_seq, max_batch, k_max, seed=0, gain_jitter=0.0, weights=None):
+    w_cpu = weights if weights is not None else inputs.make_weights(cfg, seed=seed, gain_jitter=gain_jitter)
+    w_gpu = inputs.weights_to(w_cpu, "cuda")
+    ctx = cs.Context(cfg, w_gpu, max_seq=max_seq, max_batch=max_batch, k_max=k_max)
+    model = O.Model(cfg, w_cpu, contract=True)
+    return ctx, model
+
+
+def i32(a, device="cuda"):
+    return torch.as_tensor(np.ascontiguousarray(a), dtype=torch.int32).to(device)
+
+
+def argmax_consistent(oracle_logits, gpu_ids, tol=LOGIT_TOL):
+    """GPU argmax must equal the oracle's unless the oracle's own margin over the GPU's
+    choice is below the logit tolerance."""
+    bad = []
+    for r, gid in enumerate(gpu_ids):
+        row = oracle_logits[r]
+        oid = int(np.argmax(row))
+        if gid != oid and not (row[oid] - row[gid] < tol):
+            bad.append((r, gid, oid, float(row[oid] - row[gid])))
+    return bad

@@ -1,0 +1,35 @@
+"""The tensor-core projection kernel in isolation against the plain definition
+Y = X W^T evaluated in fp64 on the CPU (building block of the forward of Sec. 3.2)."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2502_08923_b200 import inputs
+from helpers import make_pair
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c, _ = make_pair(inputs.TINY, 256, 1, 10)
+    yield c
+    c.close()
+
+
+@pytest.mark.parametrize("rows", [1, 11, 16, 17, 100, 176, 256])
+@pytest.mark.parametrize("N,K", [(128, 64), (200, 256), (768, 256), (256, 1024), (4096, 4096), (1000, 520)])
+def test_linear_matches_fp64_matmul(ctx, rows, N, K):
+    g = torch.Generator().manual_seed(rows * 7919 + N + K)
+    X = torch.randn(rows, K, generator=g).to(torch.bfloat16)
+    W = (torch.randn(N, K, generator=g) * 0.05).to(torch.bfloat16)
+    pad = (rows + 15) // 16 * 16
+    Xd = torch.zeros(pad, K, dtype=torch.bfloat16, device="cuda")
+    Xd[:rows] = X.cuda()
+    Y = ctx.cs_linear(Xd, W.cuda(), rows=rows)
+    assert ctx.cs_sync_status() == 0
+    want = X.double().numpy() @ W.double().numpy().T
+    got = Y.cpu().double().numpy()
+    # bf16 products are exact in fp32; only the fp32 summation order differs
+    tol = 1e-5 * np.sqrt(K) * max(1.0, np.abs(want).max())
+    assert np.abs(got - want).max() <= tol

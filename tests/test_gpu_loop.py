@@ -1,0 +1,114 @@
+"""cs_decode_loop on the GPU against the oracle loop, greedy decoding and the model-free
+simulator (App. B.3 steps 1, 2, 4; Sec. 3.2)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import copyspec_oracle as O
+from paper_2502_08923_b200 import binding as cs, inputs
+from helpers import i32, make_pair
+
+pytestmark = pytest.mark.gpu
+
+
+def _run_gpu(ctx, hists, lens, stride, gamma, k, max_new, policy, script=None, eos_id=-1):
+    B = len(hists)
+    h = np.zeros((B, stride), dtype=np.int32)
+    for b in range(B):
+        h[b, :lens[b]] = hists[b][:lens[b]]
+    hd, ld = i32(h), i32(lens)
+    kv = ctx.alloc_kv()
+    kv_len = torch.zeros(ctx.max_batch, dtype=torch.int32, device="cuda")[:B].contiguous()
+    ctx.cs_prefill(hd, ld, int(max(lens)), kv, kv_len)
+    st = ctx.cs_decode_loop(hd, ld, kv, kv_len, gamma, k, max_new, policy=policy, eos_id=eos_id,
+                            script=None if script is None else i32(script))
+    return hd.cpu().numpy(), ld.cpu().numpy(), kv_len.cpu().numpy(), st
+
+
+@pytest.mark.parametrize("policy", [cs.LATEST, cs.FIRST])
+def test_tiny_config_scripted_mode(policy):
+    """Small configuration: 512-token context with planted spans, gamma=3, k=10, scripted target."""
+    cfg = inputs.TINY
+    ctx, model = make_pair(cfg, 1024, 1, 10)
+    ctxt, spans = inputs.tiny_context(seed=1)
+    rng = np.random.default_rng(7)
+    max_new = 200
+    script = inputs.copy_script(rng, ctxt, max_new, 0.6, 5, 30, cfg.vocab, zipf_s=None)
+    h, n, kvl, st = _run_gpu(ctx, [ctxt], [512], 1024, 3, 10, max_new, policy, script=script[None, :])
+    steps, st_o, h_sim = O.scripted_simulator(ctxt, script, 3, 10, policy, max_new)
+    assert n[0] == 512 + max_new and kvl[0] == n[0] - 1
+    assert h[0, :n[0]].tolist() == h_sim
+    for key in ("steps", "attempts", "accepted", "emitted", "no_match"):
+        assert st[key] == st_o[key], key
+    assert st["tau_hist"][:11] == st_o["tau_hist"][:11]
+    assert st["accepted"] > 0 and len({s["tau"] for s in steps}) >= 5     # tau covers a spread of values
+    ctx.close()
+
+
+def test_tiny_config_real_mode_is_greedy_decoding():
+    """64 decode steps in real mode; the emitted tokens equal the oracle's copy loop and
+    plain greedy decoding (losslessness, Sec. 1 / App. B.2)."""
+    cfg = inputs.TINY
+    ctx, model = make_pair(cfg, 1024, 1, 10)
+    ctxt, _ = inputs.tiny_context(seed=1)
+    max_new = 64
+    h, n, kvl, st = _run_gpu(ctx, [ctxt], [512], 1024, 3, 10, max_new, cs.LATEST)
+    cache = O.KVCache(cfg, 1, 1024)
+    model.prefill(ctxt.tolist(), cache, 0)
+    h_o = ctxt.tolist()
+    trace = []
+    got_o, st_o = O.decode_loop(model, cache, 0, h_o, 3, 10, O.LATEST, max_new, trace=trace)
+    gpu_tokens = h[0, 512:n[0]].tolist()
+    if gpu_tokens != got_o:
+        # a difference is only legitimate where the oracle's top-2 margin is below tolerance
+        i = next(j for j in range(min(len(gpu_tokens), len(got_o))) if gpu_tokens[j] != got_o[j])
+        c2 = O.KVCache(cfg, 1, 1024); seq = ctxt.tolist() + got_o[:i]
+        model.prefill(seq, c2, 0)
+        lg = model.forward_block([seq[-1]], len(seq) - 1, c2, 0)[0]
+        assert lg[got_o[i]] - lg[gpu_tokens[i]] < 2e-2, "GPU decoding diverged from the oracle at a clear margin"
+        pytest.skip("near-tie divergence")
+    assert n[0] == 512 + max_new and kvl[0] == n[0] - 1
+    for key in ("steps", "attempts", "accepted", "emitted", "no_match"):
+        assert st[key] == st_o[key], key
+    # plain decoding from the same kernels (k = 0) gives the same tokens
+    h0, n0, _, st0 = _run_gpu(ctx, [ctxt], [512], 1024, 3, 0, max_new, cs.LATEST)
+    assert h0[0, 512:n0[0]].tolist() == gpu_tokens and st0["steps"] == max_new and st0["accepted"] == 0
+    ctx.close()
+
+
+def test_batch_of_sequences_with_eos_and_different_lengths():
+    cfg = inputs.ModelConfig(n_layers=2, d_model=128, n_heads=4, n_kv_heads=2, head_dim=32, d_ffn=256, vocab=64,
+                             rope_theta=10000.0, rms_eps=1e-5)
+    B, k, max_new = 4, 5, 60
+    ctx, model = make_pair(cfg, 256, B, k, seed=2)
+    rng = np.random.default_rng(2)
+    lens = [40, 25, 33, 8]
+    hists = [rng.integers(0, cfg.vocab, size=n).astype(np.int32) for n in lens]
+    # choose as EOS a token that plain decoding of sequence 0 produces somewhere in the middle
+    c0 = O.KVCache(cfg, 1, 256); model.prefill(hists[0].tolist(), c0, 0)
+    ref0 = O.greedy_decode(model, c0, 0, hists[0].tolist(), max_new)
+    eos = ref0[max_new // 2]
+    h, n, kvl, st = _run_gpu(ctx, hists, lens, 128, 3, k, max_new, cs.LATEST, eos_id=eos)
+    tot = O.new_stats()
+    for b in range(B):
+        cache = O.KVCache(cfg, 1, 256); model.prefill(hists[b].tolist(), cache, 0)
+        ho = hists[b].tolist()
+        got, so = O.decode_loop(model, cache, 0, ho, 3, k, O.LATEST, max_new, eos_id=eos)
+        assert h[b, :n[b]].tolist() == ho, b
+        assert kvl[b] == n[b] - 1
+        for key in ("steps", "attempts", "accepted", "emitted", "no_match"):
+            tot[key] += so[key]
+    for key in ("steps", "attempts", "accepted", "emitted", "no_match"):
+        assert st[key] == tot[key], key
+    ctx.close()
+
+
+def test_loop_capacity_is_reported():
+    cfg = inputs.TINY
+    ctx, _ = make_pair(cfg, 128, 1, 10)
+    hist = np.zeros((1, 64), dtype=np.int32)
+    kv = ctx.alloc_kv(); kv_len = i32([19])
+    with pytest.raises(cs.CsError) as e:
+        ctx.cs_decode_loop(i32(hist), i32([20]), kv, kv_len, 3, 10, 100)     # 20 + 100 > stride 64
+    assert e.value.code == cs.CS_ERR_CAPACITY
+    ctx.close()
