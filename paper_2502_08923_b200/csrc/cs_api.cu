@@ -206,6 +206,7 @@ cs_status cs_create(cs_ctx** out, const cs_model_config* cfg, const cs_weights* 
     return CS_ERR_UNSUPPORTED;
   }
   ctx->num_sms = prop.multiProcessorCount;
+  CREATE_OK(cudaStreamCreateWithFlags(&ctx->cap_stream, cudaStreamNonBlocking));
   char* base = static_cast<char*>(workspace);
   ctx->ws = base;
   ctx->ws_bytes = L.total;
@@ -276,6 +277,7 @@ cs_status cs_create(cs_ctx** out, const cs_model_config* cfg, const cs_weights* 
 
 void cs_destroy(cs_ctx* ctx) {
   if (ctx == nullptr) return;
+  if (ctx->cap_stream) cudaStreamDestroy(ctx->cap_stream);
   delete[] ctx->layers;
   delete ctx;
 }
@@ -375,7 +377,7 @@ cs_status cs_decode_loop(cs_ctx* ctx, int32_t* hist, int32_t* hist_len, int B, i
   cs_status s = ensure_act_maps(ctx, cs_ceil_div(B * (k + 1), 16) * 16);
   if (s != CS_OK) return s;
 
-  auto enqueue_step = [&]() -> cs_status {
+  auto enqueue_step = [&](cudaStream_t st) -> cs_status {
     cs_status r = cs_launch_find_match(hist, hist_len, B, stride, gamma, k, (int)policy, ctx->loop_mpos,
                                        ctx->loop_draft, ctx->loop_dlen, ctx->loop_last, ctx->loop_done, st);
     if (r != CS_OK) return fail(ctx, r, "match kernel launch failed");
@@ -391,9 +393,11 @@ cs_status cs_decode_loop(cs_ctx* ctx, int32_t* hist, int32_t* hist_len, int B, i
   cudaGraph_t graph = nullptr;
   cudaGraphExec_t exec = nullptr;
   if (use_graph) {
-    CS_CUDA_OK(ctx, cudaStreamBeginCapture(st, cudaStreamCaptureModeRelaxed));
-    s = enqueue_step();
-    cudaError_t e = cudaStreamEndCapture(st, &graph);
+    // captured on the context's own stream (the legacy default stream cannot capture),
+    // replayed on the caller's
+    CS_CUDA_OK(ctx, cudaStreamBeginCapture(ctx->cap_stream, cudaStreamCaptureModeRelaxed));
+    s = enqueue_step(ctx->cap_stream);
+    cudaError_t e = cudaStreamEndCapture(ctx->cap_stream, &graph);
     if (s != CS_OK) { if (graph) cudaGraphDestroy(graph); return s; }
     CS_CUDA_OK(ctx, e);
     e = cudaGraphInstantiate(&exec, graph, 0);
@@ -416,7 +420,7 @@ cs_status cs_decode_loop(cs_ctx* ctx, int32_t* hist, int32_t* hist_len, int B, i
       if (use_graph) {
         if (cudaGraphLaunch(exec, st) != cudaSuccess) s = fail(ctx, CS_ERR_CUDA, "cudaGraphLaunch failed");
       } else {
-        s = enqueue_step();
+        s = enqueue_step(st);
       }
     }
     steps += nrun;

@@ -46,6 +46,7 @@ struct cs_ctx {
   int attn_splits;   // split-KV factor
   bool gemm_simt;    // bring-up path: plain CUDA-core GEMM instead of tcgen05
   int num_sms;
+  cudaStream_t cap_stream;   // used only to capture the loop's step graph
 
   const __nv_bfloat16 *embed, *final_norm;
   LayerPlan* layers;  // host array

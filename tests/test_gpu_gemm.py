@@ -12,7 +12,9 @@ pytestmark = pytest.mark.gpu
 
 @pytest.fixture(scope="module")
 def ctx():
-    c, _ = make_pair(inputs.TINY, 256, 1, 10)
+    cfg = inputs.ModelConfig(n_layers=1, d_model=512, n_heads=4, n_kv_heads=4, head_dim=128, d_ffn=4096,
+                             vocab=512, rope_theta=10000.0, rms_eps=1e-5)   # workspace large enough for the shapes below
+    c, _ = make_pair(cfg, 256, 1, 10)
     yield c
     c.close()
 

@@ -137,7 +137,7 @@ def test_truncated_rows_do_not_leak_into_the_next_step():
     nxt = np.array([out[-1]], dtype=np.int32)
     ctx.cs_verify_step(i32(nxt), i32(draft), i32([0]), kv, kv_len, logits_dbg=logits)
     clean = O.KVCache(cfg, 1, 128)            # an oracle that only ever saw the accepted tokens
-    seq = hist[0, :41].tolist() + out
+    seq = hist[0, :40].tolist() + [int(last[0])] + out
     model.prefill(seq, clean, 0)
     lg = model.forward_block([seq[-1]], len(seq) - 1, clean, 0)
     assert np.abs(logits[0, :1].cpu().numpy() - lg).max() <= LOGIT_TOL
