@@ -1,0 +1,403 @@
+#!/usr/bin/env python
+"""Benchmark of the copy-and-verify decode step (CopySpec, arXiv 2502.08923) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One "step" is one pass of the whole hot path for one batch: suffix-match search, draft
+gather, one verification forward of the 8B-class model over the (k+1)-row block against
+the bf16 KV cache, LM-head argmax, prefix acceptance, KV truncation and the append to the
+history - i.e. one replay of the generation loop's step graph.  The workload is the
+8B-class verify configuration: batch 1, KV cache starting at 4,096 positions, gamma = 3,
+k = 10, scripted-target mode with the accepted prefix uniform in [0, 10]; every input is
+seeded and synthetic (random-init bf16 weights, N(0,1) KV fill, token paths built so that
+each step accepts a prescribed number of draft tokens).
+
+`value` is emitted tokens per second (accepted draft tokens plus the one guaranteed token
+per step) with everything resident in HBM; `e2e` drives the same steps from pinned host
+buffers through cs_find_match / cs_verify_step with the copies inside the timed region.
+With N > 1 every rank runs an independent replica (the path does not shard).
+`--impl reference` times the CPU oracle, as it stands, on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "accepted tokens/sec"
+UNIT = "tokens/s"
+GAMMA, K_DRAFT, KV_START = 3, 10, 4096
+WORKLOAD = "verify_8b_b1_kv4096_k10_scripted_tau_uniform"
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from the
+# committed ncu capture (profiles/); None until a capture of the current kernel exists.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def _peaks():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+def _taus(n_steps, seed=0):
+    """Accepted prefix per step: uniform over 0..k, each value equally often."""
+    rng = np.random.default_rng(seed)
+    reps = -(-n_steps // (K_DRAFT + 1))
+    return [int(t) for t in rng.permutation(np.repeat(np.arange(K_DRAFT + 1), reps))[:n_steps]]
+
+
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.index)],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1])); mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, v in zip(names, f[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def _dist():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+# --------------------------------------------------------------------- CPU oracle leg
+def oracle_sample(cfg8b, weights_cpu_layer0, kv_layer0, lm_head_cpu, hist, script, taus, n_steps, warmup):
+    """Times the oracle, as it stands, on a bounded sample of the workload: the verification
+    forward of ONE of the 32 decoder layers (block of k+1 rows against 4,096 cached
+    positions) per step plus the search and acceptance, and the LM head once; the full
+    step time is extrapolated as 32 * layer + LM head.  Returns tokens/s and details."""
+    from oracle import copyspec_oracle as O
+    from paper_2502_08923_b200 import inputs
+    import threadpoolctl
+    cfg1 = inputs.sliced(cfg8b, 1)
+    h = [int(t) for t in hist]
+    n = len(h)
+    p0 = O.find_match(np.asarray(h), n, GAMMA, O.LATEST)
+    draft = O.gather_draft(h, n, p0, GAMMA, K_DRAFT)
+    block = [h[-1]] + draft
+    # the forward only needs the embedding rows of the block's tokens: a small table of
+    # those rows (taken from the LM-head matrix, which has the same shape and statistics)
+    emb_small = lm_head_cpu[np.asarray(block, dtype=np.int64)]
+    w = {"embed": emb_small, "lm_head": lm_head_cpu, "final_norm": weights_cpu_layer0["final_norm"],
+         "layers": [weights_cpu_layer0["layer"]]}
+    model = O.Model(cfg1, w, contract=True, cache_weights=True)
+    cache = O.KVCache(cfg1, 1, KV_START + 64, dtype=np.float32)
+    cache.a[0, :, 0, :, :KV_START, :] = kv_layer0
+    rows = list(range(len(block)))
+    t0 = time.perf_counter()
+    logits, hidden = model.forward_block(rows, KV_START, cache, 0, return_hidden=True)
+    t_first = time.perf_counter() - t0
+    # LM head (final norm, logits, greedy token per row), weights already converted
+    t0 = time.perf_counter()
+    xn = O.rmsnorm(hidden, model._w(None, "final_norm"), cfg1.rms_eps)
+    lg = model._mm(xn, None, "lm_head")
+    am = [O.argmax_lowest(lg[r]) for r in range(len(block))]
+    t_lm = time.perf_counter() - t0
+    # per-step sample: search + one layer's forward + acceptance (an 8-row stand-in head)
+    model._cache[(None, "lm_head")] = model._cache[(None, "lm_head")][:8]
+    times = []
+    for i in range(warmup + n_steps):
+        t0 = time.perf_counter()
+        p0 = O.find_match(np.asarray(h), n, GAMMA, O.LATEST)
+        draft = O.gather_draft(h, n, p0, GAMMA, K_DRAFT)
+        model.forward_block(rows, KV_START, cache, 0)
+        O.accept_length(draft, [int(t) for t in script[:len(draft) + 1]])
+        dt = time.perf_counter() - t0
+        if i >= warmup:
+            times.append(dt)
+    t_layer = float(np.mean(times))
+    step_s = cfg8b.n_layers * t_layer + t_lm
+    tokens_per_step = float(np.mean([t + 1 for t in taus]))
+    cores = max([p.get("num_threads", 1) for p in threadpoolctl.threadpool_info()] + [1])
+    return {"value": tokens_per_step / step_s, "unit": UNIT, "cores": int(cores), "kind": "oracle",
+            "sample": (f"{n_steps} steps of search + one decoder layer (of 32) over an 11-row block and 4,096 cached "
+                       f"positions + acceptance ({t_layer * 1e3:.1f} ms each), LM head once ({t_lm * 1e3:.0f} ms); "
+                       f"step time extrapolated as 32 x layer + LM head = {step_s * 1e3:.0f} ms"),
+            "ms_per_step": step_s * 1e3, "first_call_s": t_first}
+
+
+def _oracle_inputs(cfg, seed=0):
+    """The slices the CPU sample needs, drawn on the CPU with the bench's recipe."""
+    import torch
+    from paper_2502_08923_b200 import inputs
+    g = torch.Generator().manual_seed(seed)
+
+    def normal(*shape):
+        return torch.empty(*shape, dtype=torch.float32).normal_(0.0, 0.02, generator=g).to(torch.bfloat16)
+
+    d, f = cfg.d_model, cfg.d_ffn
+    layer = {"attn_norm": torch.ones(d, dtype=torch.bfloat16), "wqkv": normal(cfg.qkv_dim, d),
+             "wo": normal(d, cfg.q_dim), "ffn_norm": torch.ones(d, dtype=torch.bfloat16),
+             "w_gate_up": normal(2 * f, d), "w_down": normal(d, f)}
+    lm = normal(cfg.vocab, d)
+    kv = torch.empty(2, cfg.n_kv_heads, KV_START, cfg.head_dim).normal_(0.0, 1.0, generator=g).to(torch.bfloat16)
+    return {"layer": layer, "final_norm": torch.ones(d, dtype=torch.bfloat16)}, kv.float().numpy(), lm
+
+
+def run_reference(args):
+    rank, world, _ = _dist()
+    if rank != 0:
+        return 0
+    from paper_2502_08923_b200 import inputs
+    cfg = inputs.LLAMA8B
+    steps = args.steps
+    taus = _taus(args.warmup + steps)
+    hist, script = inputs.tau_controlled_case(np.random.default_rng(0), taus, GAMMA, K_DRAFT, KV_START, cfg.vocab)
+    w0, kv0, lm = _oracle_inputs(cfg)
+    res = oracle_sample(cfg, w0, kv0, lm, hist, script, taus, steps, args.warmup)
+    line = {"impl": "reference", "metric": METRIC, "value": res["value"], "unit": UNIT, "n_gpus": args.gpus,
+            "steps": steps, "warmup": args.warmup, "ms_per_step": res["ms_per_step"], "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "gamma": GAMMA, "k": K_DRAFT, "batch": 1, "kv_start": KV_START},
+            "cpu_baseline": {k: res[k] for k in ("value", "unit", "cores", "kind", "sample")},
+            "e2e": {"value": res["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+# ------------------------------------------------------------------------ CUDA leg
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2502_08923_b200 import binding as cs, inputs
+
+    rank, world, local = _dist()
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the CUDA library has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+    cfg = inputs.LLAMA8B
+    W, K = args.warmup, args.steps
+    taus = _taus(W + K)
+    ctx_len = KV_START
+    while True:
+        try:
+            hist, script = inputs.tau_controlled_case(np.random.default_rng(0), taus, GAMMA, K_DRAFT, ctx_len, cfg.vocab)
+            break
+        except ValueError:
+            ctx_len += 1024            # more steps than the 4,096-token context has room for
+    max_new = len(script)
+    n0 = len(hist)
+    stride = (n0 + max_new + 64 + 3) // 4 * 4
+    max_seq = n0 + max_new + K_DRAFT + 64
+
+    weights = inputs.make_weights(cfg, seed=0, device=str(dev))
+    ctx = cs.Context(cfg, weights, max_seq=max_seq, max_batch=1, k_max=K_DRAFT)
+    kv = inputs.synthetic_kv(cfg, 1, max_seq, n0 - 1, seed=1, device=str(dev))
+    hist_h = np.zeros((1, stride), dtype=np.int32)
+    hist_h[0, :n0] = hist
+    hist_d = torch.from_numpy(hist_h).to(dev)
+    len_d = torch.tensor([n0], dtype=torch.int32, device=dev)
+    kvlen_d = torch.tensor([n0 - 1], dtype=torch.int32, device=dev)
+    script_d = torch.from_numpy(script[None, :].copy()).to(dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident loop: W warm-up steps, then exactly K timed steps ------------
+    ctx.cs_loop_begin(hist_d, len_d, kv, kvlen_d, GAMMA, K_DRAFT, max_new, script=script_d)
+    launches_per_step = ctx.cs_loop_launches_per_step()
+    ctx.cs_loop_steps(W)
+    st0, _ = ctx.cs_loop_poll()
+    sampler = ClockSampler(local)
+    barrier()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    ctx.cs_loop_steps(K)
+    e1.record()
+    barrier()
+    ms = e0.elapsed_time(e1)
+    clocks = sampler.stop()
+    st1, done = ctx.cs_loop_poll()
+    ctx.cs_loop_end()
+    emitted = st1["emitted"] - st0["emitted"]
+    steps_run = st1["steps"] - st0["steps"]
+    expect = sum(t + 1 for t in taus[W:W + K])
+    if steps_run != K or emitted != expect:
+        raise RuntimeError(f"loop ran {steps_run} steps / {emitted} tokens, expected {K} / {expect}")
+    if world > 1:
+        t = torch.tensor([ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    value = world * emitted / (ms * 1e-3)
+
+    # ---- end to end from pinned host buffers (search + verify per step, host bookkeeping)
+    Ke = min(K, 50)
+    hist_p = torch.from_numpy(hist_h.copy()).pin_memory()
+    len_p = torch.tensor([n0], dtype=torch.int32).pin_memory()
+    scr_p = torch.zeros(1, K_DRAFT + 1, dtype=torch.int32).pin_memory()
+    res_p = torch.zeros(1, K_DRAFT + 2, dtype=torch.int32).pin_memory()
+    hist_e = torch.empty_like(hist_d)
+    len_e = torch.empty_like(len_d)
+    scr_e = torch.empty(1, K_DRAFT + 1, dtype=torch.int32, device=dev)
+    res_e = torch.empty(1, K_DRAFT + 2, dtype=torch.int32, device=dev)
+    mp = torch.empty(1, dtype=torch.int32, device=dev)
+    dr = torch.empty(1, K_DRAFT, dtype=torch.int32, device=dev)
+    dl = torch.empty(1, dtype=torch.int32, device=dev)
+    am = torch.empty(1, K_DRAFT + 1, dtype=torch.int32, device=dev)
+    kvlen_d.fill_(n0 - 1)
+    script_pad = np.concatenate([script, np.full(K_DRAFT + 1, -1, dtype=np.int32)])
+    h2d = hist_p.numel() * 4 + 4 + scr_p.numel() * 4
+    d2h = res_p.numel() * 4
+
+    def host_step(n, e):
+        scr_p[0].copy_(torch.from_numpy(script_pad[e:e + K_DRAFT + 1]))
+        len_p[0] = n
+        hist_e.copy_(hist_p, non_blocking=True)
+        len_e.copy_(len_p, non_blocking=True)
+        scr_e.copy_(scr_p, non_blocking=True)
+        cs.cs_find_match(hist_e, len_e, GAMMA, K_DRAFT, out=(mp, dr, dl))
+        last = hist_e[:, n - 1].contiguous()
+        ctx.cs_verify_step(last, dr, dl, kv, kvlen_d, target_script=scr_e, out=(res_e[0, :1], res_e[:, 1:], am))
+        res_p.copy_(res_e, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+        tau = int(res_p[0, 0])
+        hist_p[0, n:n + tau + 1] = res_p[0, 1:tau + 2]
+        return n + tau + 1, e + tau + 1
+
+    n, e = n0, 0
+    for _ in range(3):
+        n, e = host_step(n, e)
+    barrier()
+    t0 = time.perf_counter()
+    e_start = e
+    for _ in range(Ke):
+        n, e = host_step(n, e)
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+    if hist_p[0, n0:n].tolist() != script[:e].tolist():
+        raise RuntimeError("host-driven steps did not reproduce the script")
+    e2e_val = world * (e - e_start) / e2e_s
+
+    # ---- roofline of the dominant kernel (the weight-streaming projection GEMM) ---------
+    kvlen_d.fill_(n0 - 1)
+    last = torch.tensor([int(hist[-1])], dtype=torch.int32, device=dev)
+    dr.copy_(torch.from_numpy(script[None, :K_DRAFT].copy()))
+    dl.fill_(K_DRAFT)
+    fam_ms, fam_n = None, None
+    for _ in range(3):
+        kvlen_d.fill_(n0 - 1)
+        fam_ms, fam_n = ctx.cs_profile_verify_step(last, dr, dl, kv, kvlen_d)
+    layer_bytes = cfg.n_layers * cfg.params_per_layer() * 2
+    gemm_launches = max(1, fam_n["gemm"])
+    peak, peak_kind = _peaks()
+    achieved = layer_bytes / gemm_launches / (fam_ms["gemm"] / gemm_launches * 1e-3) / 1e9
+    step_bytes = cfg.streamed_params() * 2 + (n0 - 1 + 0.5 * emitted) * cfg.kv_bytes_per_token()
+    step_gbs = step_bytes / (ms / K * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "k_gemm_tc (layer projections)", "achieved": achieved, "peak": peak,
+                "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind,
+                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH,
+                "bytes_per_launch": layer_bytes / gemm_launches, "launches_per_step": gemm_launches,
+                "family_ms_per_step": fam_ms,
+                "step": {"algorithmic_gb": step_bytes / 1e9, "achieved_gbs": step_gbs, "frac_of_measured_copy": step_gbs / peak,
+                         "frac_of_8tbs": step_gbs / 8000.0}}
+
+    line = None
+    if rank == 0:
+        # ---- CPU oracle on the host cores, bounded sample (rank 0, N = 1 only) ---------
+        cpu = None
+        if world == 1 and not args.no_cpu_baseline:
+            w0 = {"layer": {k2: v.cpu() for k2, v in weights["layers"][0].items()}, "final_norm": weights["final_norm"].cpu()}
+            kv0 = kv[0, :, 0, :, :KV_START, :].float().cpu().numpy()
+            res = oracle_sample(cfg, w0, kv0, weights["lm_head"].cpu(), hist, script, taus, 12, 2)
+            cpu = {k2: res[k2] for k2 in ("value", "unit", "cores", "kind", "sample")}
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+                "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": "bf16", "data": "synthetic",
+                "config": {"workload": WORKLOAD, "model_shape": "32L d4096 H32/8 Dh128 F14336 V128256", "batch": 1,
+                           "gamma": GAMMA, "k": K_DRAFT, "kv_start": n0 - 1, "kv_end": n0 - 1 + st1["emitted"],
+                           "tokens_per_step": emitted / K, "l2": "inputs larger than L2 (15 GB of weights per step)",
+                           "replicas": world, "draft_tokens_accepted_per_s": world * (emitted - K) / (ms * 1e-3)},
+                "clocks": clocks,
+                "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                        "steps": Ke, "ms_per_step": e2e_s / Ke * 1e3},
+                "gpu_launches": launches_per_step * K,
+                "roofline": roofline, "cpu_baseline": cpu}
+        print(json.dumps(line), flush=True)
+    ctx.close()
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

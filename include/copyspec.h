@@ -188,6 +188,37 @@ cs_status cs_decode_loop(cs_ctx* ctx, int32_t* hist, int32_t* hist_len, int B, i
                          cs_match_policy policy, int max_new, int eos_id,
                          const int32_t* script, cs_stats* stats_out, void* stream);
 
+/* The same loop in pieces, for callers that want to run a fixed number of steps or overlap
+ * host work (App. B.3 steps 1, 2, 4; one step = search, gather, verify, accept, truncate,
+ * append for all B sequences).  cs_loop_begin takes cs_decode_loop's arguments, checks
+ * them, resets the per-sequence counters and statistics and prepares a CUDA graph of one
+ * step; the pointers must stay valid until cs_loop_end.  cs_loop_steps enqueues n_steps
+ * steps (async; steps of finished sequences do nothing).  cs_loop_poll waits for `stream`,
+ * copies the statistics (stats_out host, may be NULL) and the number of finished sequences
+ * (n_done_out host, may be NULL) and returns the device status like cs_sync_status.
+ * cs_loop_end releases the graph (also done by cs_destroy and by the next cs_loop_begin). */
+cs_status cs_loop_begin(cs_ctx* ctx, int32_t* hist, int32_t* hist_len, int B, int stride,
+                        void* kv_cache, int32_t* kv_len, int gamma, int k,
+                        cs_match_policy policy, int max_new, int eos_id, const int32_t* script,
+                        void* stream);
+cs_status cs_loop_steps(cs_ctx* ctx, int n_steps, void* stream);
+cs_status cs_loop_poll(cs_ctx* ctx, cs_stats* stats_out, int* n_done_out, void* stream);
+void cs_loop_end(cs_ctx* ctx);
+/* Kernel launches in one step of the loop in progress (nodes of its graph; 0 if none). */
+int cs_loop_launches_per_step(const cs_ctx* ctx);
+
+/* Measurement aid (no counterpart in the paper): runs cs_verify_step once with a CUDA event
+ * pair around every kernel launch and returns, per kernel family, the summed device time
+ * in milliseconds and the number of launches.  Families: 0 = projection GEMMs of the
+ * layers, 1 = attention, 2 = LM-head GEMM with fused argmax, 3 = element-wise kernels
+ * (embedding, norms, RoPE/KV append, SwiGLU).  family_ms and family_launches are host
+ * arrays of 4.  Synchronous. */
+cs_status cs_profile_verify_step(cs_ctx* ctx, const int32_t* last_tok, const int32_t* draft,
+                                 const int32_t* draft_len, int B, int k, void* kv_cache,
+                                 int32_t* kv_len, const int32_t* target_script,
+                                 int32_t* accept_len, int32_t* out_tokens, int32_t* argmax_ids,
+                                 float* family_ms, int* family_launches, void* stream);
+
 /* Helper off the hot path: computes the KV cache of positions [0, hist_len[b] - 1) by
  * running the forward over the history in blocks with every row forced (no LM head, no
  * acceptance), and sets kv_len[b] = hist_len[b] - 1.  `max_len` (host) is an upper bound

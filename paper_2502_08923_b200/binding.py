@@ -47,7 +47,9 @@ class CsStats(C.Structure):
 
 
 EXPORTS = ("cs_workspace_bytes", "cs_create", "cs_destroy", "cs_last_error", "cs_sync_status",
-           "cs_find_match", "cs_verify_step", "cs_kv_truncate", "cs_decode_loop", "cs_prefill", "cs_linear")
+           "cs_find_match", "cs_verify_step", "cs_kv_truncate", "cs_decode_loop", "cs_prefill", "cs_linear",
+           "cs_loop_begin", "cs_loop_steps", "cs_loop_poll", "cs_loop_end", "cs_profile_verify_step",
+           "cs_loop_launches_per_step")
 
 _lib = None
 
@@ -85,6 +87,19 @@ def load(build_if_missing: bool = True) -> C.CDLL:
     lib.cs_kv_truncate.argtypes = [vp, ip, ip, i, vp]
     lib.cs_decode_loop.restype = i
     lib.cs_decode_loop.argtypes = [vp, ip, ip, i, i, vp, ip, i, i, i, i, i, ip, C.POINTER(CsStats), vp]
+    lib.cs_loop_begin.restype = i
+    lib.cs_loop_begin.argtypes = [vp, ip, ip, i, i, vp, ip, i, i, i, i, i, ip, vp]
+    lib.cs_loop_steps.restype = i
+    lib.cs_loop_steps.argtypes = [vp, i, vp]
+    lib.cs_loop_poll.restype = i
+    lib.cs_loop_poll.argtypes = [vp, C.POINTER(CsStats), C.POINTER(C.c_int), vp]
+    lib.cs_loop_launches_per_step.restype = i
+    lib.cs_loop_launches_per_step.argtypes = [vp]
+    lib.cs_loop_end.restype = None
+    lib.cs_loop_end.argtypes = [vp]
+    lib.cs_profile_verify_step.restype = i
+    lib.cs_profile_verify_step.argtypes = [vp, ip, ip, ip, i, i, vp, ip, ip, ip, ip, ip, C.POINTER(C.c_float),
+                                           C.POINTER(C.c_int), vp]
     lib.cs_prefill.restype = i
     lib.cs_prefill.argtypes = [vp, ip, ip, i, i, i, vp, ip, vp]
     lib.cs_linear.restype = i
@@ -233,6 +248,50 @@ class Context:
                                      _i32(script, "script"), C.byref(st), _stream())
         self._check(rc, "cs_decode_loop")
         return st.as_dict()
+
+    def cs_loop_begin(self, hist, hist_len, kv_cache, kv_len, gamma, k, max_new, policy=LATEST, eos_id=-1,
+                      script=None):
+        B, stride = hist.shape
+        self._loop_refs = (hist, hist_len, kv_cache, kv_len, script)     # keep the buffers alive
+        rc = self.lib.cs_loop_begin(self.handle, _i32(hist, "hist"), _i32(hist_len, "hist_len"), B, stride,
+                                    _ptr(kv_cache), _i32(kv_len, "kv_len"), gamma, k, policy, max_new, eos_id,
+                                    _i32(script, "script"), _stream())
+        self._check(rc, "cs_loop_begin")
+
+    def cs_loop_steps(self, n_steps):
+        self._check(self.lib.cs_loop_steps(self.handle, n_steps, _stream()), "cs_loop_steps")
+
+    def cs_loop_poll(self):
+        """Waits for the stream; returns (statistics dict, number of finished sequences)."""
+        st, done = CsStats(), C.c_int(0)
+        self._check(self.lib.cs_loop_poll(self.handle, C.byref(st), C.byref(done), _stream()), "cs_loop_poll")
+        return st.as_dict(), done.value
+
+    def cs_loop_launches_per_step(self):
+        return self.lib.cs_loop_launches_per_step(self.handle)
+
+    def cs_loop_end(self):
+        self.lib.cs_loop_end(self.handle)
+        self._loop_refs = None
+
+    def cs_profile_verify_step(self, last_tok, draft, draft_len, kv_cache, kv_len, target_script=None):
+        """cs_verify_step with event brackets; returns ({family: ms}, {family: launches})."""
+        B = last_tok.shape[0]
+        k = draft.shape[1] if draft is not None and draft.dim() == 2 else 0
+        dev = last_tok.device
+        al = torch.empty(B, dtype=torch.int32, device=dev)
+        ot = torch.empty(B, k + 1, dtype=torch.int32, device=dev)
+        am = torch.empty(B, k + 1, dtype=torch.int32, device=dev)
+        ms, n = (C.c_float * 4)(), (C.c_int * 4)()
+        rc = self.lib.cs_profile_verify_step(self.handle, _i32(last_tok, "last_tok"),
+                                             C.c_void_p(draft.data_ptr()) if k > 0 else None,
+                                             _i32(draft_len, "draft_len"), B, k, _ptr(kv_cache),
+                                             _i32(kv_len, "kv_len"), _i32(target_script, "target_script"),
+                                             _i32(al, "accept_len"), _i32(ot, "out_tokens"), _i32(am, "argmax_ids"),
+                                             ms, n, _stream())
+        self._check(rc, "cs_profile_verify_step")
+        names = ("gemm", "attention", "lm_head", "elementwise")
+        return dict(zip(names, list(ms))), dict(zip(names, list(n)))
 
     def cs_linear(self, X, W, rows=None):
         """Y[rows][N] fp32 = X[rows][K] bf16 @ W[N][K]^T bf16 through the tensor-core GEMM."""

@@ -102,6 +102,21 @@ cs_status ensure_act_maps(cs_ctx* ctx, int n_tok) {
   return CS_OK;
 }
 
+void prof_begin(cs_ctx* ctx, int fam, cudaStream_t st) {
+  Prof* p = ctx->prof;
+  if (p == nullptr || p->n >= CS_PROF_MAX) return;
+  cudaEventCreate(&p->ev[2 * p->n]);
+  cudaEventCreate(&p->ev[2 * p->n + 1]);
+  p->fam[p->n] = fam;
+  cudaEventRecord(p->ev[2 * p->n], st);
+}
+void prof_end(cs_ctx* ctx, cudaStream_t st) {
+  Prof* p = ctx->prof;
+  if (p == nullptr || p->n >= CS_PROF_MAX) return;
+  cudaEventRecord(p->ev[2 * p->n + 1], st);
+  p->n += 1;
+}
+
 // The forward of Sec. 3.2 over the rows prepared by a *_setup kernel: B sequences of R
 // rows each.  With `with_lm` the LM head leaves per-tile (max, id) pairs for k_accept.
 cs_status enqueue_forward(cs_ctx* ctx, int B, int R, void* kv_cache, bool with_lm, float* logits,
@@ -110,24 +125,48 @@ cs_status enqueue_forward(cs_ctx* ctx, int B, int R, void* kv_cache, bool with_l
   const int rows = B * R;
   cs_status s = ensure_act_maps(ctx, cs_ceil_div(rows, 16) * 16);
   if (s != CS_OK) return s;
+  prof_begin(ctx, CS_FAM_ELEMENTWISE, st);
   cs_launch_embed(ctx, rows, st);
+  prof_end(ctx, st);
   int prev_splits = 0;
   for (int l = 0; l < c.n_layers; ++l) {
     const LayerPlan& L = ctx->layers[l];
+    prof_begin(ctx, CS_FAM_ELEMENTWISE, st);
     cs_launch_rmsnorm(ctx, l == 0 ? nullptr : ctx->partial, prev_splits, L.attn_norm, rows, st);
-    if ((s = cs_launch_gemm(ctx, &L.qkv, &ctx->tmXn, ctx->xn, rows, 0, ctx->partial, nullptr, st)) != CS_OK) return s;
+    prof_end(ctx, st);
+    prof_begin(ctx, CS_FAM_GEMM, st);
+    if ((s = cs_launch_gemm(ctx, &L.qkv, &ctx->tmXn, ctx->xn, rows, 0, ctx->partial, nullptr, st)) != CS_OK) { prof_end(ctx, st); return s; }
+    prof_end(ctx, st);
+    prof_begin(ctx, CS_FAM_ELEMENTWISE, st);
     cs_launch_qkv_post(ctx, L.qkv.splits, kv_cache, l, B, R, st);
+    prof_end(ctx, st);
+    prof_begin(ctx, CS_FAM_ATTENTION, st);
     cs_launch_attention(ctx, kv_cache, l, B, R, st);
-    if ((s = cs_launch_gemm(ctx, &L.o, &ctx->tmAttn, ctx->attn_out, rows, 0, ctx->partial, nullptr, st)) != CS_OK) return s;
+    prof_end(ctx, st);
+    prof_begin(ctx, CS_FAM_GEMM, st);
+    if ((s = cs_launch_gemm(ctx, &L.o, &ctx->tmAttn, ctx->attn_out, rows, 0, ctx->partial, nullptr, st)) != CS_OK) { prof_end(ctx, st); return s; }
+    prof_end(ctx, st);
+    prof_begin(ctx, CS_FAM_ELEMENTWISE, st);
     cs_launch_rmsnorm(ctx, ctx->partial, L.o.splits, L.ffn_norm, rows, st);
-    if ((s = cs_launch_gemm(ctx, &L.gate_up, &ctx->tmXn, ctx->xn, rows, 0, ctx->partial, nullptr, st)) != CS_OK) return s;
+    prof_end(ctx, st);
+    prof_begin(ctx, CS_FAM_GEMM, st);
+    if ((s = cs_launch_gemm(ctx, &L.gate_up, &ctx->tmXn, ctx->xn, rows, 0, ctx->partial, nullptr, st)) != CS_OK) { prof_end(ctx, st); return s; }
+    prof_end(ctx, st);
+    prof_begin(ctx, CS_FAM_ELEMENTWISE, st);
     cs_launch_swiglu(ctx, L.gate_up.splits, rows, st);
-    if ((s = cs_launch_gemm(ctx, &L.down, &ctx->tmAct, ctx->act, rows, 0, ctx->partial, nullptr, st)) != CS_OK) return s;
+    prof_end(ctx, st);
+    prof_begin(ctx, CS_FAM_GEMM, st);
+    if ((s = cs_launch_gemm(ctx, &L.down, &ctx->tmAct, ctx->act, rows, 0, ctx->partial, nullptr, st)) != CS_OK) { prof_end(ctx, st); return s; }
+    prof_end(ctx, st);
     prev_splits = L.down.splits;
   }
   if (with_lm) {
+    prof_begin(ctx, CS_FAM_ELEMENTWISE, st);
     cs_launch_rmsnorm(ctx, ctx->partial, prev_splits, ctx->final_norm, rows, st);
-    if ((s = cs_launch_gemm(ctx, &ctx->lm, &ctx->tmXn, ctx->xn, rows, 1, nullptr, logits, st)) != CS_OK) return s;
+    prof_end(ctx, st);
+    prof_begin(ctx, CS_FAM_LMHEAD, st);
+    if ((s = cs_launch_gemm(ctx, &ctx->lm, &ctx->tmXn, ctx->xn, rows, 1, nullptr, logits, st)) != CS_OK) { prof_end(ctx, st); return s; }
+    prof_end(ctx, st);
   }
   CS_CUDA_OK(ctx, cudaGetLastError());
   return CS_OK;
@@ -140,6 +179,23 @@ __global__ void k_reduce_partial(const float* __restrict__ partial, int splits, 
   float v = 0.f;
   for (int s = 0; s < splits; ++s) v += partial[(size_t)s * rows * N + i];
   y[i] = v;
+}
+
+// One iteration of the generation loop (App. B.3 steps 1, 2, 4) on device-resident state.
+cs_status enqueue_loop_step(cs_ctx* ctx, cudaStream_t st) {
+  const LoopState& L = ctx->loop;
+  cs_status r = cs_launch_find_match(L.hist, L.hist_len, L.B, L.stride, L.gamma, L.k, L.policy, ctx->loop_mpos,
+                                     ctx->loop_draft, ctx->loop_dlen, ctx->loop_last, ctx->loop_done, st);
+  if (r != CS_OK) return fail(ctx, r, "match kernel launch failed");
+  cs_launch_block_setup(ctx, ctx->loop_last, ctx->loop_draft, ctx->loop_dlen, L.kv_len, ctx->loop_done, L.B, L.k, st);
+  r = enqueue_forward(ctx, L.B, L.k + 1, L.kv_cache, true, nullptr, st);
+  if (r != CS_OK) return r;
+  cs_launch_accept(ctx, L.B, L.k, ctx->loop_draft, ctx->loop_dlen, L.script, L.max_new, ctx->loop_emitted, L.max_new,
+                   ctx->loop_accept, ctx->loop_out, ctx->loop_argmax, L.kv_len, 0, st);
+  cs_launch_loop_commit(ctx, L.hist, L.hist_len, L.B, L.stride, L.kv_len, L.k, L.max_new, L.eos_id,
+                        L.script != nullptr, st);
+  CS_CUDA_OK(ctx, cudaGetLastError());
+  return CS_OK;
 }
 
 cs_status status_from_bits(cs_ctx* ctx, int bits) {
@@ -277,6 +333,7 @@ cs_status cs_create(cs_ctx** out, const cs_model_config* cfg, const cs_weights* 
 
 void cs_destroy(cs_ctx* ctx) {
   if (ctx == nullptr) return;
+  cs_loop_end(ctx);
   if (ctx->cap_stream) cudaStreamDestroy(ctx->cap_stream);
   delete[] ctx->layers;
   delete ctx;
@@ -357,9 +414,9 @@ cs_status cs_prefill(cs_ctx* ctx, const int32_t* hist, const int32_t* hist_len, 
   return CS_OK;
 }
 
-cs_status cs_decode_loop(cs_ctx* ctx, int32_t* hist, int32_t* hist_len, int B, int stride, void* kv_cache,
-                         int32_t* kv_len, int gamma, int k, cs_match_policy policy, int max_new, int eos_id,
-                         const int32_t* script, cs_stats* stats_out, void* stream) {
+cs_status cs_loop_begin(cs_ctx* ctx, int32_t* hist, int32_t* hist_len, int B, int stride, void* kv_cache,
+                        int32_t* kv_len, int gamma, int k, cs_match_policy policy, int max_new, int eos_id,
+                        const int32_t* script, void* stream) {
   if (ctx == nullptr) return CS_ERR_ARG;
   if (B < 1 || B > ctx->cfg.max_batch || k < 0 || k > ctx->cfg.k_max || gamma < 1 || gamma > CS_MAX_GAMMA ||
       max_new < 0 || stride < 1)
@@ -367,82 +424,124 @@ cs_status cs_decode_loop(cs_ctx* ctx, int32_t* hist, int32_t* hist_len, int B, i
   if (policy != CS_MATCH_LATEST && policy != CS_MATCH_FIRST) return fail(ctx, CS_ERR_ARG, "bad policy");
   if (hist == nullptr || hist_len == nullptr || kv_cache == nullptr || kv_len == nullptr)
     return fail(ctx, CS_ERR_ARG, "NULL argument");
+  cs_loop_end(ctx);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  LoopState& L = ctx->loop;
+  L.hist = hist; L.hist_len = hist_len; L.B = B; L.stride = stride; L.kv_cache = kv_cache; L.kv_len = kv_len;
+  L.gamma = gamma; L.k = k; L.policy = (int)policy; L.max_new = max_new; L.eos_id = eos_id; L.script = script;
   const char* env = getenv("CS_NO_GRAPH");
-  const bool use_graph = !(env != nullptr && env[0] == '1');
+  L.use_graph = !(env != nullptr && env[0] == '1');
 
   cs_launch_loop_init(ctx, hist_len, kv_len, B, stride, max_new, k, st);
   CS_CUDA_OK(ctx, cudaGetLastError());
-  // the activation maps must exist before capture (encoding is host work)
+  // the activation maps must exist before capture (encoding them is host work)
   cs_status s = ensure_act_maps(ctx, cs_ceil_div(B * (k + 1), 16) * 16);
   if (s != CS_OK) return s;
-
-  auto enqueue_step = [&](cudaStream_t st) -> cs_status {
-    cs_status r = cs_launch_find_match(hist, hist_len, B, stride, gamma, k, (int)policy, ctx->loop_mpos,
-                                       ctx->loop_draft, ctx->loop_dlen, ctx->loop_last, ctx->loop_done, st);
-    if (r != CS_OK) return fail(ctx, r, "match kernel launch failed");
-    cs_launch_block_setup(ctx, ctx->loop_last, ctx->loop_draft, ctx->loop_dlen, kv_len, ctx->loop_done, B, k, st);
-    r = enqueue_forward(ctx, B, k + 1, kv_cache, true, nullptr, st);
-    if (r != CS_OK) return r;
-    cs_launch_accept(ctx, B, k, ctx->loop_draft, ctx->loop_dlen, script, max_new, ctx->loop_emitted, max_new,
-                     ctx->loop_accept, ctx->loop_out, ctx->loop_argmax, kv_len, 0, st);
-    cs_launch_loop_commit(ctx, hist, hist_len, B, stride, kv_len, k, max_new, eos_id, script != nullptr, st);
-    return CS_OK;
-  };
-
-  cudaGraph_t graph = nullptr;
-  cudaGraphExec_t exec = nullptr;
-  if (use_graph) {
+  if (L.use_graph) {
     // captured on the context's own stream (the legacy default stream cannot capture),
     // replayed on the caller's
     CS_CUDA_OK(ctx, cudaStreamBeginCapture(ctx->cap_stream, cudaStreamCaptureModeRelaxed));
-    s = enqueue_step(ctx->cap_stream);
-    cudaError_t e = cudaStreamEndCapture(ctx->cap_stream, &graph);
-    if (s != CS_OK) { if (graph) cudaGraphDestroy(graph); return s; }
-    CS_CUDA_OK(ctx, e);
-    e = cudaGraphInstantiate(&exec, graph, 0);
-    if (e != cudaSuccess) { cudaGraphDestroy(graph); CS_CUDA_OK(ctx, e); }
+    s = enqueue_loop_step(ctx, ctx->cap_stream);
+    cudaError_t e = cudaStreamEndCapture(ctx->cap_stream, &L.graph);
+    if (s != CS_OK) { cs_loop_end(ctx); return s; }
+    if (e != cudaSuccess) { cs_loop_end(ctx); CS_CUDA_OK(ctx, e); }
+    e = cudaGraphInstantiate(&L.exec, L.graph, 0);
+    if (e != cudaSuccess) { cs_loop_end(ctx); CS_CUDA_OK(ctx, e); }
+    size_t nodes = 0;
+    if (cudaGraphGetNodes(L.graph, nullptr, &nodes) == cudaSuccess) L.graph_nodes = (int)nodes;
   }
-  int* h_done = nullptr;
-  cudaError_t e = cudaMallocHost(&h_done, sizeof(int));
-  if (e != cudaSuccess) {
-    if (exec) cudaGraphExecDestroy(exec);
-    if (graph) cudaGraphDestroy(graph);
-    CS_CUDA_OK(ctx, e);
-  }
-  *h_done = 0;
-  const int poll = 4;
-  int steps = 0;
-  s = CS_OK;
-  while (steps < max_new && s == CS_OK) {
-    const int nrun = (max_new - steps < poll) ? max_new - steps : poll;
-    for (int i = 0; i < nrun && s == CS_OK; ++i) {
-      if (use_graph) {
-        if (cudaGraphLaunch(exec, st) != cudaSuccess) s = fail(ctx, CS_ERR_CUDA, "cudaGraphLaunch failed");
-      } else {
-        s = enqueue_step(st);
-      }
+  L.active = true;
+  return CS_OK;
+}
+
+cs_status cs_loop_steps(cs_ctx* ctx, int n_steps, void* stream) {
+  if (ctx == nullptr) return CS_ERR_ARG;
+  if (!ctx->loop.active || n_steps < 0) return fail(ctx, CS_ERR_ARG, "no loop in progress");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  for (int i = 0; i < n_steps; ++i) {
+    if (ctx->loop.use_graph) {
+      CS_CUDA_OK(ctx, cudaGraphLaunch(ctx->loop.exec, st));
+    } else {
+      cs_status s = enqueue_loop_step(ctx, st);
+      if (s != CS_OK) return s;
     }
+  }
+  return CS_OK;
+}
+
+cs_status cs_loop_poll(cs_ctx* ctx, cs_stats* stats_out, int* n_done_out, void* stream) {
+  if (ctx == nullptr) return CS_ERR_ARG;
+  if (!ctx->loop.active) return fail(ctx, CS_ERR_ARG, "no loop in progress");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int done = 0;
+  CS_CUDA_OK(ctx, cudaMemcpyAsync(&done, ctx->loop_done + ctx->cfg.max_batch, sizeof(int), cudaMemcpyDeviceToHost, st));
+  if (stats_out != nullptr)
+    CS_CUDA_OK(ctx, cudaMemcpyAsync(stats_out, ctx->loop_stats, sizeof(cs_stats), cudaMemcpyDeviceToHost, st));
+  CS_CUDA_OK(ctx, cudaStreamSynchronize(st));
+  if (n_done_out != nullptr) *n_done_out = done;
+  return cs_sync_status(ctx, stream);
+}
+
+int cs_loop_launches_per_step(const cs_ctx* ctx) {
+  return (ctx != nullptr && ctx->loop.active) ? ctx->loop.graph_nodes : 0;
+}
+
+void cs_loop_end(cs_ctx* ctx) {
+  if (ctx == nullptr) return;
+  if (ctx->loop.exec) cudaGraphExecDestroy(ctx->loop.exec);
+  if (ctx->loop.graph) cudaGraphDestroy(ctx->loop.graph);
+  ctx->loop.exec = nullptr;
+  ctx->loop.graph = nullptr;
+  ctx->loop.active = false;
+}
+
+cs_status cs_decode_loop(cs_ctx* ctx, int32_t* hist, int32_t* hist_len, int B, int stride, void* kv_cache,
+                         int32_t* kv_len, int gamma, int k, cs_match_policy policy, int max_new, int eos_id,
+                         const int32_t* script, cs_stats* stats_out, void* stream) {
+  cs_status s = cs_loop_begin(ctx, hist, hist_len, B, stride, kv_cache, kv_len, gamma, k, policy, max_new, eos_id,
+                              script, stream);
+  if (s != CS_OK) return s;
+  // every live sequence emits at least one token per step, so max_new steps always suffice
+  const int poll = 4;
+  int steps = 0, done = 0;
+  while (s == CS_OK) {
+    const int nrun = (max_new - steps < poll) ? max_new - steps : poll;
+    if (nrun > 0) s = cs_loop_steps(ctx, nrun, stream);
     steps += nrun;
     if (s != CS_OK) break;
-    if (cudaMemcpyAsync(h_done, ctx->loop_done + ctx->cfg.max_batch, sizeof(int), cudaMemcpyDeviceToHost, st) !=
-            cudaSuccess ||
-        cudaStreamSynchronize(st) != cudaSuccess) {
-      s = fail(ctx, CS_ERR_CUDA, cudaGetErrorString(cudaGetLastError()));
-      break;
+    s = cs_loop_poll(ctx, stats_out, &done, stream);
+    if (done >= B || steps >= max_new) break;
+  }
+  cs_loop_end(ctx);
+  return s;
+}
+
+cs_status cs_profile_verify_step(cs_ctx* ctx, const int32_t* last_tok, const int32_t* draft,
+                                 const int32_t* draft_len, int B, int k, void* kv_cache, int32_t* kv_len,
+                                 const int32_t* target_script, int32_t* accept_len, int32_t* out_tokens,
+                                 int32_t* argmax_ids, float* family_ms, int* family_launches, void* stream) {
+  if (ctx == nullptr || family_ms == nullptr || family_launches == nullptr) return CS_ERR_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  Prof prof;
+  memset(&prof, 0, sizeof(prof));
+  ctx->prof = &prof;
+  cs_status s = cs_verify_step(ctx, last_tok, draft, draft_len, B, k, kv_cache, kv_len, target_script, accept_len,
+                               out_tokens, argmax_ids, nullptr, stream);
+  ctx->prof = nullptr;
+  cudaError_t e = cudaStreamSynchronize(st);
+  for (int f = 0; f < CS_PROF_FAMILIES; ++f) { family_ms[f] = 0.f; family_launches[f] = 0; }
+  for (int i = 0; i < prof.n; ++i) {
+    float ms = 0.f;
+    if (e == cudaSuccess && s == CS_OK && cudaEventElapsedTime(&ms, prof.ev[2 * i], prof.ev[2 * i + 1]) == cudaSuccess) {
+      family_ms[prof.fam[i]] += ms;
+      family_launches[prof.fam[i]] += 1;
     }
-    if (*h_done >= B) break;
+    cudaEventDestroy(prof.ev[2 * i]);
+    cudaEventDestroy(prof.ev[2 * i + 1]);
   }
-  if (s == CS_OK && stats_out != nullptr) {
-    if (cudaMemcpyAsync(stats_out, ctx->loop_stats, sizeof(cs_stats), cudaMemcpyDeviceToHost, st) != cudaSuccess)
-      s = fail(ctx, CS_ERR_CUDA, "copying the statistics failed");
-  }
-  if (cudaStreamSynchronize(st) != cudaSuccess && s == CS_OK) s = fail(ctx, CS_ERR_CUDA, "stream synchronize failed");
-  cudaFreeHost(h_done);
-  if (exec) cudaGraphExecDestroy(exec);
-  if (graph) cudaGraphDestroy(graph);
   if (s != CS_OK) return s;
-  return cs_sync_status(ctx, stream);
+  CS_CUDA_OK(ctx, e);
+  return CS_OK;
 }
 
 cs_status cs_linear(cs_ctx* ctx, const void* X, const void* W, int rows, int N, int K, float* Y, void* stream) {

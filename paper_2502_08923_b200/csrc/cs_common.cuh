@@ -39,6 +39,28 @@ struct LayerPlan {
   const __nv_bfloat16 *attn_norm, *ffn_norm;
 };
 
+// device-resident generation loop between cs_loop_begin and cs_loop_end
+struct LoopState {
+  bool active, use_graph;
+  int32_t *hist, *hist_len, *kv_len;
+  const int32_t* script;
+  void* kv_cache;
+  int B, stride, gamma, k, policy, max_new, eos_id;
+  int graph_nodes;   // kernel launches in one step
+  cudaGraph_t graph;
+  cudaGraphExec_t exec;
+};
+
+// event brackets around kernel families (cs_profile_verify_step)
+static constexpr int CS_PROF_MAX = 2048;
+static constexpr int CS_PROF_FAMILIES = 4;
+enum : int { CS_FAM_GEMM = 0, CS_FAM_ATTENTION = 1, CS_FAM_LMHEAD = 2, CS_FAM_ELEMENTWISE = 3 };
+struct Prof {
+  cudaEvent_t ev[2 * CS_PROF_MAX];
+  int fam[CS_PROF_MAX];
+  int n;
+};
+
 struct cs_ctx {
   cs_model_config cfg;
   int max_rows;      // max_batch * (k_max + 1)
@@ -89,6 +111,9 @@ struct cs_ctx {
   // activation operand maps, rebuilt when the block height changes
   int act_ntok;
   CUtensorMap tmXn, tmAttn, tmAct;
+
+  LoopState loop;
+  Prof* prof;   // non-NULL only inside cs_profile_verify_step
 
   char err[256];
 };

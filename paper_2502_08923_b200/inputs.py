@@ -297,3 +297,61 @@ def verify_inputs_with_tau(rng: np.random.Generator, batch: int, k: int, taus, v
     last_tok = rng.integers(0, vocab, size=batch, dtype=np.int32)
     draft_len = np.full(batch, k, dtype=np.int32)
     return last_tok, draft.astype(np.int32), draft_len, script
+
+
+def tau_controlled_case(rng: np.random.Generator, taus, gamma: int = 3, k: int = 10,
+                        context_len: int = 4096, vocab: int = 128256) -> tuple:
+    """A history and a scripted continuation on which every decode step finds a match and
+    accepts exactly `taus[i]` draft tokens at step i (0 <= taus[i] <= k).
+
+    The context holds one "path" of distinct tokens per step.  A path starts with the two
+    tokens that end the previous step's accepted run, so when the script leaves the path
+    being copied (rejecting draft token taus[i]) the extra token it emits completes the
+    opening gamma-gram of the next path, which is the only earlier occurrence of the new
+    suffix.  taus[i] == k means the whole draft is accepted and the same path goes on.
+    All tokens are distinct ids, so no chance matches occur.  Returns `(hist, script)`:
+    hist has `context_len + 1` tokens (so the KV cache holds `context_len` positions
+    before the first step), script has sum(taus) + len(taus) tokens.  Only gamma == 3."""
+    assert gamma == 3
+    taus = [int(t) for t in taus]
+    ids = rng.permutation(vocab).astype(np.int32)
+    nxt = [0]
+
+    def fresh(n):
+        out = ids[nxt[0]:nxt[0] + n].tolist()
+        nxt[0] += n
+        if nxt[0] > vocab:
+            raise ValueError("vocabulary too small for this many steps")
+        return out
+
+    paths = [fresh(3)]
+    script = []
+    tail = list(paths[0][:3])          # last tokens of history + script so far
+    cur, pos = 0, 3
+    for tau in taus:
+        need = pos + 2 * k + 2 - len(paths[cur])
+        if need > 0:
+            paths[cur].extend(fresh(need))
+        if tau >= k:
+            seg = paths[cur][pos:pos + k + 1]
+            script.extend(seg)
+            tail = (tail + seg)[-3:]
+            pos += k + 1
+        else:
+            seg = paths[cur][pos:pos + tau]
+            script.extend(seg)
+            tail = (tail + seg)[-3:]
+            new = [tail[-2], tail[-1]] + fresh(1)
+            script.append(new[2])
+            tail = (tail + [new[2]])[-3:]
+            paths.append(new)
+            cur, pos = len(paths) - 1, 3
+    need = pos + 2 * k + 2 - len(paths[cur])
+    if need > 0:
+        paths[cur].extend(fresh(need))
+    body = [t for p in paths for t in p]
+    room = context_len + 1 - 3 - len(body)
+    if room < 0:
+        raise ValueError(f"context_len {context_len} too small: the paths need {len(body) + 2} tokens")
+    hist = fresh(room) + body + list(paths[0][:3])
+    return np.asarray(hist, dtype=np.int32), np.asarray(script, dtype=np.int32)
