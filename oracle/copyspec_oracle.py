@@ -24,8 +24,9 @@ Readings taken where the paper is silent or at odds with itself:
 
 Precision contract (`contract=True`): what "bf16 weights, bf16 KV cache, fp32
 accumulation" means operationally - every contraction (projection GEMMs, q.k, LM head)
-takes its activation operand rounded to nearest-even bf16, new K/V rows are stored as
-bf16, everything else (residual stream, norms, softmax, accumulation) is wide.  With
+(projection GEMMs, q.k, softmax-weights times V, LM head) takes its activation operand
+rounded to nearest-even bf16, new K/V rows are stored as bf16, everything else (residual
+stream, norms, the softmax itself, accumulation) is wide.  With
 `contract=False` nothing is rounded: the plain fp64 definition.
 
 Pins (tests/test_oracle_*.py): brute-force enumeration of all matches; closed forms
@@ -194,11 +195,11 @@ class KVCache:
 class Model:
     """Decoder-only target model evaluated block-wise against a KV cache."""
 
-    def __init__(self, cfg, weights, contract=True, round_p=False, cache_weights=True):
+    def __init__(self, cfg, weights, contract=True, round_p=None, cache_weights=True):
         self.cfg = cfg
         self.w = weights
         self.contract = contract
-        self.round_p = round_p
+        self.round_p = contract if round_p is None else round_p
         self._cache = {} if cache_weights else None
 
     # weights are converted to fp64 on use (and kept, for small models)

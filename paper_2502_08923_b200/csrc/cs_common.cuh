@@ -165,6 +165,7 @@ void cs_launch_qkv_post(cs_ctx* ctx, int splits, void* kv_cache, int layer, int 
                         cudaStream_t st);
 void cs_launch_attention(cs_ctx* ctx, const void* kv_cache, int layer, int B, int R,
                          cudaStream_t st);
+void cs_launch_attn_merge(cs_ctx* ctx, int nsplit, int rows, cudaStream_t st);
 void cs_launch_swiglu(cs_ctx* ctx, int splits, int rows, cudaStream_t st);
 void cs_launch_accept(cs_ctx* ctx, int B, int k, const int32_t* draft, const int32_t* draft_len,
                       const int32_t* script, int script_stride, const int32_t* script_off,

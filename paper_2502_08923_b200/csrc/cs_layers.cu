@@ -170,171 +170,6 @@ __global__ void k_qkv_post(const float* __restrict__ partial, int splits, int ro
   }
 }
 
-// ------------------------------------------------------------------ attention
-// One CTA = one (sequence, KV head), one slice of the keys, up to 48 query rows (the
-// G query heads of the group times the block rows).  K/V tiles of 64 keys are staged in
-// shared memory once and reused by all rows; scores and the running softmax are fp32.
-constexpr int kAttnThreads = 256;
-constexpr int kAttnRowsPerWarp = 6;
-constexpr int kAttnRows = 8 * kAttnRowsPerWarp;   // 48
-constexpr int kAttnKeys = 64;
-
-template <int DH>
-__global__ void __launch_bounds__(kAttnThreads)
-k_attn_partial(const __nv_bfloat16* __restrict__ qbuf, const __nv_bfloat16* __restrict__ kv,
-               const int* __restrict__ row_lim, int layer, int R, int H, int Hkv, int max_batch,
-               int max_seq, int nsplit, float scale, float* __restrict__ out_o, float* __restrict__ out_ml,
-               int rows) {
-  constexpr int KSTRIDE = DH + 8;          // bf16 elements; 16 bytes of padding kill bank conflicts
-  constexpr int DPL = DH / 32;             // output dims per lane
-  extern __shared__ __align__(16) uint8_t smem[];
-  __nv_bfloat16* Ks = reinterpret_cast<__nv_bfloat16*>(smem);
-  __nv_bfloat16* Vs = Ks + kAttnKeys * KSTRIDE;
-  float* Qs = reinterpret_cast<float*>(Vs + kAttnKeys * KSTRIDE);      // [48][DH]
-  float* Ps = Qs + kAttnRows * DH;                                      // [8][6][64]
-  __shared__ int s_lim[kAttnRows];
-  __shared__ int s_grow[kAttnRows];   // global row
-  __shared__ int s_head[kAttnRows];
-
-  const int G = H / Hkv;
-  const int b = blockIdx.x / Hkv, kvh = blockIdx.x % Hkv;
-  const int split = blockIdx.y, rt = blockIdx.z;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int nq = G * R;                       // query rows of this (sequence, KV head)
-  const int q0 = rt * kAttnRows;
-  const int nrows = min(kAttnRows, nq - q0);
-
-  // query row idx -> (head g, block row r)
-  for (int i = threadIdx.x; i < kAttnRows; i += kAttnThreads) {
-    if (i < nrows) {
-      const int g = (q0 + i) / R, r = (q0 + i) % R;
-      s_grow[i] = b * R + r;
-      s_head[i] = kvh * G + g;
-      s_lim[i] = row_lim[b * R + r];
-    } else {
-      s_grow[i] = 0; s_head[i] = 0; s_lim[i] = 0;
-    }
-  }
-  __syncthreads();
-  int lmax = 0;
-  for (int i = 0; i < nrows; ++i) lmax = max(lmax, s_lim[i]);
-  for (int i = threadIdx.x; i < kAttnRows * DH; i += kAttnThreads) {
-    const int qi = i / DH, dd = i % DH;
-    Qs[i] = (qi < nrows) ? __bfloat162float(qbuf[((size_t)s_grow[qi] * H + s_head[qi]) * DH + dd]) : 0.f;
-  }
-
-  const int ntiles = (lmax + kAttnKeys - 1) / kAttnKeys;
-  const int tps = (ntiles + nsplit - 1) / nsplit;
-  const int t0 = split * tps, t1 = min(ntiles, t0 + tps);
-  const __nv_bfloat16* Kg = kv + ((((size_t)layer * 2 + 0) * max_batch + b) * Hkv + kvh) * (size_t)max_seq * DH;
-  const __nv_bfloat16* Vg = kv + ((((size_t)layer * 2 + 1) * max_batch + b) * Hkv + kvh) * (size_t)max_seq * DH;
-
-  float m[kAttnRowsPerWarp], l[kAttnRowsPerWarp], o[kAttnRowsPerWarp][DPL];
-#pragma unroll
-  for (int i = 0; i < kAttnRowsPerWarp; ++i) {
-    m[i] = -INFINITY; l[i] = 0.f;
-#pragma unroll
-    for (int dd = 0; dd < DPL; ++dd) o[i][dd] = 0.f;
-  }
-
-  for (int t = t0; t < t1; ++t) {
-    const int key0 = t * kAttnKeys;
-    __syncthreads();   // previous tile fully consumed (also covers the Q staging)
-    // stage K and V: 16-byte chunks, keys past the longest row are zero-filled
-    constexpr int CPR = DH / 8;
-    for (int c = threadIdx.x; c < kAttnKeys * CPR; c += kAttnThreads) {
-      const int j = c / CPR, cc = c % CPR;
-      uint4 kq = make_uint4(0, 0, 0, 0), vq = make_uint4(0, 0, 0, 0);
-      if (key0 + j < lmax) {
-        kq = *reinterpret_cast<const uint4*>(Kg + (size_t)(key0 + j) * DH + cc * 8);
-        vq = *reinterpret_cast<const uint4*>(Vg + (size_t)(key0 + j) * DH + cc * 8);
-      }
-      *reinterpret_cast<uint4*>(Ks + j * KSTRIDE + cc * 8) = kq;
-      *reinterpret_cast<uint4*>(Vs + j * KSTRIDE + cc * 8) = vq;
-    }
-    __syncthreads();
-    // scores: lane owns keys lane and lane + 32
-    float sc[kAttnRowsPerWarp][2];
-#pragma unroll
-    for (int i = 0; i < kAttnRowsPerWarp; ++i) { sc[i][0] = 0.f; sc[i][1] = 0.f; }
-#pragma unroll 2
-    for (int c = 0; c < CPR; ++c) {
-      const uint4 k0 = *reinterpret_cast<const uint4*>(Ks + lane * KSTRIDE + c * 8);
-      const uint4 k1 = *reinterpret_cast<const uint4*>(Ks + (lane + 32) * KSTRIDE + c * 8);
-      float kf0[8], kf1[8];
-      const __nv_bfloat162* p0 = reinterpret_cast<const __nv_bfloat162*>(&k0);
-      const __nv_bfloat162* p1 = reinterpret_cast<const __nv_bfloat162*>(&k1);
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const float2 f0 = __bfloat1622float2(p0[e]), f1 = __bfloat1622float2(p1[e]);
-        kf0[2 * e] = f0.x; kf0[2 * e + 1] = f0.y; kf1[2 * e] = f1.x; kf1[2 * e + 1] = f1.y;
-      }
-#pragma unroll
-      for (int i = 0; i < kAttnRowsPerWarp; ++i) {
-        const float* q = Qs + (warp + 8 * i) * DH + c * 8;
-        const float4 qa = *reinterpret_cast<const float4*>(q), qb = *reinterpret_cast<const float4*>(q + 4);
-        const float qv[8] = {qa.x, qa.y, qa.z, qa.w, qb.x, qb.y, qb.z, qb.w};
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          sc[i][0] = fmaf(qv[e], kf0[e], sc[i][0]);
-          sc[i][1] = fmaf(qv[e], kf1[e], sc[i][1]);
-        }
-      }
-    }
-    // running softmax per row
-    float corr[kAttnRowsPerWarp];
-#pragma unroll
-    for (int i = 0; i < kAttnRowsPerWarp; ++i) {
-      const int lim = s_lim[warp + 8 * i];
-      float s0 = (key0 + lane < lim) ? sc[i][0] * scale : -INFINITY;
-      float s1 = (key0 + lane + 32 < lim) ? sc[i][1] * scale : -INFINITY;
-      float mx = fmaxf(s0, s1);
-#pragma unroll
-      for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
-      const float mn = fmaxf(m[i], mx);
-      const float p0 = (s0 == -INFINITY) ? 0.f : expf(s0 - mn);
-      const float p1 = (s1 == -INFINITY) ? 0.f : expf(s1 - mn);
-      float ps = p0 + p1;
-#pragma unroll
-      for (int off = 16; off > 0; off >>= 1) ps += __shfl_xor_sync(0xffffffffu, ps, off);
-      corr[i] = (m[i] == -INFINITY) ? 0.f : expf(m[i] - mn);
-      l[i] = l[i] * corr[i] + ps;
-      m[i] = mn;
-      Ps[(warp * kAttnRowsPerWarp + i) * kAttnKeys + lane] = p0;
-      Ps[(warp * kAttnRowsPerWarp + i) * kAttnKeys + lane + 32] = p1;
-    }
-    __syncwarp();
-#pragma unroll
-    for (int i = 0; i < kAttnRowsPerWarp; ++i)
-#pragma unroll
-      for (int dd = 0; dd < DPL; ++dd) o[i][dd] *= corr[i];
-    // o += P V : lane owns DPL consecutive output dims
-    for (int j = 0; j < kAttnKeys; ++j) {
-      float vf[DPL];
-#pragma unroll
-      for (int dd = 0; dd < DPL; ++dd) vf[dd] = __bfloat162float(Vs[j * KSTRIDE + lane * DPL + dd]);
-#pragma unroll
-      for (int i = 0; i < kAttnRowsPerWarp; ++i) {
-        const float p = Ps[(warp * kAttnRowsPerWarp + i) * kAttnKeys + j];
-#pragma unroll
-        for (int dd = 0; dd < DPL; ++dd) o[i][dd] = fmaf(p, vf[dd], o[i][dd]);
-      }
-    }
-    __syncwarp();
-  }
-  // unnormalised partial result of this key slice
-#pragma unroll
-  for (int i = 0; i < kAttnRowsPerWarp; ++i) {
-    const int qi = warp + 8 * i;
-    if (qi < nrows) {
-      const size_t base = ((size_t)split * rows + s_grow[qi]) * H + s_head[qi];
-#pragma unroll
-      for (int dd = 0; dd < DPL; ++dd) out_o[base * DH + lane * DPL + dd] = o[i][dd];
-      if (lane == 0) { out_ml[base * 2] = m[i]; out_ml[base * 2 + 1] = l[i]; }
-    }
-  }
-}
-
 // Combine the key slices: o = sum_s o_s e^(m_s - M) / sum_s l_s e^(m_s - M).
 __global__ void k_attn_merge(const float* __restrict__ in_o, const float* __restrict__ in_ml, int nsplit,
                              int rows, int H, int Dh, __nv_bfloat16* __restrict__ attn_out) {
@@ -509,24 +344,6 @@ __global__ void k_loop_commit(int* hist, int* hist_len, int B, int stride, int* 
   }
 }
 
-template <int DH>
-void launch_attn(cs_ctx* ctx, const void* kv_cache, int layer, int B, int R, cudaStream_t st) {
-  const cs_model_config& c = ctx->cfg;
-  const int G = c.n_heads / c.n_kv_heads;
-  const int rt = cs_ceil_div(G * R, kAttnRows);
-  const size_t smem = (size_t)2 * kAttnKeys * (DH + 8) * 2 + (size_t)kAttnRows * DH * 4 +
-                      (size_t)8 * kAttnRowsPerWarp * kAttnKeys * 4;
-  static bool set = false;
-  if (!set) {
-    cudaFuncSetAttribute(k_attn_partial<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    set = true;
-  }
-  k_attn_partial<DH><<<dim3(B * c.n_kv_heads, ctx->attn_splits, rt), kAttnThreads, smem, st>>>(
-      ctx->qbuf, static_cast<const __nv_bfloat16*>(kv_cache), ctx->row_lim, layer, R, c.n_heads,
-      c.n_kv_heads, c.max_batch, c.max_seq, ctx->attn_splits, 1.0f / sqrtf((float)DH), ctx->attn_o,
-      ctx->attn_ml, B * R);
-}
-
 }  // namespace
 
 void cs_launch_block_setup(cs_ctx* ctx, const int32_t* last_tok, const int32_t* draft,
@@ -563,15 +380,10 @@ void cs_launch_qkv_post(cs_ctx* ctx, int splits, void* kv_cache, int layer, int 
       ctx->row_write, R, ctx->qbuf, static_cast<__nv_bfloat16*>(kv_cache), layer, c.max_batch, c.max_seq);
 }
 
-void cs_launch_attention(cs_ctx* ctx, const void* kv_cache, int layer, int B, int R, cudaStream_t st) {
+void cs_launch_attn_merge(cs_ctx* ctx, int nsplit, int rows, cudaStream_t st) {
   const cs_model_config& c = ctx->cfg;
-  switch (c.head_dim) {
-    case 32: launch_attn<32>(ctx, kv_cache, layer, B, R, st); break;
-    case 64: launch_attn<64>(ctx, kv_cache, layer, B, R, st); break;
-    default: launch_attn<128>(ctx, kv_cache, layer, B, R, st); break;
-  }
-  k_attn_merge<<<dim3(B * R, c.n_heads), c.head_dim, 0, st>>>(ctx->attn_o, ctx->attn_ml, ctx->attn_splits,
-                                                              B * R, c.n_heads, c.head_dim, ctx->attn_out);
+  k_attn_merge<<<dim3(rows, c.n_heads), c.head_dim, 0, st>>>(ctx->attn_o, ctx->attn_ml, nsplit, rows, c.n_heads,
+                                                             c.head_dim, ctx->attn_out);
 }
 
 void cs_launch_swiglu(cs_ctx* ctx, int splits, int rows, cudaStream_t st) {

@@ -31,3 +31,15 @@ def argmax_consistent(oracle_logits, gpu_ids, tol=LOGIT_TOL):
         if gid != oid and not (row[oid] - row[gid] < tol):
             bad.append((r, gid, oid, float(row[oid] - row[gid])))
     return bad
+
+
+def greedy_margins(model, cfg, prompt, generated):
+    """Teacher-forced check of a greedy continuation: for every generated token, how far its
+    oracle logit lies below the oracle's best logit at that position (0 = the oracle's own
+    choice).  A correct greedy decoder may only deviate where this margin is below the
+    logit tolerance."""
+    seq = [int(t) for t in prompt] + [int(t) for t in generated]
+    cache = O.KVCache(cfg, 1, len(seq) + 1)
+    logits = model.forward_block(seq[:-1], 0, cache, 0)
+    n0 = len(prompt)
+    return [float(logits[n0 - 1 + j].max() - logits[n0 - 1 + j][tok]) for j, tok in enumerate(generated)]
