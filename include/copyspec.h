@@ -33,9 +33,11 @@
  *              [0, kv_len[b]) of sequence b are meaningful (App. B.2).
  *   weights    bf16 row-major [out][in]:  embed [V][d], lm_head [V][d], final_norm [d];
  *              per layer attn_norm [d], wqkv [(H + 2 Hkv) Dh][d] (q rows, k rows, v
- *              rows), wo [d][H Dh], ffn_norm [d], w_gate_up [2 F][d] (gate rows then up
- *              rows), w_down [d][F].  All base pointers 16-byte aligned; d, H*Dh and F
- *              multiples of 8.
+ *              rows), wo [d][H Dh], ffn_norm [d], w_down [d][F], and w_gate_up
+ *              [ceil(F/64) * 128][d]: blocks of 128 rows, block t holding gate rows
+ *              64t..64t+63 followed by up rows 64t..64t+63 (rows past F are zero), so that
+ *              one GEMM tile sees both halves of SwiGLU.  All base pointers 16-byte
+ *              aligned; d, H*Dh and F multiples of 8.
  *   blocks     a verification block of sequence b has rows r = 0..draft_len[b]:
  *              row 0 is the last accepted token (whose K/V are not cached yet), row r>0
  *              is draft token r-1; row r sits at absolute position kv_len[b] + r.
@@ -229,8 +231,7 @@ cs_status cs_prefill(cs_ctx* ctx, const int32_t* hist, const int32_t* hist_len, 
 /* Building block of the forward of Sec. 3.2, exposed for testing the tensor-core path in
  * isolation: Y[rows][N] (fp32) = X[rows][K] (bf16) times W[N][K]^T (bf16), fp32
  * accumulation.  rows <= 256; K a multiple of 8; X must be readable for
- * ceil(rows/16)*16 rows.  Uses the context's workspace (so it must not overlap other
- * work of the context).  Async. */
+ * ceil(rows/16)*16 rows.  Async. */
 cs_status cs_linear(cs_ctx* ctx, const void* X, const void* W, int rows, int N, int K,
                     float* Y, void* stream);
 

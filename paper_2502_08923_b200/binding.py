@@ -144,8 +144,25 @@ def cs_find_match(hist, hist_len, gamma, k, policy=LATEST, out=None):
     return mp, dr, dl
 
 
+def pack_gate_up(w_gate_up, d_ffn):
+    """Re-lay the [2F][d] (gate rows, then up rows) matrix into the layout the library reads:
+    blocks of 128 rows, each holding 64 gate rows followed by the 64 matching up rows (rows
+    past F are zero), so that one GEMM tile sees both halves of SwiGLU."""
+    d = w_gate_up.shape[1]
+    nb = -(-d_ffn // 64)
+    out = torch.zeros(nb, 2, 64, d, dtype=w_gate_up.dtype, device=w_gate_up.device)
+    pad = torch.zeros(nb * 64, d, dtype=w_gate_up.dtype, device=w_gate_up.device)
+    pad[:d_ffn] = w_gate_up[:d_ffn]
+    out[:, 0] = pad.view(nb, 64, d)
+    pad.zero_()
+    pad[:d_ffn] = w_gate_up[d_ffn:]
+    out[:, 1] = pad.view(nb, 64, d)
+    return out.view(nb * 128, d).contiguous()
+
+
 class Context:
-    """Owns the device workspace and the cs_ctx handle for one model."""
+    """Owns the device workspace and the cs_ctx handle for one model.  `weights` uses the
+    plain layouts of `inputs.make_weights`; the gate/up matrix is re-laid here once."""
 
     def __init__(self, cfg, weights, max_seq, max_batch, k_max):
         lib = load()
@@ -164,6 +181,7 @@ class Context:
         self.weights = weights          # keeps the tensors alive
         L = cfg.n_layers
         self._arrs = {}
+        self._packed = []
         cw = CsWeights()
         for name in ("embed", "lm_head", "final_norm"):
             t = weights[name]
@@ -173,6 +191,9 @@ class Context:
             arr = (C.c_void_p * L)()
             for l in range(L):
                 t = weights["layers"][l][name]
+                if name == "w_gate_up":
+                    t = pack_gate_up(t, cfg.d_ffn)
+                    self._packed.append(t)
                 assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()
                 arr[l] = t.data_ptr()
             self._arrs[name] = arr

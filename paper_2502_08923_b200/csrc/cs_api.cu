@@ -13,7 +13,7 @@ struct WsLayout {
   size_t x, xn, attn_out, act, qbuf, partial, attn_o, attn_ml, rope_cs, inv_freq, tile_max, tile_idx,
       row_tok, row_pos, row_lim, row_write, seq_ok, status, loop_last, loop_draft, loop_dlen, loop_mpos,
       loop_emitted, loop_done, loop_accept, loop_out, loop_argmax, loop_stats, total;
-  size_t partial_elems;
+  size_t qkv_elems;
   int attn_splits;
 };
 
@@ -40,17 +40,9 @@ WsLayout ws_layout(const cs_model_config* c) {
   const size_t rows = CS_MAX_ROWS;
   const size_t d = c->d_model, qd = (size_t)c->n_heads * c->head_dim, F = c->d_ffn;
   const size_t qkv = qd + 2 * (size_t)c->n_kv_heads * c->head_dim;
-  // largest splits * N over the four projections of a layer
-  size_t pe = 0;
-  const size_t shapes[4][2] = {{qkv, d}, {d, qd}, {2 * F, d}, {d, F}};
-  for (int i = 0; i < 4; ++i) {
-    const int tiles = cs_ceil_div((int)shapes[i][0], CS_GEMM_BM), kb = cs_ceil_div((int)shapes[i][1], CS_GEMM_BK);
-    const size_t e = (size_t)cs_max_splits(tiles, kb) * shapes[i][0];
-    if (e > pe) pe = e;
-  }
-  L.partial_elems = pe * rows;
-  int as = cs_ceil_div(c->max_seq, 256);
-  L.attn_splits = as < 1 ? 1 : (as > 32 ? 32 : as);
+  L.qkv_elems = rows * (qkv > 4096 ? qkv : 4096);
+  int as = cs_ceil_div(c->max_seq, 128);
+  L.attn_splits = as < 1 ? 1 : (as > 64 ? 64 : as);
   const size_t lm_tiles = cs_ceil_div(c->vocab, CS_GEMM_BM);
   size_t off = 0;
   L.x = take(&off, rows * d * 4);
@@ -58,7 +50,7 @@ WsLayout ws_layout(const cs_model_config* c) {
   L.attn_out = take(&off, rows * qd * 2);
   L.act = take(&off, rows * F * 2);
   L.qbuf = take(&off, rows * qd * 2);
-  L.partial = take(&off, L.partial_elems * 4);
+  L.partial = take(&off, L.qkv_elems * 4);
   L.attn_o = take(&off, (size_t)L.attn_splits * rows * qd * 4);
   L.attn_ml = take(&off, (size_t)L.attn_splits * rows * c->n_heads * 2 * 4);
   L.rope_cs = take(&off, rows * c->head_dim * 4);
@@ -128,57 +120,48 @@ cs_status enqueue_forward(cs_ctx* ctx, int B, int R, void* kv_cache, bool with_l
   prof_begin(ctx, CS_FAM_ELEMENTWISE, st);
   cs_launch_embed(ctx, rows, st);
   prof_end(ctx, st);
-  int prev_splits = 0;
   for (int l = 0; l < c.n_layers; ++l) {
     const LayerPlan& L = ctx->layers[l];
     prof_begin(ctx, CS_FAM_ELEMENTWISE, st);
-    cs_launch_rmsnorm(ctx, l == 0 ? nullptr : ctx->partial, prev_splits, L.attn_norm, rows, st);
+    cs_launch_rmsnorm(ctx, L.attn_norm, rows, st);
     prof_end(ctx, st);
     prof_begin(ctx, CS_FAM_GEMM, st);
-    if ((s = cs_launch_gemm(ctx, &L.qkv, &ctx->tmXn, ctx->xn, rows, 0, ctx->partial, nullptr, st)) != CS_OK) { prof_end(ctx, st); return s; }
+    s = cs_launch_gemm(ctx, &L.qkv, &ctx->tmXn, rows, CS_EPI_STORE, ctx->qkv, nullptr, 0, st);
     prof_end(ctx, st);
+    if (s != CS_OK) return s;
     prof_begin(ctx, CS_FAM_ELEMENTWISE, st);
-    cs_launch_qkv_post(ctx, L.qkv.splits, kv_cache, l, B, R, st);
+    cs_launch_qkv_post(ctx, kv_cache, l, B, R, st);
     prof_end(ctx, st);
     prof_begin(ctx, CS_FAM_ATTENTION, st);
     cs_launch_attention(ctx, kv_cache, l, B, R, st);
     prof_end(ctx, st);
     prof_begin(ctx, CS_FAM_GEMM, st);
-    if ((s = cs_launch_gemm(ctx, &L.o, &ctx->tmAttn, ctx->attn_out, rows, 0, ctx->partial, nullptr, st)) != CS_OK) { prof_end(ctx, st); return s; }
+    s = cs_launch_gemm(ctx, &L.o, &ctx->tmAttn, rows, CS_EPI_RESIDUAL, ctx->x, nullptr, 0, st);
     prof_end(ctx, st);
+    if (s != CS_OK) return s;
     prof_begin(ctx, CS_FAM_ELEMENTWISE, st);
-    cs_launch_rmsnorm(ctx, ctx->partial, L.o.splits, L.ffn_norm, rows, st);
+    cs_launch_rmsnorm(ctx, L.ffn_norm, rows, st);
     prof_end(ctx, st);
     prof_begin(ctx, CS_FAM_GEMM, st);
-    if ((s = cs_launch_gemm(ctx, &L.gate_up, &ctx->tmXn, ctx->xn, rows, 0, ctx->partial, nullptr, st)) != CS_OK) { prof_end(ctx, st); return s; }
+    s = cs_launch_gemm(ctx, &L.gate_up, &ctx->tmXn, rows, CS_EPI_SWIGLU, nullptr, ctx->act, c.d_ffn, st);
     prof_end(ctx, st);
-    prof_begin(ctx, CS_FAM_ELEMENTWISE, st);
-    cs_launch_swiglu(ctx, L.gate_up.splits, rows, st);
-    prof_end(ctx, st);
+    if (s != CS_OK) return s;
     prof_begin(ctx, CS_FAM_GEMM, st);
-    if ((s = cs_launch_gemm(ctx, &L.down, &ctx->tmAct, ctx->act, rows, 0, ctx->partial, nullptr, st)) != CS_OK) { prof_end(ctx, st); return s; }
+    s = cs_launch_gemm(ctx, &L.down, &ctx->tmAct, rows, CS_EPI_RESIDUAL, ctx->x, nullptr, 0, st);
     prof_end(ctx, st);
-    prev_splits = L.down.splits;
+    if (s != CS_OK) return s;
   }
   if (with_lm) {
     prof_begin(ctx, CS_FAM_ELEMENTWISE, st);
-    cs_launch_rmsnorm(ctx, ctx->partial, prev_splits, ctx->final_norm, rows, st);
+    cs_launch_rmsnorm(ctx, ctx->final_norm, rows, st);
     prof_end(ctx, st);
     prof_begin(ctx, CS_FAM_LMHEAD, st);
-    if ((s = cs_launch_gemm(ctx, &ctx->lm, &ctx->tmXn, ctx->xn, rows, 1, nullptr, logits, st)) != CS_OK) { prof_end(ctx, st); return s; }
+    s = cs_launch_gemm(ctx, &ctx->lm, &ctx->tmXn, rows, CS_EPI_ARGMAX, logits, nullptr, 0, st);
     prof_end(ctx, st);
+    if (s != CS_OK) return s;
   }
   CS_CUDA_OK(ctx, cudaGetLastError());
   return CS_OK;
-}
-
-__global__ void k_reduce_partial(const float* __restrict__ partial, int splits, int rows, int N,
-                                 float* __restrict__ y) {
-  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= (size_t)rows * N) return;
-  float v = 0.f;
-  for (int s = 0; s < splits; ++s) v += partial[(size_t)s * rows * N + i];
-  y[i] = v;
 }
 
 // One iteration of the generation loop (App. B.3 steps 1, 2, 4) on device-resident state.
@@ -237,9 +220,7 @@ cs_status cs_create(cs_ctx** out, const cs_model_config* cfg, const cs_weights* 
   ctx->max_rows = cfg->max_batch * (cfg->k_max + 1);
   ctx->rows_pad = CS_MAX_ROWS;
   ctx->attn_splits = L.attn_splits;
-  ctx->partial_elems = L.partial_elems;
-  const char* env = getenv("CS_GEMM_SIMT");
-  ctx->gemm_simt = (env != nullptr && env[0] == '1');
+  ctx->qkv_elems = L.qkv_elems;
   ctx->layers = new (std::nothrow) LayerPlan[cfg->n_layers];
   cs_status s = CS_OK;
   int dev = 0;
@@ -272,7 +253,7 @@ cs_status cs_create(cs_ctx** out, const cs_model_config* cfg, const cs_weights* 
   ctx->attn_out = reinterpret_cast<__nv_bfloat16*>(base + L.attn_out);
   ctx->act = reinterpret_cast<__nv_bfloat16*>(base + L.act);
   ctx->qbuf = reinterpret_cast<__nv_bfloat16*>(base + L.qbuf);
-  ctx->partial = reinterpret_cast<float*>(base + L.partial);
+  ctx->qkv = reinterpret_cast<float*>(base + L.partial);
   ctx->attn_o = reinterpret_cast<float*>(base + L.attn_o);
   ctx->attn_ml = reinterpret_cast<float*>(base + L.attn_ml);
   ctx->rope_cs = reinterpret_cast<float*>(base + L.rope_cs);
@@ -317,7 +298,7 @@ cs_status cs_create(cs_ctx** out, const cs_model_config* cfg, const cs_weights* 
     P.ffn_norm = static_cast<const __nv_bfloat16*>(w->ffn_norm[l]);
     if ((s = cs_gemm_plan(ctx, &P.qkv, w->wqkv[l], qkv, d, true)) != CS_OK) break;
     if ((s = cs_gemm_plan(ctx, &P.o, w->wo[l], d, qd, true)) != CS_OK) break;
-    if ((s = cs_gemm_plan(ctx, &P.gate_up, w->w_gate_up[l], 2 * F, d, true)) != CS_OK) break;
+    if ((s = cs_gemm_plan(ctx, &P.gate_up, w->w_gate_up[l], cs_ceil_div(F, 64) * 128, d, true)) != CS_OK) break;
     if ((s = cs_gemm_plan(ctx, &P.down, w->w_down[l], d, F, true)) != CS_OK) break;
   }
   if (s == CS_OK) s = cs_gemm_plan(ctx, &ctx->lm, w->lm_head, cfg->vocab, d, false);
@@ -552,20 +533,10 @@ cs_status cs_linear(cs_ctx* ctx, const void* X, const void* W, int rows, int N, 
   GemmPlan g;
   cs_status s = cs_gemm_plan(ctx, &g, W, N, K, true);
   if (s != CS_OK) return s;
-  while (g.splits > 1 && (size_t)g.splits * rows * N > ctx->partial_elems) {   // fit the workspace
-    g.kb_per_split *= 2;
-    g.splits = cs_ceil_div(cs_ceil_div(K, CS_GEMM_BK), g.kb_per_split);
-  }
-  if ((size_t)g.splits * rows * N > ctx->partial_elems) return fail(ctx, CS_ERR_CAPACITY, "workspace too small for this GEMM");
   const int n_tok = cs_ceil_div(rows, 16) * 16;
   CUtensorMap tmX;
   if ((s = cs_make_act_map(ctx, &tmX, X, n_tok, K, n_tok)) != CS_OK) return s;
-  if ((s = cs_launch_gemm(ctx, &g, &tmX, static_cast<const __nv_bfloat16*>(X), rows, 0, ctx->partial, nullptr, st)) != CS_OK)
-    return s;
-  const size_t total = (size_t)rows * N;
-  k_reduce_partial<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(ctx->partial, g.splits, rows, N, Y);
-  CS_CUDA_OK(ctx, cudaGetLastError());
-  return CS_OK;
+  return cs_launch_gemm(ctx, &g, &tmX, rows, CS_EPI_STORE, Y, nullptr, 0, st);
 }
 
 }  // extern "C"

@@ -51,6 +51,7 @@ __global__ void __launch_bounds__(kThreads)
 k_attn_mma(const __nv_bfloat16* __restrict__ qbuf, const __nv_bfloat16* __restrict__ kv,
            const int* __restrict__ row_lim, int layer, int R, int H, int Hkv, int max_batch, int max_seq,
            int nsplit, float scale_log2e, float* __restrict__ out_o, float* __restrict__ out_ml, int rows) {
+  CS_PDL_PROLOGUE();
   constexpr int STRIDE = DH + 8;          // bf16 elements per shared-memory row
   constexpr int KSTEPS = DH / 16;         // MMA k-steps of the QK^T product
   constexpr int NB_S = kKeys / 8;         // 8-key column blocks of S
@@ -243,9 +244,9 @@ int launch(cs_ctx* ctx, const void* kv_cache, int layer, int B, int R, cudaStrea
     set = true;
   }
   const float scale_log2e = 1.4426950408889634f / sqrtf((float)DH);
-  k_attn_mma<DH><<<dim3(B * c.n_kv_heads, nsplit, rgs), kThreads, smem, st>>>(
-      ctx->qbuf, static_cast<const __nv_bfloat16*>(kv_cache), ctx->row_lim, layer, R, c.n_heads, c.n_kv_heads,
-      c.max_batch, c.max_seq, nsplit, scale_log2e, ctx->attn_o, ctx->attn_ml, B * R);
+  cs_launch_pdl(k_attn_mma<DH>, dim3(B * c.n_kv_heads, nsplit, rgs), dim3(kThreads), smem, st, ctx->qbuf,
+                static_cast<const __nv_bfloat16*>(kv_cache), ctx->row_lim, layer, R, c.n_heads, c.n_kv_heads,
+                c.max_batch, c.max_seq, nsplit, scale_log2e, ctx->attn_o, ctx->attn_ml, B * R);
   return nsplit;
 }
 

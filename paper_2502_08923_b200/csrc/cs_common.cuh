@@ -23,7 +23,7 @@ static constexpr int CS_MAX_ROWS = 256;   // rows of one verification block (UMM
 static constexpr int CS_GEMM_BM = 128;    // out-features per CTA tile (UMMA M)
 static constexpr int CS_GEMM_BK = 64;     // K elements per stage (one 128-byte swizzle row)
 static constexpr int CS_MAX_GAMMA = 8;
-static constexpr int CS_MAX_SPLITS = 16;  // split-K factor limit
+static constexpr int CS_MAX_SPLITS = 8;   // split-K factor limit (portable cluster size)
 static constexpr int CS_SPLIT_TILE_CAP = 640;  // tiles * splits never exceeds this (unless splits == 1)
 
 struct GemmPlan {
@@ -66,7 +66,6 @@ struct cs_ctx {
   int max_rows;      // max_batch * (k_max + 1)
   int rows_pad;      // rounded up to 16
   int attn_splits;   // split-KV factor
-  bool gemm_simt;    // bring-up path: plain CUDA-core GEMM instead of tcgen05
   int num_sms;
   cudaStream_t cap_stream;   // used only to capture the loop's step graph
 
@@ -82,8 +81,8 @@ struct cs_ctx {
   __nv_bfloat16* attn_out;   // attention output bf16 [rows_pad][H*Dh]
   __nv_bfloat16* act;        // SwiGLU output bf16 [rows_pad][F]
   __nv_bfloat16* qbuf;       // rotated queries bf16 [rows_pad][H*Dh]
-  float* partial;            // split-K partial sums fp32 [splits][rows][N]
-  size_t partial_elems;
+  float* qkv;                // QKV projection output fp32 [rows][(H+2Hkv)*Dh]; scratch of cs_linear
+  size_t qkv_elems;
   float* attn_o;             // split-KV partial outputs [splits][rows][H][Dh]
   float* attn_ml;            // split-KV (max, sum) [splits][rows][H][2]
   float* rope_cs;            // cos/sin of this block [rows][Dh/2][2]
@@ -130,6 +129,32 @@ struct cs_ctx {
 
 static inline int cs_ceil_div(int a, int b) { return (a + b - 1) / b; }
 
+// GEMM epilogues
+enum : int { CS_EPI_STORE = 0, CS_EPI_ARGMAX = 1, CS_EPI_RESIDUAL = 2, CS_EPI_SWIGLU = 3 };
+
+// Programmatic dependent launch: every kernel of the library lets its successor start
+// early and waits for its predecessor before it touches global memory the predecessor
+// (or, transitively, anything earlier in the stream) may still be using.
+#define CS_PDL_PROLOGUE()                                              \
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");     \
+  asm volatile("griddepcontrol.wait;" ::: "memory")
+
+template <typename... KArgs, typename... Args>
+static inline cudaError_t cs_launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                        cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = grid;
+  lc.blockDim = block;
+  lc.dynamicSmemBytes = smem;
+  lc.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = at;
+  lc.numAttrs = 1;
+  return cudaLaunchKernelEx(&lc, kernel, static_cast<KArgs>(args)...);
+}
+
 // split-K factor limit for a GEMM of `tiles` 128-row tiles and `kb` 64-wide K blocks
 static inline int cs_max_splits(int tiles, int kb) {
   int s = CS_SPLIT_TILE_CAP / tiles;
@@ -148,10 +173,10 @@ cs_status cs_launch_find_match(const int32_t* hist, const int32_t* hist_len, int
 cs_status cs_gemm_plan(cs_ctx* ctx, GemmPlan* g, const void* w, int N, int K, bool allow_split);
 cs_status cs_make_act_map(cs_ctx* ctx, CUtensorMap* tm, const void* base, int rows_total, int K,
                           int box_rows);
-// mode 0: partial[s][row][n] fp32; mode 1: per-tile argmax (tile_max/tile_idx) + optional logits
-cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX,
-                         const __nv_bfloat16* X, int rows, int mode, float* out, float* logits,
-                         cudaStream_t st);
+// mode = CS_EPI_*: `out` is the fp32 destination (STORE, RESIDUAL) or the optional logits dump
+// (ARGMAX); `act`/F the bf16 destination of SWIGLU
+cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX, int rows, int mode,
+                         float* out, __nv_bfloat16* act, int F, cudaStream_t st);
 // cs_layers.cu
 void cs_launch_block_setup(cs_ctx* ctx, const int32_t* last_tok, const int32_t* draft,
                            const int32_t* draft_len, const int32_t* kv_len, const int32_t* skip,
@@ -159,14 +184,11 @@ void cs_launch_block_setup(cs_ctx* ctx, const int32_t* last_tok, const int32_t* 
 void cs_launch_prefill_setup(cs_ctx* ctx, const int32_t* hist, const int32_t* hist_len, int B,
                              int stride, int start, int R, cudaStream_t st);
 void cs_launch_embed(cs_ctx* ctx, int rows, cudaStream_t st);
-void cs_launch_rmsnorm(cs_ctx* ctx, const float* partial, int splits, const __nv_bfloat16* gain,
-                       int rows, cudaStream_t st);
-void cs_launch_qkv_post(cs_ctx* ctx, int splits, void* kv_cache, int layer, int B, int R,
-                        cudaStream_t st);
+void cs_launch_rmsnorm(cs_ctx* ctx, const __nv_bfloat16* gain, int rows, cudaStream_t st);
+void cs_launch_qkv_post(cs_ctx* ctx, void* kv_cache, int layer, int B, int R, cudaStream_t st);
 void cs_launch_attention(cs_ctx* ctx, const void* kv_cache, int layer, int B, int R,
                          cudaStream_t st);
 void cs_launch_attn_merge(cs_ctx* ctx, int nsplit, int rows, cudaStream_t st);
-void cs_launch_swiglu(cs_ctx* ctx, int splits, int rows, cudaStream_t st);
 void cs_launch_accept(cs_ctx* ctx, int B, int k, const int32_t* draft, const int32_t* draft_len,
                       const int32_t* script, int script_stride, const int32_t* script_off,
                       int script_limit, int32_t* accept_len, int32_t* out_tokens,

@@ -6,14 +6,34 @@
 // 16), so even an 11-row block fills the 128 TMEM lanes.  Weights and activations arrive
 // as TMA tiles of 64 K-elements (one 128-byte swizzled row per feature / token) through an
 // mbarrier ring; one thread issues tcgen05.mma into a TMEM accumulator; four warps read
-// it back with tcgen05.ld.  K is split across CTAs (grid.y) so that every GEMM puts about
-// two CTAs on each SM; each split writes its fp32 partial sums, which the consumer kernel
-// adds in a fixed order (deterministic, no atomics).  In LM-head mode the epilogue reduces
-// each tile to (max logit, token id) per row instead of writing logits.
+// it back with tcgen05.ld.
+//
+// K is split across the CTAs of a thread-block cluster (cluster dims (1, S, 1), S <= 8) so
+// that every GEMM puts about two CTAs on each SM.  Each CTA leaves its partial tile in its
+// own shared memory; after a cluster barrier every CTA sums one slice of the features over
+// all ranks through distributed shared memory, in rank order (deterministic, no atomics,
+// no partial sums in HBM), and applies the epilogue:
+//   STORE     out[row][n]  = y                      (QKV projection, cs_linear)
+//   RESIDUAL  x[row][n]   += y                      (attention output and FFN down projections)
+//   SWIGLU    act[row][j]  = bf16(silu(gate_j) * up_j), the tile holding 64 gate rows and the
+//             64 matching up rows                   (FFN gate/up projection)
+//   ARGMAX    per 128-feature tile (max logit, lowest token id) per row; logits are only
+//             written when a debug buffer is given   (LM head)
+//
+// The kernel is launched with programmatic dependent launch: it starts while its
+// predecessor drains, fills its pipeline with weight tiles (which depend on nothing) and
+// only then waits for the predecessor before touching activations.
 //
 // Every wait is bounded: when it runs out the CTA records CS_DEV_TIMEOUT, drains its
-// copies, frees its TMEM and returns.
+// copies, still takes part in the cluster barriers, frees its TMEM and returns.
+#include <stdlib.h>
+
+#include <algorithm>
+
 #include "cs_common.cuh"
+
+using std::max;
+using std::min;
 
 namespace {
 
@@ -23,12 +43,13 @@ constexpr unsigned long long kWaitLimitNs = 2000000000ull; // 2 s
 
 struct GemmArgs {
   int rows, n_tok, N, K;
-  int num_kb, kb_per_split, stages, mode;
-  float* out;        // mode 0: partial sums [splits][rows][N]
-  float* tile_max;   // mode 1: [tiles][tile_stride]
+  int num_kb, kb_per_split, splits, stages, mode;
+  float* out;            // STORE / RESIDUAL: [rows][N] fp32; ARGMAX: optional logits [rows][N]
+  __nv_bfloat16* act;    // SWIGLU: [rows][F] bf16
+  int F;
+  float* tile_max;       // ARGMAX: [tiles][tile_stride]
   int* tile_idx;
   int tile_stride;
-  float* logits;     // mode 1, optional: [rows][N]
   int* status;
 };
 
@@ -110,9 +131,39 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
       : "r"(taddr));
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// Four consecutive floats of every rank's parked tile, summed in rank order.  All loads are
+// issued before the first add so that their latencies overlap.
+__device__ __forceinline__ float4 sum_over_ranks(uint32_t local_addr, int splits) {
+  float4 v[CS_MAX_SPLITS];
+#pragma unroll
+  for (int q = 0; q < CS_MAX_SPLITS; ++q) {
+    v[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (q < splits) {
+      uint32_t remote;
+      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(q));
+      asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+                   : "=f"(v[q].x), "=f"(v[q].y), "=f"(v[q].z), "=f"(v[q].w)
+                   : "r"(remote));
+    }
+  }
+  float4 y = v[0];
+#pragma unroll
+  for (int q = 1; q < CS_MAX_SPLITS; ++q) { y.x += v[q].x; y.y += v[q].y; y.z += v[q].z; y.w += v[q].w; }
+  return y;
+}
 
 __global__ void __launch_bounds__(kThreads, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, GemmArgs a) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   uint8_t* smem = smem_raw + (((raw + 1023u) & ~1023u) - raw);   // operand tiles need 1024-byte alignment
@@ -122,11 +173,13 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * a.stages + 1);
   volatile int* s_abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
   volatile int* s_never = reinterpret_cast<volatile int*>(tmem_slot + 2);   // stays 0: drains wait on time only
-  float* red_val = reinterpret_cast<float*>(tmem_slot + 4);       // [4][n_tok] (mode 1)
+  float* red_val = reinterpret_cast<float*>(tmem_slot + 4);       // [4][n_tok] (ARGMAX)
   int* red_idx = reinterpret_cast<int*>(red_val + 4 * a.n_tok);
+  float* dump = reinterpret_cast<float*>(smem);                   // [n_tok][128] fp32, reuses the operand ring
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int tile = blockIdx.x, split = blockIdx.y;
+  const int tile = blockIdx.x;
+  const int split = (a.splits > 1) ? (int)cluster_rank() : 0;
   const int n0 = tile * CS_GEMM_BM;
   const int kb0 = split * a.kb_per_split;
   const int kb1 = min(a.num_kb, kb0 + a.kb_per_split);
@@ -163,7 +216,17 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
   if (warp == 4) {
     // ------------------------------------------------------------- TMA producer
     if (lane == 0) {
-      int i = 0;
+      // weights depend on nothing: fill the ring with them before waiting for the predecessor
+      const int npre = min(nkb, a.stages);
+      for (int i = 0; i < npre; ++i) {
+        mbar_expect_tx(bar_full + 8 * i, (uint32_t)stage_bytes);
+        tma_load_2d(smem_u32(smem + (size_t)i * stage_bytes), &tmW, bar_full + 8 * i, (kb0 + i) * CS_GEMM_BK, n0);
+      }
+      asm volatile("griddepcontrol.wait;" ::: "memory");
+      for (int i = 0; i < npre; ++i)
+        tma_load_2d(smem_u32(smem + (size_t)i * stage_bytes) + kTileABytes, &tmX, bar_full + 8 * i,
+                    (kb0 + i) * CS_GEMM_BK, 0);
+      int i = npre;
       for (; i < nkb; ++i) {
         const int s = i % a.stages;
         const uint32_t ph = (uint32_t)(i / a.stages) & 1u;
@@ -178,7 +241,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
         atomicOr(a.status, CS_DEV_TIMEOUT);
       }
       if (*s_abort) {
-        // copies still in flight must land before this CTA's shared memory is released
+        // copies still in flight must land before this CTA's shared memory is reused or released
         for (int j = max(0, i - a.stages); j < i; ++j)
           mbar_wait(bar_full + 8 * (j % a.stages), (uint32_t)(j / a.stages) & 1u, s_never);
       }
@@ -208,49 +271,43 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
       umma_commit(bar_acc);
     }
   } else {
-    // ------------------------------------------------------------- epilogue (warps 0-3)
+    // ------------------------------------------------------------- accumulator read-out (warps 0-3)
     const int feat = n0 + warp * 32 + lane;
     if (nkb > 0) ok = mbar_wait(bar_acc, 0, s_abort);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     ok = __all_sync(0xffffffffu, ok) && (*s_abort == 0);
-    if (!ok) {
-      if (lane == 0) atomicOr(a.status, CS_DEV_TIMEOUT);
-    } else {
-      for (int c0 = 0; c0 < a.n_tok && c0 < a.rows; c0 += 16) {
-        uint32_t v[16];
-        if (nkb > 0) {
-          tmem_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
-        } else {
+    if (!ok && lane == 0) atomicOr(a.status, CS_DEV_TIMEOUT);
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    for (int c0 = 0; c0 < a.n_tok && c0 < a.rows; c0 += 16) {
+      uint32_t v[16];
+      if (nkb > 0 && ok) {
+        tmem_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
+      } else {
 #pragma unroll
-          for (int j = 0; j < 16; ++j) v[j] = 0u;
-        }
-        if (a.mode == 0) {
+        for (int j = 0; j < 16; ++j) v[j] = 0u;
+      }
+      if (a.mode != CS_EPI_ARGMAX) {
+        // the MMAs have retired, so the operand ring is free: park the tile there
 #pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const int tok = c0 + j;
-            if (tok < a.rows && feat < a.N)
-              a.out[((size_t)split * a.rows + tok) * a.N + feat] = __uint_as_float(v[j]);
+        for (int j = 0; j < 16; ++j) dump[(c0 + j) * CS_GEMM_BM + warp * 32 + lane] = __uint_as_float(v[j]);
+      } else {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const int tok = c0 + j;
+          float val = (feat < a.N) ? __uint_as_float(v[j]) : -INFINITY;
+          int idx = feat;
+          if (a.out != nullptr && tok < a.rows && feat < a.N) a.out[(size_t)tok * a.N + feat] = val;
+#pragma unroll
+          for (int off = 16; off > 0; off >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, val, off);
+            const int oi = __shfl_xor_sync(0xffffffffu, idx, off);
+            if (ov > val || (ov == val && oi < idx)) { val = ov; idx = oi; }
           }
-        } else {
-#pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const int tok = c0 + j;
-            float val = (feat < a.N) ? __uint_as_float(v[j]) : -INFINITY;
-            int idx = feat;
-            if (a.logits != nullptr && tok < a.rows && feat < a.N)
-              a.logits[(size_t)tok * a.N + feat] = val;
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) {
-              const float ov = __shfl_xor_sync(0xffffffffu, val, off);
-              const int oi = __shfl_xor_sync(0xffffffffu, idx, off);
-              if (ov > val || (ov == val && oi < idx)) { val = ov; idx = oi; }
-            }
-            if (lane == 0) { red_val[warp * a.n_tok + tok] = val; red_idx[warp * a.n_tok + tok] = idx; }
-          }
+          if (lane == 0) { red_val[warp * a.n_tok + tok] = val; red_idx[warp * a.n_tok + tok] = idx; }
         }
       }
     }
-    if (a.mode == 1) {
+    if (a.mode == CS_EPI_ARGMAX) {
       asm volatile("bar.sync 1, 128;" ::: "memory");   // the four epilogue warps only
       if (ok) {
         for (int tok = threadIdx.x; tok < a.rows; tok += 128) {
@@ -268,6 +325,67 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
       }
     }
   }
+  if (warp >= 4) asm volatile("griddepcontrol.wait;" ::: "memory");
+
+  // ---------------------------------------------------------------- split-K reduction + epilogue
+  if (a.mode != CS_EPI_ARGMAX) {
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (a.splits > 1) cluster_sync_all();          // every rank's tile is parked
+    if (warp < 4) {
+      const uint32_t dump_addr = smem_u32(dump);
+      const int e = threadIdx.x;                   // 0..127
+      if (a.mode == CS_EPI_SWIGLU) {
+        // features 0..63 of the tile are gate rows, 64..127 the matching up rows; each rank
+        // finishes a slice of j (a multiple of 4 wide), four consecutive j per thread
+        const int js = ((64 + a.splits - 1) / a.splits + 3) & ~3;
+        const int j_lo = split * js, j_n = max(0, min(64, j_lo + js) - j_lo);
+        const int per_tok = j_n >> 2;
+        for (int idx = e; idx < per_tok * a.rows; idx += 128) {
+          const int j = j_lo + 4 * (idx % per_tok), tok = idx / per_tok;
+          float4 g, u;
+          if (a.splits > 1) {
+            g = sum_over_ranks(dump_addr + 4u * (uint32_t)(tok * CS_GEMM_BM + j), a.splits);
+            u = sum_over_ranks(dump_addr + 4u * (uint32_t)(tok * CS_GEMM_BM + 64 + j), a.splits);
+          } else {
+            g = *reinterpret_cast<const float4*>(dump + tok * CS_GEMM_BM + j);
+            u = *reinterpret_cast<const float4*>(dump + tok * CS_GEMM_BM + 64 + j);
+          }
+          const float gv[4] = {g.x, g.y, g.z, g.w}, uv[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int jj = tile * 64 + j + i;
+            if (jj < a.F) a.act[(size_t)tok * a.F + jj] = __float2bfloat16_rn(gv[i] / (1.f + expf(-gv[i])) * uv[i]);
+          }
+        }
+      } else {
+        const int fs = ((CS_GEMM_BM + a.splits - 1) / a.splits + 3) & ~3;
+        const int f_lo = split * fs, f_n = max(0, min(CS_GEMM_BM, f_lo + fs) - f_lo);
+        const int per_tok = f_n >> 2;
+        for (int idx = e; idx < per_tok * a.rows; idx += 128) {
+          const int f = f_lo + 4 * (idx % per_tok), tok = idx / per_tok;
+          float4 y;
+          if (a.splits > 1) y = sum_over_ranks(dump_addr + 4u * (uint32_t)(tok * CS_GEMM_BM + f), a.splits);
+          else y = *reinterpret_cast<const float4*>(dump + tok * CS_GEMM_BM + f);
+          const float yv[4] = {y.x, y.y, y.z, y.w};
+          float* dst = a.out + (size_t)tok * a.N + n0 + f;
+          if (n0 + f + 3 < a.N && (a.N & 3) == 0) {
+            float4 o = y;
+            if (a.mode == CS_EPI_RESIDUAL) {
+              const float4 x = *reinterpret_cast<const float4*>(dst);
+              o.x += x.x; o.y += x.y; o.z += x.z; o.w += x.w;
+            }
+            *reinterpret_cast<float4*>(dst) = o;
+          } else {
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+              if (n0 + f + i < a.N) dst[i] = (a.mode == CS_EPI_RESIDUAL) ? dst[i] + yv[i] : yv[i];
+          }
+        }
+      }
+    }
+    if (a.splits > 1) cluster_sync_all();          // nobody leaves while a peer still reads its tile
+  }
   // ---------------------------------------------------------------- teardown
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
@@ -277,68 +395,6 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols)
                  : "memory");
-  }
-}
-
-// ------------------------------------------------------------------ bring-up path
-// Plain CUDA-core GEMM with the same contract (one warp per output feature).  Selected
-// with CS_GEMM_SIMT=1; it exists to check the tensor-core kernel on the device.
-__global__ void __launch_bounds__(256)
-k_gemm_simt(const __nv_bfloat16* __restrict__ X, const __nv_bfloat16* __restrict__ W, int rows, int N,
-            int K, float* __restrict__ out) {
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int feat = blockIdx.x * 8 + warp;
-  if (feat >= N) return;
-  for (int r0 = 0; r0 < rows; r0 += 16) {
-    float acc[16];
-#pragma unroll
-    for (int r = 0; r < 16; ++r) acc[r] = 0.f;
-    for (int k = lane * 8; k < K; k += 256) {
-      const uint4 wv = *reinterpret_cast<const uint4*>(W + (size_t)feat * K + k);
-      const __nv_bfloat162* w2 = reinterpret_cast<const __nv_bfloat162*>(&wv);
-#pragma unroll
-      for (int r = 0; r < 16; ++r) {
-        if (r0 + r < rows) {
-          const uint4 xv = *reinterpret_cast<const uint4*>(X + (size_t)(r0 + r) * K + k);
-          const __nv_bfloat162* x2 = reinterpret_cast<const __nv_bfloat162*>(&xv);
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const float2 wf = __bfloat1622float2(w2[e]), xf = __bfloat1622float2(x2[e]);
-            acc[r] = fmaf(wf.x, xf.x, acc[r]);
-            acc[r] = fmaf(wf.y, xf.y, acc[r]);
-          }
-        }
-      }
-    }
-#pragma unroll
-    for (int r = 0; r < 16; ++r) {
-      float v = acc[r];
-#pragma unroll
-      for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
-      if (lane == 0 && r0 + r < rows) out[(size_t)(r0 + r) * N + feat] = v;
-    }
-  }
-}
-
-// per 128-feature tile (max, lowest id) of a logits matrix, for the bring-up path
-__global__ void k_tile_argmax(const float* __restrict__ logits, int rows, int N, float* tile_max,
-                              int* tile_idx, int tile_stride) {
-  const int tile = blockIdx.x, tok = blockIdx.y;
-  const int lane = threadIdx.x;   // 32 threads
-  float val = -INFINITY;
-  int idx = INT32_MAX;
-  for (int f = tile * CS_GEMM_BM + lane; f < min(N, (tile + 1) * CS_GEMM_BM); f += 32) {
-    const float v = logits[(size_t)tok * N + f];
-    if (v > val || (v == val && f < idx)) { val = v; idx = f; }
-  }
-  for (int off = 16; off > 0; off >>= 1) {
-    const float ov = __shfl_xor_sync(0xffffffffu, val, off);
-    const int oi = __shfl_xor_sync(0xffffffffu, idx, off);
-    if (ov > val || (ov == val && oi < idx)) { val = ov; idx = oi; }
-  }
-  if (lane == 0) {
-    tile_max[(size_t)tile * tile_stride + tok] = val;
-    tile_idx[(size_t)tile * tile_stride + tok] = idx;
   }
 }
 
@@ -394,48 +450,33 @@ cs_status cs_gemm_plan(cs_ctx* ctx, GemmPlan* g, const void* w, int N, int K, bo
   g->N = N;
   g->K = K;
   const int tiles = cs_ceil_div(N, CS_GEMM_BM), kb = cs_ceil_div(K, CS_GEMM_BK);
+  // two CTAs fit on an SM; clustered launches are planned for 85 % of those slots, because
+  // a cluster must find all its CTAs free inside one GPC and a grid that needs every slot
+  // spills into a second wave
   const int slots = 2 * ctx->num_sms;
   int best = 1;
   long best_cost = -1;
   const int smax = allow_split ? cs_max_splits(tiles, kb) : 1;
   for (int s = 1; s <= smax; ++s) {
-    const long cost = (long)cs_ceil_div(tiles * s, slots) * (cs_ceil_div(kb, s) + 2);
+    const int avail = (s > 1) ? slots * 85 / 100 : slots;
+    // waves of CTAs times the K blocks each CTA streams, plus a fixed start-up/epilogue cost
+    const long cost = (long)cs_ceil_div(tiles * s, avail) * (cs_ceil_div(kb, s) + 2);
     if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = s; }
   }
+  if (allow_split && getenv("CS_TUNE_SPLITS")) best = max(1, min(CS_MAX_SPLITS, min(kb, atoi(getenv("CS_TUNE_SPLITS")))));
   g->kb_per_split = cs_ceil_div(kb, best);
   g->splits = cs_ceil_div(kb, g->kb_per_split);
-  if (ctx->gemm_simt) { g->splits = 1; g->kb_per_split = kb; return CS_OK; }
   return encode_2d(ctx, &g->tmW, w, N, K, CS_GEMM_BM, true);
 }
 
 cs_status cs_make_act_map(cs_ctx* ctx, CUtensorMap* tm, const void* base, int rows_total, int K,
                           int box_rows) {
-  if (ctx->gemm_simt) return CS_OK;
   return encode_2d(ctx, tm, base, rows_total, K, box_rows, false);
 }
 
-cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX, const __nv_bfloat16* X,
-                         int rows, int mode, float* out, float* logits, cudaStream_t st) {
+cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX, int rows, int mode,
+                         float* out, __nv_bfloat16* act, int F, cudaStream_t st) {
   const int tiles = cs_ceil_div(g->N, CS_GEMM_BM);
-  if (ctx->gemm_simt) {
-    float* dst = out;
-    if (mode == 1) {
-      dst = logits;
-      if (dst == nullptr) {
-        if ((size_t)rows * g->N > ctx->partial_elems) {
-          snprintf(ctx->err, sizeof(ctx->err), "bring-up GEMM: logits do not fit the workspace");
-          return CS_ERR_UNSUPPORTED;
-        }
-        dst = ctx->partial;
-      }
-    }
-    k_gemm_simt<<<cs_ceil_div(g->N, 8), 256, 0, st>>>(X, g->W, rows, g->N, g->K, dst);
-    if (mode == 1)
-      k_tile_argmax<<<dim3(tiles, rows), 32, 0, st>>>(dst, rows, g->N, ctx->tile_max, ctx->tile_idx,
-                                                      ctx->rows_pad);
-    CS_CUDA_OK(ctx, cudaGetLastError());
-    return CS_OK;
-  }
   GemmArgs a;
   a.rows = rows;
   a.n_tok = cs_ceil_div(rows, 16) * 16;
@@ -443,12 +484,14 @@ cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX,
   a.K = g->K;
   a.num_kb = cs_ceil_div(g->K, CS_GEMM_BK);
   a.kb_per_split = g->kb_per_split;
+  a.splits = g->splits;
   a.mode = mode;
   a.out = out;
+  a.act = act;
+  a.F = F;
   a.tile_max = ctx->tile_max;
   a.tile_idx = ctx->tile_idx;
   a.tile_stride = ctx->rows_pad;
-  a.logits = logits;
   a.status = ctx->d_status;
   const int stage_bytes = kTileABytes + a.n_tok * 128;
   const int fixed = 1024 /*alignment slack*/ + (2 * 8 + 1) * 8 + 16 + 8 * a.n_tok * 4;
@@ -456,18 +499,38 @@ cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX,
   int stages = (100 * 1024 - fixed) / stage_bytes;
   if (stages < 4) stages = (220 * 1024 - fixed) / stage_bytes;
   if (stages > 8) stages = 8;
-  if (stages < 2) {
+  if (getenv("CS_TUNE_SMEM_KB")) stages = min(12, (atoi(getenv("CS_TUNE_SMEM_KB")) * 1024 - fixed) / stage_bytes);
+  // the parked tile ([n_tok][128] fp32) reuses the ring
+  if (stages < 2 || (size_t)stages * stage_bytes < (size_t)a.n_tok * CS_GEMM_BM * 4) {
     snprintf(ctx->err, sizeof(ctx->err), "GEMM stage of %d bytes does not fit shared memory", stage_bytes);
     return CS_ERR_UNSUPPORTED;
   }
   a.stages = stages;
   const size_t smem = (size_t)fixed + (size_t)stages * stage_bytes;
-  static size_t smem_set = 0;
-  if (smem > smem_set) {
+  static bool attr_set = false;
+  if (!attr_set) {
     CS_CUDA_OK(ctx, cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-    smem_set = 227 * 1024;
+    attr_set = true;
   }
-  k_gemm_tc<<<dim3(tiles, g->splits), kThreads, smem, st>>>(g->tmW, *tmX, a);
-  CS_CUDA_OK(ctx, cudaGetLastError());
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = dim3(tiles, g->splits, 1);
+  lc.blockDim = dim3(kThreads, 1, 1);
+  lc.dynamicSmemBytes = smem;
+  lc.stream = st;
+  cudaLaunchAttribute at[2];
+  int na = 0;
+  at[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[na].val.programmaticStreamSerializationAllowed = 1;
+  ++na;
+  if (g->splits > 1) {
+    at[na].id = cudaLaunchAttributeClusterDimension;
+    at[na].val.clusterDim.x = 1;
+    at[na].val.clusterDim.y = g->splits;
+    at[na].val.clusterDim.z = 1;
+    ++na;
+  }
+  lc.attrs = at;
+  lc.numAttrs = na;
+  CS_CUDA_OK(ctx, cudaLaunchKernelEx(&lc, k_gemm_tc, g->tmW, *tmX, a));
   return CS_OK;
 }

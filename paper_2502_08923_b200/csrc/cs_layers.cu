@@ -17,6 +17,7 @@ __global__ void k_block_setup(const int* __restrict__ last_tok, const int* __res
                               const int* __restrict__ skip, int B, int k, int max_seq, int vocab,
                               int half, const double* __restrict__ inv_freq, int* row_tok, int* row_pos,
                               int* row_lim, int* row_write, int* seq_ok, float* rope_cs, int* status) {
+  CS_PDL_PROLOGUE();
   const int R = k + 1, rows = B * R;
   for (int row = threadIdx.x; row < rows; row += blockDim.x) {
     const int b = row / R, r = row % R;
@@ -56,6 +57,7 @@ __global__ void k_prefill_setup(const int* __restrict__ hist, const int* __restr
                                 int stride, int start, int R, int max_seq, int vocab, int half,
                                 const double* __restrict__ inv_freq, int* row_tok, int* row_pos,
                                 int* row_lim, int* row_write, int* seq_ok, float* rope_cs, int* status) {
+  CS_PDL_PROLOGUE();
   const int rows = B * R;
   for (int row = threadIdx.x; row < rows; row += blockDim.x) {
     const int b = row / R, r = row % R;
@@ -86,6 +88,7 @@ __global__ void k_prefill_setup(const int* __restrict__ hist, const int* __restr
 
 __global__ void k_embed(const __nv_bfloat16* __restrict__ E, const int* __restrict__ row_tok, int d,
                         float* __restrict__ x) {
+  CS_PDL_PROLOGUE();
   const int row = blockIdx.x;
   const __nv_bfloat16* e = E + (size_t)row_tok[row] * d;
   for (int i = threadIdx.x * 2; i < d; i += blockDim.x * 2) {
@@ -94,21 +97,16 @@ __global__ void k_embed(const __nv_bfloat16* __restrict__ E, const int* __restri
   }
 }
 
-// x += sum_s partial[s] (the projection that closed the previous sub-layer), then
 // xn = bf16(x * rsqrt(mean(x^2) + eps) * g).  One CTA per row.
 __global__ void __launch_bounds__(256)
-k_rmsnorm(float* __restrict__ x, const float* __restrict__ partial, int splits, int rows, int d,
-          const __nv_bfloat16* __restrict__ gain, float eps, __nv_bfloat16* __restrict__ xn) {
+k_rmsnorm(const float* __restrict__ x, int d, const __nv_bfloat16* __restrict__ gain, float eps,
+          __nv_bfloat16* __restrict__ xn) {
+  CS_PDL_PROLOGUE();
   const int row = blockIdx.x;
-  float* xr = x + (size_t)row * d;
+  const float* xr = x + (size_t)row * d;
   float ss = 0.f;
   for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
-    float4 v = *reinterpret_cast<const float4*>(xr + i);
-    for (int s = 0; s < splits; ++s) {
-      const float4 p = *reinterpret_cast<const float4*>(partial + ((size_t)s * rows + row) * d + i);
-      v.x += p.x; v.y += p.y; v.z += p.z; v.w += p.w;
-    }
-    if (splits > 0) *reinterpret_cast<float4*>(xr + i) = v;
+    const float4 v = *reinterpret_cast<const float4*>(xr + i);
     ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
   }
   __shared__ float red[8];
@@ -134,20 +132,17 @@ k_rmsnorm(float* __restrict__ x, const float* __restrict__ partial, int splits, 
   }
 }
 
-// Sum the QKV split-K partials, rotate q and k (rotate-half pairing) at the row's
+// Rotate q and k of the QKV projection (rotate-half pairing) at the row's
 // absolute position, store q as the bf16 attention operand and append k, v to the cache.
-__global__ void k_qkv_post(const float* __restrict__ partial, int splits, int rows, int H, int Hkv, int Dh,
+__global__ void k_qkv_post(const float* __restrict__ qkv, int H, int Hkv, int Dh,
                            const float* __restrict__ rope_cs, const int* __restrict__ row_pos,
                            const int* __restrict__ row_write, int R, __nv_bfloat16* __restrict__ qbuf,
                            __nv_bfloat16* __restrict__ kv, int layer, int max_batch, int max_seq) {
   const int row = blockIdx.x, head = blockIdx.y, i = threadIdx.x;
   const int half = Dh >> 1, N = (H + 2 * Hkv) * Dh;
-  float a = 0.f, b = 0.f;
-  for (int s = 0; s < splits; ++s) {
-    const float* p = partial + ((size_t)s * rows + row) * N + (size_t)head * Dh;
-    a += p[i];
-    b += p[i + half];
-  }
+  CS_PDL_PROLOGUE();
+  const float* p = qkv + (size_t)row * N + (size_t)head * Dh;
+  const float a = p[i], b = p[i + half];
   const float c = rope_cs[2 * (row * half + i)], sn = rope_cs[2 * (row * half + i) + 1];
   if (head < H) {
     __nv_bfloat16* q = qbuf + (size_t)row * H * Dh + (size_t)head * Dh;
@@ -173,34 +168,35 @@ __global__ void k_qkv_post(const float* __restrict__ partial, int splits, int ro
 // Combine the key slices: o = sum_s o_s e^(m_s - M) / sum_s l_s e^(m_s - M).
 __global__ void k_attn_merge(const float* __restrict__ in_o, const float* __restrict__ in_ml, int nsplit,
                              int rows, int H, int Dh, __nv_bfloat16* __restrict__ attn_out) {
+  CS_PDL_PROLOGUE();
   const int row = blockIdx.x, h = blockIdx.y, dd = threadIdx.x;
-  float M = -INFINITY;
-  for (int s = 0; s < nsplit; ++s) M = fmaxf(M, in_ml[(((size_t)s * rows + row) * H + h) * 2]);
-  float L = 0.f, acc = 0.f;
+  const int lane = threadIdx.x & 31;
+  // every warp works out the slice weights e^(m_s - M) / L itself: lane s owns slices s, s+32
+  float m0 = -INFINITY, l0 = 0.f, m1 = -INFINITY, l1 = 0.f;
+  if (lane < nsplit) {
+    const size_t base = ((size_t)lane * rows + row) * H + h;
+    m0 = in_ml[base * 2]; l0 = in_ml[base * 2 + 1];
+  }
+  if (lane + 32 < nsplit) {
+    const size_t base = ((size_t)(lane + 32) * rows + row) * H + h;
+    m1 = in_ml[base * 2]; l1 = in_ml[base * 2 + 1];
+  }
+  float M = fmaxf(m0, m1);
+  for (int off = 16; off > 0; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
+  float w0 = (m0 == -INFINITY) ? 0.f : expf(m0 - M), w1 = (m1 == -INFINITY) ? 0.f : expf(m1 - M);
+  float L = l0 * w0 + l1 * w1;
+  for (int off = 16; off > 0; off >>= 1) L += __shfl_xor_sync(0xffffffffu, L, off);
+  const float inv = L > 0.f ? 1.f / L : 0.f;
+  w0 *= inv; w1 *= inv;
+  float acc = 0.f;
+  const size_t stride = (size_t)rows * H * Dh;
+  const float* src = in_o + ((size_t)row * H + h) * Dh + dd;
+#pragma unroll 8
   for (int s = 0; s < nsplit; ++s) {
-    const size_t base = ((size_t)s * rows + row) * H + h;
-    const float ms = in_ml[base * 2];
-    if (ms == -INFINITY) continue;
-    const float w = expf(ms - M);
-    L += in_ml[base * 2 + 1] * w;
-    acc += in_o[base * Dh + dd] * w;
+    const float w = __shfl_sync(0xffffffffu, s < 32 ? w0 : w1, s & 31);
+    acc = fmaf(src[(size_t)s * stride], w, acc);
   }
-  attn_out[((size_t)row * H + h) * Dh + dd] = __float2bfloat16_rn(L > 0.f ? acc / L : 0.f);
-}
-
-// act = bf16( silu(gate) * up ), gate/up summed over the split-K partials
-__global__ void k_swiglu(const float* __restrict__ partial, int splits, int rows, int F,
-                         __nv_bfloat16* __restrict__ act) {
-  const int row = blockIdx.y;
-  const int j = blockIdx.x * blockDim.x + threadIdx.x;
-  if (j >= F) return;
-  float g = 0.f, u = 0.f;
-  for (int s = 0; s < splits; ++s) {
-    const float* p = partial + ((size_t)s * rows + row) * (2 * (size_t)F);
-    g += p[j];
-    u += p[F + j];
-  }
-  act[(size_t)row * F + j] = __float2bfloat16_rn(g / (1.f + expf(-g)) * u);
+  attn_out[((size_t)row * H + h) * Dh + dd] = __float2bfloat16_rn(acc);
 }
 
 // ------------------------------------------------------------------ acceptance
@@ -214,6 +210,7 @@ k_accept(const float* __restrict__ tile_max, const int* __restrict__ tile_idx, i
          const int* __restrict__ script_off, int script_limit, int* __restrict__ accept_len,
          int* __restrict__ out_tokens, int* __restrict__ argmax_ids, int* __restrict__ kv_len,
          int update_kv) {
+  CS_PDL_PROLOGUE();
   const int b = blockIdx.x, R = k + 1;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   __shared__ int s_arg[CS_MAX_ROWS];
@@ -265,6 +262,7 @@ k_accept(const float* __restrict__ tile_max, const int* __restrict__ tile_idx, i
 }
 
 __global__ void k_truncate(int* kv_len, const int* new_len, int B, int* status) {
+  CS_PDL_PROLOGUE();
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= B) return;
   const int nl = new_len[b];
@@ -273,6 +271,7 @@ __global__ void k_truncate(int* kv_len, const int* new_len, int B, int* status) 
 }
 
 __global__ void k_prefill_finish(const int* hist_len, const int* seq_ok, int* kv_len, int B) {
+  CS_PDL_PROLOGUE();
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b < B && seq_ok[b]) kv_len[b] = max(0, hist_len[b] - 1);
 }
@@ -281,6 +280,7 @@ __global__ void k_prefill_finish(const int* hist_len, const int* seq_ok, int* kv
 __global__ void k_loop_init(const int* hist_len, const int* kv_len, int B, int stride, int max_new, int k,
                             int max_seq, int max_batch, int* emitted, int* done,
                             unsigned long long* stats, int* status) {
+  CS_PDL_PROLOGUE();
   const int t = threadIdx.x;
   for (int i = t; i < (int)(sizeof(cs_stats) / 8); i += blockDim.x) stats[i] = 0ull;
   __shared__ int s_done;
@@ -307,6 +307,7 @@ __global__ void k_loop_init(const int* hist_len, const int* kv_len, int B, int s
 __global__ void k_loop_commit(int* hist, int* hist_len, int B, int stride, int* kv_len, int k, int max_new,
                               int eos_id, int scripted, const int* accept, const int* out, const int* mpos,
                               int* emitted, int* done, int max_batch, unsigned long long* stats) {
+  CS_PDL_PROLOGUE();
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= B || done[b]) return;
   cs_stats* st = reinterpret_cast<cs_stats*>(stats);
@@ -350,75 +351,66 @@ void cs_launch_block_setup(cs_ctx* ctx, const int32_t* last_tok, const int32_t* 
                            const int32_t* draft_len, const int32_t* kv_len, const int32_t* skip, int B,
                            int k, cudaStream_t st) {
   const cs_model_config& c = ctx->cfg;
-  k_block_setup<<<1, 256, 0, st>>>(last_tok, draft, draft_len, kv_len, skip, B, k, c.max_seq, c.vocab,
-                                   c.head_dim / 2, ctx->inv_freq, ctx->row_tok, ctx->row_pos, ctx->row_lim,
-                                   ctx->row_write, ctx->seq_ok, ctx->rope_cs, ctx->d_status);
+  cs_launch_pdl(k_block_setup, dim3(1), dim3(256), 0, st, last_tok, draft, draft_len, kv_len, skip, B, k, c.max_seq,
+                c.vocab, c.head_dim / 2, ctx->inv_freq, ctx->row_tok, ctx->row_pos, ctx->row_lim, ctx->row_write,
+                ctx->seq_ok, ctx->rope_cs, ctx->d_status);
 }
 
 void cs_launch_prefill_setup(cs_ctx* ctx, const int32_t* hist, const int32_t* hist_len, int B, int stride,
                              int start, int R, cudaStream_t st) {
   const cs_model_config& c = ctx->cfg;
-  k_prefill_setup<<<1, 256, 0, st>>>(hist, hist_len, B, stride, start, R, c.max_seq, c.vocab, c.head_dim / 2,
-                                     ctx->inv_freq, ctx->row_tok, ctx->row_pos, ctx->row_lim, ctx->row_write,
-                                     ctx->seq_ok, ctx->rope_cs, ctx->d_status);
+  cs_launch_pdl(k_prefill_setup, dim3(1), dim3(256), 0, st, hist, hist_len, B, stride, start, R, c.max_seq, c.vocab,
+                c.head_dim / 2, ctx->inv_freq, ctx->row_tok, ctx->row_pos, ctx->row_lim, ctx->row_write, ctx->seq_ok,
+                ctx->rope_cs, ctx->d_status);
 }
 
 void cs_launch_embed(cs_ctx* ctx, int rows, cudaStream_t st) {
-  k_embed<<<rows, 128, 0, st>>>(ctx->embed, ctx->row_tok, ctx->cfg.d_model, ctx->x);
+  cs_launch_pdl(k_embed, dim3(rows), dim3(128), 0, st, ctx->embed, ctx->row_tok, ctx->cfg.d_model, ctx->x);
 }
 
-void cs_launch_rmsnorm(cs_ctx* ctx, const float* partial, int splits, const __nv_bfloat16* gain, int rows,
-                       cudaStream_t st) {
-  k_rmsnorm<<<rows, 256, 0, st>>>(ctx->x, partial, partial ? splits : 0, rows, ctx->cfg.d_model, gain,
-                                  ctx->cfg.rms_eps, ctx->xn);
+void cs_launch_rmsnorm(cs_ctx* ctx, const __nv_bfloat16* gain, int rows, cudaStream_t st) {
+  cs_launch_pdl(k_rmsnorm, dim3(rows), dim3(256), 0, st, ctx->x, ctx->cfg.d_model, gain, ctx->cfg.rms_eps, ctx->xn);
 }
 
-void cs_launch_qkv_post(cs_ctx* ctx, int splits, void* kv_cache, int layer, int B, int R, cudaStream_t st) {
+void cs_launch_qkv_post(cs_ctx* ctx, void* kv_cache, int layer, int B, int R, cudaStream_t st) {
   const cs_model_config& c = ctx->cfg;
-  k_qkv_post<<<dim3(B * R, c.n_heads + 2 * c.n_kv_heads), c.head_dim / 2, 0, st>>>(
-      ctx->partial, splits, B * R, c.n_heads, c.n_kv_heads, c.head_dim, ctx->rope_cs, ctx->row_pos,
-      ctx->row_write, R, ctx->qbuf, static_cast<__nv_bfloat16*>(kv_cache), layer, c.max_batch, c.max_seq);
+  cs_launch_pdl(k_qkv_post, dim3(B * R, c.n_heads + 2 * c.n_kv_heads), dim3(c.head_dim / 2), 0, st, ctx->qkv,
+                c.n_heads, c.n_kv_heads, c.head_dim, ctx->rope_cs, ctx->row_pos, ctx->row_write, R, ctx->qbuf,
+                static_cast<__nv_bfloat16*>(kv_cache), layer, c.max_batch, c.max_seq);
 }
 
 void cs_launch_attn_merge(cs_ctx* ctx, int nsplit, int rows, cudaStream_t st) {
   const cs_model_config& c = ctx->cfg;
-  k_attn_merge<<<dim3(rows, c.n_heads), c.head_dim, 0, st>>>(ctx->attn_o, ctx->attn_ml, nsplit, rows, c.n_heads,
-                                                             c.head_dim, ctx->attn_out);
-}
-
-void cs_launch_swiglu(cs_ctx* ctx, int splits, int rows, cudaStream_t st) {
-  k_swiglu<<<dim3(cs_ceil_div(ctx->cfg.d_ffn, 256), rows), 256, 0, st>>>(ctx->partial, splits, rows,
-                                                                         ctx->cfg.d_ffn, ctx->act);
+  cs_launch_pdl(k_attn_merge, dim3(rows, c.n_heads), dim3(c.head_dim), 0, st, ctx->attn_o, ctx->attn_ml, nsplit, rows,
+                c.n_heads, c.head_dim, ctx->attn_out);
 }
 
 void cs_launch_accept(cs_ctx* ctx, int B, int k, const int32_t* draft, const int32_t* draft_len,
                       const int32_t* script, int script_stride, const int32_t* script_off, int script_limit,
                       int32_t* accept_len, int32_t* out_tokens, int32_t* argmax_ids, int32_t* kv_len,
                       int update_kv, cudaStream_t st) {
-  k_accept<<<B, 128, 0, st>>>(ctx->tile_max, ctx->tile_idx, cs_ceil_div(ctx->cfg.vocab, CS_GEMM_BM),
-                              ctx->rows_pad, k, draft, draft_len, ctx->seq_ok, script, script_stride,
-                              script_off, script_limit, accept_len, out_tokens, argmax_ids, kv_len, update_kv);
+  cs_launch_pdl(k_accept, dim3(B), dim3(128), 0, st, ctx->tile_max, ctx->tile_idx,
+                cs_ceil_div(ctx->cfg.vocab, CS_GEMM_BM), ctx->rows_pad, k, draft, draft_len, ctx->seq_ok, script,
+                script_stride, script_off, script_limit, accept_len, out_tokens, argmax_ids, kv_len, update_kv);
 }
 
 void cs_launch_truncate(cs_ctx* ctx, int32_t* kv_len, const int32_t* new_len, int B, cudaStream_t st) {
-  k_truncate<<<cs_ceil_div(B, 128), 128, 0, st>>>(kv_len, new_len, B, ctx->d_status);
+  cs_launch_pdl(k_truncate, dim3(cs_ceil_div(B, 128)), dim3(128), 0, st, kv_len, new_len, B, ctx->d_status);
 }
 
 void cs_launch_prefill_finish(cs_ctx* ctx, const int32_t* hist_len, int32_t* kv_len, int B, cudaStream_t st) {
-  k_prefill_finish<<<cs_ceil_div(B, 128), 128, 0, st>>>(hist_len, ctx->seq_ok, kv_len, B);
+  cs_launch_pdl(k_prefill_finish, dim3(cs_ceil_div(B, 128)), dim3(128), 0, st, hist_len, ctx->seq_ok, kv_len, B);
 }
 
 void cs_launch_loop_init(cs_ctx* ctx, const int32_t* hist_len, const int32_t* kv_len, int B, int stride,
                          int max_new, int k, cudaStream_t st) {
-  k_loop_init<<<1, 256, 0, st>>>(hist_len, kv_len, B, stride, max_new, k, ctx->cfg.max_seq,
-                                 ctx->cfg.max_batch, ctx->loop_emitted, ctx->loop_done, ctx->loop_stats,
-                                 ctx->d_status);
+  cs_launch_pdl(k_loop_init, dim3(1), dim3(256), 0, st, hist_len, kv_len, B, stride, max_new, k, ctx->cfg.max_seq,
+                ctx->cfg.max_batch, ctx->loop_emitted, ctx->loop_done, ctx->loop_stats, ctx->d_status);
 }
 
 void cs_launch_loop_commit(cs_ctx* ctx, int32_t* hist, int32_t* hist_len, int B, int stride, int32_t* kv_len,
                            int k, int max_new, int eos_id, int scripted, cudaStream_t st) {
-  k_loop_commit<<<cs_ceil_div(B, 128), 128, 0, st>>>(hist, hist_len, B, stride, kv_len, k, max_new, eos_id,
-                                                     scripted, ctx->loop_accept, ctx->loop_out, ctx->loop_mpos,
-                                                     ctx->loop_emitted, ctx->loop_done, ctx->cfg.max_batch,
-                                                     ctx->loop_stats);
+  cs_launch_pdl(k_loop_commit, dim3(cs_ceil_div(B, 128)), dim3(128), 0, st, hist, hist_len, B, stride, kv_len, k,
+                max_new, eos_id, scripted, ctx->loop_accept, ctx->loop_out, ctx->loop_mpos, ctx->loop_emitted,
+                ctx->loop_done, ctx->cfg.max_batch, ctx->loop_stats);
 }

@@ -26,6 +26,7 @@ k_find_match(const int* __restrict__ hist, const int* __restrict__ hist_len, int
              int k, int policy, int* __restrict__ match_pos, int* __restrict__ draft,
              int* __restrict__ draft_len, int* __restrict__ last_tok,
              const int* __restrict__ skip) {
+  CS_PDL_PROLOGUE();
   cg::cluster_group cluster = cg::this_cluster();
   const int b = blockIdx.y;
   const int rank = (int)cluster.block_rank();
@@ -126,13 +127,15 @@ cs_status cs_launch_find_match(const int32_t* hist, const int32_t* hist_len, int
   lc.blockDim = dim3(kThreads, 1, 1);
   lc.dynamicSmemBytes = 0;
   lc.stream = st;
-  cudaLaunchAttribute at[1];
+  cudaLaunchAttribute at[2];
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[1].val.programmaticStreamSerializationAllowed = 1;
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = cl;
   at[0].val.clusterDim.y = 1;
   at[0].val.clusterDim.z = 1;
   lc.attrs = at;
-  lc.numAttrs = 1;
+  lc.numAttrs = 2;
   cudaError_t e = cudaLaunchKernelEx(&lc, k_find_match, (const int*)hist, (const int*)hist_len,
                                      stride, gamma, k, policy, (int*)match_pos, (int*)draft,
                                      (int*)draft_len, (int*)last_tok, (const int*)skip);
