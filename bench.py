@@ -40,7 +40,7 @@ WORKLOAD = "verify_8b_b1_kv4096_k10_scripted_tau_uniform"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from the
 # committed ncu capture (profiles/); None until a capture of the current kernel exists.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 111.65e6   # profiles/k_gemm_tc_verify8b_2layer_ncu_full.md
 
 
 def _peaks():
@@ -226,7 +226,7 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     dev = torch.device("cuda", local)
-    cfg = inputs.LLAMA8B
+    cfg = inputs.LLAMA8B if args.layers <= 0 else inputs.sliced(inputs.LLAMA8B, args.layers)
     W, K = args.warmup, args.steps
     taus = _taus(W + K)
     ctx_len = KV_START
@@ -367,7 +367,7 @@ def run_ours(args):
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
                 "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                 "dtype": "bf16", "data": "synthetic",
-                "config": {"workload": WORKLOAD, "model_shape": "32L d4096 H32/8 Dh128 F14336 V128256", "batch": 1,
+                "config": {"workload": WORKLOAD, "model_shape": f"{cfg.n_layers}L d4096 H32/8 Dh128 F14336 V128256", "batch": 1,
                            "gamma": GAMMA, "k": K_DRAFT, "kv_start": n0 - 1, "kv_end": n0 - 1 + st1["emitted"],
                            "tokens_per_step": emitted / K, "l2": "inputs larger than L2 (15 GB of weights per step)",
                            "replicas": world, "draft_tokens_accepted_per_s": world * (emitted - K) / (ms * 1e-3)},
@@ -391,6 +391,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="profiling aid: keep only this many of the 32 layers (small case for ncu captures; "
+                         "not the benchmark workload)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
