@@ -235,6 +235,15 @@ cs_status cs_prefill(cs_ctx* ctx, const int32_t* hist, const int32_t* hist_len, 
 cs_status cs_linear(cs_ctx* ctx, const void* X, const void* W, int rows, int N, int K,
                     float* Y, void* stream);
 
+/* The LM-head stage of the verification forward on its own (Sec. 3.2; App. B.2: greedy
+ * token at temperature 0): ids[r] = the lowest token id with the largest logit of
+ * X[r] . lm_head^T, for rows already normalised and rounded to bf16.  X bf16 [rows][d_model],
+ * readable for ceil(rows/16)*16 rows; ids int32 [rows]; logits_dbg fp32 [rows][vocab] or
+ * NULL.  Uses the context's workspace for the per-tile maxima, so it must not overlap other
+ * work of the context.  rows <= 256.  Async. */
+cs_status cs_lm_head(cs_ctx* ctx, const void* X, int rows, int32_t* ids, float* logits_dbg,
+                     void* stream);
+
 #ifdef __cplusplus
 }
 #endif

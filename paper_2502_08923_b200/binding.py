@@ -49,7 +49,7 @@ class CsStats(C.Structure):
 EXPORTS = ("cs_workspace_bytes", "cs_create", "cs_destroy", "cs_last_error", "cs_sync_status",
            "cs_find_match", "cs_verify_step", "cs_kv_truncate", "cs_decode_loop", "cs_prefill", "cs_linear",
            "cs_loop_begin", "cs_loop_steps", "cs_loop_poll", "cs_loop_end", "cs_profile_verify_step",
-           "cs_loop_launches_per_step")
+           "cs_loop_launches_per_step", "cs_lm_head")
 
 _lib = None
 
@@ -102,6 +102,8 @@ def load(build_if_missing: bool = True) -> C.CDLL:
                                            C.POINTER(C.c_int), vp]
     lib.cs_prefill.restype = i
     lib.cs_prefill.argtypes = [vp, ip, ip, i, i, i, vp, ip, vp]
+    lib.cs_lm_head.restype = i
+    lib.cs_lm_head.argtypes = [vp, vp, i, ip, vp, vp]
     lib.cs_linear.restype = i
     lib.cs_linear.argtypes = [vp, vp, vp, i, i, i, vp, vp]
     _lib = lib
@@ -313,6 +315,14 @@ class Context:
         self._check(rc, "cs_profile_verify_step")
         names = ("gemm", "attention", "lm_head", "elementwise")
         return dict(zip(names, list(ms))), dict(zip(names, list(n)))
+
+    def cs_lm_head(self, X, rows=None, logits_dbg=None):
+        """Greedy token ids of bf16 rows X[rows][d_model] under the model's LM head."""
+        rows = X.shape[0] if rows is None else rows
+        ids = torch.empty(rows, dtype=torch.int32, device=X.device)
+        rc = self.lib.cs_lm_head(self.handle, _ptr(X), rows, _i32(ids, "ids"), _ptr(logits_dbg), _stream())
+        self._check(rc, "cs_lm_head")
+        return ids
 
     def cs_linear(self, X, W, rows=None):
         """Y[rows][N] fp32 = X[rows][K] bf16 @ W[N][K]^T bf16 through the tensor-core GEMM."""

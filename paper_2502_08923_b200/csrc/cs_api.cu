@@ -539,4 +539,18 @@ cs_status cs_linear(cs_ctx* ctx, const void* X, const void* W, int rows, int N, 
   return cs_launch_gemm(ctx, &g, &tmX, rows, CS_EPI_STORE, Y, nullptr, 0, st);
 }
 
+cs_status cs_lm_head(cs_ctx* ctx, const void* X, int rows, int32_t* ids, float* logits_dbg, void* stream) {
+  if (ctx == nullptr) return CS_ERR_ARG;
+  if (X == nullptr || ids == nullptr || rows < 1 || rows > CS_MAX_ROWS) return fail(ctx, CS_ERR_ARG, "bad argument");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int n_tok = cs_ceil_div(rows, 16) * 16;
+  CUtensorMap tmX;
+  cs_status s = cs_make_act_map(ctx, &tmX, X, n_tok, ctx->cfg.d_model, n_tok);
+  if (s != CS_OK) return s;
+  if ((s = cs_launch_gemm(ctx, &ctx->lm, &tmX, rows, CS_EPI_ARGMAX, logits_dbg, nullptr, 0, st)) != CS_OK) return s;
+  cs_launch_tile_reduce(ctx, rows, ids, st);
+  CS_CUDA_OK(ctx, cudaGetLastError());
+  return CS_OK;
+}
+
 }  // extern "C"

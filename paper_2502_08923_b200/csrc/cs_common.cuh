@@ -193,6 +193,7 @@ void cs_launch_accept(cs_ctx* ctx, int B, int k, const int32_t* draft, const int
                       const int32_t* script, int script_stride, const int32_t* script_off,
                       int script_limit, int32_t* accept_len, int32_t* out_tokens,
                       int32_t* argmax_ids, int32_t* kv_len, int update_kv, cudaStream_t st);
+void cs_launch_tile_reduce(cs_ctx* ctx, int rows, int32_t* ids, cudaStream_t st);
 void cs_launch_truncate(cs_ctx* ctx, int32_t* kv_len, const int32_t* new_len, int B,
                         cudaStream_t st);
 void cs_launch_prefill_finish(cs_ctx* ctx, const int32_t* hist_len, int32_t* kv_len, int B,

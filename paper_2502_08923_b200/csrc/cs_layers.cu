@@ -261,6 +261,35 @@ k_accept(const float* __restrict__ tile_max, const int* __restrict__ tile_idx, i
   }
 }
 
+// Greedy token of each row from the LM head's per-tile (max, id) pairs (lowest id on ties).
+__global__ void __launch_bounds__(128)
+k_tile_reduce(const float* __restrict__ tile_max, const int* __restrict__ tile_idx, int tiles, int tile_stride,
+              int* __restrict__ ids) {
+  CS_PDL_PROLOGUE();
+  const int row = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  float val = -INFINITY;
+  int idx = INT32_MAX;
+  for (int t = threadIdx.x; t < tiles; t += 128) {
+    const float v = tile_max[(size_t)t * tile_stride + row];
+    const int id = tile_idx[(size_t)t * tile_stride + row];
+    if (v > val || (v == val && id < idx)) { val = v; idx = id; }
+  }
+  __shared__ float sv[4];
+  __shared__ int si[4];
+  for (int off = 16; off > 0; off >>= 1) {
+    const float ov = __shfl_xor_sync(0xffffffffu, val, off);
+    const int oi = __shfl_xor_sync(0xffffffffu, idx, off);
+    if (ov > val || (ov == val && oi < idx)) { val = ov; idx = oi; }
+  }
+  if (lane == 0) { sv[warp] = val; si[warp] = idx; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < 4; ++w)
+      if (sv[w] > val || (sv[w] == val && si[w] < idx)) { val = sv[w]; idx = si[w]; }
+    ids[row] = (idx == INT32_MAX) ? -1 : idx;
+  }
+}
+
 __global__ void k_truncate(int* kv_len, const int* new_len, int B, int* status) {
   CS_PDL_PROLOGUE();
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
@@ -392,6 +421,11 @@ void cs_launch_accept(cs_ctx* ctx, int B, int k, const int32_t* draft, const int
   cs_launch_pdl(k_accept, dim3(B), dim3(128), 0, st, ctx->tile_max, ctx->tile_idx,
                 cs_ceil_div(ctx->cfg.vocab, CS_GEMM_BM), ctx->rows_pad, k, draft, draft_len, ctx->seq_ok, script,
                 script_stride, script_off, script_limit, accept_len, out_tokens, argmax_ids, kv_len, update_kv);
+}
+
+void cs_launch_tile_reduce(cs_ctx* ctx, int rows, int32_t* ids, cudaStream_t st) {
+  cs_launch_pdl(k_tile_reduce, dim3(rows), dim3(128), 0, st, ctx->tile_max, ctx->tile_idx,
+                cs_ceil_div(ctx->cfg.vocab, CS_GEMM_BM), ctx->rows_pad, ids);
 }
 
 void cs_launch_truncate(cs_ctx* ctx, int32_t* kv_len, const int32_t* new_len, int B, cudaStream_t st) {

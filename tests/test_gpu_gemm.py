@@ -35,3 +35,26 @@ def test_linear_matches_fp64_matmul(ctx, rows, N, K):
     # bf16 products are exact in fp32; only the fp32 summation order differs
     tol = 1e-5 * np.sqrt(K) * max(1.0, np.abs(want).max())
     assert np.abs(got - want).max() <= tol
+
+
+@pytest.mark.parametrize("rows", [1, 11, 40])
+def test_lm_head_argmax_matches_fp64(rows):
+    """LM-head stage alone: tile argmax in the GEMM epilogue + final reduction."""
+    from helpers import argmax_consistent
+    cfg = inputs.ModelConfig(n_layers=1, d_model=256, n_heads=8, n_kv_heads=8, head_dim=32, d_ffn=512,
+                             vocab=5000, rope_theta=10000.0, rms_eps=1e-5)      # 5000 = 39 tiles + ragged tail
+    c, _ = make_pair(cfg, 64, 4, 10, seed=3)
+    g = torch.Generator().manual_seed(rows)
+    X = torch.randn(rows, cfg.d_model, generator=g).to(torch.bfloat16)
+    pad = (rows + 15) // 16 * 16
+    Xd = torch.zeros(pad, cfg.d_model, dtype=torch.bfloat16, device="cuda")
+    Xd[:rows] = X.cuda()
+    logits = torch.zeros(rows, cfg.vocab, dtype=torch.float32, device="cuda")
+    ids = c.cs_lm_head(Xd, rows=rows, logits_dbg=logits)
+    assert c.cs_sync_status() == 0
+    want = X.double().numpy() @ c.weights["lm_head"].cpu().double().numpy().T
+    assert np.abs(logits.cpu().double().numpy() - want).max() <= 1e-4
+    assert not argmax_consistent(want, ids.cpu().tolist(), tol=1e-4)
+    ids2 = c.cs_lm_head(Xd, rows=rows)          # without the debug dump
+    assert ids2.cpu().tolist() == ids.cpu().tolist()
+    c.close()
