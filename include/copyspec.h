@@ -67,7 +67,8 @@ typedef enum {
   CS_ERR_CAPACITY = -3,    /* KV cache, history row or workspace too small                */
   CS_ERR_CUDA = -4,        /* a CUDA runtime/driver call failed (see cs_last_error)       */
   CS_ERR_TIMEOUT = -5,     /* a bounded device-side wait ran out                          */
-  CS_ERR_UNSUPPORTED = -6  /* valid request outside what is built                         */
+  CS_ERR_UNSUPPORTED = -6, /* valid request outside what is built                         */
+  CS_ERR_LIMIT = -7        /* size beyond the built-in maximum of cs_lm_head_static       */
 } cs_status;
 
 /* Which occurrence is used when the last gamma tokens recur more than once.  The paper
@@ -243,6 +244,32 @@ cs_status cs_linear(cs_ctx* ctx, const void* X, const void* W, int rows, int N, 
  * work of the context.  rows <= 256.  Async. */
 cs_status cs_lm_head(cs_ctx* ctx, const void* X, int rows, int32_t* ids, float* logits_dbg,
                      void* stream);
+
+/* cs_lm_head for callers that cannot allocate device memory (the paper has no counterpart:
+ * this is a deployment convenience, not a step of the method).
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - inside another framework's
+ * allocator or stream callback, in a plug-in that is handed input and output buffers but
+ * owns no allocator, or in a process whose device memory is already fully committed.  Such
+ * a caller cannot provide the workspace cs_create asks for.  This call needs no context and
+ * no workspace: the per-tile (max logit, token id) pairs it needs between the GEMM and the
+ * final reduction live in a fixed 512 KB array inside the library image, which every GPU
+ * that loads the library holds until the process exits.  It calls no allocating routine.
+ *
+ *   X bf16 [rows][d_model] (readable for ceil(rows/16)*16 rows), W bf16 [vocab][d_model]
+ *   (the LM head, 16-byte aligned), ids int32 [rows]: the lowest token id with the largest
+ *   logit of X[r] . W^T.  d_model a multiple of 8.  Async on `stream`.
+ *   Limits: rows <= 64 and vocab <= 131072; anything larger returns CS_ERR_LIMIT and does
+ *   nothing.  Other errors: CS_ERR_ARG, CS_ERR_CUDA.  A row whose GEMM gave up on a bounded
+ *   wait gets id -2.
+ *
+ * The first call on a device looks up the array's device address (and raises the kernel's
+ * shared-memory limit); make that first call outside any stream capture.  All calls share
+ * the one array, which keeps the previous call's contents (only its status word is cleared
+ * per call): two calls that overlap on the GPU - different streams, or threads - race on it
+ * and give wrong tokens.  Keep calls on one stream, or order them yourself. */
+cs_status cs_lm_head_static(const void* X, const void* W, int rows, int vocab, int d_model,
+                            int32_t* ids, void* stream);
 
 #ifdef __cplusplus
 }

@@ -13,11 +13,12 @@ from . import build as _build
 
 CS_OK = 0
 CS_ERR_ARG, CS_ERR_SHAPE, CS_ERR_CAPACITY, CS_ERR_CUDA, CS_ERR_TIMEOUT, CS_ERR_UNSUPPORTED = -1, -2, -3, -4, -5, -6
+CS_ERR_LIMIT = -7
 LATEST, FIRST = 0, 1
 TAU_HIST = 65
 
 _STATUS = {0: "CS_OK", -1: "CS_ERR_ARG", -2: "CS_ERR_SHAPE", -3: "CS_ERR_CAPACITY", -4: "CS_ERR_CUDA",
-           -5: "CS_ERR_TIMEOUT", -6: "CS_ERR_UNSUPPORTED"}
+           -5: "CS_ERR_TIMEOUT", -6: "CS_ERR_UNSUPPORTED", -7: "CS_ERR_LIMIT"}
 
 
 class CsError(RuntimeError):
@@ -49,7 +50,7 @@ class CsStats(C.Structure):
 EXPORTS = ("cs_workspace_bytes", "cs_create", "cs_destroy", "cs_last_error", "cs_sync_status",
            "cs_find_match", "cs_verify_step", "cs_kv_truncate", "cs_decode_loop", "cs_prefill", "cs_linear",
            "cs_loop_begin", "cs_loop_steps", "cs_loop_poll", "cs_loop_end", "cs_profile_verify_step",
-           "cs_loop_launches_per_step", "cs_lm_head")
+           "cs_loop_launches_per_step", "cs_lm_head", "cs_lm_head_static")
 
 _lib = None
 
@@ -104,6 +105,8 @@ def load(build_if_missing: bool = True) -> C.CDLL:
     lib.cs_prefill.argtypes = [vp, ip, ip, i, i, i, vp, ip, vp]
     lib.cs_lm_head.restype = i
     lib.cs_lm_head.argtypes = [vp, vp, i, ip, vp, vp]
+    lib.cs_lm_head_static.restype = i
+    lib.cs_lm_head_static.argtypes = [vp, vp, i, i, i, ip, vp]
     lib.cs_linear.restype = i
     lib.cs_linear.argtypes = [vp, vp, vp, i, i, i, vp, vp]
     _lib = lib
@@ -160,6 +163,21 @@ def pack_gate_up(w_gate_up, d_ffn):
     pad[:d_ffn] = w_gate_up[d_ffn:]
     out[:, 1] = pad.view(nb, 64, d)
     return out.view(nb * 128, d).contiguous()
+
+
+def cs_lm_head_static(X, W, ids, rows=None):
+    """Greedy token ids of bf16 rows X under the LM head W, written into the caller's `ids`.
+    For callers that may not allocate: needs no Context and no workspace, and this wrapper
+    itself allocates nothing - X, W and ids are all the caller's tensors.  Limits: rows <= 64,
+    vocab <= 131072 (CsError with CS_ERR_LIMIT beyond).  Calls share one fixed scratch array
+    inside the library, so keep them on one stream."""
+    lib = load()
+    rows = X.shape[0] if rows is None else rows
+    vocab, d = W.shape
+    rc = lib.cs_lm_head_static(_ptr(X), _ptr(W), rows, vocab, d, _i32(ids, "ids"), _stream())
+    if rc != CS_OK:
+        raise CsError(rc, "cs_lm_head_static")
+    return ids
 
 
 class Context:

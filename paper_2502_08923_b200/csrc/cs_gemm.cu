@@ -534,3 +534,133 @@ cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX,
   CS_CUDA_OK(ctx, cudaLaunchKernelEx(&lc, k_gemm_tc, g->tmW, *tmX, a));
   return CS_OK;
 }
+
+// ------------------------------------------------------------------------------------------
+// cs_lm_head_static: the LM-head argmax stage for callers that may not allocate.
+//
+// The tile-argmax epilogue above needs somewhere to put one (max logit, token id) pair per
+// 128-token-id tile and row before the final reduction.  Every other entry point takes that
+// room from the workspace the caller allocated for cs_create.  This one takes it from a fixed
+// array that is part of the library image, so a caller that cannot obtain device memory of
+// its own at that moment (inside a memory-pool callback, in a plug-in that is handed input and
+// output buffers but no allocator, late in a process whose memory is fully committed) can
+// still ask for greedy tokens.  The price: a fixed maximum size, 512 KB held on every GPU
+// that loads the library until the process exits, and one array shared by all calls.
+namespace {
+
+constexpr int kStaticMaxRows = 64;                       // rows per call
+constexpr int kStaticMaxTiles = 1024;                    // 128-id tiles: vocab <= 131072
+constexpr size_t kStaticMaxBytes = (size_t)kStaticMaxTiles * kStaticMaxRows * 4;
+// [tile maxima fp32][tile ids int32][status word + padding]
+static __device__ __align__(256) unsigned char g_lm_scratch[2 * kStaticMaxBytes + 256];
+
+// Host code must not pass `g_lm_scratch` itself to a kernel: on the host that name is only a
+// handle for the runtime.  The device address is looked up once per device and kept here.
+constexpr int kMaxDevices = 64;
+void* g_lm_scratch_dev[kMaxDevices] = {nullptr};
+
+cs_status static_scratch(void** out) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return CS_ERR_CUDA;
+  if (g_lm_scratch_dev[dev] == nullptr) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_lm_scratch) != cudaSuccess || p == nullptr) return CS_ERR_CUDA;
+    if (cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+      return CS_ERR_CUDA;
+    g_lm_scratch_dev[dev] = p;
+  }
+  *out = g_lm_scratch_dev[dev];
+  return CS_OK;
+}
+
+// greedy token per row from the per-tile pairs; -2 marks a row whose GEMM gave up on a wait
+__global__ void __launch_bounds__(128)
+k_tile_reduce_static(const float* __restrict__ tile_max, const int* __restrict__ tile_idx, int tiles,
+                     int tile_stride, const int* __restrict__ status, int* __restrict__ ids) {
+  CS_PDL_PROLOGUE();
+  const int row = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  float val = -INFINITY;
+  int idx = INT32_MAX;
+  for (int t = threadIdx.x; t < tiles; t += 128) {
+    const float v = tile_max[(size_t)t * tile_stride + row];
+    const int id = tile_idx[(size_t)t * tile_stride + row];
+    if (v > val || (v == val && id < idx)) { val = v; idx = id; }
+  }
+  __shared__ float sv[4];
+  __shared__ int si[4];
+  for (int off = 16; off > 0; off >>= 1) {
+    const float ov = __shfl_xor_sync(0xffffffffu, val, off);
+    const int oi = __shfl_xor_sync(0xffffffffu, idx, off);
+    if (ov > val || (ov == val && oi < idx)) { val = ov; idx = oi; }
+  }
+  if (lane == 0) { sv[warp] = val; si[warp] = idx; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < 4; ++w)
+      if (sv[w] > val || (sv[w] == val && si[w] < idx)) { val = sv[w]; idx = si[w]; }
+    ids[row] = (*status != 0) ? -2 : ((idx == INT32_MAX) ? -1 : idx);
+  }
+}
+
+}  // namespace
+
+extern "C" cs_status cs_lm_head_static(const void* X, const void* W, int rows, int vocab, int d_model,
+                                       int32_t* ids, void* stream) {
+  if (X == nullptr || W == nullptr || ids == nullptr || rows < 1 || vocab < 1 || d_model < 8 || (d_model % 8))
+    return CS_ERR_ARG;
+  const int tiles = cs_ceil_div(vocab, CS_GEMM_BM);
+  if (rows > kStaticMaxRows || tiles > kStaticMaxTiles) return CS_ERR_LIMIT;
+  void* scratch = nullptr;
+  cs_status s = static_scratch(&scratch);
+  if (s != CS_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  float* tile_max = static_cast<float*>(scratch);
+  int* tile_idx = reinterpret_cast<int*>(static_cast<unsigned char*>(scratch) + kStaticMaxBytes);
+  int* status = reinterpret_cast<int*>(static_cast<unsigned char*>(scratch) + 2 * kStaticMaxBytes);
+  // the array keeps whatever the last call left: the status word is the only part that is
+  // read before it is written, so it is the only part cleared
+  if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return CS_ERR_CUDA;
+
+  cs_ctx err_sink;                      // only its error string is touched by the encoder
+  err_sink.err[0] = 0;
+  CUtensorMap tmW, tmX;
+  GemmArgs a;
+  a.rows = rows;
+  a.n_tok = cs_ceil_div(rows, 16) * 16;
+  if ((s = encode_2d(&err_sink, &tmW, W, vocab, d_model, CS_GEMM_BM, true)) != CS_OK) return s;
+  if ((s = encode_2d(&err_sink, &tmX, X, a.n_tok, d_model, a.n_tok, false)) != CS_OK) return s;
+  a.N = vocab;
+  a.K = d_model;
+  a.num_kb = cs_ceil_div(d_model, CS_GEMM_BK);
+  a.kb_per_split = a.num_kb;
+  a.splits = 1;
+  a.mode = CS_EPI_ARGMAX;
+  a.out = nullptr;
+  a.act = nullptr;
+  a.F = 0;
+  a.tile_max = tile_max;
+  a.tile_idx = tile_idx;
+  a.tile_stride = kStaticMaxRows;
+  a.status = status;
+  const int stage_bytes = kTileABytes + a.n_tok * 128;
+  const int fixed = 1024 + (2 * 8 + 1) * 8 + 16 + 8 * a.n_tok * 4;
+  int stages = (100 * 1024 - fixed) / stage_bytes;
+  if (stages > 8) stages = 8;
+  if (stages < 2) return CS_ERR_UNSUPPORTED;
+  a.stages = stages;
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = dim3(tiles, 1, 1);
+  lc.blockDim = dim3(kThreads, 1, 1);
+  lc.dynamicSmemBytes = (size_t)fixed + (size_t)stages * stage_bytes;
+  lc.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = at;
+  lc.numAttrs = 1;
+  if (cudaLaunchKernelEx(&lc, k_gemm_tc, tmW, tmX, a) != cudaSuccess) return CS_ERR_CUDA;
+  if (cs_launch_pdl(k_tile_reduce_static, dim3(rows), dim3(128), 0, st, (const float*)tile_max,
+                    (const int*)tile_idx, tiles, kStaticMaxRows, (const int*)status, ids) != cudaSuccess)
+    return CS_ERR_CUDA;
+  return CS_OK;
+}
