@@ -213,6 +213,20 @@ def run_reference(args):
     return 0
 
 
+def aggregate_replicas(ms_local, emitted_local, world, device):
+    """Replicas share nothing: the job's time is the slowest rank's, its tokens the sum over
+    ranks.  Returns (ms, tokens per second of the whole job)."""
+    import torch
+    import torch.distributed as dist
+    if world == 1:
+        return ms_local, emitted_local / (ms_local * 1e-3)
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    n = torch.tensor([float(emitted_local)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(n, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(n.item()) / (float(t.item()) * 1e-3)
+
+
 # ------------------------------------------------------------------------ CUDA leg
 def run_ours(args):
     import torch
@@ -278,11 +292,7 @@ def run_ours(args):
     expect = sum(t + 1 for t in taus[W:W + K])
     if steps_run != K or emitted != expect:
         raise RuntimeError(f"loop ran {steps_run} steps / {emitted} tokens, expected {K} / {expect}")
-    if world > 1:
-        t = torch.tensor([ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    value = world * emitted / (ms * 1e-3)
+    ms, value = aggregate_replicas(ms, emitted, world, dev)
 
     # ---- end to end from pinned host buffers (search + verify per step, host bookkeeping)
     Ke = min(K, 50)
