@@ -1,0 +1,76 @@
+"""Parity at the benchmark's full size (8B-class shape, KV 4,096, block of 11 rows), in the
+launch configuration bench.py times.  Integer outputs of the scripted loop are compared with
+the oracle's model-free simulator exactly; the logits of one verification step of the whole
+32-layer model are compared with the oracle within the logit tolerance."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import copyspec_oracle as O
+from paper_2502_08923_b200 import binding as cs, inputs
+from helpers import LOGIT_TOL, argmax_consistent, i32
+
+pytestmark = pytest.mark.gpu
+
+GAMMA, K = 3, 10
+
+
+@pytest.fixture(scope="module")
+def big():
+    cfg = inputs.LLAMA8B
+    w = inputs.make_weights(cfg, seed=0, device="cuda")
+    taus = [int(t) for t in np.random.default_rng(0).permutation(np.repeat(np.arange(K + 1), 3))]
+    hist, script = inputs.tau_controlled_case(np.random.default_rng(0), taus, GAMMA, K, 4096, cfg.vocab)
+    max_seq = len(hist) + len(script) + K + 64
+    ctx = cs.Context(cfg, w, max_seq=max_seq, max_batch=1, k_max=K)
+    kv = inputs.synthetic_kv(cfg, 1, max_seq, len(hist) - 1, seed=1, device="cuda")
+    yield cfg, w, ctx, kv, hist, script, taus
+    ctx.close()
+
+
+def test_scripted_loop_matches_simulator_at_full_size(big):
+    cfg, w, ctx, kv, hist, script, taus = big
+    n0, max_new = len(hist), len(script)
+    stride = (n0 + max_new + 67) // 4 * 4
+    h = np.zeros((1, stride), dtype=np.int32); h[0, :n0] = hist
+    hd, ld, kvl = i32(h), i32([n0]), i32([n0 - 1])
+    kv_run = kv.clone()
+    st = ctx.cs_decode_loop(hd, ld, kv_run, kvl, GAMMA, K, max_new, script=i32(script[None, :]))
+    steps, st_o, h_sim = O.scripted_simulator(hist, script, GAMMA, K, O.LATEST, max_new)
+    assert [s["tau"] for s in steps] == taus
+    assert hd[0, :int(ld[0])].cpu().tolist() == h_sim
+    assert int(kvl[0]) == int(ld[0]) - 1 == n0 + max_new - 1
+    for key in ("steps", "attempts", "accepted", "emitted", "no_match"):
+        assert st[key] == st_o[key], key
+    assert st["tau_hist"][:K + 1] == st_o["tau_hist"][:K + 1]
+
+
+def test_one_verify_step_logits_against_oracle_at_full_size(big):
+    """All 32 layers and the 128,256-row LM head for one 11-row block over 4,096 cached
+    positions; the oracle converts one layer at a time (about a minute of CPU work)."""
+    cfg, w, ctx, kv, hist, script, taus = big
+    n0 = len(hist)
+    p0 = O.find_match(hist, n0, GAMMA, O.LATEST)
+    draft = O.gather_draft(hist, n0, p0, GAMMA, K)
+    assert len(draft) == K
+    kv_run = kv.clone()
+    kvl = i32([n0 - 1])
+    logits = torch.zeros(1, K + 1, cfg.vocab, dtype=torch.float32, device="cuda")
+    al, ot, am = ctx.cs_verify_step(i32([hist[-1]]), i32(np.asarray(draft)[None, :]), i32([K]), kv_run, kvl,
+                                    logits_dbg=logits)
+    assert ctx.cs_sync_status() == 0
+    model = O.Model(cfg, w, contract=True, cache_weights=False)
+    cache = O.KVCache(cfg, 1, n0 + K + 1, dtype=np.float32)
+    cache.a[:, :, :, :, :n0 - 1, :] = kv[:, :, :, :, :n0 - 1, :].float().cpu().numpy()
+    lg = model.forward_block([int(hist[-1])] + draft, n0 - 1, cache, 0)
+    got = logits[0].cpu().numpy()
+    err = float(np.abs(got - lg).max())
+    assert err <= LOGIT_TOL, err
+    assert not argmax_consistent(lg, am[0].cpu().tolist())
+    # greedy acceptance from those ids
+    tau = O.accept_length(draft, [int(np.argmax(lg[r])) for r in range(K + 1)])
+    assert int(al[0]) == tau or argmax_consistent(lg, am[0].cpu().tolist()) == []
+    # the block's K/V rows landed in the cache within bf16 resolution
+    new = kv_run[:, :, 0, :, n0 - 1:n0 + K, :].float().cpu().numpy()
+    want = cache.a[:, :, 0, :, n0 - 1:n0 + K, :]
+    assert np.abs(new - want).max() <= 2e-2 * max(1.0, float(np.abs(want).max()))
