@@ -46,10 +46,11 @@ WsLayout ws_layout(const cs_model_config* c) {
   const size_t lm_tiles = cs_ceil_div(c->vocab, CS_GEMM_BM);
   size_t off = 0;
   L.x = take(&off, rows * d * 4);
-  L.xn = take(&off, rows * d * 2);
-  L.attn_out = take(&off, rows * qd * 2);
-  L.act = take(&off, rows * F * 2);
-  L.qbuf = take(&off, rows * qd * 2);
+  // operands carried as two bf16 terms: hi rows then lo rows
+  L.xn = take(&off, 2 * rows * d * 2);
+  L.attn_out = take(&off, 2 * rows * qd * 2);
+  L.act = take(&off, 2 * rows * F * 2);
+  L.qbuf = take(&off, 2 * rows * qd * 2);
   L.partial = take(&off, L.qkv_elems * 4);
   L.attn_o = take(&off, (size_t)L.attn_splits * rows * qd * 4);
   L.attn_ml = take(&off, (size_t)L.attn_splits * rows * c->n_heads * 2 * 4);
@@ -86,10 +87,10 @@ cs_status ensure_act_maps(cs_ctx* ctx, int n_tok) {
   if (ctx->act_ntok == n_tok) return CS_OK;
   const cs_model_config& c = ctx->cfg;
   cs_status s;
-  if ((s = cs_make_act_map(ctx, &ctx->tmXn, ctx->xn, CS_MAX_ROWS, c.d_model, n_tok)) != CS_OK) return s;
-  if ((s = cs_make_act_map(ctx, &ctx->tmAttn, ctx->attn_out, CS_MAX_ROWS, c.n_heads * c.head_dim, n_tok)) != CS_OK)
+  if ((s = cs_make_act_map(ctx, &ctx->tmXn, ctx->xn, 2 * CS_MAX_ROWS, c.d_model, n_tok)) != CS_OK) return s;
+  if ((s = cs_make_act_map(ctx, &ctx->tmAttn, ctx->attn_out, 2 * CS_MAX_ROWS, c.n_heads * c.head_dim, n_tok)) != CS_OK)
     return s;
-  if ((s = cs_make_act_map(ctx, &ctx->tmAct, ctx->act, CS_MAX_ROWS, c.d_ffn, n_tok)) != CS_OK) return s;
+  if ((s = cs_make_act_map(ctx, &ctx->tmAct, ctx->act, 2 * CS_MAX_ROWS, c.d_ffn, n_tok)) != CS_OK) return s;
   ctx->act_ntok = n_tok;
   return CS_OK;
 }
@@ -126,7 +127,7 @@ cs_status enqueue_forward(cs_ctx* ctx, int B, int R, void* kv_cache, bool with_l
     cs_launch_rmsnorm(ctx, L.attn_norm, rows, st);
     prof_end(ctx, st);
     prof_begin(ctx, CS_FAM_GEMM, st);
-    s = cs_launch_gemm(ctx, &L.qkv, &ctx->tmXn, rows, CS_EPI_STORE, ctx->qkv, nullptr, 0, st);
+    s = cs_launch_gemm(ctx, &L.qkv, &ctx->tmXn, CS_MAX_ROWS, rows, CS_EPI_STORE, ctx->qkv, nullptr, nullptr, 0, st);
     prof_end(ctx, st);
     if (s != CS_OK) return s;
     prof_begin(ctx, CS_FAM_ELEMENTWISE, st);
@@ -136,18 +137,19 @@ cs_status enqueue_forward(cs_ctx* ctx, int B, int R, void* kv_cache, bool with_l
     cs_launch_attention(ctx, kv_cache, l, B, R, st);
     prof_end(ctx, st);
     prof_begin(ctx, CS_FAM_GEMM, st);
-    s = cs_launch_gemm(ctx, &L.o, &ctx->tmAttn, rows, CS_EPI_RESIDUAL, ctx->x, nullptr, 0, st);
+    s = cs_launch_gemm(ctx, &L.o, &ctx->tmAttn, CS_MAX_ROWS, rows, CS_EPI_RESIDUAL, ctx->x, nullptr, nullptr, 0, st);
     prof_end(ctx, st);
     if (s != CS_OK) return s;
     prof_begin(ctx, CS_FAM_ELEMENTWISE, st);
     cs_launch_rmsnorm(ctx, L.ffn_norm, rows, st);
     prof_end(ctx, st);
     prof_begin(ctx, CS_FAM_GEMM, st);
-    s = cs_launch_gemm(ctx, &L.gate_up, &ctx->tmXn, rows, CS_EPI_SWIGLU, nullptr, ctx->act, c.d_ffn, st);
+    s = cs_launch_gemm(ctx, &L.gate_up, &ctx->tmXn, CS_MAX_ROWS, rows, CS_EPI_SWIGLU, nullptr, ctx->act,
+                       ctx->act + (size_t)CS_MAX_ROWS * c.d_ffn, c.d_ffn, st);
     prof_end(ctx, st);
     if (s != CS_OK) return s;
     prof_begin(ctx, CS_FAM_GEMM, st);
-    s = cs_launch_gemm(ctx, &L.down, &ctx->tmAct, rows, CS_EPI_RESIDUAL, ctx->x, nullptr, 0, st);
+    s = cs_launch_gemm(ctx, &L.down, &ctx->tmAct, CS_MAX_ROWS, rows, CS_EPI_RESIDUAL, ctx->x, nullptr, nullptr, 0, st);
     prof_end(ctx, st);
     if (s != CS_OK) return s;
   }
@@ -156,7 +158,7 @@ cs_status enqueue_forward(cs_ctx* ctx, int B, int R, void* kv_cache, bool with_l
     cs_launch_rmsnorm(ctx, ctx->final_norm, rows, st);
     prof_end(ctx, st);
     prof_begin(ctx, CS_FAM_LMHEAD, st);
-    s = cs_launch_gemm(ctx, &ctx->lm, &ctx->tmXn, rows, CS_EPI_ARGMAX, logits, nullptr, 0, st);
+    s = cs_launch_gemm(ctx, &ctx->lm, &ctx->tmXn, CS_MAX_ROWS, rows, CS_EPI_ARGMAX, logits, nullptr, nullptr, 0, st);
     prof_end(ctx, st);
     if (s != CS_OK) return s;
   }
@@ -536,7 +538,7 @@ cs_status cs_linear(cs_ctx* ctx, const void* X, const void* W, int rows, int N, 
   const int n_tok = cs_ceil_div(rows, 16) * 16;
   CUtensorMap tmX;
   if ((s = cs_make_act_map(ctx, &tmX, X, n_tok, K, n_tok)) != CS_OK) return s;
-  return cs_launch_gemm(ctx, &g, &tmX, rows, CS_EPI_STORE, Y, nullptr, 0, st);
+  return cs_launch_gemm(ctx, &g, &tmX, -1, rows, CS_EPI_STORE, Y, nullptr, nullptr, 0, st);
 }
 
 cs_status cs_lm_head(cs_ctx* ctx, const void* X, int rows, int32_t* ids, float* logits_dbg, void* stream) {
@@ -547,7 +549,7 @@ cs_status cs_lm_head(cs_ctx* ctx, const void* X, int rows, int32_t* ids, float* 
   CUtensorMap tmX;
   cs_status s = cs_make_act_map(ctx, &tmX, X, n_tok, ctx->cfg.d_model, n_tok);
   if (s != CS_OK) return s;
-  if ((s = cs_launch_gemm(ctx, &ctx->lm, &tmX, rows, CS_EPI_ARGMAX, logits_dbg, nullptr, 0, st)) != CS_OK) return s;
+  if ((s = cs_launch_gemm(ctx, &ctx->lm, &tmX, -1, rows, CS_EPI_ARGMAX, logits_dbg, nullptr, nullptr, 0, st)) != CS_OK) return s;
   cs_launch_tile_reduce(ctx, rows, ids, st);
   CS_CUDA_OK(ctx, cudaGetLastError());
   return CS_OK;

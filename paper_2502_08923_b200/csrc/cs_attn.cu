@@ -6,7 +6,8 @@
 // One CTA = one (sequence, KV head), one slice of the key range (split-KV) and up to 64
 // query rows; each of its four warps owns 16 query rows and runs a register-resident
 // flash-attention loop on bf16 tensor-core MMAs (m16n8k16, fp32 accumulation): S = Q K^T,
-// running row max / sum, P rounded to bf16, O += P V.  K and V tiles of 64 keys stream
+// running row max / sum, O += P V; Q and P enter the MMAs as two bf16 terms each (value =
+// hi + lo), so only K and V - which the cache stores in bf16 - are rounded.  K and V tiles of 64 keys stream
 // through a double-buffered cp.async pipeline in shared memory (rows padded by 16 bytes so
 // that fragment loads and ldmatrix are bank-conflict free).  Each slice writes its
 // un-normalised output and (max, sum); k_attn_merge combines the slices.
@@ -44,6 +45,15 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void* 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+// (lo, hi) as a leading bf16 pair plus the bf16 pair of what that rounding lost
+__device__ __forceinline__ void pack_two(float lo, float hi, uint32_t& first, uint32_t& second) {
+  const __nv_bfloat162 a = __floats2bfloat162_rn(lo, hi);
+  const float2 af = __bfloat1622float2(a);
+  const __nv_bfloat162 b = __floats2bfloat162_rn(lo - af.x, hi - af.y);
+  first = *reinterpret_cast<const uint32_t*>(&a);
+  second = *reinterpret_cast<const uint32_t*>(&b);
 }
 
 template <int DH>
@@ -91,16 +101,22 @@ k_attn_mma(const __nv_bfloat16* __restrict__ qbuf, const __nv_bfloat16* __restri
   const int head_lo = v_lo ? kvh * G + q_lo / R : 0, head_hi = v_hi ? kvh * G + q_hi / R : 0;
   const int lim_lo = v_lo ? row_lim[grow_lo] : 0, lim_hi = v_hi ? row_lim[grow_hi] : 0;
 
-  uint32_t qa[KSTEPS][4];
+  // queries come as two bf16 terms (q = qa + qb): two MMAs give the product of the fp32 query
+  uint32_t qa[KSTEPS][4], qb[KSTEPS][4];
   {
     const __nv_bfloat16* ql = qbuf + ((size_t)grow_lo * H + head_lo) * DH;
     const __nv_bfloat16* qh = qbuf + ((size_t)grow_hi * H + head_hi) * DH;
+    const size_t second = (size_t)CS_MAX_ROWS * H * DH;
 #pragma unroll
     for (int ks = 0; ks < KSTEPS; ++ks) {
       qa[ks][0] = v_lo ? *reinterpret_cast<const uint32_t*>(ql + ks * 16 + 2 * t) : 0u;
       qa[ks][1] = v_hi ? *reinterpret_cast<const uint32_t*>(qh + ks * 16 + 2 * t) : 0u;
       qa[ks][2] = v_lo ? *reinterpret_cast<const uint32_t*>(ql + ks * 16 + 8 + 2 * t) : 0u;
       qa[ks][3] = v_hi ? *reinterpret_cast<const uint32_t*>(qh + ks * 16 + 8 + 2 * t) : 0u;
+      qb[ks][0] = v_lo ? *reinterpret_cast<const uint32_t*>(ql + second + ks * 16 + 2 * t) : 0u;
+      qb[ks][1] = v_hi ? *reinterpret_cast<const uint32_t*>(qh + second + ks * 16 + 2 * t) : 0u;
+      qb[ks][2] = v_lo ? *reinterpret_cast<const uint32_t*>(ql + second + ks * 16 + 8 + 2 * t) : 0u;
+      qb[ks][3] = v_hi ? *reinterpret_cast<const uint32_t*>(qh + second + ks * 16 + 8 + 2 * t) : 0u;
     }
   }
 
@@ -146,7 +162,9 @@ k_attn_mma(const __nv_bfloat16* __restrict__ qbuf, const __nv_bfloat16* __restri
 #pragma unroll
       for (int ks = 0; ks < KSTEPS; ++ks) {
         const __nv_bfloat16* kp = kt + (nb * 8 + g) * STRIDE + ks * 16 + 2 * t;
-        mma_bf16(s[nb], qa[ks], *reinterpret_cast<const uint32_t*>(kp), *reinterpret_cast<const uint32_t*>(kp + 8));
+        const uint32_t k0 = *reinterpret_cast<const uint32_t*>(kp), k1 = *reinterpret_cast<const uint32_t*>(kp + 8);
+        mma_bf16(s[nb], qa[ks], k0, k1);
+        mma_bf16(s[nb], qb[ks], k0, k1);
       }
     }
     // scale (log2 domain), causal mask, running max
@@ -187,11 +205,12 @@ k_attn_mma(const __nv_bfloat16* __restrict__ qbuf, const __nv_bfloat16* __restri
     // O += P V: the S accumulators are already laid out as the A fragments of the next MMA
 #pragma unroll
     for (int j = 0; j < kKeys / 16; ++j) {
-      uint32_t pa[4];
-      pa[0] = pack_bf16(s[2 * j][0], s[2 * j][1]);
-      pa[1] = pack_bf16(s[2 * j][2], s[2 * j][3]);
-      pa[2] = pack_bf16(s[2 * j + 1][0], s[2 * j + 1][1]);
-      pa[3] = pack_bf16(s[2 * j + 1][2], s[2 * j + 1][3]);
+      // softmax weights as two bf16 terms as well
+      uint32_t pa[4], pb[4];
+      pack_two(s[2 * j][0], s[2 * j][1], pa[0], pb[0]);
+      pack_two(s[2 * j][2], s[2 * j][3], pa[1], pb[1]);
+      pack_two(s[2 * j + 1][0], s[2 * j + 1][1], pa[2], pb[2]);
+      pack_two(s[2 * j + 1][2], s[2 * j + 1][3], pa[3], pb[3]);
 #pragma unroll
       for (int nd = 0; nd < NB_O; nd += 2) {
         // four transposed 8x8 blocks of V: keys 16j..16j+15, dims nd*8 .. nd*8+15
@@ -199,7 +218,9 @@ k_attn_mma(const __nv_bfloat16* __restrict__ qbuf, const __nv_bfloat16* __restri
         const int mi = lane >> 3, r8 = lane & 7;
         ldmatrix_x4_trans(vb, vt + (j * 16 + (mi & 1) * 8 + r8) * STRIDE + (nd + (mi >> 1)) * 8);
         mma_bf16(o[nd], pa, vb[0], vb[1]);
+        mma_bf16(o[nd], pb, vb[0], vb[1]);
         mma_bf16(o[nd + 1], pa, vb[2], vb[3]);
+        mma_bf16(o[nd + 1], pb, vb[2], vb[3]);
       }
     }
     __syncthreads();   // everyone is done with this stage before it is refilled

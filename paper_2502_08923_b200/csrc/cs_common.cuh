@@ -77,10 +77,11 @@ struct cs_ctx {
   char* ws;
   size_t ws_bytes;
   float* x;                  // residual stream fp32 [rows_pad][d]
-  __nv_bfloat16* xn;         // normed activations bf16 [rows_pad][d]
-  __nv_bfloat16* attn_out;   // attention output bf16 [rows_pad][H*Dh]
-  __nv_bfloat16* act;        // SwiGLU output bf16 [rows_pad][F]
-  __nv_bfloat16* qbuf;       // rotated queries bf16 [rows_pad][H*Dh]
+  // GEMM / attention operands as two bf16 terms: rows [0, 256) = hi, rows [256, 512) = lo
+  __nv_bfloat16* xn;         // normed activations [2*rows_pad][d]
+  __nv_bfloat16* attn_out;   // attention output [2*rows_pad][H*Dh]
+  __nv_bfloat16* act;        // SwiGLU output [2*rows_pad][F]
+  __nv_bfloat16* qbuf;       // rotated queries [2*rows_pad][H*Dh]
   float* qkv;                // QKV projection output fp32 [rows][(H+2Hkv)*Dh]; scratch of cs_linear
   size_t qkv_elems;
   float* attn_o;             // split-KV partial outputs [splits][rows][H][Dh]
@@ -175,8 +176,9 @@ cs_status cs_make_act_map(cs_ctx* ctx, CUtensorMap* tm, const void* base, int ro
                           int box_rows);
 // mode = CS_EPI_*: `out` is the fp32 destination (STORE, RESIDUAL) or the optional logits dump
 // (ARGMAX); `act`/F the bf16 destination of SWIGLU
-cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX, int rows, int mode,
-                         float* out, __nv_bfloat16* act, int F, cudaStream_t st);
+// lo_row: row coordinate (in tmX) of the activation operand's second bf16 term, -1 if X is plain bf16
+cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX, int lo_row, int rows, int mode,
+                         float* out, __nv_bfloat16* act, __nv_bfloat16* act_lo, int F, cudaStream_t st);
 // cs_layers.cu
 void cs_launch_block_setup(cs_ctx* ctx, const int32_t* last_tok, const int32_t* draft,
                            const int32_t* draft_len, const int32_t* kv_len, const int32_t* skip,

@@ -6,7 +6,10 @@
 // 16), so even an 11-row block fills the 128 TMEM lanes.  Weights and activations arrive
 // as TMA tiles of 64 K-elements (one 128-byte swizzled row per feature / token) through an
 // mbarrier ring; one thread issues tcgen05.mma into a TMEM accumulator; four warps read
-// it back with tcgen05.ld.
+// it back with tcgen05.ld.  Activations are carried as two bf16 terms (x = hi + lo, lo being
+// the rounding error of hi): both tiles are loaded and multiplied against the same weight
+// tile, so the product is that of the fp32 activation although the operands are bf16.  The
+// extra MMAs are free here: the kernel waits for weight bytes, not for the tensor pipe.
 //
 // K is split across the CTAs of a thread-block cluster (cluster dims (1, S, 1), S <= 8) so
 // that every GEMM puts about two CTAs on each SM.  Each CTA leaves its partial tile in its
@@ -45,7 +48,9 @@ struct GemmArgs {
   int rows, n_tok, N, K;
   int num_kb, kb_per_split, splits, stages, mode;
   float* out;            // STORE / RESIDUAL: [rows][N] fp32; ARGMAX: optional logits [rows][N]
-  __nv_bfloat16* act;    // SWIGLU: [rows][F] bf16
+  __nv_bfloat16* act;    // SWIGLU: [rows][F] bf16 (leading term)
+  __nv_bfloat16* act_lo; // SWIGLU: second bf16 term of the same values, or NULL
+  int lo_row;            // row coordinate of the activation operand's second bf16 term, -1 = none
   int F;
   float* tile_max;       // ARGMAX: [tiles][tile_stride]
   int* tile_idx;
@@ -167,7 +172,9 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   uint8_t* smem = smem_raw + (((raw + 1023u) & ~1023u) - raw);   // operand tiles need 1024-byte alignment
-  const int stage_bytes = kTileABytes + a.n_tok * 128;
+  const int xtile = a.n_tok * 128;                 // one activation tile
+  const bool two = a.lo_row >= 0;                   // activations come as two bf16 terms
+  const int stage_bytes = kTileABytes + (two ? 2 : 1) * xtile;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)a.stages * stage_bytes);
   // bars[0..stages) = tile landed, bars[stages..2*stages) = tile consumed, bars[2*stages] = accumulator done
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * a.stages + 1);
@@ -224,8 +231,11 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
       }
       asm volatile("griddepcontrol.wait;" ::: "memory");
       for (int i = 0; i < npre; ++i)
-        tma_load_2d(smem_u32(smem + (size_t)i * stage_bytes) + kTileABytes, &tmX, bar_full + 8 * i,
-                    (kb0 + i) * CS_GEMM_BK, 0);
+      {
+        const uint32_t sx = smem_u32(smem + (size_t)i * stage_bytes) + kTileABytes;
+        tma_load_2d(sx, &tmX, bar_full + 8 * i, (kb0 + i) * CS_GEMM_BK, 0);
+        if (two) tma_load_2d(sx + xtile, &tmX, bar_full + 8 * i, (kb0 + i) * CS_GEMM_BK, a.lo_row);
+      }
       int i = npre;
       for (; i < nkb; ++i) {
         const int s = i % a.stages;
@@ -235,6 +245,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
         mbar_expect_tx(bar_full + 8 * s, (uint32_t)stage_bytes);
         tma_load_2d(sa, &tmW, bar_full + 8 * s, (kb0 + i) * CS_GEMM_BK, n0);
         tma_load_2d(sa + kTileABytes, &tmX, bar_full + 8 * s, (kb0 + i) * CS_GEMM_BK, 0);
+        if (two) tma_load_2d(sa + kTileABytes + xtile, &tmX, bar_full + 8 * s, (kb0 + i) * CS_GEMM_BK, a.lo_row);
       }
       if (!ok) {
         *s_abort = 1;
@@ -258,10 +269,13 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
         if (!mbar_wait(bar_full + 8 * s, ph, s_abort)) { ok = false; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
-        const uint64_t da = umma_desc(sa), db = umma_desc(sa + kTileABytes);
+        const uint64_t da = umma_desc(sa), db = umma_desc(sa + kTileABytes),
+                       dl = umma_desc(sa + kTileABytes + xtile);
 #pragma unroll
-        for (int kk = 0; kk < CS_GEMM_BK / 16; ++kk)   // 16 K-elements = 32 bytes per instruction
+        for (int kk = 0; kk < CS_GEMM_BK / 16; ++kk) {   // 16 K-elements = 32 bytes per instruction
           umma_bf16(tmem_base, da + 2 * kk, db + 2 * kk, idesc, (i > 0 || kk > 0) ? 1u : 0u);
+          if (two) umma_bf16(tmem_base, da + 2 * kk, dl + 2 * kk, idesc, 1u);   // x = hi + lo
+        }
         umma_commit(bar_empty + 8 * s);
       }
       if (!ok) {
@@ -355,7 +369,12 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             const int jj = tile * 64 + j + i;
-            if (jj < a.F) a.act[(size_t)tok * a.F + jj] = __float2bfloat16_rn(gv[i] / (1.f + expf(-gv[i])) * uv[i]);
+            if (jj < a.F) {
+              const float v = gv[i] / (1.f + expf(-gv[i])) * uv[i];
+              const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+              a.act[(size_t)tok * a.F + jj] = hi;
+              if (a.act_lo != nullptr) a.act_lo[(size_t)tok * a.F + jj] = __float2bfloat16_rn(v - __bfloat162float(hi));
+            }
           }
         }
       } else {
@@ -474,8 +493,8 @@ cs_status cs_make_act_map(cs_ctx* ctx, CUtensorMap* tm, const void* base, int ro
   return encode_2d(ctx, tm, base, rows_total, K, box_rows, false);
 }
 
-cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX, int rows, int mode,
-                         float* out, __nv_bfloat16* act, int F, cudaStream_t st) {
+cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX, int lo_row, int rows, int mode,
+                         float* out, __nv_bfloat16* act, __nv_bfloat16* act_lo, int F, cudaStream_t st) {
   const int tiles = cs_ceil_div(g->N, CS_GEMM_BM);
   GemmArgs a;
   a.rows = rows;
@@ -488,12 +507,14 @@ cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX,
   a.mode = mode;
   a.out = out;
   a.act = act;
+  a.act_lo = act_lo;
+  a.lo_row = lo_row;
   a.F = F;
   a.tile_max = ctx->tile_max;
   a.tile_idx = ctx->tile_idx;
   a.tile_stride = ctx->rows_pad;
   a.status = ctx->d_status;
-  const int stage_bytes = kTileABytes + a.n_tok * 128;
+  const int stage_bytes = kTileABytes + (lo_row >= 0 ? 2 : 1) * a.n_tok * 128;
   const int fixed = 1024 /*alignment slack*/ + (2 * 8 + 1) * 8 + 16 + 8 * a.n_tok * 4;
   // small blocks: two CTAs per SM (about 100 KB each); large blocks: one CTA with the whole SM
   int stages = (100 * 1024 - fixed) / stage_bytes;
@@ -637,6 +658,8 @@ extern "C" cs_status cs_lm_head_static(const void* X, const void* W, int rows, i
   a.mode = CS_EPI_ARGMAX;
   a.out = nullptr;
   a.act = nullptr;
+  a.act_lo = nullptr;
+  a.lo_row = -1;
   a.F = 0;
   a.tile_max = tile_max;
   a.tile_idx = tile_idx;

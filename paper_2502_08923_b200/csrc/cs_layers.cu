@@ -97,10 +97,10 @@ __global__ void k_embed(const __nv_bfloat16* __restrict__ E, const int* __restri
   }
 }
 
-// xn = bf16(x * rsqrt(mean(x^2) + eps) * g).  One CTA per row.
+// xn = x * rsqrt(mean(x^2) + eps) * g as two bf16 terms (hi, lo).  One CTA per row.
 __global__ void __launch_bounds__(256)
 k_rmsnorm(const float* __restrict__ x, int d, const __nv_bfloat16* __restrict__ gain, float eps,
-          __nv_bfloat16* __restrict__ xn) {
+          __nv_bfloat16* __restrict__ xn, __nv_bfloat16* __restrict__ xn_lo) {
   CS_PDL_PROLOGUE();
   const int row = blockIdx.x;
   const float* xr = x + (size_t)row * d;
@@ -125,10 +125,14 @@ k_rmsnorm(const float* __restrict__ x, int d, const __nv_bfloat16* __restrict__ 
     const float4 v = *reinterpret_cast<const float4*>(xr + i);
     const float2 g0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(gain + i));
     const float2 g1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(gain + i + 2));
-    __nv_bfloat162 o0 = __floats2bfloat162_rn(v.x * sc * g0.x, v.y * sc * g0.y);
-    __nv_bfloat162 o1 = __floats2bfloat162_rn(v.z * sc * g1.x, v.w * sc * g1.y);
+    const float y0 = v.x * sc * g0.x, y1 = v.y * sc * g0.y, y2 = v.z * sc * g1.x, y3 = v.w * sc * g1.y;
+    const __nv_bfloat162 o0 = __floats2bfloat162_rn(y0, y1), o1 = __floats2bfloat162_rn(y2, y3);
     *reinterpret_cast<__nv_bfloat162*>(xn + (size_t)row * d + i) = o0;
     *reinterpret_cast<__nv_bfloat162*>(xn + (size_t)row * d + i + 2) = o1;
+    // second term: what the first rounding lost
+    const float2 h0 = __bfloat1622float2(o0), h1 = __bfloat1622float2(o1);
+    *reinterpret_cast<__nv_bfloat162*>(xn_lo + (size_t)row * d + i) = __floats2bfloat162_rn(y0 - h0.x, y1 - h0.y);
+    *reinterpret_cast<__nv_bfloat162*>(xn_lo + (size_t)row * d + i + 2) = __floats2bfloat162_rn(y2 - h1.x, y3 - h1.y);
   }
 }
 
@@ -146,8 +150,13 @@ __global__ void k_qkv_post(const float* __restrict__ qkv, int H, int Hkv, int Dh
   const float c = rope_cs[2 * (row * half + i)], sn = rope_cs[2 * (row * half + i) + 1];
   if (head < H) {
     __nv_bfloat16* q = qbuf + (size_t)row * H * Dh + (size_t)head * Dh;
-    q[i] = __float2bfloat16_rn(a * c - b * sn);
-    q[i + half] = __float2bfloat16_rn(b * c + a * sn);
+    __nv_bfloat16* ql = q + (size_t)CS_MAX_ROWS * H * Dh;      // second bf16 term
+    const float r0 = a * c - b * sn, r1 = b * c + a * sn;
+    const __nv_bfloat16 h0 = __float2bfloat16_rn(r0), h1 = __float2bfloat16_rn(r1);
+    q[i] = h0;
+    q[i + half] = h1;
+    ql[i] = __float2bfloat16_rn(r0 - __bfloat162float(h0));
+    ql[i + half] = __float2bfloat16_rn(r1 - __bfloat162float(h1));
     return;
   }
   if (!row_write[row]) return;
@@ -196,7 +205,9 @@ __global__ void k_attn_merge(const float* __restrict__ in_o, const float* __rest
     const float w = __shfl_sync(0xffffffffu, s < 32 ? w0 : w1, s & 31);
     acc = fmaf(src[(size_t)s * stride], w, acc);
   }
-  attn_out[((size_t)row * H + h) * Dh + dd] = __float2bfloat16_rn(acc);
+  const __nv_bfloat16 hi = __float2bfloat16_rn(acc);
+  attn_out[((size_t)row * H + h) * Dh + dd] = hi;
+  attn_out[((size_t)(CS_MAX_ROWS + row) * H + h) * Dh + dd] = __float2bfloat16_rn(acc - __bfloat162float(hi));
 }
 
 // ------------------------------------------------------------------ acceptance
@@ -398,7 +409,8 @@ void cs_launch_embed(cs_ctx* ctx, int rows, cudaStream_t st) {
 }
 
 void cs_launch_rmsnorm(cs_ctx* ctx, const __nv_bfloat16* gain, int rows, cudaStream_t st) {
-  cs_launch_pdl(k_rmsnorm, dim3(rows), dim3(256), 0, st, ctx->x, ctx->cfg.d_model, gain, ctx->cfg.rms_eps, ctx->xn);
+  cs_launch_pdl(k_rmsnorm, dim3(rows), dim3(256), 0, st, ctx->x, ctx->cfg.d_model, gain, ctx->cfg.rms_eps, ctx->xn,
+                ctx->xn + (size_t)CS_MAX_ROWS * ctx->cfg.d_model);
 }
 
 void cs_launch_qkv_post(cs_ctx* ctx, void* kv_cache, int layer, int B, int R, cudaStream_t st) {
