@@ -372,7 +372,7 @@ def run_ours(args):
         if world == 1 and not args.no_cpu_baseline:
             w0 = {"layer": {k2: v.cpu() for k2, v in weights["layers"][0].items()}, "final_norm": weights["final_norm"].cpu()}
             kv0 = kv[0, :, 0, :, :KV_START, :].float().cpu().numpy()
-            res = oracle_sample(cfg, w0, kv0, weights["lm_head"].cpu(), hist, script, taus, 12, 2)
+            res = oracle_sample(cfg, w0, kv0, weights["lm_head"].cpu(), hist, script, taus, 150, 3)
             cpu = {k2: res[k2] for k2 in ("value", "unit", "cores", "kind", "sample")}
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
                 "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
