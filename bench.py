@@ -394,6 +394,112 @@ def run_ours(args):
     return 0
 
 
+
+# ------------------------------------------------------------- the other workloads
+def run_workload(args):
+    """Additional measurements (not the headline line): the long-context and multi-turn loops
+    at full shape, plain one-token decoding from the same kernels, and the search alone."""
+    import torch
+    from paper_2502_08923_b200 import binding as cs, inputs
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    name = args.workload
+    W, K = args.warmup, args.steps
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    if name == "match_search":
+        hist, kinds, _ = inputs.match_search_histories()
+        hd = torch.from_numpy(hist).to(dev)
+        ld = torch.full((64,), 32768, dtype=torch.int32, device=dev)
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+        out = {}
+        for gamma in (3, 5):
+            bufs = cs.cs_find_match(hd, ld, gamma, K_DRAFT)
+            for mode in ("warm", "cold"):
+                ts = []
+                for i in range(W + K):
+                    if mode == "cold":
+                        flush.fill_(i & 1)
+                    e0, e1 = ev(), ev()
+                    e0.record()
+                    cs.cs_find_match(hd, ld, gamma, K_DRAFT, out=bufs)
+                    e1.record()
+                    torch.cuda.synchronize()
+                    if i >= W:
+                        ts.append(e0.elapsed_time(e1) * 1e3)
+                out[f"gamma{gamma}_{mode}_us_per_batch"] = float(np.median(ts))
+        us = out["gamma3_cold_us_per_batch"]
+        line = {"metric": "match-search us/seq", "value": us / 64, "unit": "us", "higher_is_better": False,
+                "n_gpus": 1, "steps": K, "warmup": W, "dtype": "int32", "data": "synthetic",
+                "config": {"workload": "match_search_64x32768_zipf", "k": K_DRAFT, "bytes_per_batch": 64 * 32768 * 4,
+                           "gbs_cold": 64 * 32768 * 4 / us / 1e3, **out}}
+        print(json.dumps(line), flush=True)
+        return 0
+    cfg = inputs.LLAMA8B
+    if name == "long_context_b1_k10":
+        cases, k = [inputs.long_context_case(100)], 10
+    elif name == "long_context_b8_k20":
+        cases, k = [inputs.long_context_case(100 + b) for b in range(8)], 20
+    elif name == "multi_turn_b16_k10":
+        cases, k = [inputs.multi_turn_case(200 + b)[:2] for b in range(16)], 10
+    elif name == "verify_plain_decode":
+        taus = _taus(W + K)
+        cases, k = [inputs.tau_controlled_case(np.random.default_rng(0), taus, GAMMA, K_DRAFT, KV_START, cfg.vocab)], 10
+    else:
+        raise SystemExit(f"unknown workload {name}")
+    B = len(cases)
+    n0 = max(len(h) for h, _ in cases)
+    max_new = min(len(s) for _, s in cases)
+    stride = (n0 + max_new + 67) // 4 * 4
+    max_seq = n0 + max_new + k + 64
+    weights = inputs.make_weights(cfg, seed=0, device=str(dev))
+    ctx = cs.Context(cfg, weights, max_seq=max_seq, max_batch=B, k_max=k)
+    kv = torch.zeros(cfg.n_layers, 2, B, cfg.n_kv_heads, max_seq, cfg.head_dim, dtype=torch.bfloat16, device=dev)
+    g = torch.Generator(device=dev); g.manual_seed(1)
+    for layer in range(cfg.n_layers):
+        kv[layer, :, :, :, :n0 - 1, :] = torch.randn(2, B, cfg.n_kv_heads, n0 - 1, cfg.head_dim, device=dev,
+                                                      generator=g).to(torch.bfloat16)
+    h = np.zeros((B, stride), dtype=np.int32)
+    lens = np.array([len(hh) for hh, _ in cases], dtype=np.int32)
+    for b, (hh, _) in enumerate(cases):
+        h[b, :len(hh)] = hh
+    script_d = torch.from_numpy(np.stack([s[:max_new] for _, s in cases]).astype(np.int32)).to(dev)
+    res = {}
+    for kk in ((k, 0) if name != "verify_plain_decode" else (0,)):
+        steps = K if kk else min(4 * K, max_new - W - 1)
+        steps = min(steps, (max_new // (kk + 1)) - W - 1)
+        hd, ld = torch.from_numpy(h).to(dev), torch.from_numpy(lens).to(dev)
+        kvl = torch.from_numpy(lens - 1).to(dev)
+        ctx.cs_loop_begin(hd, ld, kv, kvl, GAMMA, kk, max_new, script=script_d)
+        ctx.cs_loop_steps(W)
+        st0, _ = ctx.cs_loop_poll()
+        e0, e1 = ev(), ev()
+        e0.record()
+        ctx.cs_loop_steps(steps)
+        e1.record()
+        torch.cuda.synchronize()
+        st1, _ = ctx.cs_loop_poll()
+        ctx.cs_loop_end()
+        ms = e0.elapsed_time(e1)
+        em = st1["emitted"] - st0["emitted"]
+        att = max(1, st1["attempts"] - st0["attempts"])
+        res[kk] = {"tokens_per_s": em / (ms * 1e-3), "ms_per_step": ms / steps, "steps": steps,
+                   "tokens_per_step": em / steps / B, "mean_tau": (st1["accepted"] - st0["accepted"]) / att,
+                   "copied_frac": (st1["accepted"] - st0["accepted"]) / max(1, em)}
+    main = res[k] if k in res and name != "verify_plain_decode" else res[0]
+    kv_bytes = float(np.sum(lens)) * cfg.kv_bytes_per_token()
+    step_bytes = cfg.streamed_params() * 2 + kv_bytes
+    line = {"metric": METRIC, "value": main["tokens_per_s"], "unit": UNIT, "n_gpus": 1, "steps": main["steps"],
+            "warmup": W, "ms_per_step": main["ms_per_step"], "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": name, "batch": B, "gamma": GAMMA, "k": k if name != "verify_plain_decode" else 0,
+                       "context": int(n0), "algorithmic_gb_per_step": step_bytes / 1e9,
+                       "achieved_gbs": step_bytes / (main["ms_per_step"] * 1e-3) / 1e9, **{f"k{kk}": v for kk, v in res.items()}}}
+    if 0 in res and k in res and name != "verify_plain_decode":
+        line["config"]["speedup_vs_plain_decode"] = res[k]["tokens_per_s"] / res[0]["tokens_per_s"]
+    print(json.dumps(line), flush=True)
+    ctx.close()
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -401,6 +507,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", default="verify",
+                    choices=["verify", "verify_plain_decode", "long_context_b1_k10", "long_context_b8_k20",
+                             "multi_turn_b16_k10", "match_search"],
+                    help="verify = the benchmark; the others are additional single-GPU measurements")
     ap.add_argument("--layers", type=int, default=0,
                     help="profiling aid: keep only this many of the 32 layers (small case for ncu captures; "
                          "not the benchmark workload)")
@@ -409,6 +519,8 @@ def main():
         args.warmup = 3
     if args.impl == "reference":
         return run_reference(args)
+    if args.workload != "verify":
+        return run_workload(args)
     return run_ours(args)
 
 
