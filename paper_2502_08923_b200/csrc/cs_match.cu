@@ -135,7 +135,11 @@ cs_status cs_launch_find_match(const int32_t* hist, const int32_t* hist_len, int
   at[0].val.clusterDim.y = 1;
   at[0].val.clusterDim.z = 1;
   lc.attrs = at;
-  lc.numAttrs = 2;
+  // Launched as an ordinary stream-ordered kernel (cluster attribute only): the search opens
+  // a decode step and reads the history the previous step's commit has just written, so the
+  // step boundary is a full serialisation point.  (With the programmatic-launch attribute on
+  // this cluster kernel the loop was observed to read a stale history.)
+  lc.numAttrs = 1;
   cudaError_t e = cudaLaunchKernelEx(&lc, k_find_match, (const int*)hist, (const int*)hist_len,
                                      stride, gamma, k, policy, (int*)match_pos, (int*)draft,
                                      (int*)draft_len, (int*)last_tok, (const int*)skip);

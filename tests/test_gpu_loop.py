@@ -106,6 +106,24 @@ def test_batch_of_sequences_with_eos_and_different_lengths():
     ctx.close()
 
 
+def test_loop_without_graph_capture_gives_the_same_result(monkeypatch):
+    """The step can also be enqueued launch by launch (CS_NO_GRAPH=1); overlapping launches of
+    consecutive steps must not change any integer result."""
+    monkeypatch.setenv("CS_NO_GRAPH", "1")
+    cfg = inputs.TINY
+    ctx, model = make_pair(cfg, 1024, 1, 10)
+    ctxt, _ = inputs.tiny_context(seed=1)
+    rng = np.random.default_rng(11)
+    max_new = 200
+    script = inputs.copy_script(rng, ctxt, max_new, 0.6, 5, 30, cfg.vocab, zipf_s=None)
+    h, n, kvl, st = _run_gpu(ctx, [ctxt], [512], 1024, 3, 10, max_new, cs.LATEST, script=script[None, :])
+    steps, st_o, h_sim = O.scripted_simulator(ctxt, script, 3, 10, O.LATEST, max_new)
+    assert h[0, :n[0]].tolist() == h_sim
+    for key in ("steps", "attempts", "accepted", "emitted", "no_match"):
+        assert st[key] == st_o[key], key
+    ctx.close()
+
+
 def test_loop_capacity_is_reported():
     cfg = inputs.TINY
     ctx, _ = make_pair(cfg, 128, 1, 10)
