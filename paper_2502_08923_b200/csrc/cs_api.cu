@@ -127,17 +127,16 @@ cs_status enqueue_forward(cs_ctx* ctx, int B, int R, void* kv_cache, bool with_l
     cs_launch_rmsnorm(ctx, L.attn_norm, rows, st);
     prof_end(ctx, st);
     prof_begin(ctx, CS_FAM_GEMM, st);
-    s = cs_launch_gemm(ctx, &L.qkv, &ctx->tmXn, CS_MAX_ROWS, rows, CS_EPI_STORE, ctx->qkv, nullptr, nullptr, 0, st);
+    const QkvEpi qe = {ctx->rope_cs, ctx->row_pos, ctx->row_write, ctx->qbuf, static_cast<__nv_bfloat16*>(kv_cache),
+                       R, l, c.n_heads, c.n_kv_heads, c.head_dim, c.max_batch, c.max_seq};
+    s = cs_launch_gemm(ctx, &L.qkv, &ctx->tmXn, CS_MAX_ROWS, rows, CS_EPI_QKV, nullptr, nullptr, nullptr, 0, &qe, st);
     prof_end(ctx, st);
     if (s != CS_OK) return s;
-    prof_begin(ctx, CS_FAM_ELEMENTWISE, st);
-    cs_launch_qkv_post(ctx, kv_cache, l, B, R, st);
-    prof_end(ctx, st);
     prof_begin(ctx, CS_FAM_ATTENTION, st);
     cs_launch_attention(ctx, kv_cache, l, B, R, st);
     prof_end(ctx, st);
     prof_begin(ctx, CS_FAM_GEMM, st);
-    s = cs_launch_gemm(ctx, &L.o, &ctx->tmAttn, CS_MAX_ROWS, rows, CS_EPI_RESIDUAL, ctx->x, nullptr, nullptr, 0, st);
+    s = cs_launch_gemm(ctx, &L.o, &ctx->tmAttn, CS_MAX_ROWS, rows, CS_EPI_RESIDUAL, ctx->x, nullptr, nullptr, 0, nullptr, st);
     prof_end(ctx, st);
     if (s != CS_OK) return s;
     prof_begin(ctx, CS_FAM_ELEMENTWISE, st);
@@ -145,11 +144,11 @@ cs_status enqueue_forward(cs_ctx* ctx, int B, int R, void* kv_cache, bool with_l
     prof_end(ctx, st);
     prof_begin(ctx, CS_FAM_GEMM, st);
     s = cs_launch_gemm(ctx, &L.gate_up, &ctx->tmXn, CS_MAX_ROWS, rows, CS_EPI_SWIGLU, nullptr, ctx->act,
-                       ctx->act + (size_t)CS_MAX_ROWS * c.d_ffn, c.d_ffn, st);
+                       ctx->act + (size_t)CS_MAX_ROWS * c.d_ffn, c.d_ffn, nullptr, st);
     prof_end(ctx, st);
     if (s != CS_OK) return s;
     prof_begin(ctx, CS_FAM_GEMM, st);
-    s = cs_launch_gemm(ctx, &L.down, &ctx->tmAct, CS_MAX_ROWS, rows, CS_EPI_RESIDUAL, ctx->x, nullptr, nullptr, 0, st);
+    s = cs_launch_gemm(ctx, &L.down, &ctx->tmAct, CS_MAX_ROWS, rows, CS_EPI_RESIDUAL, ctx->x, nullptr, nullptr, 0, nullptr, st);
     prof_end(ctx, st);
     if (s != CS_OK) return s;
   }
@@ -158,7 +157,7 @@ cs_status enqueue_forward(cs_ctx* ctx, int B, int R, void* kv_cache, bool with_l
     cs_launch_rmsnorm(ctx, ctx->final_norm, rows, st);
     prof_end(ctx, st);
     prof_begin(ctx, CS_FAM_LMHEAD, st);
-    s = cs_launch_gemm(ctx, &ctx->lm, &ctx->tmXn, CS_MAX_ROWS, rows, CS_EPI_ARGMAX, logits, nullptr, nullptr, 0, st);
+    s = cs_launch_gemm(ctx, &ctx->lm, &ctx->tmXn, CS_MAX_ROWS, rows, CS_EPI_ARGMAX, logits, nullptr, nullptr, 0, nullptr, st);
     prof_end(ctx, st);
     if (s != CS_OK) return s;
   }
@@ -538,7 +537,7 @@ cs_status cs_linear(cs_ctx* ctx, const void* X, const void* W, int rows, int N, 
   const int n_tok = cs_ceil_div(rows, 16) * 16;
   CUtensorMap tmX;
   if ((s = cs_make_act_map(ctx, &tmX, X, n_tok, K, n_tok)) != CS_OK) return s;
-  return cs_launch_gemm(ctx, &g, &tmX, -1, rows, CS_EPI_STORE, Y, nullptr, nullptr, 0, st);
+  return cs_launch_gemm(ctx, &g, &tmX, -1, rows, CS_EPI_STORE, Y, nullptr, nullptr, 0, nullptr, st);
 }
 
 cs_status cs_lm_head(cs_ctx* ctx, const void* X, int rows, int32_t* ids, float* logits_dbg, void* stream) {
@@ -549,7 +548,7 @@ cs_status cs_lm_head(cs_ctx* ctx, const void* X, int rows, int32_t* ids, float* 
   CUtensorMap tmX;
   cs_status s = cs_make_act_map(ctx, &tmX, X, n_tok, ctx->cfg.d_model, n_tok);
   if (s != CS_OK) return s;
-  if ((s = cs_launch_gemm(ctx, &ctx->lm, &tmX, -1, rows, CS_EPI_ARGMAX, logits_dbg, nullptr, nullptr, 0, st)) != CS_OK) return s;
+  if ((s = cs_launch_gemm(ctx, &ctx->lm, &tmX, -1, rows, CS_EPI_ARGMAX, logits_dbg, nullptr, nullptr, 0, nullptr, st)) != CS_OK) return s;
   cs_launch_tile_reduce(ctx, rows, ids, st);
   CS_CUDA_OK(ctx, cudaGetLastError());
   return CS_OK;

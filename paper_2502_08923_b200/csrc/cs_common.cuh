@@ -132,7 +132,17 @@ struct cs_ctx {
 static inline int cs_ceil_div(int a, int b) { return (a + b - 1) / b; }
 
 // GEMM epilogues
-enum : int { CS_EPI_STORE = 0, CS_EPI_ARGMAX = 1, CS_EPI_RESIDUAL = 2, CS_EPI_SWIGLU = 3 };
+enum : int { CS_EPI_STORE = 0, CS_EPI_ARGMAX = 1, CS_EPI_RESIDUAL = 2, CS_EPI_SWIGLU = 3, CS_EPI_QKV = 4 };
+
+// destination of the QKV epilogue
+struct QkvEpi {
+  const float* rope_cs;
+  const int* row_pos;
+  const int* row_write;
+  __nv_bfloat16* qbuf;
+  __nv_bfloat16* kv;
+  int R, layer, H, Hkv, Dh, max_batch, max_seq;
+};
 
 // Programmatic dependent launch: every kernel of the library lets its successor start
 // early and waits for its predecessor before it touches global memory the predecessor
@@ -179,7 +189,8 @@ cs_status cs_make_act_map(cs_ctx* ctx, CUtensorMap* tm, const void* base, int ro
 // (ARGMAX); `act`/F the bf16 destination of SWIGLU
 // lo_row: row coordinate (in tmX) of the activation operand's second bf16 term, -1 if X is plain bf16
 cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX, int lo_row, int rows, int mode,
-                         float* out, __nv_bfloat16* act, __nv_bfloat16* act_lo, int F, cudaStream_t st);
+                         float* out, __nv_bfloat16* act, __nv_bfloat16* act_lo, int F, const QkvEpi* q,
+                         cudaStream_t st);
 // cs_layers.cu
 void cs_launch_block_setup(cs_ctx* ctx, const int32_t* last_tok, const int32_t* draft,
                            const int32_t* draft_len, const int32_t* kv_len, const int32_t* skip,
@@ -188,7 +199,6 @@ void cs_launch_prefill_setup(cs_ctx* ctx, const int32_t* hist, const int32_t* hi
                              int stride, int start, int R, cudaStream_t st);
 void cs_launch_embed(cs_ctx* ctx, int rows, cudaStream_t st);
 void cs_launch_rmsnorm(cs_ctx* ctx, const __nv_bfloat16* gain, int rows, cudaStream_t st);
-void cs_launch_qkv_post(cs_ctx* ctx, void* kv_cache, int layer, int B, int R, cudaStream_t st);
 void cs_launch_attention(cs_ctx* ctx, const void* kv_cache, int layer, int B, int R,
                          cudaStream_t st);
 void cs_launch_attn_merge(cs_ctx* ctx, int nsplit, int rows, cudaStream_t st);

@@ -16,7 +16,9 @@
 // own shared memory; after a cluster barrier every CTA sums one slice of the features over
 // all ranks through distributed shared memory, in rank order (deterministic, no atomics,
 // no partial sums in HBM), and applies the epilogue:
-//   STORE     out[row][n]  = y                      (QKV projection, cs_linear)
+//   STORE     out[row][n]  = y                      (cs_linear)
+//   QKV       rotates q and k (RoPE), writes q as the attention operand and appends the new
+//             K/V rows to the bf16 cache            (QKV projection)
 //   RESIDUAL  x[row][n]   += y                      (attention output and FFN down projections)
 //   SWIGLU    act[row][j]  = bf16(silu(gate_j) * up_j), the tile holding 64 gate rows and the
 //             64 matching up rows                   (FFN gate/up projection)
@@ -52,6 +54,7 @@ struct GemmArgs {
   __nv_bfloat16* act_lo; // SWIGLU: second bf16 term of the same values, or NULL
   int lo_row;            // row coordinate of the activation operand's second bf16 term, -1 = none
   int F;
+  QkvEpi q;              // QKV: where the rotated queries and the new K/V rows go
   float* tile_max;       // ARGMAX: [tiles][tile_stride]
   int* tile_idx;
   int tile_stride;
@@ -349,7 +352,62 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
     if (warp < 4) {
       const uint32_t dump_addr = smem_u32(dump);
       const int e = threadIdx.x;                   // 0..127
-      if (a.mode == CS_EPI_SWIGLU) {
+      if (a.mode == CS_EPI_QKV) {
+        // RoPE pairs feature i of a head with i + Dh/2: both lie in this tile.  j in [0,64) walks
+        // the first halves of the tile's heads; each rank finishes a slice of j, four at a time.
+        const QkvEpi& Q = a.q;
+        const int half = Q.Dh >> 1;
+        const int js = ((64 + a.splits - 1) / a.splits + 3) & ~3;
+        const int j_lo = split * js, j_n = max(0, min(64, j_lo + js) - j_lo);
+        const int per_tok = j_n >> 2;
+        for (int idx = e; idx < per_tok * a.rows; idx += 128) {
+          const int j = j_lo + 4 * (idx % per_tok), tok = idx / per_tok;
+          const int i = j % half, f1 = (j / half) * Q.Dh + i, f2 = f1 + half;
+          const int head = (n0 + f1) / Q.Dh;
+          if (head >= Q.H + 2 * Q.Hkv) continue;
+          float4 av, bv;
+          if (a.splits > 1) {
+            av = sum_over_ranks(dump_addr + 4u * (uint32_t)(tok * CS_GEMM_BM + f1), a.splits);
+            bv = sum_over_ranks(dump_addr + 4u * (uint32_t)(tok * CS_GEMM_BM + f2), a.splits);
+          } else {
+            av = *reinterpret_cast<const float4*>(dump + tok * CS_GEMM_BM + f1);
+            bv = *reinterpret_cast<const float4*>(dump + tok * CS_GEMM_BM + f2);
+          }
+          const float a4[4] = {av.x, av.y, av.z, av.w}, b4[4] = {bv.x, bv.y, bv.z, bv.w};
+          float r0[4], r1[4];
+          const bool is_v = head >= Q.H + Q.Hkv;
+#pragma unroll
+          for (int t4 = 0; t4 < 4; ++t4) {
+            const float2 cs2 = *reinterpret_cast<const float2*>(Q.rope_cs + 2 * ((size_t)tok * half + i + t4));
+            r0[t4] = is_v ? a4[t4] : a4[t4] * cs2.x - b4[t4] * cs2.y;
+            r1[t4] = is_v ? b4[t4] : b4[t4] * cs2.x + a4[t4] * cs2.y;
+          }
+          __nv_bfloat162 h0[2], h1[2];
+          h0[0] = __floats2bfloat162_rn(r0[0], r0[1]); h0[1] = __floats2bfloat162_rn(r0[2], r0[3]);
+          h1[0] = __floats2bfloat162_rn(r1[0], r1[1]); h1[1] = __floats2bfloat162_rn(r1[2], r1[3]);
+          if (head < Q.H) {
+            // rotated query as two bf16 terms, the attention kernel's operand
+            __nv_bfloat16* qd = Q.qbuf + ((size_t)tok * Q.H + head) * Q.Dh + i;
+            __nv_bfloat16* ql = qd + (size_t)CS_MAX_ROWS * Q.H * Q.Dh;
+            *reinterpret_cast<uint2*>(qd) = *reinterpret_cast<const uint2*>(h0);
+            *reinterpret_cast<uint2*>(qd + half) = *reinterpret_cast<const uint2*>(h1);
+            const float2 f00 = __bfloat1622float2(h0[0]), f01 = __bfloat1622float2(h0[1]);
+            const float2 f10 = __bfloat1622float2(h1[0]), f11 = __bfloat1622float2(h1[1]);
+            __nv_bfloat162 l0[2], l1[2];
+            l0[0] = __floats2bfloat162_rn(r0[0] - f00.x, r0[1] - f00.y); l0[1] = __floats2bfloat162_rn(r0[2] - f01.x, r0[3] - f01.y);
+            l1[0] = __floats2bfloat162_rn(r1[0] - f10.x, r1[1] - f10.y); l1[1] = __floats2bfloat162_rn(r1[2] - f11.x, r1[3] - f11.y);
+            *reinterpret_cast<uint2*>(ql) = *reinterpret_cast<const uint2*>(l0);
+            *reinterpret_cast<uint2*>(ql + half) = *reinterpret_cast<const uint2*>(l1);
+          } else if (Q.row_write[tok]) {
+            // new K (rotated) / V row of the cache, stored in bf16
+            const int kvh = is_v ? head - Q.H - Q.Hkv : head - Q.H;
+            __nv_bfloat16* dst = Q.kv + ((((size_t)Q.layer * 2 + (is_v ? 1 : 0)) * Q.max_batch + tok / Q.R) * Q.Hkv + kvh) *
+                                            (size_t)Q.max_seq * Q.Dh + (size_t)Q.row_pos[tok] * Q.Dh + i;
+            *reinterpret_cast<uint2*>(dst) = *reinterpret_cast<const uint2*>(h0);
+            *reinterpret_cast<uint2*>(dst + half) = *reinterpret_cast<const uint2*>(h1);
+          }
+        }
+      } else if (a.mode == CS_EPI_SWIGLU) {
         // features 0..63 of the tile are gate rows, 64..127 the matching up rows; each rank
         // finishes a slice of j (a multiple of 4 wide), four consecutive j per thread
         const int js = ((64 + a.splits - 1) / a.splits + 3) & ~3;
@@ -494,7 +552,8 @@ cs_status cs_make_act_map(cs_ctx* ctx, CUtensorMap* tm, const void* base, int ro
 }
 
 cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX, int lo_row, int rows, int mode,
-                         float* out, __nv_bfloat16* act, __nv_bfloat16* act_lo, int F, cudaStream_t st) {
+                         float* out, __nv_bfloat16* act, __nv_bfloat16* act_lo, int F, const QkvEpi* q,
+                         cudaStream_t st) {
   const int tiles = cs_ceil_div(g->N, CS_GEMM_BM);
   GemmArgs a;
   a.rows = rows;
@@ -510,6 +569,7 @@ cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX,
   a.act_lo = act_lo;
   a.lo_row = lo_row;
   a.F = F;
+  if (q != nullptr) a.q = *q;
   a.tile_max = ctx->tile_max;
   a.tile_idx = ctx->tile_idx;
   a.tile_stride = ctx->rows_pad;

@@ -136,44 +136,6 @@ k_rmsnorm(const float* __restrict__ x, int d, const __nv_bfloat16* __restrict__ 
   }
 }
 
-// Rotate q and k of the QKV projection (rotate-half pairing) at the row's
-// absolute position, store q as the bf16 attention operand and append k, v to the cache.
-__global__ void k_qkv_post(const float* __restrict__ qkv, int H, int Hkv, int Dh,
-                           const float* __restrict__ rope_cs, const int* __restrict__ row_pos,
-                           const int* __restrict__ row_write, int R, __nv_bfloat16* __restrict__ qbuf,
-                           __nv_bfloat16* __restrict__ kv, int layer, int max_batch, int max_seq) {
-  const int row = blockIdx.x, head = blockIdx.y, i = threadIdx.x;
-  const int half = Dh >> 1, N = (H + 2 * Hkv) * Dh;
-  CS_PDL_PROLOGUE();
-  const float* p = qkv + (size_t)row * N + (size_t)head * Dh;
-  const float a = p[i], b = p[i + half];
-  const float c = rope_cs[2 * (row * half + i)], sn = rope_cs[2 * (row * half + i) + 1];
-  if (head < H) {
-    __nv_bfloat16* q = qbuf + (size_t)row * H * Dh + (size_t)head * Dh;
-    __nv_bfloat16* ql = q + (size_t)CS_MAX_ROWS * H * Dh;      // second bf16 term
-    const float r0 = a * c - b * sn, r1 = b * c + a * sn;
-    const __nv_bfloat16 h0 = __float2bfloat16_rn(r0), h1 = __float2bfloat16_rn(r1);
-    q[i] = h0;
-    q[i + half] = h1;
-    ql[i] = __float2bfloat16_rn(r0 - __bfloat162float(h0));
-    ql[i + half] = __float2bfloat16_rn(r1 - __bfloat162float(h1));
-    return;
-  }
-  if (!row_write[row]) return;
-  const int bseq = row / R;
-  const bool is_k = head < H + Hkv;
-  const int kvh = is_k ? head - H : head - H - Hkv;
-  __nv_bfloat16* dst = kv + ((((size_t)layer * 2 + (is_k ? 0 : 1)) * max_batch + bseq) * Hkv + kvh) *
-                                (size_t)max_seq * Dh + (size_t)row_pos[row] * Dh;
-  if (is_k) {
-    dst[i] = __float2bfloat16_rn(a * c - b * sn);
-    dst[i + half] = __float2bfloat16_rn(b * c + a * sn);
-  } else {
-    dst[i] = __float2bfloat16_rn(a);
-    dst[i + half] = __float2bfloat16_rn(b);
-  }
-}
-
 // Combine the key slices: o = sum_s o_s e^(m_s - M) / sum_s l_s e^(m_s - M).
 __global__ void k_attn_merge(const float* __restrict__ in_o, const float* __restrict__ in_ml, int nsplit,
                              int rows, int H, int Dh, __nv_bfloat16* __restrict__ attn_out) {
@@ -411,13 +373,6 @@ void cs_launch_embed(cs_ctx* ctx, int rows, cudaStream_t st) {
 void cs_launch_rmsnorm(cs_ctx* ctx, const __nv_bfloat16* gain, int rows, cudaStream_t st) {
   cs_launch_pdl(k_rmsnorm, dim3(rows), dim3(256), 0, st, ctx->x, ctx->cfg.d_model, gain, ctx->cfg.rms_eps, ctx->xn,
                 ctx->xn + (size_t)CS_MAX_ROWS * ctx->cfg.d_model);
-}
-
-void cs_launch_qkv_post(cs_ctx* ctx, void* kv_cache, int layer, int B, int R, cudaStream_t st) {
-  const cs_model_config& c = ctx->cfg;
-  cs_launch_pdl(k_qkv_post, dim3(B * R, c.n_heads + 2 * c.n_kv_heads), dim3(c.head_dim / 2), 0, st, ctx->qkv,
-                c.n_heads, c.n_kv_heads, c.head_dim, ctx->rope_cs, ctx->row_pos, ctx->row_write, R, ctx->qbuf,
-                static_cast<__nv_bfloat16*>(kv_cache), layer, c.max_batch, c.max_seq);
 }
 
 void cs_launch_attn_merge(cs_ctx* ctx, int nsplit, int rows, cudaStream_t st) {
