@@ -101,25 +101,6 @@ k_attn_mma(const __nv_bfloat16* __restrict__ qbuf, const __nv_bfloat16* __restri
   const int head_lo = v_lo ? kvh * G + q_lo / R : 0, head_hi = v_hi ? kvh * G + q_hi / R : 0;
   const int lim_lo = v_lo ? row_lim[grow_lo] : 0, lim_hi = v_hi ? row_lim[grow_hi] : 0;
 
-  // queries come as two bf16 terms (q = qa + qb): two MMAs give the product of the fp32 query
-  uint32_t qa[KSTEPS][4], qb[KSTEPS][4];
-  {
-    const __nv_bfloat16* ql = qbuf + ((size_t)grow_lo * H + head_lo) * DH;
-    const __nv_bfloat16* qh = qbuf + ((size_t)grow_hi * H + head_hi) * DH;
-    const size_t second = (size_t)CS_MAX_ROWS * H * DH;
-#pragma unroll
-    for (int ks = 0; ks < KSTEPS; ++ks) {
-      qa[ks][0] = v_lo ? *reinterpret_cast<const uint32_t*>(ql + ks * 16 + 2 * t) : 0u;
-      qa[ks][1] = v_hi ? *reinterpret_cast<const uint32_t*>(qh + ks * 16 + 2 * t) : 0u;
-      qa[ks][2] = v_lo ? *reinterpret_cast<const uint32_t*>(ql + ks * 16 + 8 + 2 * t) : 0u;
-      qa[ks][3] = v_hi ? *reinterpret_cast<const uint32_t*>(qh + ks * 16 + 8 + 2 * t) : 0u;
-      qb[ks][0] = v_lo ? *reinterpret_cast<const uint32_t*>(ql + second + ks * 16 + 2 * t) : 0u;
-      qb[ks][1] = v_hi ? *reinterpret_cast<const uint32_t*>(qh + second + ks * 16 + 2 * t) : 0u;
-      qb[ks][2] = v_lo ? *reinterpret_cast<const uint32_t*>(ql + second + ks * 16 + 8 + 2 * t) : 0u;
-      qb[ks][3] = v_hi ? *reinterpret_cast<const uint32_t*>(qh + second + ks * 16 + 8 + 2 * t) : 0u;
-    }
-  }
-
   const __nv_bfloat16* Kg = kv + ((((size_t)layer * 2 + 0) * max_batch + b) * Hkv + kvh) * (size_t)max_seq * DH;
   const __nv_bfloat16* Vg = kv + ((((size_t)layer * 2 + 1) * max_batch + b) * Hkv + kvh) * (size_t)max_seq * DH;
 
@@ -144,6 +125,26 @@ k_attn_mma(const __nv_bfloat16* __restrict__ qbuf, const __nv_bfloat16* __restri
 
   if (t0 < t1) load_tile(t0, 0);
   cp_async_commit();
+  // (the first K/V tile is already on its way while the query fragments are fetched)
+  // queries come as two bf16 terms (q = qa + qb): two MMAs give the product of the fp32 query
+  uint32_t qa[KSTEPS][4], qb[KSTEPS][4];
+  {
+    const __nv_bfloat16* ql = qbuf + ((size_t)grow_lo * H + head_lo) * DH;
+    const __nv_bfloat16* qh = qbuf + ((size_t)grow_hi * H + head_hi) * DH;
+    const size_t second = (size_t)CS_MAX_ROWS * H * DH;
+#pragma unroll
+    for (int ks = 0; ks < KSTEPS; ++ks) {
+      qa[ks][0] = v_lo ? *reinterpret_cast<const uint32_t*>(ql + ks * 16 + 2 * t) : 0u;
+      qa[ks][1] = v_hi ? *reinterpret_cast<const uint32_t*>(qh + ks * 16 + 2 * t) : 0u;
+      qa[ks][2] = v_lo ? *reinterpret_cast<const uint32_t*>(ql + ks * 16 + 8 + 2 * t) : 0u;
+      qa[ks][3] = v_hi ? *reinterpret_cast<const uint32_t*>(qh + ks * 16 + 8 + 2 * t) : 0u;
+      qb[ks][0] = v_lo ? *reinterpret_cast<const uint32_t*>(ql + second + ks * 16 + 2 * t) : 0u;
+      qb[ks][1] = v_hi ? *reinterpret_cast<const uint32_t*>(qh + second + ks * 16 + 2 * t) : 0u;
+      qb[ks][2] = v_lo ? *reinterpret_cast<const uint32_t*>(ql + second + ks * 16 + 8 + 2 * t) : 0u;
+      qb[ks][3] = v_hi ? *reinterpret_cast<const uint32_t*>(qh + second + ks * 16 + 8 + 2 * t) : 0u;
+    }
+  }
+
   for (int tile = t0; tile < t1; ++tile) {
     const int stage = (tile - t0) & 1;
     if (tile + 1 < t1) load_tile(tile + 1, stage ^ 1);

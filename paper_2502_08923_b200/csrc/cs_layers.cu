@@ -97,35 +97,43 @@ __global__ void k_embed(const __nv_bfloat16* __restrict__ E, const int* __restri
   }
 }
 
-// xn = x * rsqrt(mean(x^2) + eps) * g as two bf16 terms (hi, lo).  One CTA per row.
-__global__ void __launch_bounds__(256)
+// xn = x * rsqrt(mean(x^2) + eps) * g as two bf16 terms (hi, lo).  One CTA per row; the row is
+// read once and kept in registers (up to 4 float4 per thread).
+constexpr int kNormThreads = 1024;
+__global__ void __launch_bounds__(kNormThreads)
 k_rmsnorm(const float* __restrict__ x, int d, const __nv_bfloat16* __restrict__ gain, float eps,
           __nv_bfloat16* __restrict__ xn, __nv_bfloat16* __restrict__ xn_lo) {
   CS_PDL_PROLOGUE();
   const int row = blockIdx.x;
   const float* xr = x + (size_t)row * d;
+  float4 v[4];
   float ss = 0.f;
-  for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
-    const float4 v = *reinterpret_cast<const float4*>(xr + i);
-    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int i = (q * kNormThreads + threadIdx.x) * 4;
+    v[q] = (i < d) ? *reinterpret_cast<const float4*>(xr + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+    ss += v[q].x * v[q].x + v[q].y * v[q].y + v[q].z * v[q].z + v[q].w * v[q].w;
   }
-  __shared__ float red[8];
+  for (int i = 4 * kNormThreads * 4 + threadIdx.x * 4; i < d; i += kNormThreads * 4) {   // d > 16384
+    const float4 w = *reinterpret_cast<const float4*>(xr + i);
+    ss += w.x * w.x + w.y * w.y + w.z * w.z + w.w * w.w;
+  }
+  __shared__ float red[32];
   __shared__ float s_scale;
   for (int off = 16; off > 0; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
   __syncthreads();
-  if (threadIdx.x == 0) {
-    float t = 0.f;
-    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t += red[w];
-    s_scale = rsqrtf(t / (float)d + eps);
+  if (threadIdx.x < 32) {
+    float t = red[threadIdx.x];
+    for (int off = 16; off > 0; off >>= 1) t += __shfl_xor_sync(0xffffffffu, t, off);
+    if (threadIdx.x == 0) s_scale = rsqrtf(t / (float)d + eps);
   }
   __syncthreads();
   const float sc = s_scale;
-  for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
-    const float4 v = *reinterpret_cast<const float4*>(xr + i);
+  auto emit = [&](int i, const float4& w) {
     const float2 g0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(gain + i));
     const float2 g1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(gain + i + 2));
-    const float y0 = v.x * sc * g0.x, y1 = v.y * sc * g0.y, y2 = v.z * sc * g1.x, y3 = v.w * sc * g1.y;
+    const float y0 = w.x * sc * g0.x, y1 = w.y * sc * g0.y, y2 = w.z * sc * g1.x, y3 = w.w * sc * g1.y;
     const __nv_bfloat162 o0 = __floats2bfloat162_rn(y0, y1), o1 = __floats2bfloat162_rn(y2, y3);
     *reinterpret_cast<__nv_bfloat162*>(xn + (size_t)row * d + i) = o0;
     *reinterpret_cast<__nv_bfloat162*>(xn + (size_t)row * d + i + 2) = o1;
@@ -133,7 +141,14 @@ k_rmsnorm(const float* __restrict__ x, int d, const __nv_bfloat16* __restrict__ 
     const float2 h0 = __bfloat1622float2(o0), h1 = __bfloat1622float2(o1);
     *reinterpret_cast<__nv_bfloat162*>(xn_lo + (size_t)row * d + i) = __floats2bfloat162_rn(y0 - h0.x, y1 - h0.y);
     *reinterpret_cast<__nv_bfloat162*>(xn_lo + (size_t)row * d + i + 2) = __floats2bfloat162_rn(y2 - h1.x, y3 - h1.y);
+  };
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int i = (q * kNormThreads + threadIdx.x) * 4;
+    if (i < d) emit(i, v[q]);
   }
+  for (int i = 4 * kNormThreads * 4 + threadIdx.x * 4; i < d; i += kNormThreads * 4)
+    emit(i, *reinterpret_cast<const float4*>(xr + i));
 }
 
 // Combine the key slices: o = sum_s o_s e^(m_s - M) / sum_s l_s e^(m_s - M).
@@ -142,6 +157,15 @@ __global__ void k_attn_merge(const float* __restrict__ in_o, const float* __rest
   CS_PDL_PROLOGUE();
   const int row = blockIdx.x, h = blockIdx.y, dd = threadIdx.x;
   const int lane = threadIdx.x & 31;
+  // all partial outputs of this (row, head, dim) are requested at once, so their latencies
+  // overlap each other and the weight computation below (at most 64 key slices)
+  float v[64];
+  {
+    const size_t stride = (size_t)rows * H * Dh;
+    const float* src = in_o + ((size_t)row * H + h) * Dh + dd;
+#pragma unroll
+    for (int s = 0; s < 64; ++s) v[s] = (s < nsplit) ? src[(size_t)s * stride] : 0.f;
+  }
   // every warp works out the slice weights e^(m_s - M) / L itself: lane s owns slices s, s+32
   float m0 = -INFINITY, l0 = 0.f, m1 = -INFINITY, l1 = 0.f;
   if (lane < nsplit) {
@@ -160,12 +184,10 @@ __global__ void k_attn_merge(const float* __restrict__ in_o, const float* __rest
   const float inv = L > 0.f ? 1.f / L : 0.f;
   w0 *= inv; w1 *= inv;
   float acc = 0.f;
-  const size_t stride = (size_t)rows * H * Dh;
-  const float* src = in_o + ((size_t)row * H + h) * Dh + dd;
-#pragma unroll 8
-  for (int s = 0; s < nsplit; ++s) {
+#pragma unroll
+  for (int s = 0; s < 64; ++s) {
     const float w = __shfl_sync(0xffffffffu, s < 32 ? w0 : w1, s & 31);
-    acc = fmaf(src[(size_t)s * stride], w, acc);
+    acc = fmaf(v[s], w, acc);
   }
   const __nv_bfloat16 hi = __float2bfloat16_rn(acc);
   attn_out[((size_t)row * H + h) * Dh + dd] = hi;
@@ -371,7 +393,7 @@ void cs_launch_embed(cs_ctx* ctx, int rows, cudaStream_t st) {
 }
 
 void cs_launch_rmsnorm(cs_ctx* ctx, const __nv_bfloat16* gain, int rows, cudaStream_t st) {
-  cs_launch_pdl(k_rmsnorm, dim3(rows), dim3(256), 0, st, ctx->x, ctx->cfg.d_model, gain, ctx->cfg.rms_eps, ctx->xn,
+  cs_launch_pdl(k_rmsnorm, dim3(rows), dim3(kNormThreads), 0, st, ctx->x, ctx->cfg.d_model, gain, ctx->cfg.rms_eps, ctx->xn,
                 ctx->xn + (size_t)CS_MAX_ROWS * ctx->cfg.d_model);
 }
 
