@@ -10,7 +10,7 @@
 namespace {
 
 struct WsLayout {
-  size_t x, xn, attn_out, act, qbuf, partial, attn_o, attn_ml, rope_cs, inv_freq, tile_max, tile_idx,
+  size_t x, xn, attn_out, act, qbuf, partial, attn_o, attn_ml, ssq, rope_cs, inv_freq, tile_max, tile_idx,
       row_tok, row_pos, row_lim, row_write, seq_ok, status, loop_last, loop_draft, loop_dlen, loop_mpos,
       loop_emitted, loop_done, loop_accept, loop_out, loop_argmax, loop_stats, total;
   size_t qkv_elems;
@@ -54,6 +54,7 @@ WsLayout ws_layout(const cs_model_config* c) {
   L.partial = take(&off, L.qkv_elems * 4);
   L.attn_o = take(&off, (size_t)L.attn_splits * rows * qd * 4);
   L.attn_ml = take(&off, (size_t)L.attn_splits * rows * c->n_heads * 2 * 4);
+  L.ssq = take(&off, rows * (size_t)cs_ceil_div(c->d_model, CS_GEMM_BM) * CS_MAX_SPLITS * 4);
   L.rope_cs = take(&off, rows * c->head_dim * 4);
   L.inv_freq = take(&off, (size_t)c->head_dim / 2 * 8);
   L.tile_max = take(&off, lm_tiles * rows * 4);
@@ -121,43 +122,62 @@ cs_status enqueue_forward(cs_ctx* ctx, int B, int R, void* kv_cache, bool with_l
   prof_begin(ctx, CS_FAM_ELEMENTWISE, st);
   cs_launch_embed(ctx, rows, st);
   prof_end(ctx, st);
+  // Only the first RMSNorm runs as a kernel.  Every later one is folded into the GEMMs around
+  // it: the residual GEMM before it writes gain * x (two bf16 terms) and sums of squares, the
+  // GEMM after it scales its accumulators by 1/rms.
+  NormFuse take_norm = {};           // how the next norm-consuming GEMM finds its 1/rms
   for (int l = 0; l < c.n_layers; ++l) {
     const LayerPlan& L = ctx->layers[l];
-    prof_begin(ctx, CS_FAM_ELEMENTWISE, st);
-    cs_launch_rmsnorm(ctx, L.attn_norm, rows, st);
-    prof_end(ctx, st);
+    if (l == 0) {
+      prof_begin(ctx, CS_FAM_ELEMENTWISE, st);
+      cs_launch_rmsnorm(ctx, L.attn_norm, rows, st);
+      prof_end(ctx, st);
+    }
     prof_begin(ctx, CS_FAM_GEMM, st);
     const QkvEpi qe = {ctx->rope_cs, ctx->row_pos, ctx->row_write, ctx->qbuf, static_cast<__nv_bfloat16*>(kv_cache),
                        R, l, c.n_heads, c.n_kv_heads, c.head_dim, c.max_batch, c.max_seq};
-    s = cs_launch_gemm(ctx, &L.qkv, &ctx->tmXn, CS_MAX_ROWS, rows, CS_EPI_QKV, nullptr, nullptr, nullptr, 0, &qe, st);
+    s = cs_launch_gemm(ctx, &L.qkv, &ctx->tmXn, CS_MAX_ROWS, rows, CS_EPI_QKV, nullptr, nullptr, nullptr, 0, &qe,
+                       &take_norm, st);
     prof_end(ctx, st);
     if (s != CS_OK) return s;
     prof_begin(ctx, CS_FAM_ATTENTION, st);
     cs_launch_attention(ctx, kv_cache, l, B, R, st);
     prof_end(ctx, st);
     prof_begin(ctx, CS_FAM_GEMM, st);
-    s = cs_launch_gemm(ctx, &L.o, &ctx->tmAttn, CS_MAX_ROWS, rows, CS_EPI_RESIDUAL, ctx->x, nullptr, nullptr, 0, nullptr, st);
+    NormFuse give = {};
+    give.gain_out = L.ffn_norm;
+    give.xn_out = ctx->xn;
+    give.ssq_out = ctx->ssq;
+    give.slot_stride = ctx->ssq_stride;
+    s = cs_launch_gemm(ctx, &L.o, &ctx->tmAttn, CS_MAX_ROWS, rows, CS_EPI_RESIDUAL, ctx->x, nullptr, nullptr, 0, nullptr,
+                       &give, st);
     prof_end(ctx, st);
     if (s != CS_OK) return s;
-    prof_begin(ctx, CS_FAM_ELEMENTWISE, st);
-    cs_launch_rmsnorm(ctx, L.ffn_norm, rows, st);
-    prof_end(ctx, st);
+    take_norm = NormFuse{};
+    take_norm.ssq_in = ctx->ssq;
+    take_norm.slots_in = cs_ceil_div(L.o.N, CS_GEMM_BM) * L.o.splits;
+    take_norm.slot_stride = ctx->ssq_stride;
+    take_norm.inv_d = 1.f / (float)c.d_model;
+    take_norm.eps = c.rms_eps;
     prof_begin(ctx, CS_FAM_GEMM, st);
     s = cs_launch_gemm(ctx, &L.gate_up, &ctx->tmXn, CS_MAX_ROWS, rows, CS_EPI_SWIGLU, nullptr, ctx->act,
-                       ctx->act + (size_t)CS_MAX_ROWS * c.d_ffn, c.d_ffn, nullptr, st);
+                       ctx->act + (size_t)CS_MAX_ROWS * c.d_ffn, c.d_ffn, nullptr, &take_norm, st);
     prof_end(ctx, st);
     if (s != CS_OK) return s;
+    // the norm after this layer: the next layer's, or the final one before the LM head
+    const __nv_bfloat16* next_gain = (l + 1 < c.n_layers) ? ctx->layers[l + 1].attn_norm : (with_lm ? ctx->final_norm : nullptr);
+    give.gain_out = next_gain;
     prof_begin(ctx, CS_FAM_GEMM, st);
-    s = cs_launch_gemm(ctx, &L.down, &ctx->tmAct, CS_MAX_ROWS, rows, CS_EPI_RESIDUAL, ctx->x, nullptr, nullptr, 0, nullptr, st);
+    s = cs_launch_gemm(ctx, &L.down, &ctx->tmAct, CS_MAX_ROWS, rows, CS_EPI_RESIDUAL, ctx->x, nullptr, nullptr, 0, nullptr,
+                       &give, st);
     prof_end(ctx, st);
     if (s != CS_OK) return s;
+    take_norm.slots_in = cs_ceil_div(L.down.N, CS_GEMM_BM) * L.down.splits;
   }
   if (with_lm) {
-    prof_begin(ctx, CS_FAM_ELEMENTWISE, st);
-    cs_launch_rmsnorm(ctx, ctx->final_norm, rows, st);
-    prof_end(ctx, st);
     prof_begin(ctx, CS_FAM_LMHEAD, st);
-    s = cs_launch_gemm(ctx, &ctx->lm, &ctx->tmXn, CS_MAX_ROWS, rows, CS_EPI_ARGMAX, logits, nullptr, nullptr, 0, nullptr, st);
+    s = cs_launch_gemm(ctx, &ctx->lm, &ctx->tmXn, CS_MAX_ROWS, rows, CS_EPI_ARGMAX, logits, nullptr, nullptr, 0, nullptr,
+                       &take_norm, st);
     prof_end(ctx, st);
     if (s != CS_OK) return s;
   }
@@ -257,6 +277,8 @@ cs_status cs_create(cs_ctx** out, const cs_model_config* cfg, const cs_weights* 
   ctx->qkv = reinterpret_cast<float*>(base + L.partial);
   ctx->attn_o = reinterpret_cast<float*>(base + L.attn_o);
   ctx->attn_ml = reinterpret_cast<float*>(base + L.attn_ml);
+  ctx->ssq = reinterpret_cast<float*>(base + L.ssq);
+  ctx->ssq_stride = cs_ceil_div(ctx->cfg.d_model, CS_GEMM_BM) * CS_MAX_SPLITS;
   ctx->rope_cs = reinterpret_cast<float*>(base + L.rope_cs);
   ctx->inv_freq = reinterpret_cast<double*>(base + L.inv_freq);
   ctx->tile_max = reinterpret_cast<float*>(base + L.tile_max);
@@ -537,7 +559,7 @@ cs_status cs_linear(cs_ctx* ctx, const void* X, const void* W, int rows, int N, 
   const int n_tok = cs_ceil_div(rows, 16) * 16;
   CUtensorMap tmX;
   if ((s = cs_make_act_map(ctx, &tmX, X, n_tok, K, n_tok)) != CS_OK) return s;
-  return cs_launch_gemm(ctx, &g, &tmX, -1, rows, CS_EPI_STORE, Y, nullptr, nullptr, 0, nullptr, st);
+  return cs_launch_gemm(ctx, &g, &tmX, -1, rows, CS_EPI_STORE, Y, nullptr, nullptr, 0, nullptr, nullptr, st);
 }
 
 cs_status cs_lm_head(cs_ctx* ctx, const void* X, int rows, int32_t* ids, float* logits_dbg, void* stream) {
@@ -548,7 +570,7 @@ cs_status cs_lm_head(cs_ctx* ctx, const void* X, int rows, int32_t* ids, float* 
   CUtensorMap tmX;
   cs_status s = cs_make_act_map(ctx, &tmX, X, n_tok, ctx->cfg.d_model, n_tok);
   if (s != CS_OK) return s;
-  if ((s = cs_launch_gemm(ctx, &ctx->lm, &tmX, -1, rows, CS_EPI_ARGMAX, logits_dbg, nullptr, nullptr, 0, nullptr, st)) != CS_OK) return s;
+  if ((s = cs_launch_gemm(ctx, &ctx->lm, &tmX, -1, rows, CS_EPI_ARGMAX, logits_dbg, nullptr, nullptr, 0, nullptr, nullptr, st)) != CS_OK) return s;
   cs_launch_tile_reduce(ctx, rows, ids, st);
   CS_CUDA_OK(ctx, cudaGetLastError());
   return CS_OK;

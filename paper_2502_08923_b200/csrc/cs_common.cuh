@@ -87,6 +87,8 @@ struct cs_ctx {
   size_t qkv_elems;
   float* attn_o;             // split-KV partial outputs [splits][rows][H][Dh]
   float* attn_ml;            // split-KV (max, sum) [splits][rows][H][2]
+  float* ssq;                // sum-of-squares slots of the folded RMSNorm [rows][ssq_stride]
+  int ssq_stride;
   float* rope_cs;            // cos/sin of this block [rows][Dh/2][2]
   double* inv_freq;          // theta^(-2i/Dh) [Dh/2]
   float* tile_max;           // LM-head tile maxima [tiles][rows_pad]
@@ -144,6 +146,20 @@ struct QkvEpi {
   int R, layer, H, Hkv, Dh, max_batch, max_seq;
 };
 
+// RMSNorm folded into the GEMMs on either side of it.  A residual GEMM that feeds a norm
+// (`gain_out` set) also writes gain * x_new as the next GEMM's two-term bf16 operand and, per
+// (tile, split-K rank) slot, the sum of squares of the features it finished; the GEMM that
+// consumes the norm (`ssq_in` set) adds the slots up in a fixed order and scales its
+// accumulators by rsqrt(sum / d + eps), which commutes with the contraction.
+struct NormFuse {
+  const float* ssq_in;            // [rows][slot_stride], NULL = operand already normalised
+  int slots_in, slot_stride;
+  float inv_d, eps;
+  const __nv_bfloat16* gain_out;  // NULL = no norm follows
+  __nv_bfloat16* xn_out;          // [2 * CS_MAX_ROWS][N]: leading terms, then second terms
+  float* ssq_out;
+};
+
 // Programmatic dependent launch: every kernel of the library lets its successor start
 // early and waits for its predecessor before it touches global memory the predecessor
 // (or, transitively, anything earlier in the stream) may still be using.
@@ -189,7 +205,7 @@ cs_status cs_make_act_map(cs_ctx* ctx, CUtensorMap* tm, const void* base, int ro
 // (ARGMAX); `act`/F the bf16 destination of SWIGLU
 // lo_row: row coordinate (in tmX) of the activation operand's second bf16 term, -1 if X is plain bf16
 cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX, int lo_row, int rows, int mode,
-                         float* out, __nv_bfloat16* act, __nv_bfloat16* act_lo, int F, const QkvEpi* q,
+                         float* out, __nv_bfloat16* act, __nv_bfloat16* act_lo, int F, const QkvEpi* q, const NormFuse* nf,
                          cudaStream_t st);
 // cs_layers.cu
 void cs_launch_block_setup(cs_ctx* ctx, const int32_t* last_tok, const int32_t* draft,

@@ -55,6 +55,7 @@ struct GemmArgs {
   int lo_row;            // row coordinate of the activation operand's second bf16 term, -1 = none
   int F;
   QkvEpi q;              // QKV: where the rotated queries and the new K/V rows go
+  NormFuse nf;           // RMSNorm folded into this GEMM's read-out (consumer) or residual update (producer)
   float* tile_max;       // ARGMAX: [tiles][tile_stride]
   int* tile_idx;
   int tile_stride;
@@ -185,6 +186,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
   volatile int* s_never = reinterpret_cast<volatile int*>(tmem_slot + 2);   // stays 0: drains wait on time only
   float* red_val = reinterpret_cast<float*>(tmem_slot + 4);       // [4][n_tok] (ARGMAX)
   int* red_idx = reinterpret_cast<int*>(red_val + 4 * a.n_tok);
+  float* rstd_s = reinterpret_cast<float*>(red_idx + 4 * a.n_tok);   // [n_tok] (folded RMSNorm)
   float* dump = reinterpret_cast<float*>(smem);                   // [n_tok][128] fp32, reuses the operand ring
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -290,11 +292,23 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
   } else {
     // ------------------------------------------------------------- accumulator read-out (warps 0-3)
     const int feat = n0 + warp * 32 + lane;
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const bool scaled = a.nf.ssq_in != nullptr;
+    if (scaled) {
+      // 1/rms of every token row while the main loop runs: slots summed in a fixed order
+      for (int tok = warp; tok < a.rows; tok += 4) {
+        float ss = 0.f;
+        for (int sl = lane; sl < a.nf.slots_in; sl += 32) ss += a.nf.ssq_in[(size_t)tok * a.nf.slot_stride + sl];
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
+        if (lane == 0) rstd_s[tok] = rsqrtf(ss * a.nf.inv_d + a.nf.eps);
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+    }
     if (nkb > 0) ok = mbar_wait(bar_acc, 0, s_abort);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     ok = __all_sync(0xffffffffu, ok) && (*s_abort == 0);
     if (!ok && lane == 0) atomicOr(a.status, CS_DEV_TIMEOUT);
-    asm volatile("griddepcontrol.wait;" ::: "memory");
     for (int c0 = 0; c0 < a.n_tok && c0 < a.rows; c0 += 16) {
       uint32_t v[16];
       if (nkb > 0 && ok) {
@@ -302,6 +316,11 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
       } else {
 #pragma unroll
         for (int j = 0; j < 16; ++j) v[j] = 0u;
+      }
+      if (scaled) {
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+          if (c0 + j < a.rows) v[j] = __float_as_uint(__uint_as_float(v[j]) * rstd_s[c0 + j]);
       }
       if (a.mode != CS_EPI_ARGMAX) {
         // the MMAs have retired, so the operand ring is free: park the tile there
@@ -439,8 +458,11 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
         const int fs = ((CS_GEMM_BM + a.splits - 1) / a.splits + 3) & ~3;
         const int f_lo = split * fs, f_n = max(0, min(CS_GEMM_BM, f_lo + fs) - f_lo);
         const int per_tok = f_n >> 2;
+        const bool feeds_norm = a.mode == CS_EPI_RESIDUAL && a.nf.gain_out != nullptr;
+        float* part = dump + a.n_tok * CS_GEMM_BM;   // [rows][32] sums of squares, behind the parked tile
         for (int idx = e; idx < per_tok * a.rows; idx += 128) {
           const int f = f_lo + 4 * (idx % per_tok), tok = idx / per_tok;
+          if (feeds_norm) part[tok * 32 + idx % per_tok] = 0.f;
           float4 y;
           if (a.splits > 1) y = sum_over_ranks(dump_addr + 4u * (uint32_t)(tok * CS_GEMM_BM + f), a.splits);
           else y = *reinterpret_cast<const float4*>(dump + tok * CS_GEMM_BM + f);
@@ -453,10 +475,32 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
               o.x += x.x; o.y += x.y; o.z += x.z; o.w += x.w;
             }
             *reinterpret_cast<float4*>(dst) = o;
+            if (feeds_norm) {
+              const uint2 gw = *reinterpret_cast<const uint2*>(a.nf.gain_out + n0 + f);
+              const float2 g01 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&gw.x));
+              const float2 g23 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&gw.y));
+              const float w0 = o.x * g01.x, w1 = o.y * g01.y, w2 = o.z * g23.x, w3 = o.w * g23.y;
+              __nv_bfloat162 h[2], l[2];
+              h[0] = __floats2bfloat162_rn(w0, w1); h[1] = __floats2bfloat162_rn(w2, w3);
+              const float2 h0 = __bfloat1622float2(h[0]), h1 = __bfloat1622float2(h[1]);
+              l[0] = __floats2bfloat162_rn(w0 - h0.x, w1 - h0.y); l[1] = __floats2bfloat162_rn(w2 - h1.x, w3 - h1.y);
+              __nv_bfloat16* xo = a.nf.xn_out + (size_t)tok * a.N + n0 + f;
+              *reinterpret_cast<uint2*>(xo) = *reinterpret_cast<const uint2*>(h);
+              *reinterpret_cast<uint2*>(xo + (size_t)CS_MAX_ROWS * a.N) = *reinterpret_cast<const uint2*>(l);
+              part[tok * 32 + idx % per_tok] = (o.x * o.x + o.y * o.y) + (o.z * o.z + o.w * o.w);
+            }
           } else {
 #pragma unroll
             for (int i = 0; i < 4; ++i)
               if (n0 + f + i < a.N) dst[i] = (a.mode == CS_EPI_RESIDUAL) ? dst[i] + yv[i] : yv[i];
+          }
+        }
+        if (feeds_norm) {
+          asm volatile("bar.sync 1, 128;" ::: "memory");
+          for (int tok = e; tok < a.rows; tok += 128) {
+            float ss = 0.f;
+            for (int q = 0; q < per_tok; ++q) ss += part[tok * 32 + q];
+            a.nf.ssq_out[(size_t)tok * a.nf.slot_stride + tile * a.splits + split] = ss;
           }
         }
       }
@@ -553,7 +597,7 @@ cs_status cs_make_act_map(cs_ctx* ctx, CUtensorMap* tm, const void* base, int ro
 
 cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX, int lo_row, int rows, int mode,
                          float* out, __nv_bfloat16* act, __nv_bfloat16* act_lo, int F, const QkvEpi* q,
-                         cudaStream_t st) {
+                         const NormFuse* nf, cudaStream_t st) {
   const int tiles = cs_ceil_div(g->N, CS_GEMM_BM);
   GemmArgs a;
   a.rows = rows;
@@ -570,19 +614,26 @@ cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX,
   a.lo_row = lo_row;
   a.F = F;
   if (q != nullptr) a.q = *q;
+  a.nf = NormFuse{};
+  if (nf != nullptr) a.nf = *nf;
+  if (a.nf.gain_out != nullptr && (mode != CS_EPI_RESIDUAL || (g->N & 3) != 0)) {
+    snprintf(ctx->err, sizeof(ctx->err), "a norm can only be folded into a residual GEMM whose width is a multiple of 4");
+    return CS_ERR_UNSUPPORTED;
+  }
   a.tile_max = ctx->tile_max;
   a.tile_idx = ctx->tile_idx;
   a.tile_stride = ctx->rows_pad;
   a.status = ctx->d_status;
   const int stage_bytes = kTileABytes + (lo_row >= 0 ? 2 : 1) * a.n_tok * 128;
-  const int fixed = 1024 /*alignment slack*/ + (2 * 8 + 1) * 8 + 16 + 8 * a.n_tok * 4;
+  const int fixed = 1024 /*alignment slack*/ + (2 * 8 + 1) * 8 + 16 + 9 * a.n_tok * 4;
   // small blocks: two CTAs per SM (about 100 KB each); large blocks: one CTA with the whole SM
   int stages = (100 * 1024 - fixed) / stage_bytes;
   if (stages < 4) stages = (220 * 1024 - fixed) / stage_bytes;
   if (stages > 8) stages = 8;
   if (getenv("CS_TUNE_SMEM_KB")) stages = min(12, (atoi(getenv("CS_TUNE_SMEM_KB")) * 1024 - fixed) / stage_bytes);
   // the parked tile ([n_tok][128] fp32) reuses the ring
-  if (stages < 2 || (size_t)stages * stage_bytes < (size_t)a.n_tok * CS_GEMM_BM * 4) {
+  // (a GEMM that feeds a norm keeps [n_tok][32] more floats behind it)
+  if (stages < 2 || (size_t)stages * stage_bytes < (size_t)a.n_tok * (CS_GEMM_BM + 32) * 4) {
     snprintf(ctx->err, sizeof(ctx->err), "GEMM stage of %d bytes does not fit shared memory", stage_bytes);
     return CS_ERR_UNSUPPORTED;
   }
@@ -721,12 +772,13 @@ extern "C" cs_status cs_lm_head_static(const void* X, const void* W, int rows, i
   a.act_lo = nullptr;
   a.lo_row = -1;
   a.F = 0;
+  a.nf = NormFuse{};
   a.tile_max = tile_max;
   a.tile_idx = tile_idx;
   a.tile_stride = kStaticMaxRows;
   a.status = status;
   const int stage_bytes = kTileABytes + a.n_tok * 128;
-  const int fixed = 1024 + (2 * 8 + 1) * 8 + 16 + 8 * a.n_tok * 4;
+  const int fixed = 1024 + (2 * 8 + 1) * 8 + 16 + 9 * a.n_tok * 4;
   int stages = (100 * 1024 - fixed) / stage_bytes;
   if (stages > 8) stages = 8;
   if (stages < 2) return CS_ERR_UNSUPPORTED;
