@@ -11,6 +11,8 @@
 // through a double-buffered cp.async pipeline in shared memory (rows padded by 16 bytes so
 // that fragment loads and ldmatrix are bank-conflict free).  Each slice writes its
 // un-normalised output and (max, sum); k_attn_merge combines the slices.
+#include <stdlib.h>
+
 #include "cs_common.cuh"
 
 namespace {
@@ -275,7 +277,11 @@ int launch(cs_ctx* ctx, const void* kv_cache, int layer, int B, int R, cudaStrea
 }  // namespace
 
 void cs_launch_attention(cs_ctx* ctx, const void* kv_cache, int layer, int B, int R, cudaStream_t st) {
-  int nsplit;
+  int nsplit = getenv("CS_ATTN_LEGACY") ? 0 : cs_launch_attention_tc(ctx, kv_cache, layer, B, R, st);
+  if (nsplit > 0) {
+    cs_launch_attn_merge(ctx, nsplit, B * R, st);
+    return;
+  }
   switch (ctx->cfg.head_dim) {
     case 32: nsplit = launch<32>(ctx, kv_cache, layer, B, R, st); break;
     case 64: nsplit = launch<64>(ctx, kv_cache, layer, B, R, st); break;

@@ -1,0 +1,441 @@
+// Causal block attention over the bf16 KV cache on the 5th-generation tensor cores
+// (Sec. 3.2; App. B.2), for head_dim 128 and up to 128 query rows per KV head.
+//
+// One CTA = one (sequence, KV head) and one slice of the key range.  The query rows (the
+// (k+1) block rows of the G query heads sharing the KV head) are the M dimension of both
+// products, so that TMEM lane i belongs to query row i and the whole online softmax of a
+// row is private to one thread:
+//     S [128 x 128 keys]  = Q_hi K_tile^T + Q_lo K_tile^T     (tcgen05.mma, A and B K-major)
+//     O [128 x 128 dims] += P_hi V_tile  + P_lo V_tile        (tcgen05.mma, B MN-major)
+// Queries and softmax weights enter as two bf16 terms each, so they are fp32-equivalent and
+// only K and V - which the cache stores in bf16 - are rounded.  Only the first nq of the 128
+// rows are real: the A-operand buffers hold just those rows and the MMAs read on into the
+// shared memory behind them; whatever they find there only reaches accumulator rows that
+// nobody reads.  K and V tiles arrive by TMA (128-byte swizzle, two 64-wide halves) through
+// an mbarrier ring.  Each CTA writes its un-normalised (O, max, sum); k_attn_merge combines
+// the slices.  Every wait is bounded (2 s): on expiry the CTA flags CS_DEV_TIMEOUT, drains
+// its copies, frees its TMEM and returns.
+#include <stdlib.h>
+
+#include "cs_common.cuh"
+
+namespace {
+
+constexpr int kThreads = 192;   // warps 0-3 softmax/epilogue, warp 4 TMA producer, warp 5 MMA
+constexpr int kTileKeys = 128;
+constexpr int kDh = 128;
+constexpr int kHalfBytes = kTileKeys * 128;          // one [128 keys x 64 dims] half tile
+constexpr int kNQMax = 128;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+
+struct AttnArgs {
+  const int* row_lim;
+  int layer, R, G, H, Hkv, max_batch, max_seq, nsplit, NQ, rows, stages;
+  float scale_log2e;
+  float* out_o;
+  float* out_ml;
+  int* status;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  unsigned long long t0 = 0;
+  for (uint32_t it = 0;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 1023u) == 1023u) {
+      if (*abort_flag) return false;
+      const unsigned long long now = globaltimer_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > kWaitLimitNs) return false;
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+// operand descriptors, 128-byte swizzle.  K-major: rows of 128 bytes, 8-row groups 1024 bytes
+// apart.  MN-major: rows (one per K index) of 128 bytes holding 64 contiguous MN elements,
+// 8-row groups 1024 bytes apart (stride field), the next 64 MN elements `lbo` bytes further.
+__device__ __forceinline__ uint64_t desc_kmajor(uint32_t saddr) {
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
+         ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+__device__ __forceinline__ uint64_t desc_mnmajor(uint32_t saddr, uint32_t lbo) {
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
+         ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const float (&v)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
+        "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])),
+        "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])),
+        "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])),
+        "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])),
+        "r"(__float_as_uint(v[15]))
+      : "memory");
+}
+// eight values as eight leading bf16 terms and the eight bf16 terms of what that rounding lost
+__device__ __forceinline__ void split8(const float* p, uint4& hi, uint4& lo) {
+  uint32_t h[4], l[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const __nv_bfloat162 a = __floats2bfloat162_rn(p[2 * i], p[2 * i + 1]);
+    const float2 af = __bfloat1622float2(a);
+    const __nv_bfloat162 b = __floats2bfloat162_rn(p[2 * i] - af.x, p[2 * i + 1] - af.y);
+    h[i] = *reinterpret_cast<const uint32_t*>(&a);
+    l[i] = *reinterpret_cast<const uint32_t*>(&b);
+  }
+  hi = make_uint4(h[0], h[1], h[2], h[3]);
+  lo = make_uint4(l[0], l[1], l[2], l[3]);
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUtensorMap tmQ, AttnArgs a) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  uint8_t* smem = smem_raw + (((raw + 1023u) & ~1023u) - raw);
+  const int NQ = a.NQ, G = a.G, R = a.R, nq = G * R, stages = a.stages;
+  const uint32_t qhalf = (uint32_t)NQ * 128u;          // [NQ rows x 64 elements] of one term
+  const uint32_t qterm = 2u * qhalf;
+  // A operands first, K/V behind them: the MMAs' reads past row NQ stay inside the allocation
+  uint8_t* sQ = smem;                                  // [term][half][NQ][128 B]
+  uint8_t* sP = sQ + 2 * qterm;                        // same shape, 64 keys per half
+  uint8_t* sK = sP + 2 * qterm;                        // [stage][half][128 keys][128 B]
+  uint8_t* sV = sK + (size_t)stages * 2 * kHalfBytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sV + (size_t)stages * 2 * kHalfBytes);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 10);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  volatile int* s_never = reinterpret_cast<volatile int*>(tmem_slot + 2);
+  int* s_lmax = reinterpret_cast<int*>(tmem_slot + 3);
+  const uint32_t b_kfull = smem_u32(bars), b_vfull = smem_u32(bars + 2), b_free = smem_u32(bars + 4),
+                 b_qfull = smem_u32(bars + 6), b_sready = smem_u32(bars + 7), b_pready = smem_u32(bars + 8),
+                 b_odone = smem_u32(bars + 9);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int b = blockIdx.x / a.Hkv, kvh = blockIdx.x % a.Hkv, split = blockIdx.y;
+  const int nact = (nq + 31) >> 5;                     // softmax warps that own real rows
+  constexpr uint32_t kTmemCols = 256, kOCol = 128;     // S in columns 0..127, O in 128..255
+
+  if (tid == 128) {
+    for (int s = 0; s < 2; ++s) { mbar_init(b_kfull + 8 * s, 1); mbar_init(b_vfull + 8 * s, 1); mbar_init(b_free + 8 * s, 1); }
+    mbar_init(b_qfull, 1);
+    mbar_init(b_sready, 1);
+    mbar_init(b_pready, (uint32_t)nact * 32u);
+    mbar_init(b_odone, 1);
+    *s_abort = 0; *s_never = 0; *s_lmax = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmKV) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmQ) : "memory");
+  }
+  if (warp == 5) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot;
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+
+  if (warp < 4) {
+    int lm = 0;
+    for (int r = tid; r < R; r += 128) lm = max(lm, a.row_lim[b * R + r]);
+    lm = __reduce_max_sync(0xffffffffu, lm);
+    if (lane == 0 && lm > 0) atomicMax(s_lmax, lm);
+  }
+  __syncthreads();
+  const int lmax = *s_lmax;
+  const int ntiles = (lmax + kTileKeys - 1) / kTileKeys;
+  // tiles dealt out evenly over the slices
+  const int t0 = (int)((long long)ntiles * split / a.nsplit), t1 = (int)((long long)ntiles * (split + 1) / a.nsplit);
+  const int ntl = t1 - t0;
+
+  if (warp == 4) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0 && ntl > 0) {
+      mbar_expect_tx(b_qfull, (uint32_t)(4 * nq * 128));
+      for (int term = 0; term < 2; ++term)
+        for (int dh = 0; dh < 2; ++dh)
+          tma_load_3d(smem_u32(sQ + term * qterm + dh * qhalf), &tmQ, b_qfull, dh * 64, kvh * G, term * CS_MAX_ROWS + b * R);
+      const long long krow = ((((long long)a.layer * 2 + 0) * a.max_batch + b) * a.Hkv + kvh) * (long long)a.max_seq;
+      const long long vrow = ((((long long)a.layer * 2 + 1) * a.max_batch + b) * a.Hkv + kvh) * (long long)a.max_seq;
+      int i = 0;
+      bool ok = true;
+      for (; i < ntl; ++i) {
+        const int s = i % stages;
+        const uint32_t ph = (uint32_t)(i / stages) & 1u;
+        if (!mbar_wait(b_free + 8 * s, ph ^ 1u, s_abort)) { ok = false; break; }
+        const int key0 = (t0 + i) * kTileKeys;
+        const uint32_t dk = smem_u32(sK + (size_t)s * 2 * kHalfBytes), dv = smem_u32(sV + (size_t)s * 2 * kHalfBytes);
+        mbar_expect_tx(b_kfull + 8 * s, 2u * kHalfBytes);
+        tma_load_2d(dk, &tmKV, b_kfull + 8 * s, 0, (int)(krow + key0));
+        tma_load_2d(dk + kHalfBytes, &tmKV, b_kfull + 8 * s, 64, (int)(krow + key0));
+        mbar_expect_tx(b_vfull + 8 * s, 2u * kHalfBytes);
+        tma_load_2d(dv, &tmKV, b_vfull + 8 * s, 0, (int)(vrow + key0));
+        tma_load_2d(dv + kHalfBytes, &tmKV, b_vfull + 8 * s, 64, (int)(vrow + key0));
+      }
+      if (!ok) { *s_abort = 1; atomicOr(a.status, CS_DEV_TIMEOUT); }
+      if (*s_abort) {   // let the copies land before the shared memory goes away
+        mbar_wait(b_qfull, 0, s_never);
+        for (int j = max(0, i - stages); j < i; ++j) {
+          mbar_wait(b_kfull + 8 * (j % stages), (uint32_t)(j / stages) & 1u, s_never);
+          mbar_wait(b_vfull + 8 * (j % stages), (uint32_t)(j / stages) & 1u, s_never);
+        }
+      }
+    }
+  } else if (warp == 5) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0 && ntl > 0) {
+      const uint32_t idesc1 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+      const uint32_t idesc2 = idesc1 | (1u << 16);      // B (= V) is MN-major
+      bool ok = mbar_wait(b_qfull, 0, s_abort);
+      for (int i = 0; i < ntl && ok; ++i) {
+        const int s = i % stages;
+        const uint32_t ph = (uint32_t)(i / stages) & 1u;
+        if (!mbar_wait(b_kfull + 8 * s, ph, s_abort)) { ok = false; break; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t ak = smem_u32(sK + (size_t)s * 2 * kHalfBytes), aq = smem_u32(sQ);
+#pragma unroll
+        for (int term = 0; term < 2; ++term)
+#pragma unroll
+          for (int dh = 0; dh < 2; ++dh)
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+              umma_bf16(tmem_base, desc_kmajor(aq + term * qterm + dh * qhalf) + 2 * kk, desc_kmajor(ak + dh * kHalfBytes) + 2 * kk,
+                        idesc1, (term | dh | kk) ? 1u : 0u);
+        umma_commit(b_sready);
+        if (!mbar_wait(b_pready, (uint32_t)i & 1u, s_abort) || !mbar_wait(b_vfull + 8 * s, ph, s_abort)) { ok = false; break; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t av = smem_u32(sV + (size_t)s * 2 * kHalfBytes), ap = smem_u32(sP);
+#pragma unroll
+        for (int term = 0; term < 2; ++term)
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk)   // 16 keys per instruction
+            umma_bf16(tmem_base + kOCol, desc_kmajor(ap + term * qterm + (kk >> 2) * qhalf) + 2 * (kk & 3),
+                      desc_mnmajor(av + kk * 2048, kHalfBytes), idesc2, (i > 0 || term > 0 || kk > 0) ? 1u : 0u);
+        umma_commit(b_free + 8 * s);
+        umma_commit(b_odone);
+      }
+      if (!ok) { *s_abort = 1; atomicOr(a.status, CS_DEV_TIMEOUT); }
+    }
+  } else if (warp < nact) {
+    // ------------------------------------------------------------------ softmax + epilogue (thread = query row)
+    const int q = tid;
+    const bool valid = q < nq;
+    const int lim = valid ? a.row_lim[b * R + q / G] : 0;
+    const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
+    const float sc = a.scale_log2e;
+    float m = -INFINITY, l = 0.f;                      // running max (log2 domain) and sum of this row
+    bool have = ntl > 0;
+    for (int i = 0; i < ntl; ++i) {
+      const int s = i % stages;
+      const uint32_t ph = (uint32_t)(i / stages) & 1u;
+      const int key0 = (t0 + i) * kTileKeys;
+      // (S of this tile complete also means the previous tile's P V product has retired:
+      //  P may be overwritten and O is up to date)
+      bool ok = mbar_wait(b_sready, (uint32_t)i & 1u, s_abort);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) { *s_abort = 1; have = false; break; }
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      float mx = -INFINITY;
+#pragma unroll 1
+      for (int c = 0; c < 8; ++c) {
+        float v[16];
+        tmem_ld16(lane_base + (uint32_t)(c * 16), v);
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+          if (key0 + c * 16 + j < lim) mx = fmaxf(mx, v[j] * sc);
+      }
+      const float m_new = fmaxf(m, mx);
+      const float corr = (m == -INFINITY) ? 0.f : exp2f(m - m_new);
+      if (i > 0 && __any_sync(0xffffffffu, m_new > m)) {
+#pragma unroll 1
+        for (int c = 0; c < 8; ++c) {
+          float o[16];
+          tmem_ld16(lane_base + kOCol + (uint32_t)(c * 16), o);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) o[j] *= corr;
+          tmem_st16(lane_base + kOCol + (uint32_t)(c * 16), o);
+        }
+        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+      }
+      l *= corr;
+      m = m_new;
+      uint8_t* prow = sP + (size_t)q * 128;
+#pragma unroll 1
+      for (int c = 0; c < 8; ++c) {
+        float v[16];
+        tmem_ld16(lane_base + (uint32_t)(c * 16), v);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          v[j] = (key0 + c * 16 + j < lim) ? exp2f(v[j] * sc - m_new) : 0.f;
+          l += v[j];
+        }
+        if (valid) {
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            uint4 hi, lo;
+            split8(v + 8 * h, hi, lo);
+            const uint32_t off = (uint32_t)(c >> 2) * qhalf + ((((uint32_t)(2 * c + h) & 7u) ^ ((uint32_t)q & 7u)) << 4);
+            *reinterpret_cast<uint4*>(prow + off) = hi;
+            *reinterpret_cast<uint4*>(prow + qterm + off) = lo;
+          }
+        }
+      }
+      // keys past the longest row of this sequence hold whatever the cache held: zero their V rows
+      if (key0 + kTileKeys > lmax) {
+        if (!mbar_wait(b_vfull + 8 * s, ph, s_abort)) *s_abort = 1;
+        uint8_t* vs = sV + (size_t)s * 2 * kHalfBytes;
+        for (int rr = max(lmax - key0, 0) + tid; rr < kTileKeys; rr += nact * 32) {
+#pragma unroll
+          for (int c = 0; c < 8; ++c) {
+            *reinterpret_cast<uint4*>(vs + (size_t)rr * 128 + c * 16) = make_uint4(0u, 0u, 0u, 0u);
+            *reinterpret_cast<uint4*>(vs + kHalfBytes + (size_t)rr * 128 + c * 16) = make_uint4(0u, 0u, 0u, 0u);
+          }
+        }
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      mbar_arrive(b_pready);
+    }
+    // ---- un-normalised result of this key slice
+    if (have) {
+      bool ok = mbar_wait(b_odone, (uint32_t)(ntl - 1) & 1u, s_abort);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) { *s_abort = 1; have = false; }
+    }
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const size_t obase = valid ? ((size_t)split * a.rows + (b * R + q / G)) * a.H + (kvh * G + q % G) : 0;
+#pragma unroll 1
+    for (int c = 0; c < 8; ++c) {
+      float o[16];
+      if (have) {
+        tmem_ld16(lane_base + kOCol + (uint32_t)(c * 16), o);
+      } else {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) o[j] = 0.f;
+      }
+      if (valid) {
+        float4* dst = reinterpret_cast<float4*>(a.out_o + obase * kDh + c * 16);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) dst[j] = make_float4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+      }
+    }
+    if (valid) {
+      constexpr float kLn2 = 0.6931471805599453f;
+      a.out_ml[obase * 2] = have ? m * kLn2 : -INFINITY;
+      a.out_ml[obase * 2 + 1] = have ? l : 0.f;
+    }
+    if (*s_abort && lane == 0) atomicOr(a.status, CS_DEV_TIMEOUT);
+  }
+  // ---------------------------------------------------------------------- teardown
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 5) {
+    if (*s_abort && lane == 0 && ntl > 0) mbar_wait(b_odone, (uint32_t)(ntl - 1) & 1u, s_never);   // MMAs retired (bounded)
+    __syncwarp();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+}
+
+}  // namespace
+
+int cs_launch_attention_tc(cs_ctx* ctx, const void* kv_cache, int layer, int B, int R, cudaStream_t st) {
+  const cs_model_config& c = ctx->cfg;
+  const int G = c.n_heads / c.n_kv_heads, nq = G * R;
+  if (c.head_dim != kDh || nq > kNQMax || R < 1 || R > 256 || G > 256) return 0;
+  const int NQ = (nq + 15) / 16 * 16;
+  if (ctx->tmKV_base != kv_cache) {
+    const unsigned long long rows = (unsigned long long)c.n_layers * 2 * c.max_batch * c.n_kv_heads * c.max_seq;
+    if (rows > 0x7fffffffull) return 0;
+    const unsigned long long dims[2] = {(unsigned long long)kDh, rows}, strides[1] = {kDh * 2};
+    const unsigned box[2] = {64, (unsigned)kTileKeys};
+    if (cs_encode_tiled(ctx, &ctx->tmKV, kv_cache, 2, dims, strides, box) != CS_OK) return -1;
+    ctx->tmKV_base = kv_cache;
+  }
+  if (ctx->tmQ_R != R) {
+    const unsigned long long dims[3] = {(unsigned long long)kDh, (unsigned long long)c.n_heads, 2ull * CS_MAX_ROWS};
+    const unsigned long long strides[2] = {kDh * 2, (unsigned long long)c.n_heads * kDh * 2};
+    const unsigned box[3] = {64, (unsigned)G, (unsigned)R};
+    if (cs_encode_tiled(ctx, &ctx->tmQ, ctx->qbuf, 3, dims, strides, box) != CS_OK) return -1;
+    ctx->tmQ_R = R;
+  }
+  int nsplit = ctx->num_sms / (B * c.n_kv_heads);
+  if (nsplit > ctx->attn_splits) nsplit = ctx->attn_splits;
+  if (nsplit < 1) nsplit = 1;
+  const size_t ab = (size_t)8 * NQ * 128;                       // Q and P, two terms of two halves each
+  const size_t misc = 10 * 8 + 16, limit = 227 * 1024;
+  const int stages = (1024 + ab + (size_t)2 * 4 * kHalfBytes + misc <= limit) ? 2 : 1;
+  const size_t smem = 1024 + ab + (size_t)stages * 4 * kHalfBytes + misc;
+  static size_t smem_set = 0;
+  if (smem > smem_set) {
+    if (cudaFuncSetAttribute(k_attn_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+      snprintf(ctx->err, sizeof(ctx->err), "attention needs %zu bytes of shared memory", smem);
+      return -1;
+    }
+    smem_set = smem;
+  }
+  AttnArgs a;
+  a.row_lim = ctx->row_lim;
+  a.layer = layer; a.R = R; a.G = G; a.H = c.n_heads; a.Hkv = c.n_kv_heads;
+  a.max_batch = c.max_batch; a.max_seq = c.max_seq; a.nsplit = nsplit; a.NQ = NQ; a.rows = B * R; a.stages = stages;
+  a.scale_log2e = 1.4426950408889634f / sqrtf((float)kDh);
+  a.out_o = ctx->attn_o; a.out_ml = ctx->attn_ml; a.status = ctx->d_status;
+  if (cs_launch_pdl(k_attn_tc, dim3(B * c.n_kv_heads, nsplit), dim3(kThreads), smem, st, ctx->tmKV, ctx->tmQ, a) != cudaSuccess) {
+    snprintf(ctx->err, sizeof(ctx->err), "attention launch failed");
+    return -1;
+  }
+  return nsplit;
+}

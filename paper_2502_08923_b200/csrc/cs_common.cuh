@@ -115,6 +115,12 @@ struct cs_ctx {
   int act_ntok;
   CUtensorMap tmXn, tmAttn, tmAct;
 
+  // tensor-core attention: maps over the whole KV cache (rebuilt when the cache pointer
+  // changes) and over the rotated queries (rebuilt when the block height changes)
+  CUtensorMap tmKV, tmQ;
+  const void* tmKV_base;
+  int tmQ_R;
+
   LoopState loop;
   Prof* prof;   // non-NULL only inside cs_profile_verify_step
 
@@ -218,6 +224,12 @@ void cs_launch_rmsnorm(cs_ctx* ctx, const __nv_bfloat16* gain, int rows, cudaStr
 void cs_launch_attention(cs_ctx* ctx, const void* kv_cache, int layer, int B, int R,
                          cudaStream_t st);
 void cs_launch_attn_merge(cs_ctx* ctx, int nsplit, int rows, cudaStream_t st);
+// tcgen05 path (head_dim 128, at most 128 query rows per KV head); returns the number of key
+// slices written, 0 when the shape is not covered, -1 on a host error (ctx->err set)
+int cs_launch_attention_tc(cs_ctx* ctx, const void* kv_cache, int layer, int B, int R, cudaStream_t st);
+// bf16 tensor map of rank <= 5, 128-byte swizzle; dims/box innermost first, strides for dims 1..
+cs_status cs_encode_tiled(cs_ctx* ctx, CUtensorMap* tm, const void* base, int rank, const unsigned long long* dims,
+                          const unsigned long long* strides_bytes, const unsigned* box);
 void cs_launch_accept(cs_ctx* ctx, int B, int k, const int32_t* draft, const int32_t* draft_len,
                       const int32_t* script, int script_stride, const int32_t* script_off,
                       int script_limit, int32_t* accept_len, int32_t* out_tokens,

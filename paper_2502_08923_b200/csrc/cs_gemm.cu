@@ -566,6 +566,31 @@ cs_status encode_2d(cs_ctx* ctx, CUtensorMap* tm, const void* base, int rows, in
 
 }  // namespace
 
+cs_status cs_encode_tiled(cs_ctx* ctx, CUtensorMap* tm, const void* base, int rank, const unsigned long long* dims,
+                          const unsigned long long* strides_bytes, const unsigned* box) {
+  EncodeTiledFn enc = get_encode();
+  if (enc == nullptr) {
+    snprintf(ctx->err, sizeof(ctx->err), "cuTensorMapEncodeTiled is not available");
+    return CS_ERR_CUDA;
+  }
+  if (rank < 1 || rank > 5 || (reinterpret_cast<uintptr_t>(base) & 15) != 0) {
+    snprintf(ctx->err, sizeof(ctx->err), "tensor map needs rank 1..5 and a 16-byte aligned base");
+    return CS_ERR_SHAPE;
+  }
+  cuuint64_t d[5], sb[4];
+  cuuint32_t bx[5], estr[5];
+  for (int i = 0; i < rank; ++i) { d[i] = dims[i]; bx[i] = box[i]; estr[i] = 1; }
+  for (int i = 0; i + 1 < rank; ++i) sb[i] = strides_bytes[i];
+  CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), d, sb, bx, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    snprintf(ctx->err, sizeof(ctx->err), "cuTensorMapEncodeTiled (rank %d) failed with %d", rank, (int)r);
+    return CS_ERR_CUDA;
+  }
+  return CS_OK;
+}
+
 cs_status cs_gemm_plan(cs_ctx* ctx, GemmPlan* g, const void* w, int N, int K, bool allow_split) {
   g->W = static_cast<const __nv_bfloat16*>(w);
   g->N = N;
