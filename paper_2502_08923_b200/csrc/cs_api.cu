@@ -5,6 +5,8 @@
 
 #include <new>
 
+#include <string.h>
+
 #include "cs_common.cuh"
 
 namespace {
@@ -241,6 +243,10 @@ cs_status cs_create(cs_ctx** out, const cs_model_config* cfg, const cs_weights* 
   ctx->max_rows = cfg->max_batch * (cfg->k_max + 1);
   ctx->rows_pad = CS_MAX_ROWS;
   ctx->attn_splits = L.attn_splits;
+  {
+    const char* k = getenv("CS_ATTN_KERNEL");
+    ctx->attn_force = (k == nullptr) ? 0 : (strcmp(k, "mma") == 0 ? 1 : (strcmp(k, "tc") == 0 ? 2 : 0));
+  }
   ctx->qkv_elems = L.qkv_elems;
   ctx->layers = new (std::nothrow) LayerPlan[cfg->n_layers];
   cs_status s = CS_OK;

@@ -120,6 +120,7 @@ struct cs_ctx {
   CUtensorMap tmKV, tmQ;
   const void* tmKV_base;
   int tmQ_R;
+  int attn_force;            // 0 = choose by shape, 1 = mma.sync kernel, 2 = tcgen05 kernel
 
   LoopState loop;
   Prof* prof;   // non-NULL only inside cs_profile_verify_step

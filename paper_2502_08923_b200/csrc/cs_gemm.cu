@@ -144,6 +144,16 @@ __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+// the two halves of the cluster barrier; like every barrier they count whole warps, so each
+// warp executes each half exactly once, with all its lanes converged
+__device__ __forceinline__ void cluster_arrive() {
+  __syncwarp();
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_wait() {
+  __syncwarp();
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 __device__ __forceinline__ uint32_t cluster_rank() {
   uint32_t r;
   asm volatile("mov.u32 %0, %cluster_ctarank;" : "=r"(r));
@@ -168,6 +178,12 @@ __device__ __forceinline__ float4 sum_over_ranks(uint32_t local_addr, int splits
 #pragma unroll
   for (int q = 1; q < CS_MAX_SPLITS; ++q) { y.x += v[q].x; y.y += v[q].y; y.z += v[q].z; y.w += v[q].w; }
   return y;
+}
+
+// The remote loads behind two sums must have returned before what follows is issued: an
+// empty asm that takes the sums as inputs cannot be scheduled before they exist.
+__device__ __forceinline__ void keep_alive(const float4& p, const float4& q) {
+  asm volatile("" ::"f"(p.x), "f"(p.y), "f"(p.z), "f"(p.w), "f"(q.x), "f"(q.y), "f"(q.z), "f"(q.w) : "memory");
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -367,10 +383,24 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
   if (a.mode != CS_EPI_ARGMAX) {
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
-    if (a.splits > 1) cluster_sync_all();          // every rank's tile is parked
+    // Cluster barrier 1: every rank's tile is parked.  Barrier 2 (nobody leaves while a peer
+    // still reads its tile) is split: a warp arrives as soon as the last remote reads of its lanes
+    // have returned and only waits after its global stores, which hides the barrier behind them.
+    if (a.splits > 1) cluster_arrive();
+    const int e = threadIdx.x;
+    // residual update: the first item's x (and gain) can be on their way during the barrier
+    const int r_fs = ((CS_GEMM_BM + a.splits - 1) / a.splits + 3) & ~3;
+    const int r_flo = split * r_fs, r_per_tok = max(0, min(CS_GEMM_BM, r_flo + r_fs) - r_flo) >> 2;
+    const bool r_vec = (a.N & 3) == 0;
+    float4 x_pre = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (warp < 4 && a.mode == CS_EPI_RESIDUAL && r_vec && e < r_per_tok * a.rows) {
+      const int f = r_flo + 4 * (e % r_per_tok), tok = e / r_per_tok;
+      if (n0 + f + 3 < a.N) x_pre = *reinterpret_cast<const float4*>(a.out + (size_t)tok * a.N + n0 + f);
+    }
+    if (a.splits > 1) cluster_wait();
+    bool arrived = a.splits <= 1;                  // this thread's half of barrier 2
     if (warp < 4) {
       const uint32_t dump_addr = smem_u32(dump);
-      const int e = threadIdx.x;                   // 0..127
       if (a.mode == CS_EPI_QKV) {
         // RoPE pairs feature i of a head with i + Dh/2: both lie in this tile.  j in [0,64) walks
         // the first halves of the tile's heads; each rank finishes a slice of j, four at a time.
@@ -379,19 +409,26 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
         const int js = ((64 + a.splits - 1) / a.splits + 3) & ~3;
         const int j_lo = split * js, j_n = max(0, min(64, j_lo + js) - j_lo);
         const int per_tok = j_n >> 2;
-        for (int idx = e; idx < per_tok * a.rows; idx += 128) {
-          const int j = j_lo + 4 * (idx % per_tok), tok = idx / per_tok;
+        const int total = per_tok * a.rows, iters = (total + 127) >> 7;   // same trip count for every thread
+        for (int it = 0; it < iters; ++it) {
+          const int idx = e + (it << 7);
+          const int idc = idx < total ? idx : 0;
+          const int j = j_lo + 4 * (idc % per_tok), tok = idc / per_tok;
           const int i = j % half, f1 = (j / half) * Q.Dh + i, f2 = f1 + half;
           const int head = (n0 + f1) / Q.Dh;
-          if (head >= Q.H + 2 * Q.Hkv) continue;
-          float4 av, bv;
+          const bool act = idx < total && head < Q.H + 2 * Q.Hkv;
+          float4 av = make_float4(0.f, 0.f, 0.f, 0.f), bv = av;
           if (a.splits > 1) {
-            av = sum_over_ranks(dump_addr + 4u * (uint32_t)(tok * CS_GEMM_BM + f1), a.splits);
-            bv = sum_over_ranks(dump_addr + 4u * (uint32_t)(tok * CS_GEMM_BM + f2), a.splits);
-          } else {
+            if (act) {
+              av = sum_over_ranks(dump_addr + 4u * (uint32_t)(tok * CS_GEMM_BM + f1), a.splits);
+              bv = sum_over_ranks(dump_addr + 4u * (uint32_t)(tok * CS_GEMM_BM + f2), a.splits);
+            }
+            if (it == iters - 1) { keep_alive(av, bv); cluster_arrive(); arrived = true; }
+          } else if (act) {
             av = *reinterpret_cast<const float4*>(dump + tok * CS_GEMM_BM + f1);
             bv = *reinterpret_cast<const float4*>(dump + tok * CS_GEMM_BM + f2);
           }
+          if (!act) continue;
           const float a4[4] = {av.x, av.y, av.z, av.w}, b4[4] = {bv.x, bv.y, bv.z, bv.w};
           float r0[4], r1[4];
           const bool is_v = head >= Q.H + Q.Hkv;
@@ -432,17 +469,38 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
         const int js = ((64 + a.splits - 1) / a.splits + 3) & ~3;
         const int j_lo = split * js, j_n = max(0, min(64, j_lo + js) - j_lo);
         const int per_tok = j_n >> 2;
-        for (int idx = e; idx < per_tok * a.rows; idx += 128) {
-          const int j = j_lo + 4 * (idx % per_tok), tok = idx / per_tok;
-          float4 g, u;
+        const int total = per_tok * a.rows, iters = (total + 127) >> 7;
+        for (int it = 0; it < iters; ++it) {
+          const int idx = e + (it << 7);
+          const bool act = idx < total;
+          const int idc = act ? idx : 0;
+          const int j = j_lo + 4 * (idc % per_tok), tok = idc / per_tok;
+          float4 g = make_float4(0.f, 0.f, 0.f, 0.f), u = g;
           if (a.splits > 1) {
-            g = sum_over_ranks(dump_addr + 4u * (uint32_t)(tok * CS_GEMM_BM + j), a.splits);
-            u = sum_over_ranks(dump_addr + 4u * (uint32_t)(tok * CS_GEMM_BM + 64 + j), a.splits);
-          } else {
+            if (act) {
+              g = sum_over_ranks(dump_addr + 4u * (uint32_t)(tok * CS_GEMM_BM + j), a.splits);
+              u = sum_over_ranks(dump_addr + 4u * (uint32_t)(tok * CS_GEMM_BM + 64 + j), a.splits);
+            }
+            if (it == iters - 1) { keep_alive(g, u); cluster_arrive(); arrived = true; }
+          } else if (act) {
             g = *reinterpret_cast<const float4*>(dump + tok * CS_GEMM_BM + j);
             u = *reinterpret_cast<const float4*>(dump + tok * CS_GEMM_BM + 64 + j);
           }
+          if (!act) continue;
           const float gv[4] = {g.x, g.y, g.z, g.w}, uv[4] = {u.x, u.y, u.z, u.w};
+          const int jj0 = tile * 64 + j;
+          if ((a.F & 3) == 0 && jj0 + 3 < a.F) {
+            float v4[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) v4[i] = gv[i] / (1.f + expf(-gv[i])) * uv[i];
+            __nv_bfloat162 h[2], l[2];
+            h[0] = __floats2bfloat162_rn(v4[0], v4[1]); h[1] = __floats2bfloat162_rn(v4[2], v4[3]);
+            const float2 h0 = __bfloat1622float2(h[0]), h1 = __bfloat1622float2(h[1]);
+            l[0] = __floats2bfloat162_rn(v4[0] - h0.x, v4[1] - h0.y); l[1] = __floats2bfloat162_rn(v4[2] - h1.x, v4[3] - h1.y);
+            *reinterpret_cast<uint2*>(a.act + (size_t)tok * a.F + jj0) = *reinterpret_cast<const uint2*>(h);
+            if (a.act_lo != nullptr) *reinterpret_cast<uint2*>(a.act_lo + (size_t)tok * a.F + jj0) = *reinterpret_cast<const uint2*>(l);
+            continue;
+          }
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             const int jj = tile * 64 + j + i;
@@ -460,18 +518,27 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
         const int per_tok = f_n >> 2;
         const bool feeds_norm = a.mode == CS_EPI_RESIDUAL && a.nf.gain_out != nullptr;
         float* part = dump + a.n_tok * CS_GEMM_BM;   // [rows][32] sums of squares, behind the parked tile
-        for (int idx = e; idx < per_tok * a.rows; idx += 128) {
-          const int f = f_lo + 4 * (idx % per_tok), tok = idx / per_tok;
+        const int total = per_tok * a.rows, iters = (total + 127) >> 7;
+        for (int it = 0; it < iters; ++it) {
+          const int idx = e + (it << 7);
+          const bool act = idx < total;
+          const int idc = act ? idx : 0;
+          const int f = f_lo + 4 * (idc % per_tok), tok = idc / per_tok;
+          float4 y = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (a.splits > 1) {
+            if (act) y = sum_over_ranks(dump_addr + 4u * (uint32_t)(tok * CS_GEMM_BM + f), a.splits);
+            if (it == iters - 1) { keep_alive(y, y); cluster_arrive(); arrived = true; }
+          } else if (act) {
+            y = *reinterpret_cast<const float4*>(dump + tok * CS_GEMM_BM + f);
+          }
+          if (!act) continue;
           if (feeds_norm) part[tok * 32 + idx % per_tok] = 0.f;
-          float4 y;
-          if (a.splits > 1) y = sum_over_ranks(dump_addr + 4u * (uint32_t)(tok * CS_GEMM_BM + f), a.splits);
-          else y = *reinterpret_cast<const float4*>(dump + tok * CS_GEMM_BM + f);
           const float yv[4] = {y.x, y.y, y.z, y.w};
           float* dst = a.out + (size_t)tok * a.N + n0 + f;
           if (n0 + f + 3 < a.N && (a.N & 3) == 0) {
             float4 o = y;
             if (a.mode == CS_EPI_RESIDUAL) {
-              const float4 x = *reinterpret_cast<const float4*>(dst);
+              const float4 x = (it == 0) ? x_pre : *reinterpret_cast<const float4*>(dst);
               o.x += x.x; o.y += x.y; o.z += x.z; o.w += x.w;
             }
             *reinterpret_cast<float4*>(dst) = o;
@@ -505,7 +572,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
         }
       }
     }
-    if (a.splits > 1) cluster_sync_all();          // nobody leaves while a peer still reads its tile
+    if (a.splits > 1) {
+      if (!arrived) cluster_arrive();
+      cluster_wait();                              // nobody leaves while a peer still reads its tile
+    }
   }
   // ---------------------------------------------------------------- teardown
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");

@@ -21,11 +21,15 @@ def _kv_close(kv_gpu, cache, b_gpu, b_or, n, tol=2e-2):
     return np.abs(got - want).max() <= tol, float(np.abs(got - want).max())
 
 
-@pytest.mark.parametrize("cfg_name", ["tiny", "gqa"])
-def test_prefill_and_verify_steps(cfg_name):
+@pytest.mark.parametrize("cfg_name", ["tiny", "gqa", "gqa-tc", "gqa-mma"])
+def test_prefill_and_verify_steps(cfg_name, monkeypatch):
     if cfg_name == "tiny":
         cfg = inputs.TINY
     else:   # grouped-query attention with 128-wide heads, odd sizes that leave ragged tiles
+        # (the library picks the attention kernel by shape; the suffix forces one of the two
+        #  for contexts created from here on, so both are checked on the same case)
+        if "-" in cfg_name:
+            monkeypatch.setenv("CS_ATTN_KERNEL", cfg_name.split("-")[1])
         cfg = inputs.ModelConfig(n_layers=2, d_model=320, n_heads=4, n_kv_heads=2, head_dim=128, d_ffn=1000,
                                  vocab=1000, rope_theta=500000.0, rms_eps=1e-5)
     B, k, max_seq = 3, 10, 700
