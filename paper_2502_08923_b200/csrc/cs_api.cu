@@ -12,7 +12,7 @@
 namespace {
 
 struct WsLayout {
-  size_t x, xn, attn_out, act, qbuf, partial, attn_o, attn_ml, ssq, chain_bar, chain_scratch, rope_cs, inv_freq, tile_max, tile_idx,
+  size_t x, xn, attn_out, act, qbuf, partial, attn_o, attn_ml, ssq, rope_cs, inv_freq, tile_max, tile_idx,
       row_tok, row_pos, row_lim, row_write, seq_ok, status, loop_last, loop_draft, loop_dlen, loop_mpos,
       loop_emitted, loop_done, loop_accept, loop_out, loop_argmax, loop_stats, total;
   size_t qkv_elems;
@@ -57,8 +57,6 @@ WsLayout ws_layout(const cs_model_config* c) {
   L.attn_o = take(&off, (size_t)L.attn_splits * rows * qd * 4);
   L.attn_ml = take(&off, (size_t)L.attn_splits * rows * c->n_heads * 2 * 4);
   L.ssq = take(&off, rows * (size_t)cs_ceil_div(c->d_model, CS_GEMM_BM) * CS_MAX_SPLITS * 4);
-  L.chain_bar = take(&off, CS_CHAIN_BAR_WORDS * 4);
-  L.chain_scratch = take(&off, (size_t)cs_ceil_div(c->d_model, CS_GEMM_BM) * CS_MAX_SPLITS * CS_CHAIN_MAX_TOK * CS_GEMM_BM * 4);
   L.rope_cs = take(&off, rows * c->head_dim * 4);
   L.inv_freq = take(&off, (size_t)c->head_dim / 2 * 8);
   L.tile_max = take(&off, lm_tiles * rows * 4);
@@ -108,13 +106,6 @@ void prof_begin(cs_ctx* ctx, int fam, cudaStream_t st) {
   p->fam[p->n] = fam;
   cudaEventRecord(p->ev[2 * p->n], st);
 }
-// forget a bracket that was opened for a launch that did not happen
-void prof_drop(cs_ctx* ctx) {
-  Prof* p = ctx->prof;
-  if (p == nullptr || p->n >= CS_PROF_MAX) return;
-  cudaEventDestroy(p->ev[2 * p->n]);
-  cudaEventDestroy(p->ev[2 * p->n + 1]);
-}
 void prof_end(cs_ctx* ctx, cudaStream_t st) {
   Prof* p = ctx->prof;
   if (p == nullptr || p->n >= CS_PROF_MAX) return;
@@ -154,42 +145,34 @@ cs_status enqueue_forward(cs_ctx* ctx, int B, int R, void* kv_cache, bool with_l
     prof_begin(ctx, CS_FAM_ATTENTION, st);
     cs_launch_attention(ctx, kv_cache, l, B, R, st);
     prof_end(ctx, st);
+    prof_begin(ctx, CS_FAM_GEMM, st);
     NormFuse give = {};
     give.gain_out = L.ffn_norm;
     give.xn_out = ctx->xn;
     give.ssq_out = ctx->ssq;
     give.slot_stride = ctx->ssq_stride;
+    s = cs_launch_gemm(ctx, &L.o, &ctx->tmAttn, CS_MAX_ROWS, rows, CS_EPI_RESIDUAL, ctx->x, nullptr, nullptr, 0, nullptr,
+                       &give, st);
+    prof_end(ctx, st);
+    if (s != CS_OK) return s;
     take_norm = NormFuse{};
     take_norm.ssq_in = ctx->ssq;
     take_norm.slots_in = cs_ceil_div(L.o.N, CS_GEMM_BM) * L.o.splits;
     take_norm.slot_stride = ctx->ssq_stride;
     take_norm.inv_d = 1.f / (float)c.d_model;
     take_norm.eps = c.rms_eps;
-    // the norm after this layer: the next layer's, or the final one before the LM head
-    NormFuse give_next = give;
-    give_next.gain_out = (l + 1 < c.n_layers) ? ctx->layers[l + 1].attn_norm : (with_lm ? ctx->final_norm : nullptr);
-    // the three projections as one launch where the plans allow it, else one by one
     prof_begin(ctx, CS_FAM_GEMM, st);
-    s = cs_launch_gemm_chain(ctx, &L, rows, &give, &take_norm, &give_next, st);
-    if (s == CS_ERR_UNSUPPORTED) {
-      prof_drop(ctx);
-      prof_begin(ctx, CS_FAM_GEMM, st);
-      s = cs_launch_gemm(ctx, &L.o, &ctx->tmAttn, CS_MAX_ROWS, rows, CS_EPI_RESIDUAL, ctx->x, nullptr, nullptr, 0, nullptr,
-                         &give, st);
-      prof_end(ctx, st);
-      if (s != CS_OK) return s;
-      prof_begin(ctx, CS_FAM_GEMM, st);
-      s = cs_launch_gemm(ctx, &L.gate_up, &ctx->tmXn, CS_MAX_ROWS, rows, CS_EPI_SWIGLU, nullptr, ctx->act,
-                         ctx->act + (size_t)CS_MAX_ROWS * c.d_ffn, c.d_ffn, nullptr, &take_norm, st);
-      prof_end(ctx, st);
-      if (s != CS_OK) return s;
-      prof_begin(ctx, CS_FAM_GEMM, st);
-      s = cs_launch_gemm(ctx, &L.down, &ctx->tmAct, CS_MAX_ROWS, rows, CS_EPI_RESIDUAL, ctx->x, nullptr, nullptr, 0, nullptr,
-                         &give_next, st);
-      prof_end(ctx, st);
-    } else {
-      prof_end(ctx, st);
-    }
+    s = cs_launch_gemm(ctx, &L.gate_up, &ctx->tmXn, CS_MAX_ROWS, rows, CS_EPI_SWIGLU, nullptr, ctx->act,
+                       ctx->act + (size_t)CS_MAX_ROWS * c.d_ffn, c.d_ffn, nullptr, &take_norm, st);
+    prof_end(ctx, st);
+    if (s != CS_OK) return s;
+    // the norm after this layer: the next layer's, or the final one before the LM head
+    const __nv_bfloat16* next_gain = (l + 1 < c.n_layers) ? ctx->layers[l + 1].attn_norm : (with_lm ? ctx->final_norm : nullptr);
+    give.gain_out = next_gain;
+    prof_begin(ctx, CS_FAM_GEMM, st);
+    s = cs_launch_gemm(ctx, &L.down, &ctx->tmAct, CS_MAX_ROWS, rows, CS_EPI_RESIDUAL, ctx->x, nullptr, nullptr, 0, nullptr,
+                       &give, st);
+    prof_end(ctx, st);
     if (s != CS_OK) return s;
     take_norm.slots_in = cs_ceil_div(L.down.N, CS_GEMM_BM) * L.down.splits;
   }
@@ -302,9 +285,6 @@ cs_status cs_create(cs_ctx** out, const cs_model_config* cfg, const cs_weights* 
   ctx->attn_ml = reinterpret_cast<float*>(base + L.attn_ml);
   ctx->ssq = reinterpret_cast<float*>(base + L.ssq);
   ctx->ssq_stride = cs_ceil_div(ctx->cfg.d_model, CS_GEMM_BM) * CS_MAX_SPLITS;
-  ctx->chain_bar = reinterpret_cast<unsigned*>(base + L.chain_bar);
-  ctx->chain_scratch = reinterpret_cast<float*>(base + L.chain_scratch);
-  ctx->chain_state = getenv("CS_NO_CHAIN") ? -1 : 0;
   ctx->rope_cs = reinterpret_cast<float*>(base + L.rope_cs);
   ctx->inv_freq = reinterpret_cast<double*>(base + L.inv_freq);
   ctx->tile_max = reinterpret_cast<float*>(base + L.tile_max);
@@ -357,7 +337,6 @@ cs_status cs_create(cs_ctx** out, const cs_model_config* cfg, const cs_weights* 
     return s;
   }
 #undef CREATE_OK
-  cs_gemm_chain_probe(ctx, nullptr);
   *out = ctx;
   return CS_OK;
 }

@@ -35,9 +35,6 @@ struct GemmPlan {
   int kb_per_split;     // 64-wide K blocks per split
 };
 
-constexpr int CS_CHAIN_BAR_WORDS = 1024;   // 2 grid barriers + 2 x (d_model / 128) tile counters
-constexpr int CS_CHAIN_MAX_TOK = 64;       // tallest block the projection chain takes
-
 struct LayerPlan {
   GemmPlan qkv, o, gate_up, down;
   const __nv_bfloat16 *attn_norm, *ffn_norm;
@@ -124,11 +121,6 @@ struct cs_ctx {
   const void* tmKV_base;
   int tmQ_R;
   int attn_force;            // 0 = choose by shape, 1 = mma.sync kernel, 2 = tcgen05 kernel
-
-  // O / gate-up / down projections as one launch with grid barriers
-  unsigned* chain_bar;       // [CS_CHAIN_BAR_WORDS] barrier and tile counters, zeroed by k_attn_merge of the same layer
-  float* chain_scratch;      // split-K partial tiles [d/128 * CS_MAX_SPLITS][CS_CHAIN_MAX_TOK][128]
-  int chain_state;           // 0 = not probed yet, 1 = usable, -1 = not on this GPU / switched off
 
   LoopState loop;
   Prof* prof;   // non-NULL only inside cs_profile_verify_step
@@ -233,9 +225,6 @@ void cs_launch_rmsnorm(cs_ctx* ctx, const __nv_bfloat16* gain, int rows, cudaStr
 void cs_launch_attention(cs_ctx* ctx, const void* kv_cache, int layer, int B, int R,
                          cudaStream_t st);
 void cs_launch_attn_merge(cs_ctx* ctx, int nsplit, int rows, cudaStream_t st);
-cs_status cs_launch_gemm_chain(cs_ctx* ctx, const LayerPlan* L, int rows, const NormFuse* nf_o, const NormFuse* nf_gate_up,
-                               const NormFuse* nf_down, cudaStream_t st);
-void cs_gemm_chain_probe(cs_ctx* ctx, cudaStream_t st);
 // tcgen05 path (head_dim 128, at most 128 query rows per KV head); returns the number of key
 // slices written, 0 when the shape is not covered, -1 on a host error (ctx->err set)
 int cs_launch_attention_tc(cs_ctx* ctx, const void* kv_cache, int layer, int B, int R, cudaStream_t st);

@@ -153,11 +153,8 @@ k_rmsnorm(const float* __restrict__ x, int d, const __nv_bfloat16* __restrict__ 
 
 // Combine the key slices: o = sum_s o_s e^(m_s - M) / sum_s l_s e^(m_s - M).
 __global__ void k_attn_merge(const float* __restrict__ in_o, const float* __restrict__ in_ml, int nsplit,
-                             int rows, int H, int Dh, __nv_bfloat16* __restrict__ attn_out, unsigned* chain_bar) {
+                             int rows, int H, int Dh, __nv_bfloat16* __restrict__ attn_out) {
   CS_PDL_PROLOGUE();
-  // the grid-barrier counters of the projection chain that follows start from zero
-  if (blockIdx.x == 0 && blockIdx.y == 0)
-    for (int i = threadIdx.x; i < CS_CHAIN_BAR_WORDS; i += blockDim.x) chain_bar[i] = 0u;
   const int row = blockIdx.x, h = blockIdx.y, dd = threadIdx.x;
   const int lane = threadIdx.x & 31;
   // all partial outputs of this (row, head, dim) are requested at once, so their latencies
@@ -403,7 +400,7 @@ void cs_launch_rmsnorm(cs_ctx* ctx, const __nv_bfloat16* gain, int rows, cudaStr
 void cs_launch_attn_merge(cs_ctx* ctx, int nsplit, int rows, cudaStream_t st) {
   const cs_model_config& c = ctx->cfg;
   cs_launch_pdl(k_attn_merge, dim3(rows, c.n_heads), dim3(c.head_dim), 0, st, ctx->attn_o, ctx->attn_ml, nsplit, rows,
-                c.n_heads, c.head_dim, ctx->attn_out, ctx->chain_bar);
+                c.n_heads, c.head_dim, ctx->attn_out);
 }
 
 void cs_launch_accept(cs_ctx* ctx, int B, int k, const int32_t* draft, const int32_t* draft_len,
