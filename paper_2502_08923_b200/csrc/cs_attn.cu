@@ -277,11 +277,10 @@ int launch(cs_ctx* ctx, const void* kv_cache, int layer, int B, int R, cudaStrea
 }  // namespace
 
 void cs_launch_attention(cs_ctx* ctx, const void* kv_cache, int layer, int B, int R, cudaStream_t st) {
-  // The tcgen05 kernel wins once the query tile of a KV head no longer fits one 64-row
-  // mma.sync CTA; below that the register-resident kernel is faster (CS_ATTN_KERNEL=tc|mma,
-  // read when the context is created, forces one of them).
-  const int nq = ctx->cfg.n_heads / ctx->cfg.n_kv_heads * R;
-  const bool want_tc = ctx->attn_force == 2 || (ctx->attn_force == 0 && nq > 64);
+  // The tcgen05 kernel takes every shape it covers (head_dim 128, at most 128 query rows per KV
+  // head); the register-resident mma.sync kernel takes the rest.  CS_ATTN_KERNEL=tc|mma, read
+  // when the context is created, forces one of them (tests run both on the same inputs).
+  const bool want_tc = ctx->attn_force != 1;
   int nsplit = want_tc ? cs_launch_attention_tc(ctx, kv_cache, layer, B, R, st) : 0;
   if (nsplit > 0) {
     cs_launch_attn_merge(ctx, nsplit, B * R, st);

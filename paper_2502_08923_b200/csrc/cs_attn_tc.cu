@@ -112,6 +112,31 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
 #pragma unroll
   for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
+// 32 accumulator columns with one wait (two loads in flight)
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr + 16u));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+// 2^x, hardware approximation (relative error about 2^-22; -inf gives 0)
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const float (&v)[16]) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
@@ -153,7 +178,9 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
   uint8_t* sP = sQ + 2 * qterm;                        // same shape, 64 keys per half
   uint8_t* sK = sP + 2 * qterm;                        // [stage][half][128 keys][128 B]
   uint8_t* sV = sK + (size_t)stages * 2 * kHalfBytes;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(sV + (size_t)stages * 2 * kHalfBytes);
+  // barriers and flags live in the alignment slack: in front of the aligned area when it is at
+  // least 96 bytes, else in what is then left behind it
+  uint64_t* bars = reinterpret_cast<uint64_t*>((smem - smem_raw >= 96) ? smem_raw : sV + (size_t)stages * 2 * kHalfBytes);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 10);
   volatile int* s_abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
   volatile int* s_never = reinterpret_cast<volatile int*>(tmem_slot + 2);
@@ -194,29 +221,40 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
     lm = __reduce_max_sync(0xffffffffu, lm);
     if (lane == 0 && lm > 0) atomicMax(s_lmax, lm);
   }
+  // Slice `split` works on key tiles split, split + nsplit, ...: its first tile is known before
+  // the key range is, so the queries and that tile are requested while the range is worked out
+  // (a slice beyond the range only has to let them land).
+  const long long krow = ((((long long)a.layer * 2 + 0) * a.max_batch + b) * a.Hkv + kvh) * (long long)a.max_seq;
+  const long long vrow = ((((long long)a.layer * 2 + 1) * a.max_batch + b) * a.Hkv + kvh) * (long long)a.max_seq;
+  if (warp == 4 && lane == 0) {
+    mbar_expect_tx(b_qfull, (uint32_t)(4 * nq * 128));
+    for (int term = 0; term < 2; ++term)
+      for (int dh = 0; dh < 2; ++dh)
+        tma_load_3d(smem_u32(sQ + term * qterm + dh * qhalf), &tmQ, b_qfull, dh * 64, kvh * G, term * CS_MAX_ROWS + b * R);
+    const int key0 = split * kTileKeys;
+    const uint32_t dk = smem_u32(sK), dv = smem_u32(sV);
+    mbar_expect_tx(b_kfull, 2u * kHalfBytes);
+    tma_load_2d(dk, &tmKV, b_kfull, 0, (int)(krow + key0));
+    tma_load_2d(dk + kHalfBytes, &tmKV, b_kfull, 64, (int)(krow + key0));
+    mbar_expect_tx(b_vfull, 2u * kHalfBytes);
+    tma_load_2d(dv, &tmKV, b_vfull, 0, (int)(vrow + key0));
+    tma_load_2d(dv + kHalfBytes, &tmKV, b_vfull, 64, (int)(vrow + key0));
+  }
   __syncthreads();
   const int lmax = *s_lmax;
   const int ntiles = (lmax + kTileKeys - 1) / kTileKeys;
-  // tiles dealt out evenly over the slices
-  const int t0 = (int)((long long)ntiles * split / a.nsplit), t1 = (int)((long long)ntiles * (split + 1) / a.nsplit);
-  const int ntl = t1 - t0;
+  const int ntl = (ntiles > split) ? (ntiles - split + a.nsplit - 1) / a.nsplit : 0;
 
   if (warp == 4) {
     // ------------------------------------------------------------------ TMA producer
-    if (lane == 0 && ntl > 0) {
-      mbar_expect_tx(b_qfull, (uint32_t)(4 * nq * 128));
-      for (int term = 0; term < 2; ++term)
-        for (int dh = 0; dh < 2; ++dh)
-          tma_load_3d(smem_u32(sQ + term * qterm + dh * qhalf), &tmQ, b_qfull, dh * 64, kvh * G, term * CS_MAX_ROWS + b * R);
-      const long long krow = ((((long long)a.layer * 2 + 0) * a.max_batch + b) * a.Hkv + kvh) * (long long)a.max_seq;
-      const long long vrow = ((((long long)a.layer * 2 + 1) * a.max_batch + b) * a.Hkv + kvh) * (long long)a.max_seq;
-      int i = 0;
+    if (lane == 0) {
+      int i = 1;        // tile 0 of this slice is already on its way
       bool ok = true;
       for (; i < ntl; ++i) {
         const int s = i % stages;
         const uint32_t ph = (uint32_t)(i / stages) & 1u;
         if (!mbar_wait(b_free + 8 * s, ph ^ 1u, s_abort)) { ok = false; break; }
-        const int key0 = (t0 + i) * kTileKeys;
+        const int key0 = (split + i * a.nsplit) * kTileKeys;
         const uint32_t dk = smem_u32(sK + (size_t)s * 2 * kHalfBytes), dv = smem_u32(sV + (size_t)s * 2 * kHalfBytes);
         mbar_expect_tx(b_kfull + 8 * s, 2u * kHalfBytes);
         tma_load_2d(dk, &tmKV, b_kfull + 8 * s, 0, (int)(krow + key0));
@@ -226,7 +264,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
         tma_load_2d(dv + kHalfBytes, &tmKV, b_vfull + 8 * s, 64, (int)(vrow + key0));
       }
       if (!ok) { *s_abort = 1; atomicOr(a.status, CS_DEV_TIMEOUT); }
-      if (*s_abort) {   // let the copies land before the shared memory goes away
+      if (*s_abort || ntl == 0) {   // let the copies land before the shared memory goes away
         mbar_wait(b_qfull, 0, s_never);
         for (int j = max(0, i - stages); j < i; ++j) {
           mbar_wait(b_kfull + 8 * (j % stages), (uint32_t)(j / stages) & 1u, s_never);
@@ -281,7 +319,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
     for (int i = 0; i < ntl; ++i) {
       const int s = i % stages;
       const uint32_t ph = (uint32_t)(i / stages) & 1u;
-      const int key0 = (t0 + i) * kTileKeys;
+      const int key0 = (split + i * a.nsplit) * kTileKeys;
       // (S of this tile complete also means the previous tile's P V product has retired:
       //  P may be overwritten and O is up to date)
       bool ok = mbar_wait(b_sready, (uint32_t)i & 1u, s_abort);
@@ -289,16 +327,23 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
       if (!ok) { *s_abort = 1; have = false; break; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       float mx = -INFINITY;
+      const bool whole = key0 + kTileKeys <= lim;      // no key of this tile is masked for this row
 #pragma unroll 1
-      for (int c = 0; c < 8; ++c) {
-        float v[16];
-        tmem_ld16(lane_base + (uint32_t)(c * 16), v);
+      for (int c = 0; c < 4; ++c) {
+        float v[32];
+        tmem_ld32(lane_base + (uint32_t)(c * 32), v);
+        if (whole) {
 #pragma unroll
-        for (int j = 0; j < 16; ++j)
-          if (key0 + c * 16 + j < lim) mx = fmaxf(mx, v[j] * sc);
+          for (int j = 0; j < 32; ++j) mx = fmaxf(mx, v[j]);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (key0 + c * 32 + j < lim) mx = fmaxf(mx, v[j]);
+        }
       }
+      mx *= sc;                                        // sc > 0: scaling commutes with the maximum
       const float m_new = fmaxf(m, mx);
-      const float corr = (m == -INFINITY) ? 0.f : exp2f(m - m_new);
+      const float corr = (m == -INFINITY) ? 0.f : ex2(m - m_new);
       if (i > 0 && __any_sync(0xffffffffu, m_new > m)) {
 #pragma unroll 1
         for (int c = 0; c < 8; ++c) {
@@ -314,20 +359,20 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
       m = m_new;
       uint8_t* prow = sP + (size_t)q * 128;
 #pragma unroll 1
-      for (int c = 0; c < 8; ++c) {
-        float v[16];
-        tmem_ld16(lane_base + (uint32_t)(c * 16), v);
+      for (int c = 0; c < 4; ++c) {
+        float v[32];
+        tmem_ld32(lane_base + (uint32_t)(c * 32), v);
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          v[j] = (key0 + c * 16 + j < lim) ? exp2f(v[j] * sc - m_new) : 0.f;
+        for (int j = 0; j < 32; ++j) {
+          v[j] = (whole || key0 + c * 32 + j < lim) ? ex2(fmaf(v[j], sc, -m_new)) : 0.f;
           l += v[j];
         }
         if (valid) {
 #pragma unroll
-          for (int h = 0; h < 2; ++h) {
+          for (int h = 0; h < 4; ++h) {      // 8 keys = one 16-byte chunk of the operand row
             uint4 hi, lo;
             split8(v + 8 * h, hi, lo);
-            const uint32_t off = (uint32_t)(c >> 2) * qhalf + ((((uint32_t)(2 * c + h) & 7u) ^ ((uint32_t)q & 7u)) << 4);
+            const uint32_t off = (uint32_t)(c >> 1) * qhalf + ((((uint32_t)(4 * c + h) & 7u) ^ ((uint32_t)q & 7u)) << 4);
             *reinterpret_cast<uint4*>(prow + off) = hi;
             *reinterpret_cast<uint4*>(prow + qterm + off) = lo;
           }
@@ -412,13 +457,17 @@ int cs_launch_attention_tc(cs_ctx* ctx, const void* kv_cache, int layer, int B, 
     if (cs_encode_tiled(ctx, &ctx->tmQ, ctx->qbuf, 3, dims, strides, box) != CS_OK) return -1;
     ctx->tmQ_R = R;
   }
-  int nsplit = ctx->num_sms / (B * c.n_kv_heads);
+  // 1 KB of slack for the 1024-byte alignment; the barriers (96 bytes) fit inside it.  Small
+  // query tiles take one K/V stage and two CTAs per SM - short key slices, twice the CTAs -
+  // larger ones two stages and the whole SM.
+  const size_t ab = (size_t)8 * NQ * 128;                       // Q and P, two terms of two halves each
+  const size_t two_per_sm = 113 * 1024, limit = 227 * 1024;
+  const bool small = 1024 + ab + (size_t)4 * kHalfBytes <= two_per_sm;
+  const int stages = small ? 1 : ((1024 + ab + (size_t)2 * 4 * kHalfBytes <= limit) ? 2 : 1);
+  const size_t smem = 1024 + ab + (size_t)stages * 4 * kHalfBytes;
+  int nsplit = (small ? 2 : 1) * ctx->num_sms / (B * c.n_kv_heads);
   if (nsplit > ctx->attn_splits) nsplit = ctx->attn_splits;
   if (nsplit < 1) nsplit = 1;
-  const size_t ab = (size_t)8 * NQ * 128;                       // Q and P, two terms of two halves each
-  const size_t misc = 10 * 8 + 16, limit = 227 * 1024;
-  const int stages = (1024 + ab + (size_t)2 * 4 * kHalfBytes + misc <= limit) ? 2 : 1;
-  const size_t smem = 1024 + ab + (size_t)stages * 4 * kHalfBytes + misc;
   static size_t smem_set = 0;
   if (smem > smem_set) {
     if (cudaFuncSetAttribute(k_attn_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
