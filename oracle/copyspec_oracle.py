@@ -345,7 +345,7 @@ def decode_loop(model, cache, b, hist, gamma, k, policy, max_new, eos_id=-1, scr
         if p0 >= 0:
             st["attempts"] += 1
             st["accepted"] += c - 1
-            st["tau_hist"][c - 1] += 1
+            st["tau_hist"][min(c - 1, len(st["tau_hist"]) - 1)] += 1   # the last bin also takes longer prefixes
         else:
             st["no_match"] += 1
         if trace is not None:
@@ -393,7 +393,7 @@ def scripted_simulator(hist, script, gamma, k, policy, max_new):
         if p0 >= 0:
             st["attempts"] += 1
             st["accepted"] += c - 1
-            st["tau_hist"][c - 1] += 1
+            st["tau_hist"][min(c - 1, len(st["tau_hist"]) - 1)] += 1   # the last bin also takes longer prefixes
         else:
             st["no_match"] += 1
         steps.append({"n": n, "p0": p0, "draft": draft, "tau": c - 1, "out": out})

@@ -277,8 +277,8 @@ int launch(cs_ctx* ctx, const void* kv_cache, int layer, int B, int R, cudaStrea
 }  // namespace
 
 void cs_launch_attention(cs_ctx* ctx, const void* kv_cache, int layer, int B, int R, cudaStream_t st) {
-  // The tcgen05 kernel takes every shape it covers (head_dim 128, at most 128 query rows per KV
-  // head); the register-resident mma.sync kernel takes the rest.  CS_ATTN_KERNEL=tc|mma, read
+  // The tcgen05 kernel takes every shape it covers (head_dim 128); the register-resident
+  // mma.sync kernel takes the other head sizes.  CS_ATTN_KERNEL=tc|mma, read
   // when the context is created, forces one of them (tests run both on the same inputs).
   const bool want_tc = ctx->attn_force != 1;
   int nsplit = want_tc ? cs_launch_attention_tc(ctx, kv_cache, layer, B, R, st) : 0;

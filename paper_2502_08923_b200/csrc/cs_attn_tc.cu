@@ -1,5 +1,6 @@
 // Causal block attention over the bf16 KV cache on the 5th-generation tensor cores
-// (Sec. 3.2; App. B.2), for head_dim 128 and up to 128 query rows per KV head.
+// (Sec. 3.2; App. B.2), for head_dim 128.  Up to 128 query rows per KV head form one query
+// tile; taller blocks are cut into groups of block rows, one group per CTA.
 //
 // One CTA = one (sequence, KV head) and one slice of the key range.  The query rows (the
 // (k+1) block rows of the G query heads sharing the KV head) are the M dimension of both
@@ -30,7 +31,7 @@ constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 struct AttnArgs {
   const int* row_lim;
-  int layer, R, G, H, Hkv, max_batch, max_seq, nsplit, NQ, rows, stages;
+  int layer, R, Rg, G, H, Hkv, max_batch, max_seq, nsplit, NQ, rows, stages;   // Rg = block rows per row group
   float scale_log2e;
   float* out_o;
   float* out_ml;
@@ -170,7 +171,9 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   uint8_t* smem = smem_raw + (((raw + 1023u) & ~1023u) - raw);
-  const int NQ = a.NQ, G = a.G, R = a.R, nq = G * R, stages = a.stages;
+  // blockIdx.z picks a group of Rg consecutive block rows (blocks taller than 128 / G rows)
+  const int NQ = a.NQ, G = a.G, R = a.R, r0 = blockIdx.z * a.Rg, Rcur = min(a.Rg, R - r0);
+  const int nq = G * Rcur, nq_box = G * a.Rg, stages = a.stages;
   const uint32_t qhalf = (uint32_t)NQ * 128u;          // [NQ rows x 64 elements] of one term
   const uint32_t qterm = 2u * qhalf;
   // A operands first, K/V behind them: the MMAs' reads past row NQ stay inside the allocation
@@ -217,7 +220,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
 
   if (warp < 4) {
     int lm = 0;
-    for (int r = tid; r < R; r += 128) lm = max(lm, a.row_lim[b * R + r]);
+    for (int r = tid; r < Rcur; r += 128) lm = max(lm, a.row_lim[b * R + r0 + r]);
     lm = __reduce_max_sync(0xffffffffu, lm);
     if (lane == 0 && lm > 0) atomicMax(s_lmax, lm);
   }
@@ -227,10 +230,11 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
   const long long krow = ((((long long)a.layer * 2 + 0) * a.max_batch + b) * a.Hkv + kvh) * (long long)a.max_seq;
   const long long vrow = ((((long long)a.layer * 2 + 1) * a.max_batch + b) * a.Hkv + kvh) * (long long)a.max_seq;
   if (warp == 4 && lane == 0) {
-    mbar_expect_tx(b_qfull, (uint32_t)(4 * nq * 128));
+    mbar_expect_tx(b_qfull, (uint32_t)(4 * nq_box * 128));
     for (int term = 0; term < 2; ++term)
       for (int dh = 0; dh < 2; ++dh)
-        tma_load_3d(smem_u32(sQ + term * qterm + dh * qhalf), &tmQ, b_qfull, dh * 64, kvh * G, term * CS_MAX_ROWS + b * R);
+        tma_load_3d(smem_u32(sQ + term * qterm + dh * qhalf), &tmQ, b_qfull, dh * 64, kvh * G,
+                    term * CS_MAX_ROWS + b * R + r0);   // the box is always Rg rows tall; rows past the group are never used
     const int key0 = split * kTileKeys;
     const uint32_t dk = smem_u32(sK), dv = smem_u32(sV);
     mbar_expect_tx(b_kfull, 2u * kHalfBytes);
@@ -311,7 +315,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
     // ------------------------------------------------------------------ softmax + epilogue (thread = query row)
     const int q = tid;
     const bool valid = q < nq;
-    const int lim = valid ? a.row_lim[b * R + q / G] : 0;
+    const int lim = valid ? a.row_lim[b * R + r0 + q / G] : 0;
     const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
     const float sc = a.scale_log2e;
     float m = -INFINITY, l = 0.f;                      // running max (log2 domain) and sum of this row
@@ -401,7 +405,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
       if (!ok) { *s_abort = 1; have = false; }
     }
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    const size_t obase = valid ? ((size_t)split * a.rows + (b * R + q / G)) * a.H + (kvh * G + q % G) : 0;
+    const size_t obase = valid ? ((size_t)split * a.rows + (b * R + r0 + q / G)) * a.H + (kvh * G + q % G) : 0;
 #pragma unroll 1
     for (int c = 0; c < 8; ++c) {
       float o[16];
@@ -439,8 +443,12 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
 
 int cs_launch_attention_tc(cs_ctx* ctx, const void* kv_cache, int layer, int B, int R, cudaStream_t st) {
   const cs_model_config& c = ctx->cfg;
-  const int G = c.n_heads / c.n_kv_heads, nq = G * R;
-  if (c.head_dim != kDh || nq > kNQMax || R < 1 || R > 256 || G > 256) return 0;
+  const int G = c.n_heads / c.n_kv_heads;
+  if (c.head_dim != kDh || G > kNQMax || R < 1 || R > 256) return 0;
+  // blocks with more than 128 query rows per KV head are cut into groups of block rows
+  const int ngroups = cs_ceil_div(G * R, kNQMax), Rg = cs_ceil_div(R, ngroups);
+  if (G * Rg > kNQMax) return 0;
+  const int nq = G * Rg;
   const int NQ = (nq + 15) / 16 * 16;
   if (ctx->tmKV_base != kv_cache) {
     const unsigned long long rows = (unsigned long long)c.n_layers * 2 * c.max_batch * c.n_kv_heads * c.max_seq;
@@ -450,12 +458,12 @@ int cs_launch_attention_tc(cs_ctx* ctx, const void* kv_cache, int layer, int B, 
     if (cs_encode_tiled(ctx, &ctx->tmKV, kv_cache, 2, dims, strides, box) != CS_OK) return -1;
     ctx->tmKV_base = kv_cache;
   }
-  if (ctx->tmQ_R != R) {
+  if (ctx->tmQ_R != Rg) {
     const unsigned long long dims[3] = {(unsigned long long)kDh, (unsigned long long)c.n_heads, 2ull * CS_MAX_ROWS};
     const unsigned long long strides[2] = {kDh * 2, (unsigned long long)c.n_heads * kDh * 2};
-    const unsigned box[3] = {64, (unsigned)G, (unsigned)R};
+    const unsigned box[3] = {64, (unsigned)G, (unsigned)Rg};
     if (cs_encode_tiled(ctx, &ctx->tmQ, ctx->qbuf, 3, dims, strides, box) != CS_OK) return -1;
-    ctx->tmQ_R = R;
+    ctx->tmQ_R = Rg;
   }
   // 1 KB of slack for the 1024-byte alignment; the barriers (96 bytes) fit inside it.  Small
   // query tiles take one K/V stage and two CTAs per SM - short key slices, twice the CTAs -
@@ -465,7 +473,7 @@ int cs_launch_attention_tc(cs_ctx* ctx, const void* kv_cache, int layer, int B, 
   const bool small = 1024 + ab + (size_t)4 * kHalfBytes <= two_per_sm;
   const int stages = small ? 1 : ((1024 + ab + (size_t)2 * 4 * kHalfBytes <= limit) ? 2 : 1);
   const size_t smem = 1024 + ab + (size_t)stages * 4 * kHalfBytes;
-  int nsplit = (small ? 2 : 1) * ctx->num_sms / (B * c.n_kv_heads);
+  int nsplit = (small ? 2 : 1) * ctx->num_sms / (B * c.n_kv_heads * ngroups);
   if (nsplit > ctx->attn_splits) nsplit = ctx->attn_splits;
   if (nsplit < 1) nsplit = 1;
   static size_t smem_set = 0;
@@ -478,11 +486,11 @@ int cs_launch_attention_tc(cs_ctx* ctx, const void* kv_cache, int layer, int B, 
   }
   AttnArgs a;
   a.row_lim = ctx->row_lim;
-  a.layer = layer; a.R = R; a.G = G; a.H = c.n_heads; a.Hkv = c.n_kv_heads;
+  a.layer = layer; a.R = R; a.Rg = Rg; a.G = G; a.H = c.n_heads; a.Hkv = c.n_kv_heads;
   a.max_batch = c.max_batch; a.max_seq = c.max_seq; a.nsplit = nsplit; a.NQ = NQ; a.rows = B * R; a.stages = stages;
   a.scale_log2e = 1.4426950408889634f / sqrtf((float)kDh);
   a.out_o = ctx->attn_o; a.out_ml = ctx->attn_ml; a.status = ctx->d_status;
-  if (cs_launch_pdl(k_attn_tc, dim3(B * c.n_kv_heads, nsplit), dim3(kThreads), smem, st, ctx->tmKV, ctx->tmQ, a) != cudaSuccess) {
+  if (cs_launch_pdl(k_attn_tc, dim3(B * c.n_kv_heads, nsplit, ngroups), dim3(kThreads), smem, st, ctx->tmKV, ctx->tmQ, a) != cudaSuccess) {
     snprintf(ctx->err, sizeof(ctx->err), "attention launch failed");
     return -1;
   }

@@ -225,7 +225,7 @@ void cs_launch_rmsnorm(cs_ctx* ctx, const __nv_bfloat16* gain, int rows, cudaStr
 void cs_launch_attention(cs_ctx* ctx, const void* kv_cache, int layer, int B, int R,
                          cudaStream_t st);
 void cs_launch_attn_merge(cs_ctx* ctx, int nsplit, int rows, cudaStream_t st);
-// tcgen05 path (head_dim 128, at most 128 query rows per KV head); returns the number of key
+// tcgen05 path (head_dim 128, at most 128 query heads per KV head); returns the number of key
 // slices written, 0 when the shape is not covered, -1 on a host error (ctx->err set)
 int cs_launch_attention_tc(cs_ctx* ctx, const void* kv_cache, int layer, int B, int R, cudaStream_t st);
 // bf16 tensor map of rank <= 5, 128-byte swizzle; dims/box innermost first, strides for dims 1..

@@ -133,3 +133,23 @@ def test_loop_capacity_is_reported():
         ctx.cs_decode_loop(i32(hist), i32([20]), kv, kv_len, 3, 10, 100)     # 20 + 100 > stride 64
     assert e.value.code == cs.CS_ERR_CAPACITY
     ctx.close()
+
+
+@pytest.mark.parametrize("k", [50, 100])
+def test_wide_blocks_match_the_simulator(k):
+    """Copy windows of 50 and 100 tokens (the sweep of Sec. 4 / App. B.1): blocks of 51 and 101
+    rows through the same kernels; every integer of the scripted loop equals the simulator's."""
+    cfg = inputs.TINY
+    ctx, model = make_pair(cfg, 1536, 1, k)
+    ctxt, spans = inputs.tiny_context(seed=1)
+    rng = np.random.default_rng(11)
+    max_new = 420
+    script = inputs.copy_script(rng, ctxt, max_new, 0.7, 20, 160, cfg.vocab, zipf_s=None)
+    h, n, kvl, st = _run_gpu(ctx, [ctxt], [512], 1024, 3, k, max_new, cs.LATEST, script=script[None, :])
+    steps, st_o, h_sim = O.scripted_simulator(ctxt, script, 3, k, O.LATEST, max_new)
+    assert n[0] == 512 + max_new and kvl[0] == n[0] - 1
+    assert h[0, :n[0]].tolist() == h_sim
+    for key in ("steps", "attempts", "accepted", "emitted", "no_match"):
+        assert st[key] == st_o[key], key
+    assert max(s["tau"] for s in steps) > 20          # the wide window is actually used
+    ctx.close()

@@ -146,3 +146,34 @@ def test_truncated_rows_do_not_leak_into_the_next_step():
     lg = model.forward_block([seq[-1]], len(seq) - 1, clean, 0)
     assert np.abs(logits[0, :1].cpu().numpy() - lg).max() <= LOGIT_TOL
     ctx.close()
+
+
+@pytest.mark.parametrize("k", [50, 100])
+def test_wide_block_logits(k):
+    """One verification step with a 51- / 101-row block on the 128-wide-head configuration:
+    102 query rows per KV head still go to the tcgen05 attention kernel, 202 to the mma.sync
+    one; logits and the appended K/V rows against the oracle."""
+    cfg = inputs.ModelConfig(n_layers=2, d_model=320, n_heads=4, n_kv_heads=2, head_dim=128, d_ffn=1000,
+                             vocab=1000, rope_theta=500000.0, rms_eps=1e-5)
+    max_seq = 512
+    ctx, model = make_pair(cfg, max_seq, 1, k, seed=2, gain_jitter=0.1)
+    rng = np.random.default_rng(4)
+    n0 = 301
+    hist = rng.integers(0, cfg.vocab, size=(1, 320), dtype=np.int32)
+    kv = ctx.alloc_kv()
+    kv_len = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ctx.cs_prefill(i32(hist), i32([n0]), n0, kv, kv_len)
+    cache = O.KVCache(cfg, 1, max_seq)
+    model.prefill(hist[0, :n0].tolist(), cache, 0)
+    last, draft, dl, script = inputs.verify_inputs_with_tau(rng, 1, k, [k - 7], cfg.vocab)
+    logits = torch.zeros(1, k + 1, cfg.vocab, dtype=torch.float32, device="cuda")
+    al, ot, am = ctx.cs_verify_step(i32(last), i32(draft), i32(dl), kv, kv_len, target_script=i32(script), logits_dbg=logits)
+    assert ctx.cs_sync_status() == 0
+    tau, out, am_o, new_len, lg_o = O.verify_step(model, cache, 0, last[0], draft[0], n0 - 1, script_row=script[0])
+    assert int(al[0]) == tau == k - 7 and ot[0, :tau + 1].cpu().tolist() == out
+    assert np.abs(logits[0].cpu().numpy() - lg_o).max() <= LOGIT_TOL
+    assert not argmax_consistent(lg_o, am[0].cpu().tolist())
+    assert int(kv_len[0]) == new_len
+    ok, err = _kv_close(kv, cache, 0, 0, new_len)
+    assert ok, err
+    ctx.close()
