@@ -104,7 +104,8 @@ typedef struct {
   uint64_t accepted;  /* draft tokens accepted (sum of tau)                              */
   uint64_t emitted;   /* tokens appended to the histories                                */
   uint64_t no_match;  /* steps without a match (plain one-token decode)                  */
-  uint64_t tau_hist[CS_TAU_HIST]; /* attempts by accepted length                         */
+  uint64_t tau_hist[CS_TAU_HIST]; /* attempts by accepted length; the last bin also takes
+                                     every length beyond CS_TAU_HIST - 1                  */
 } cs_stats;
 
 /* Bytes of device workspace cs_create needs for this configuration (0 on a bad config).
