@@ -435,6 +435,33 @@ def run_workload(args):
         print(json.dumps(line), flush=True)
         return 0
     cfg = inputs.LLAMA8B
+    if name == "prefill_b1_4096":
+        # context ingestion through cs_prefill (chunks of 256 block rows through the same kernels)
+        n_ctx = 4096
+        weights = inputs.make_weights(cfg, seed=0, device=str(dev))
+        ctx = cs.Context(cfg, weights, max_seq=n_ctx + 64, max_batch=1, k_max=K_DRAFT)
+        kv = ctx.alloc_kv()
+        hist = torch.from_numpy(inputs.zipf_tokens(np.random.default_rng(0), n_ctx, cfg.vocab, 1.1).astype(np.int32)[None, :]).to(dev)
+        ld = torch.tensor([n_ctx], dtype=torch.int32, device=dev)
+        kvl = torch.zeros(1, dtype=torch.int32, device=dev)
+        ts = []
+        for i in range(3 + min(K, 10)):
+            e0, e1 = ev(), ev()
+            e0.record()
+            ctx.cs_prefill(hist, ld, n_ctx, kv, kvl)
+            e1.record()
+            torch.cuda.synchronize()
+            if i >= 3:
+                ts.append(e0.elapsed_time(e1))
+        ms = float(np.median(ts))
+        flops = 2.0 * cfg.streamed_params() * n_ctx
+        line = {"metric": "prefill tokens/sec", "value": n_ctx / (ms * 1e-3), "unit": "tokens/s", "n_gpus": 1,
+                "steps": len(ts), "warmup": 3, "ms_per_step": ms, "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
+                "config": {"workload": name, "batch": 1, "context": n_ctx, "chunk_rows": 256,
+                           "weight_passes": n_ctx // 256, "dense_tflops": flops / (ms * 1e-3) / 1e12}}
+        print(json.dumps(line), flush=True)
+        ctx.close()
+        return 0
     if name == "long_context_b1_k10":
         cases, k = [inputs.long_context_case(100)], 10
     elif name == "long_context_b8_k20":
@@ -518,7 +545,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--workload", default="verify",
-                    choices=["verify", "verify_plain_decode", "long_context_b1_k10", "long_context_b8_k20", "k_sweep_long_context_b1",
+                    choices=["verify", "verify_plain_decode", "long_context_b1_k10", "long_context_b8_k20", "k_sweep_long_context_b1", "prefill_b1_4096",
                              "multi_turn_b16_k10", "match_search"],
                     help="verify = the benchmark; the others are additional single-GPU measurements")
     ap.add_argument("--layers", type=int, default=0,

@@ -44,11 +44,6 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void* 
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
                : "r"(s));
 }
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<const uint32_t*>(&v);
-}
-
 // (lo, hi) as a leading bf16 pair plus the bf16 pair of what that rounding lost
 __device__ __forceinline__ void pack_two(float lo, float hi, uint32_t& first, uint32_t& second) {
   const __nv_bfloat162 a = __floats2bfloat162_rn(lo, hi);
