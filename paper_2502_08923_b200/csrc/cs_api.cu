@@ -244,6 +244,8 @@ cs_status cs_create(cs_ctx** out, const cs_model_config* cfg, const cs_weights* 
   ctx->rows_pad = CS_MAX_ROWS;
   ctx->attn_splits = L.attn_splits;
   {
+    const char* kb = getenv("CS_TUNE_SMEM_KB");
+    ctx->tune_smem_kb = (kb != nullptr) ? atoi(kb) : 0;
     const char* k = getenv("CS_ATTN_KERNEL");
     ctx->attn_force = (k == nullptr) ? 0 : (strcmp(k, "mma") == 0 ? 1 : (strcmp(k, "tc") == 0 ? 2 : 0));
   }

@@ -230,16 +230,18 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
   const long long krow = ((((long long)a.layer * 2 + 0) * a.max_batch + b) * a.Hkv + kvh) * (long long)a.max_seq;
   const long long vrow = ((((long long)a.layer * 2 + 1) * a.max_batch + b) * a.Hkv + kvh) * (long long)a.max_seq;
   if (warp == 4 && lane == 0) {
-    mbar_expect_tx(b_qfull, (uint32_t)(4 * nq_box * 128));
-    for (int term = 0; term < 2; ++term)
-      for (int dh = 0; dh < 2; ++dh)
-        tma_load_3d(smem_u32(sQ + term * qterm + dh * qhalf), &tmQ, b_qfull, dh * 64, kvh * G,
-                    term * CS_MAX_ROWS + b * R + r0);   // the box is always Rg rows tall; rows past the group are never used
+    // K first (it comes from HBM and the first product waits for it), then the queries (fresh in
+    // L2), V last: it is not needed before the softmax of the tile is done
     const int key0 = split * kTileKeys;
     const uint32_t dk = smem_u32(sK), dv = smem_u32(sV);
     mbar_expect_tx(b_kfull, 2u * kHalfBytes);
     tma_load_2d(dk, &tmKV, b_kfull, 0, (int)(krow + key0));
     tma_load_2d(dk + kHalfBytes, &tmKV, b_kfull, 64, (int)(krow + key0));
+    mbar_expect_tx(b_qfull, (uint32_t)(4 * nq_box * 128));
+    for (int term = 0; term < 2; ++term)
+      for (int dh = 0; dh < 2; ++dh)
+        tma_load_3d(smem_u32(sQ + term * qterm + dh * qhalf), &tmQ, b_qfull, dh * 64, kvh * G,
+                    term * CS_MAX_ROWS + b * R + r0);   // the box is always Rg rows tall; rows past the group are never used
     mbar_expect_tx(b_vfull, 2u * kHalfBytes);
     tma_load_2d(dv, &tmKV, b_vfull, 0, (int)(vrow + key0));
     tma_load_2d(dv + kHalfBytes, &tmKV, b_vfull, 64, (int)(vrow + key0));

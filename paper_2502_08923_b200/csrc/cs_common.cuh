@@ -121,6 +121,7 @@ struct cs_ctx {
   const void* tmKV_base;
   int tmQ_R;
   int attn_force;            // 0 = choose by shape, 1 = mma.sync kernel, 2 = tcgen05 kernel
+  int tune_smem_kb;          // > 0: shared memory budget of a GEMM CTA (CS_TUNE_SMEM_KB, read at creation)
 
   LoopState loop;
   Prof* prof;   // non-NULL only inside cs_profile_verify_step

@@ -721,7 +721,7 @@ cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX,
   int stages = (100 * 1024 - fixed) / stage_bytes;
   if (stages < 4) stages = (220 * 1024 - fixed) / stage_bytes;
   if (stages > 8) stages = 8;
-  if (getenv("CS_TUNE_SMEM_KB")) stages = min(12, (atoi(getenv("CS_TUNE_SMEM_KB")) * 1024 - fixed) / stage_bytes);
+  if (ctx->tune_smem_kb > 0) stages = min(12, (ctx->tune_smem_kb * 1024 - fixed) / stage_bytes);
   // the parked tile ([n_tok][128] fp32) reuses the ring
   // (a GEMM that feeds a norm keeps [n_tok][32] more floats behind it)
   if (stages < 2 || (size_t)stages * stage_bytes < (size_t)a.n_tok * (CS_GEMM_BM + 32) * 4) {
