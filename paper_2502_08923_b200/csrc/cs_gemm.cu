@@ -488,7 +488,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
           if ((a.F & 3) == 0 && jj0 + 3 < a.F) {
             float v4[4];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) v4[i] = gv[i] / (1.f + expf(-gv[i])) * uv[i];
+            for (int i = 0; i < 4; ++i) v4[i] = __fdividef(gv[i], 1.f + __expf(-gv[i])) * uv[i];
             __nv_bfloat162 h[2], l[2];
             h[0] = __floats2bfloat162_rn(v4[0], v4[1]); h[1] = __floats2bfloat162_rn(v4[2], v4[3]);
             const float2 h0 = __bfloat1622float2(h[0]), h1 = __bfloat1622float2(h[1]);
@@ -501,7 +501,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
           for (int i = 0; i < 4; ++i) {
             const int jj = tile * 64 + j + i;
             if (jj < a.F) {
-              const float v = gv[i] / (1.f + expf(-gv[i])) * uv[i];
+              const float v = __fdividef(gv[i], 1.f + __expf(-gv[i])) * uv[i];
               const __nv_bfloat16 hi = __float2bfloat16_rn(v);
               a.act[(size_t)tok * a.F + jj] = hi;
               if (a.act_lo != nullptr) a.act_lo[(size_t)tok * a.F + jj] = __float2bfloat16_rn(v - __bfloat162float(hi));
