@@ -121,9 +121,6 @@ cs_status enqueue_forward(cs_ctx* ctx, int B, int R, void* kv_cache, bool with_l
   const int rows = B * R;
   cs_status s = ensure_act_maps(ctx, cs_ceil_div(rows, 16) * 16);
   if (s != CS_OK) return s;
-  prof_begin(ctx, CS_FAM_ELEMENTWISE, st);
-  cs_launch_embed(ctx, rows, st);
-  prof_end(ctx, st);
   // Only the first RMSNorm runs as a kernel.  Every later one is folded into the GEMMs around
   // it: the residual GEMM before it writes gain * x (two bf16 terms) and sums of squares, the
   // GEMM after it scales its accumulators by 1/rms.
@@ -132,7 +129,7 @@ cs_status enqueue_forward(cs_ctx* ctx, int B, int R, void* kv_cache, bool with_l
     const LayerPlan& L = ctx->layers[l];
     if (l == 0) {
       prof_begin(ctx, CS_FAM_ELEMENTWISE, st);
-      cs_launch_rmsnorm(ctx, L.attn_norm, rows, st);
+      cs_launch_embed_rmsnorm(ctx, L.attn_norm, rows, st);
       prof_end(ctx, st);
     }
     prof_begin(ctx, CS_FAM_GEMM, st);

@@ -221,8 +221,7 @@ void cs_launch_block_setup(cs_ctx* ctx, const int32_t* last_tok, const int32_t* 
                            int B, int k, cudaStream_t st);
 void cs_launch_prefill_setup(cs_ctx* ctx, const int32_t* hist, const int32_t* hist_len, int B,
                              int stride, int start, int R, cudaStream_t st);
-void cs_launch_embed(cs_ctx* ctx, int rows, cudaStream_t st);
-void cs_launch_rmsnorm(cs_ctx* ctx, const __nv_bfloat16* gain, int rows, cudaStream_t st);
+void cs_launch_embed_rmsnorm(cs_ctx* ctx, const __nv_bfloat16* gain, int rows, cudaStream_t st);
 void cs_launch_attention(cs_ctx* ctx, const void* kv_cache, int layer, int B, int R,
                          cudaStream_t st);
 void cs_launch_attn_merge(cs_ctx* ctx, int nsplit, int rows, cudaStream_t st);

@@ -86,36 +86,37 @@ __global__ void k_prefill_setup(const int* __restrict__ hist, const int* __restr
   }
 }
 
-__global__ void k_embed(const __nv_bfloat16* __restrict__ E, const int* __restrict__ row_tok, int d,
-                        float* __restrict__ x) {
-  CS_PDL_PROLOGUE();
-  const int row = blockIdx.x;
-  const __nv_bfloat16* e = E + (size_t)row_tok[row] * d;
-  for (int i = threadIdx.x * 2; i < d; i += blockDim.x * 2) {
-    const float2 v = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(e + i));
-    *reinterpret_cast<float2*>(x + (size_t)row * d + i) = v;
-  }
-}
-
+// Embedding lookup and the first RMSNorm in one pass: x = E[token] (fp32 residual stream) and
 // xn = x * rsqrt(mean(x^2) + eps) * g as two bf16 terms (hi, lo).  One CTA per row; the row is
-// read once and kept in registers (up to 4 float4 per thread).
+// read once and kept in registers (up to 4 float4 per thread).  Every later norm is folded
+// into the GEMMs around it.
 constexpr int kNormThreads = 1024;
 __global__ void __launch_bounds__(kNormThreads)
-k_rmsnorm(const float* __restrict__ x, int d, const __nv_bfloat16* __restrict__ gain, float eps,
-          __nv_bfloat16* __restrict__ xn, __nv_bfloat16* __restrict__ xn_lo) {
+k_embed_rmsnorm(const __nv_bfloat16* __restrict__ E, const int* __restrict__ row_tok, float* __restrict__ x, int d,
+                const __nv_bfloat16* __restrict__ gain, float eps, __nv_bfloat16* __restrict__ xn,
+                __nv_bfloat16* __restrict__ xn_lo) {
   CS_PDL_PROLOGUE();
   const int row = blockIdx.x;
-  const float* xr = x + (size_t)row * d;
+  const __nv_bfloat16* er = E + (size_t)row_tok[row] * d;
+  float* xr = x + (size_t)row * d;
+  auto fetch = [&](int i) {
+    const uint2 w = *reinterpret_cast<const uint2*>(er + i);          // four bf16
+    const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w.x));
+    const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w.y));
+    const float4 v = make_float4(a.x, a.y, b.x, b.y);
+    *reinterpret_cast<float4*>(xr + i) = v;
+    return v;
+  };
   float4 v[4];
   float ss = 0.f;
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
     const int i = (q * kNormThreads + threadIdx.x) * 4;
-    v[q] = (i < d) ? *reinterpret_cast<const float4*>(xr + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+    v[q] = (i < d) ? fetch(i) : make_float4(0.f, 0.f, 0.f, 0.f);
     ss += v[q].x * v[q].x + v[q].y * v[q].y + v[q].z * v[q].z + v[q].w * v[q].w;
   }
   for (int i = 4 * kNormThreads * 4 + threadIdx.x * 4; i < d; i += kNormThreads * 4) {   // d > 16384
-    const float4 w = *reinterpret_cast<const float4*>(xr + i);
+    const float4 w = fetch(i);
     ss += w.x * w.x + w.y * w.y + w.z * w.z + w.w * w.w;
   }
   __shared__ float red[32];
@@ -198,7 +199,7 @@ __global__ void k_attn_merge(const float* __restrict__ in_o, const float* __rest
 // Reduce the LM-head tile maxima to the greedy token of each row (lowest id on ties),
 // then accept the longest prefix of the draft that agrees with the target tokens and
 // emit it plus one extra token (Sec. 3.2; App. B.2).  One CTA per sequence.
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(512)
 k_accept(const float* __restrict__ tile_max, const int* __restrict__ tile_idx, int tiles, int tile_stride,
          int k, const int* __restrict__ draft, const int* __restrict__ draft_len,
          const int* __restrict__ seq_ok, const int* __restrict__ script, int script_stride,
@@ -207,30 +208,49 @@ k_accept(const float* __restrict__ tile_max, const int* __restrict__ tile_idx, i
          int update_kv) {
   CS_PDL_PROLOGUE();
   const int b = blockIdx.x, R = k + 1;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
   __shared__ int s_arg[CS_MAX_ROWS];
+  __shared__ float s_val[32][16];
+  __shared__ int s_idx[32][16];
   int dl = draft_len[b];
   dl = dl < 0 ? 0 : (dl > k ? k : dl);
   const bool ok = seq_ok[b] != 0;
-  for (int r = warp; r < R; r += 4) {
-    float val = -INFINITY;
-    int idx = INT32_MAX;
-    if (ok && r <= dl) {
-      const int row = b * R + r;
-      for (int t = lane; t < tiles; t += 32) {
-        const float v = tile_max[(size_t)t * tile_stride + row];
-        const int id = tile_idx[(size_t)t * tile_stride + row];
-        if (v > val || (v == val && id < idx)) { val = v; idx = id; }
+  // Greedy token of every live row: the whole block scans the tile maxima of 16 rows at a time
+  // (one or two independent loads per thread and row), then one warp per row finishes.
+  for (int r0 = 0; r0 < R; r0 += 16) {
+    for (int rr = 0; rr < 16; ++rr) {
+      const int r = r0 + rr;
+      float val = -INFINITY;
+      int idx = INT32_MAX;
+      if (ok && r <= dl && r < R) {
+        const int row = b * R + r;
+        for (int t = threadIdx.x; t < tiles; t += blockDim.x) {
+          const float v = tile_max[(size_t)t * tile_stride + row];
+          const int id = tile_idx[(size_t)t * tile_stride + row];
+          if (v > val || (v == val && id < idx)) { val = v; idx = id; }
+        }
+        for (int off = 16; off > 0; off >>= 1) {
+          const float ov = __shfl_xor_sync(0xffffffffu, val, off);
+          const int oi = __shfl_xor_sync(0xffffffffu, idx, off);
+          if (ov > val || (ov == val && oi < idx)) { val = ov; idx = oi; }
+        }
       }
+      if (lane == 0) { s_val[warp][rr] = val; s_idx[warp][rr] = idx; }
+    }
+    __syncthreads();
+    if (warp < 16 && r0 + warp < R) {
+      const int r = r0 + warp;
+      float val = (lane < nwarps) ? s_val[lane][warp] : -INFINITY;
+      int idx = (lane < nwarps) ? s_idx[lane][warp] : INT32_MAX;
       for (int off = 16; off > 0; off >>= 1) {
         const float ov = __shfl_xor_sync(0xffffffffu, val, off);
         const int oi = __shfl_xor_sync(0xffffffffu, idx, off);
         if (ov > val || (ov == val && oi < idx)) { val = ov; idx = oi; }
       }
+      if (lane == 0) s_arg[r] = (ok && r <= dl && idx != INT32_MAX) ? idx : -1;
     }
-    if (lane == 0) s_arg[r] = (ok && r <= dl && idx != INT32_MAX) ? idx : -1;
+    __syncthreads();
   }
-  __syncthreads();
   for (int r = threadIdx.x; r < R; r += blockDim.x) argmax_ids[(size_t)b * R + r] = s_arg[r];
   if (threadIdx.x == 0) {
     if (!ok) {
@@ -388,13 +408,9 @@ void cs_launch_prefill_setup(cs_ctx* ctx, const int32_t* hist, const int32_t* hi
                 ctx->rope_cs, ctx->d_status);
 }
 
-void cs_launch_embed(cs_ctx* ctx, int rows, cudaStream_t st) {
-  cs_launch_pdl(k_embed, dim3(rows), dim3(128), 0, st, ctx->embed, ctx->row_tok, ctx->cfg.d_model, ctx->x);
-}
-
-void cs_launch_rmsnorm(cs_ctx* ctx, const __nv_bfloat16* gain, int rows, cudaStream_t st) {
-  cs_launch_pdl(k_rmsnorm, dim3(rows), dim3(kNormThreads), 0, st, ctx->x, ctx->cfg.d_model, gain, ctx->cfg.rms_eps, ctx->xn,
-                ctx->xn + (size_t)CS_MAX_ROWS * ctx->cfg.d_model);
+void cs_launch_embed_rmsnorm(cs_ctx* ctx, const __nv_bfloat16* gain, int rows, cudaStream_t st) {
+  cs_launch_pdl(k_embed_rmsnorm, dim3(rows), dim3(kNormThreads), 0, st, ctx->embed, ctx->row_tok, ctx->x, ctx->cfg.d_model, gain,
+                ctx->cfg.rms_eps, ctx->xn, ctx->xn + (size_t)CS_MAX_ROWS * ctx->cfg.d_model);
 }
 
 void cs_launch_attn_merge(cs_ctx* ctx, int nsplit, int rows, cudaStream_t st) {
@@ -407,7 +423,7 @@ void cs_launch_accept(cs_ctx* ctx, int B, int k, const int32_t* draft, const int
                       const int32_t* script, int script_stride, const int32_t* script_off, int script_limit,
                       int32_t* accept_len, int32_t* out_tokens, int32_t* argmax_ids, int32_t* kv_len,
                       int update_kv, cudaStream_t st) {
-  cs_launch_pdl(k_accept, dim3(B), dim3(128), 0, st, ctx->tile_max, ctx->tile_idx,
+  cs_launch_pdl(k_accept, dim3(B), dim3(512), 0, st, ctx->tile_max, ctx->tile_idx,
                 cs_ceil_div(ctx->cfg.vocab, CS_GEMM_BM), ctx->rows_pad, k, draft, draft_len, ctx->seq_ok, script,
                 script_stride, script_off, script_limit, accept_len, out_tokens, argmax_ids, kv_len, update_kv);
 }
