@@ -40,7 +40,7 @@ WORKLOAD = "verify_8b_b1_kv4096_k10_scripted_tau_uniform"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from the
 # committed ncu capture (profiles/); None until a capture of the current kernel exists.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 111.5e6   # profiles/k_gemm_tc_verify8b_2layer_ncu_full.md
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 111.8e6   # profiles/k_gemm_tc_verify8b_2layer_ncu_full.md
 
 
 def _peaks():
