@@ -427,6 +427,51 @@ def run_workload(args):
                     if i >= W:
                         ts.append(e0.elapsed_time(e1) * 1e3)
                 out[f"gamma{gamma}_{mode}_us_per_batch"] = float(np.median(ts))
+        # the gamma-gram index (Sec. 3.1) on the same batch: bulk build once, then one step's worth
+        # of update (10 appended tokens per sequence) + lookup
+        idx = cs.GramIndex(64, 32768, 3)
+        ld0 = torch.full((64,), 32758, dtype=torch.int32, device=dev)
+        e0, e1 = ev(), ev()
+        e0.record(); idx.cs_gram_index_update(hd, ld0); e1.record(); torch.cuda.synchronize()
+        out["index_build_us_per_batch"] = e0.elapsed_time(e1) * 1e3
+        bufs = idx.cs_find_match_indexed(hd, ld, K_DRAFT)
+        ts = []
+        for i in range(W + K):
+            flush.fill_(i & 1)
+            e0, e1 = ev(), ev()
+            e0.record()
+            idx.cs_gram_index_update(hd, ld)
+            idx.cs_find_match_indexed(hd, ld, K_DRAFT, out=bufs)
+            e1.record()
+            torch.cuda.synchronize()
+            if i >= W:
+                ts.append(e0.elapsed_time(e1) * 1e3)
+        out["index_update_lookup_cold_us_per_batch"] = float(np.median(ts))
+        # where the index pays: the same comparison on 8 histories of 262,144 tokens
+        hist_l, _, _ = inputs.match_search_histories(batch=8, n=262144, n_spans=4, span_lo=64, span_hi=256)
+        hl = torch.from_numpy(hist_l).to(dev)
+        ll = torch.full((8,), 262144, dtype=torch.int32, device=dev)
+        idx_l = cs.GramIndex(8, 262144, 3)
+        idx_l.cs_gram_index_update(hl, torch.full((8,), 262134, dtype=torch.int32, device=dev))
+        bs, bi = cs.cs_find_match(hl, ll, 3, K_DRAFT), idx_l.cs_find_match_indexed(hl, ll, K_DRAFT)
+        t_scan, t_idx = [], []
+        for i in range(W + K):
+            flush.fill_(i & 1)
+            e0, e1, e2 = ev(), ev(), ev()
+            e0.record()
+            cs.cs_find_match(hl, ll, 3, K_DRAFT, out=bs)
+            e1.record()
+            idx_l.cs_gram_index_update(hl, ll)
+            idx_l.cs_find_match_indexed(hl, ll, K_DRAFT, out=bi)
+            e2.record()
+            torch.cuda.synchronize()
+            if i >= W:
+                t_scan.append(e0.elapsed_time(e1) * 1e3)
+                t_idx.append(e1.elapsed_time(e2) * 1e3)
+        if not all(torch.equal(x, y) for x, y in zip(bs, bi)):
+            raise RuntimeError("index and scan disagree")
+        out["long_8x262144_scan_cold_us"] = float(np.median(t_scan))
+        out["long_8x262144_index_update_lookup_cold_us"] = float(np.median(t_idx))
         us = out["gamma3_cold_us_per_batch"]
         line = {"metric": "match-search us/seq", "value": us / 64, "unit": "us", "higher_is_better": False,
                 "n_gpus": 1, "steps": K, "warmup": W, "dtype": "int32", "data": "synthetic",

@@ -142,6 +142,30 @@ cs_status cs_find_match(const int32_t* hist, const int32_t* hist_len, int B, int
                         int gamma, int k, cs_match_policy policy, int32_t* match_pos,
                         int32_t* draft, int32_t* draft_len, void* stream);
 
+/* Index of all gamma-grams of the accepted sequences (Sec. 3.1: a hash map from every
+ * gamma-token subsequence to where it occurs, O(gamma) work per appended token and per
+ * lookup).  An alternative to the scan of cs_find_match whose cost does not grow with the
+ * history; results are identical (tokens are compared, not hashes).
+ *   index: caller-allocated DEVICE buffer of cs_gram_index_bytes(B, capacity_tokens) bytes,
+ *          one table per sequence sized for histories of up to capacity_tokens tokens;
+ *   cs_gram_index_reset   empties it (async);
+ *   cs_gram_index_update  inserts the gamma-grams that have become admissible since the last
+ *          update: starts p <= hist_len[b] - 2*gamma (a match must end before the key starts,
+ *          App. B.3 step 1(c)).  Histories only grow; one index serves one gamma.  Async;
+ *   cs_find_match_indexed same outputs as cs_find_match for the history lengths of the last
+ *          update (call update first whenever tokens were appended).  Async;
+ *   cs_gram_index_status  synchronises the stream; CS_ERR_CAPACITY if a table overflowed.
+ * Errors on the host: CS_ERR_ARG, CS_ERR_CUDA. */
+size_t cs_gram_index_bytes(int B, int capacity_tokens);
+cs_status cs_gram_index_reset(void* index, int B, int capacity_tokens, void* stream);
+cs_status cs_gram_index_update(void* index, int B, int capacity_tokens, const int32_t* hist,
+                               const int32_t* hist_len, int stride, int gamma, void* stream);
+cs_status cs_find_match_indexed(const void* index, int B, int capacity_tokens, const int32_t* hist,
+                                const int32_t* hist_len, int stride, int gamma, int k,
+                                cs_match_policy policy, int32_t* match_pos, int32_t* draft,
+                                int32_t* draft_len, void* stream);
+cs_status cs_gram_index_status(const void* index, int B, int capacity_tokens, void* stream);
+
 /* One verification forward plus acceptance (Sec. 3.2; App. B.2; App. B.3 step 2). Async.
  * Evaluates the block [last_tok[b], draft[b][0 .. draft_len[b])] of every sequence at
  * positions kv_len[b].. in one forward, appends the block's K/V rows to the cache,

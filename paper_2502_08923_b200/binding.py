@@ -50,7 +50,8 @@ class CsStats(C.Structure):
 EXPORTS = ("cs_workspace_bytes", "cs_create", "cs_destroy", "cs_last_error", "cs_sync_status",
            "cs_find_match", "cs_verify_step", "cs_kv_truncate", "cs_decode_loop", "cs_prefill", "cs_linear",
            "cs_loop_begin", "cs_loop_steps", "cs_loop_poll", "cs_loop_end", "cs_profile_verify_step",
-           "cs_loop_launches_per_step", "cs_lm_head", "cs_lm_head_static")
+           "cs_loop_launches_per_step", "cs_lm_head", "cs_lm_head_static", "cs_gram_index_bytes",
+           "cs_gram_index_reset", "cs_gram_index_update", "cs_find_match_indexed", "cs_gram_index_status")
 
 _lib = None
 
@@ -147,6 +148,50 @@ def cs_find_match(hist, hist_len, gamma, k, policy=LATEST, out=None):
     if rc != CS_OK:
         raise CsError(rc, "cs_find_match")
     return mp, dr, dl
+
+
+class GramIndex:
+    """Device-resident gamma-gram index (argument marshalling only).  One per batch of sequences."""
+
+    def __init__(self, B, capacity_tokens, gamma, device="cuda"):
+        self.lib = load()
+        self.B, self.cap, self.gamma = B, capacity_tokens, gamma
+        self.lib.cs_gram_index_bytes.restype = C.c_size_t
+        nbytes = self.lib.cs_gram_index_bytes(B, capacity_tokens)
+        self.buf = torch.empty(nbytes, dtype=torch.uint8, device=device)
+        self.cs_gram_index_reset()
+
+    def _p(self):
+        return C.c_void_p(self.buf.data_ptr())
+
+    def cs_gram_index_reset(self):
+        rc = self.lib.cs_gram_index_reset(self._p(), self.B, self.cap, _stream())
+        if rc != CS_OK:
+            raise CsError(rc, "cs_gram_index_reset")
+
+    def cs_gram_index_update(self, hist, hist_len):
+        B, stride = hist.shape
+        rc = self.lib.cs_gram_index_update(self._p(), B, self.cap, _i32(hist, "hist"), _i32(hist_len, "hist_len"), stride,
+                                           self.gamma, _stream())
+        if rc != CS_OK:
+            raise CsError(rc, "cs_gram_index_update")
+
+    def cs_find_match_indexed(self, hist, hist_len, k, policy=LATEST, out=None):
+        B, stride = hist.shape
+        if out is None:
+            out = (torch.empty(B, dtype=torch.int32, device=hist.device),
+                   torch.empty(B, max(k, 1), dtype=torch.int32, device=hist.device)[:, :k].contiguous(),
+                   torch.empty(B, dtype=torch.int32, device=hist.device))
+        mp, dr, dl = out
+        rc = self.lib.cs_find_match_indexed(self._p(), B, self.cap, _i32(hist, "hist"), _i32(hist_len, "hist_len"), stride,
+                                            self.gamma, k, policy, _i32(mp, "match_pos"),
+                                            C.c_void_p(dr.data_ptr()) if k > 0 else None, _i32(dl, "draft_len"), _stream())
+        if rc != CS_OK:
+            raise CsError(rc, "cs_find_match_indexed")
+        return mp, dr, dl
+
+    def cs_gram_index_status(self):
+        return self.lib.cs_gram_index_status(self._p(), self.B, self.cap, _stream())
 
 
 def pack_gate_up(w_gate_up, d_ffn):
