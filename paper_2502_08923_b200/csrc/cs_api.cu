@@ -154,7 +154,11 @@ cs_status enqueue_forward(cs_ctx* ctx, int B, int R, void* kv_cache, bool with_l
     if (s != CS_OK) return s;
     take_norm = NormFuse{};
     take_norm.ssq_in = ctx->ssq;
-    take_norm.slots_in = cs_ceil_div(L.o.N, CS_GEMM_BM) * L.o.splits;
+    {
+      int sp, kbs;
+      cs_gemm_splits(ctx, &L.o, rows, &sp, &kbs);
+      take_norm.slots_in = cs_ceil_div(L.o.N, CS_GEMM_BM) * sp;
+    }
     take_norm.slot_stride = ctx->ssq_stride;
     take_norm.inv_d = 1.f / (float)c.d_model;
     take_norm.eps = c.rms_eps;
@@ -171,7 +175,11 @@ cs_status enqueue_forward(cs_ctx* ctx, int B, int R, void* kv_cache, bool with_l
                        &give, st);
     prof_end(ctx, st);
     if (s != CS_OK) return s;
-    take_norm.slots_in = cs_ceil_div(L.down.N, CS_GEMM_BM) * L.down.splits;
+    {
+      int sp, kbs;
+      cs_gemm_splits(ctx, &L.down, rows, &sp, &kbs);
+      take_norm.slots_in = cs_ceil_div(L.down.N, CS_GEMM_BM) * sp;
+    }
   }
   if (with_lm) {
     prof_begin(ctx, CS_FAM_LMHEAD, st);

@@ -207,6 +207,7 @@ cs_status cs_launch_find_match(const int32_t* hist, const int32_t* hist_len, int
                                cudaStream_t st);
 // cs_gemm.cu
 cs_status cs_gemm_plan(cs_ctx* ctx, GemmPlan* g, const void* w, int N, int K, bool allow_split);
+void cs_gemm_splits(const cs_ctx* ctx, const GemmPlan* g, int rows, int* splits, int* kb_per_split);
 cs_status cs_make_act_map(cs_ctx* ctx, CUtensorMap* tm, const void* base, int rows_total, int K,
                           int box_rows);
 // mode = CS_EPI_*: `out` is the fp32 destination (STORE, RESIDUAL) or the optional logits dump

@@ -681,6 +681,20 @@ cs_status cs_gemm_plan(cs_ctx* ctx, GemmPlan* g, const void* w, int N, int K, bo
   return encode_2d(ctx, &g->tmW, w, N, K, CS_GEMM_BM, true);
 }
 
+// Split-K factor and K blocks per split for a block of `rows` token rows.  The plan's factor is
+// made for two CTAs per SM; blocks too tall for that run one CTA per SM, and their grid is kept
+// within one wave where the tile count allows it.
+void cs_gemm_splits(const cs_ctx* ctx, const GemmPlan* g, int rows, int* splits, int* kb_per_split) {
+  const int n_tok = cs_ceil_div(rows, 16) * 16;
+  const int tiles = cs_ceil_div(g->N, CS_GEMM_BM), kb = cs_ceil_div(g->K, CS_GEMM_BK);
+  int s = g->splits;
+  const int stage_bytes = CS_GEMM_BM * CS_GEMM_BK * 2 + 2 * n_tok * 128;
+  const bool one_per_sm = (113 * 1024 - 2048) / stage_bytes < 2;
+  if (one_per_sm && s > 1 && tiles * s > ctx->num_sms) s = max(1, ctx->num_sms / tiles);
+  *kb_per_split = cs_ceil_div(kb, s);
+  *splits = cs_ceil_div(kb, *kb_per_split);
+}
+
 cs_status cs_make_act_map(cs_ctx* ctx, CUtensorMap* tm, const void* base, int rows_total, int K,
                           int box_rows) {
   return encode_2d(ctx, tm, base, rows_total, K, box_rows, false);
@@ -696,8 +710,7 @@ cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX,
   a.N = g->N;
   a.K = g->K;
   a.num_kb = cs_ceil_div(g->K, CS_GEMM_BK);
-  a.kb_per_split = g->kb_per_split;
-  a.splits = g->splits;
+  cs_gemm_splits(ctx, g, rows, &a.splits, &a.kb_per_split);
   a.mode = mode;
   a.out = out;
   a.act = act;
@@ -717,9 +730,15 @@ cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX,
   a.status = ctx->d_status;
   const int stage_bytes = kTileABytes + (lo_row >= 0 ? 2 : 1) * a.n_tok * 128;
   const int fixed = 1024 /*alignment slack*/ + (2 * 8 + 1) * 8 + 16 + 9 * a.n_tok * 4;
-  // small blocks: two CTAs per SM (about 100 KB each); large blocks: one CTA with the whole SM
+  // Two CTAs per SM wherever two stages fit into half an SM: the grids (224-240 CTAs) are
+  // sized for the 296 slots that gives, and a one-CTA-per-SM launch would run them in two
+  // waves.  Only blocks too tall for that take the whole SM.
   int stages = (100 * 1024 - fixed) / stage_bytes;
-  if (stages < 4) stages = (220 * 1024 - fixed) / stage_bytes;
+  if (stages < 4) {
+    const int two = (113 * 1024 - fixed) / stage_bytes;
+    const bool park_fits = (size_t)two * stage_bytes >= (size_t)a.n_tok * (CS_GEMM_BM + 32) * 4;
+    stages = (two >= 2 && park_fits) ? two : (220 * 1024 - fixed) / stage_bytes;
+  }
   if (stages > 8) stages = 8;
   if (ctx->tune_smem_kb > 0) stages = min(12, (ctx->tune_smem_kb * 1024 - fixed) / stage_bytes);
   // the parked tile ([n_tok][128] fp32) reuses the ring
@@ -736,7 +755,7 @@ cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX,
     attr_set = true;
   }
   cudaLaunchConfig_t lc = {};
-  lc.gridDim = dim3(tiles, g->splits, 1);
+  lc.gridDim = dim3(tiles, a.splits, 1);
   lc.blockDim = dim3(kThreads, 1, 1);
   lc.dynamicSmemBytes = smem;
   lc.stream = st;
@@ -745,10 +764,10 @@ cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX,
   at[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   at[na].val.programmaticStreamSerializationAllowed = 1;
   ++na;
-  if (g->splits > 1) {
+  if (a.splits > 1) {
     at[na].id = cudaLaunchAttributeClusterDimension;
     at[na].val.clusterDim.x = 1;
-    at[na].val.clusterDim.y = g->splits;
+    at[na].val.clusterDim.y = a.splits;
     at[na].val.clusterDim.z = 1;
     ++na;
   }
