@@ -539,7 +539,7 @@ def run_workload(args):
         h[b, :len(hh)] = hh
     script_d = torch.from_numpy(np.stack([s[:max_new] for _, s in cases]).astype(np.int32)).to(dev)
     res = {}
-    sweep = (100, 50, 20, 10, 0) if name == "k_sweep_long_context_b1" else ((k, 0) if name != "verify_plain_decode" else (0,))
+    sweep = (100, 50, 20, 10, 5, 0) if name == "k_sweep_long_context_b1" else ((k, 0) if name != "verify_plain_decode" else (0,))
     for kk in sweep:
         steps = K if kk else min(4 * K, max_new - W - 1)
         steps = min(steps, (max_new // (kk + 1)) - W - 1)
