@@ -199,7 +199,10 @@ cs_status enqueue_loop_step(cs_ctx* ctx, cudaStream_t st) {
                                      ctx->loop_draft, ctx->loop_dlen, ctx->loop_last, ctx->loop_done, st);
   if (r != CS_OK) return fail(ctx, r, "match kernel launch failed");
   cs_launch_block_setup(ctx, ctx->loop_last, ctx->loop_draft, ctx->loop_dlen, L.kv_len, ctx->loop_done, L.B, L.k, st);
+  // the step opened with a stream-ordered launch and nothing before k_loop_commit changes kv_len
+  ctx->kv_len_early = L.kv_len;
   r = enqueue_forward(ctx, L.B, L.k + 1, L.kv_cache, true, nullptr, st);
+  ctx->kv_len_early = nullptr;
   if (r != CS_OK) return r;
   cs_launch_accept(ctx, L.B, L.k, ctx->loop_draft, ctx->loop_dlen, L.script, L.max_new, ctx->loop_emitted, L.max_new,
                    ctx->loop_accept, ctx->loop_out, ctx->loop_argmax, L.kv_len, 0, st);

@@ -14,8 +14,13 @@
 // shared memory behind them; whatever they find there only reaches accumulator rows that
 // nobody reads.  K and V tiles arrive by TMA (128-byte swizzle, two 64-wide halves) through
 // an mbarrier ring.  Each CTA writes its un-normalised (O, max, sum); k_attn_merge combines
-// the slices.  Every wait is bounded (2 s): on expiry the CTA flags CS_DEV_TIMEOUT, drains
-// its copies, frees its TMEM and returns.
+// the slices.  A K buffer is handed back to the producer as soon as the score product that
+// read it has retired and a V buffer after the P V product, so with a single stage the next
+// tile's K lands during the softmax and its V during the next score product.  When the caller
+// vouches for the cached lengths (kv_len_early), a slice whose first tile lies wholly below
+// the cached length requests that tile before it waits for the preceding kernel: those rows
+// were written by earlier steps.  Every wait is bounded (2 s): on expiry the CTA flags
+// CS_DEV_TIMEOUT, drains its copies, frees its TMEM and returns.
 #include <stdlib.h>
 
 #include "cs_common.cuh"
@@ -31,6 +36,7 @@ constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 struct AttnArgs {
   const int* row_lim;
+  const int* kv_len_early;   // cached lengths that no kernel in flight changes, or NULL
   int layer, R, Rg, G, H, Hkv, max_batch, max_seq, nsplit, NQ, rows, stages;   // Rg = block rows per row group
   float scale_log2e;
   float* out_o;
@@ -183,14 +189,14 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
   uint8_t* sV = sK + (size_t)stages * 2 * kHalfBytes;
   // barriers and flags live in the alignment slack: in front of the aligned area when it is at
   // least 96 bytes, else in what is then left behind it
-  uint64_t* bars = reinterpret_cast<uint64_t*>((smem - smem_raw >= 96) ? smem_raw : sV + (size_t)stages * 2 * kHalfBytes);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 10);
+  uint64_t* bars = reinterpret_cast<uint64_t*>((smem - smem_raw >= 128) ? smem_raw : sV + (size_t)stages * 2 * kHalfBytes);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 12);
   volatile int* s_abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
   volatile int* s_never = reinterpret_cast<volatile int*>(tmem_slot + 2);
   int* s_lmax = reinterpret_cast<int*>(tmem_slot + 3);
-  const uint32_t b_kfull = smem_u32(bars), b_vfull = smem_u32(bars + 2), b_free = smem_u32(bars + 4),
-                 b_qfull = smem_u32(bars + 6), b_sready = smem_u32(bars + 7), b_pready = smem_u32(bars + 8),
-                 b_odone = smem_u32(bars + 9);
+  const uint32_t b_kfull = smem_u32(bars), b_vfull = smem_u32(bars + 2), b_kfree = smem_u32(bars + 4),
+                 b_vfree = smem_u32(bars + 6), b_qfull = smem_u32(bars + 8), b_sready = smem_u32(bars + 9),
+                 b_pready = smem_u32(bars + 10), b_odone = smem_u32(bars + 11);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int b = blockIdx.x / a.Hkv, kvh = blockIdx.x % a.Hkv, split = blockIdx.y;
@@ -198,7 +204,10 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
   constexpr uint32_t kTmemCols = 256, kOCol = 128;     // S in columns 0..127, O in 128..255
 
   if (tid == 128) {
-    for (int s = 0; s < 2; ++s) { mbar_init(b_kfull + 8 * s, 1); mbar_init(b_vfull + 8 * s, 1); mbar_init(b_free + 8 * s, 1); }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(b_kfull + 8 * s, 1); mbar_init(b_vfull + 8 * s, 1);
+      mbar_init(b_kfree + 8 * s, 1); mbar_init(b_vfree + 8 * s, 1);
+    }
     mbar_init(b_qfull, 1);
     mbar_init(b_sready, 1);
     mbar_init(b_pready, (uint32_t)nact * 32u);
@@ -216,6 +225,26 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
+  // Slice `split` works on key tiles split, split + nsplit, ...: its first tile is known before
+  // the key range is, so the queries and that tile are requested while the range is worked out
+  // (a slice beyond the range only has to let them land).
+  const long long krow = ((((long long)a.layer * 2 + 0) * a.max_batch + b) * a.Hkv + kvh) * (long long)a.max_seq;
+  const long long vrow = ((((long long)a.layer * 2 + 1) * a.max_batch + b) * a.Hkv + kvh) * (long long)a.max_seq;
+  const int key_first = split * kTileKeys;
+  bool early = false;
+  if (warp == 4 && lane == 0 && a.kv_len_early != nullptr) {
+    // a tile of cached keys only: nothing in flight writes it, so it need not wait
+    if (key_first + kTileKeys <= min(a.kv_len_early[b], a.max_seq)) {
+      early = true;
+      const uint32_t dk = smem_u32(sK), dv = smem_u32(sV);
+      mbar_expect_tx(b_kfull, 2u * kHalfBytes);
+      tma_load_2d(dk, &tmKV, b_kfull, 0, (int)(krow + key_first));
+      tma_load_2d(dk + kHalfBytes, &tmKV, b_kfull, 64, (int)(krow + key_first));
+      mbar_expect_tx(b_vfull, 2u * kHalfBytes);
+      tma_load_2d(dv, &tmKV, b_vfull, 0, (int)(vrow + key_first));
+      tma_load_2d(dv + kHalfBytes, &tmKV, b_vfull, 64, (int)(vrow + key_first));
+    }
+  }
   asm volatile("griddepcontrol.wait;" ::: "memory");
 
   if (warp < 4) {
@@ -224,27 +253,25 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
     lm = __reduce_max_sync(0xffffffffu, lm);
     if (lane == 0 && lm > 0) atomicMax(s_lmax, lm);
   }
-  // Slice `split` works on key tiles split, split + nsplit, ...: its first tile is known before
-  // the key range is, so the queries and that tile are requested while the range is worked out
-  // (a slice beyond the range only has to let them land).
-  const long long krow = ((((long long)a.layer * 2 + 0) * a.max_batch + b) * a.Hkv + kvh) * (long long)a.max_seq;
-  const long long vrow = ((((long long)a.layer * 2 + 1) * a.max_batch + b) * a.Hkv + kvh) * (long long)a.max_seq;
   if (warp == 4 && lane == 0) {
     // K first (it comes from HBM and the first product waits for it), then the queries (fresh in
     // L2), V last: it is not needed before the softmax of the tile is done
-    const int key0 = split * kTileKeys;
     const uint32_t dk = smem_u32(sK), dv = smem_u32(sV);
-    mbar_expect_tx(b_kfull, 2u * kHalfBytes);
-    tma_load_2d(dk, &tmKV, b_kfull, 0, (int)(krow + key0));
-    tma_load_2d(dk + kHalfBytes, &tmKV, b_kfull, 64, (int)(krow + key0));
+    if (!early) {
+      mbar_expect_tx(b_kfull, 2u * kHalfBytes);
+      tma_load_2d(dk, &tmKV, b_kfull, 0, (int)(krow + key_first));
+      tma_load_2d(dk + kHalfBytes, &tmKV, b_kfull, 64, (int)(krow + key_first));
+    }
     mbar_expect_tx(b_qfull, (uint32_t)(4 * nq_box * 128));
     for (int term = 0; term < 2; ++term)
       for (int dh = 0; dh < 2; ++dh)
         tma_load_3d(smem_u32(sQ + term * qterm + dh * qhalf), &tmQ, b_qfull, dh * 64, kvh * G,
                     term * CS_MAX_ROWS + b * R + r0);   // the box is always Rg rows tall; rows past the group are never used
-    mbar_expect_tx(b_vfull, 2u * kHalfBytes);
-    tma_load_2d(dv, &tmKV, b_vfull, 0, (int)(vrow + key0));
-    tma_load_2d(dv + kHalfBytes, &tmKV, b_vfull, 64, (int)(vrow + key0));
+    if (!early) {
+      mbar_expect_tx(b_vfull, 2u * kHalfBytes);
+      tma_load_2d(dv, &tmKV, b_vfull, 0, (int)(vrow + key_first));
+      tma_load_2d(dv + kHalfBytes, &tmKV, b_vfull, 64, (int)(vrow + key_first));
+    }
   }
   __syncthreads();
   const int lmax = *s_lmax;
@@ -254,28 +281,29 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
   if (warp == 4) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      int i = 1;        // tile 0 of this slice is already on its way
+      int ik = 1, iv = 1;   // K and V tiles requested so far (tile 0 of this slice is already on its way)
       bool ok = true;
-      for (; i < ntl; ++i) {
+      for (int i = 1; i < ntl; ++i) {
         const int s = i % stages;
         const uint32_t ph = (uint32_t)(i / stages) & 1u;
-        if (!mbar_wait(b_free + 8 * s, ph ^ 1u, s_abort)) { ok = false; break; }
         const int key0 = (split + i * a.nsplit) * kTileKeys;
         const uint32_t dk = smem_u32(sK + (size_t)s * 2 * kHalfBytes), dv = smem_u32(sV + (size_t)s * 2 * kHalfBytes);
+        if (!mbar_wait(b_kfree + 8 * s, ph ^ 1u, s_abort)) { ok = false; break; }
         mbar_expect_tx(b_kfull + 8 * s, 2u * kHalfBytes);
         tma_load_2d(dk, &tmKV, b_kfull + 8 * s, 0, (int)(krow + key0));
         tma_load_2d(dk + kHalfBytes, &tmKV, b_kfull + 8 * s, 64, (int)(krow + key0));
+        ik = i + 1;
+        if (!mbar_wait(b_vfree + 8 * s, ph ^ 1u, s_abort)) { ok = false; break; }
         mbar_expect_tx(b_vfull + 8 * s, 2u * kHalfBytes);
         tma_load_2d(dv, &tmKV, b_vfull + 8 * s, 0, (int)(vrow + key0));
         tma_load_2d(dv + kHalfBytes, &tmKV, b_vfull + 8 * s, 64, (int)(vrow + key0));
+        iv = i + 1;
       }
       if (!ok) { *s_abort = 1; atomicOr(a.status, CS_DEV_TIMEOUT); }
       if (*s_abort || ntl == 0) {   // let the copies land before the shared memory goes away
         mbar_wait(b_qfull, 0, s_never);
-        for (int j = max(0, i - stages); j < i; ++j) {
-          mbar_wait(b_kfull + 8 * (j % stages), (uint32_t)(j / stages) & 1u, s_never);
-          mbar_wait(b_vfull + 8 * (j % stages), (uint32_t)(j / stages) & 1u, s_never);
-        }
+        for (int j = max(0, ik - stages); j < ik; ++j) mbar_wait(b_kfull + 8 * (j % stages), (uint32_t)(j / stages) & 1u, s_never);
+        for (int j = max(0, iv - stages); j < iv; ++j) mbar_wait(b_vfull + 8 * (j % stages), (uint32_t)(j / stages) & 1u, s_never);
       }
     }
   } else if (warp == 5) {
@@ -283,13 +311,13 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
     if (lane == 0 && ntl > 0) {
       const uint32_t idesc1 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
       const uint32_t idesc2 = idesc1 | (1u << 16);      // B (= V) is MN-major
-      bool ok = mbar_wait(b_qfull, 0, s_abort);
-      for (int i = 0; i < ntl && ok; ++i) {
+      const uint32_t aq = smem_u32(sQ), ap = smem_u32(sP);
+      // S of tile i: issued behind the P V product of tile i - 1, so one commit covers both
+      auto issue_scores = [&](int i) -> bool {
         const int s = i % stages;
-        const uint32_t ph = (uint32_t)(i / stages) & 1u;
-        if (!mbar_wait(b_kfull + 8 * s, ph, s_abort)) { ok = false; break; }
+        if (!mbar_wait(b_kfull + 8 * s, (uint32_t)(i / stages) & 1u, s_abort)) return false;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t ak = smem_u32(sK + (size_t)s * 2 * kHalfBytes), aq = smem_u32(sQ);
+        const uint32_t ak = smem_u32(sK + (size_t)s * 2 * kHalfBytes);
 #pragma unroll
         for (int term = 0; term < 2; ++term)
 #pragma unroll
@@ -298,18 +326,26 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
             for (int kk = 0; kk < 4; ++kk)
               umma_bf16(tmem_base, desc_kmajor(aq + term * qterm + dh * qhalf) + 2 * kk, desc_kmajor(ak + dh * kHalfBytes) + 2 * kk,
                         idesc1, (term | dh | kk) ? 1u : 0u);
+        umma_commit(b_kfree + 8 * s);
         umma_commit(b_sready);
+        return true;
+      };
+      bool ok = mbar_wait(b_qfull, 0, s_abort) && issue_scores(0);
+      for (int i = 0; i < ntl && ok; ++i) {
+        const int s = i % stages;
+        const uint32_t ph = (uint32_t)(i / stages) & 1u;
         if (!mbar_wait(b_pready, (uint32_t)i & 1u, s_abort) || !mbar_wait(b_vfull + 8 * s, ph, s_abort)) { ok = false; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t av = smem_u32(sV + (size_t)s * 2 * kHalfBytes), ap = smem_u32(sP);
+        const uint32_t av = smem_u32(sV + (size_t)s * 2 * kHalfBytes);
 #pragma unroll
         for (int term = 0; term < 2; ++term)
 #pragma unroll
           for (int kk = 0; kk < 8; ++kk)   // 16 keys per instruction
             umma_bf16(tmem_base + kOCol, desc_kmajor(ap + term * qterm + (kk >> 2) * qhalf) + 2 * (kk & 3),
                       desc_mnmajor(av + kk * 2048, kHalfBytes), idesc2, (i > 0 || term > 0 || kk > 0) ? 1u : 0u);
-        umma_commit(b_free + 8 * s);
+        umma_commit(b_vfree + 8 * s);
         umma_commit(b_odone);
+        if (i + 1 < ntl && !issue_scores(i + 1)) { ok = false; break; }
       }
       if (!ok) { *s_abort = 1; atomicOr(a.status, CS_DEV_TIMEOUT); }
     }
@@ -488,6 +524,7 @@ int cs_launch_attention_tc(cs_ctx* ctx, const void* kv_cache, int layer, int B, 
   }
   AttnArgs a;
   a.row_lim = ctx->row_lim;
+  a.kv_len_early = ctx->kv_len_early;
   a.layer = layer; a.R = R; a.Rg = Rg; a.G = G; a.H = c.n_heads; a.Hkv = c.n_kv_heads;
   a.max_batch = c.max_batch; a.max_seq = c.max_seq; a.nsplit = nsplit; a.NQ = NQ; a.rows = B * R; a.stages = stages;
   a.scale_log2e = 1.4426950408889634f / sqrtf((float)kDh);

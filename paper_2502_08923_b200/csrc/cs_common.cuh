@@ -120,6 +120,11 @@ struct cs_ctx {
   CUtensorMap tmKV, tmQ;
   const void* tmKV_base;
   int tmQ_R;
+  // Cached lengths [max_batch] that stay as they are until the forward being enqueued has
+  // finished, and whose cache rows are complete: set only where the step opens with an
+  // ordinary stream-ordered launch (the generation loop); NULL elsewhere.  The attention
+  // kernel may then fetch tiles of cached keys before it waits for the preceding kernel.
+  const int* kv_len_early;
   int attn_force;            // 0 = choose by shape, 1 = mma.sync kernel, 2 = tcgen05 kernel
   int tune_smem_kb;          // > 0: shared memory budget of a GEMM CTA (CS_TUNE_SMEM_KB, read at creation)
 
