@@ -215,6 +215,7 @@ cs_status enqueue_loop_step(cs_ctx* ctx, cudaStream_t st) {
 cs_status status_from_bits(cs_ctx* ctx, int bits) {
   if (bits & CS_DEV_TIMEOUT) return fail(ctx, CS_ERR_TIMEOUT, "a bounded device-side wait ran out");
   if (bits & CS_DEV_CAPACITY) return fail(ctx, CS_ERR_CAPACITY, "KV cache or history row too small for a sequence");
+  if (bits & CS_DEV_SMEM) return fail(ctx, CS_ERR_UNSUPPORTED, "attention kernel could not place its barriers in shared memory");
   if (bits & CS_DEV_BADARG) return fail(ctx, CS_ERR_ARG, "device-side argument check failed (lengths inconsistent)");
   return CS_OK;
 }

@@ -4,8 +4,10 @@
 //
 // One CTA = one (sequence, KV head) and one slice of the key range.  The query rows (the
 // (k+1) block rows of the G query heads sharing the KV head) are the M dimension of both
-// products, so that TMEM lane i belongs to query row i and the whole online softmax of a
-// row is private to one thread:
+// products, so that TMEM lane i belongs to query row i and the online softmax of a row is
+// shared by just two threads (warps w and w + 4 both reach TMEM lanes 32 w .. 32 w + 31; one
+// takes keys 0-63 of a tile and output dims 0-63, the other the upper halves; they exchange
+// their row maxima and sums through shared memory and a bounded mbarrier wait):
 //     S [128 x 128 keys]  = Q_hi K_tile^T + Q_lo K_tile^T     (tcgen05.mma, A and B K-major)
 //     O [128 x 128 dims] += P_hi V_tile  + P_lo V_tile        (tcgen05.mma, B MN-major)
 // Queries and softmax weights enter as two bf16 terms each, so they are fp32-equivalent and
@@ -27,7 +29,9 @@
 
 namespace {
 
-constexpr int kThreads = 192;   // warps 0-3 softmax/epilogue, warp 4 TMA producer, warp 5 MMA
+constexpr int kThreads = 320;   // warps 0-7 softmax/epilogue, warp 8 TMA producer, warp 9 MMA
+constexpr int kProdWarp = 8, kMmaWarp = 9;
+constexpr int kCtlBytes = 160;  // 16 mbarriers + TMEM slot + flags
 constexpr int kTileKeys = 128;
 constexpr int kDh = 128;
 constexpr int kHalfBytes = kTileKeys * 128;          // one [128 keys x 64 dims] half tile
@@ -38,6 +42,7 @@ struct AttnArgs {
   const int* row_lim;
   const int* kv_len_early;   // cached lengths that no kernel in flight changes, or NULL
   int layer, R, Rg, G, H, Hkv, max_batch, max_seq, nsplit, NQ, rows, stages;   // Rg = block rows per row group
+  int smem_bytes;            // dynamic shared memory of the launch
   float scale_log2e;
   float* out_o;
   float* out_ml;
@@ -171,7 +176,7 @@ __device__ __forceinline__ void split8(const float* p, uint4& hi, uint4& lo) {
   lo = make_uint4(l[0], l[1], l[2], l[3]);
 }
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, 2)
 k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUtensorMap tmQ, AttnArgs a) {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   extern __shared__ uint8_t smem_raw[];
@@ -187,37 +192,47 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
   uint8_t* sP = sQ + 2 * qterm;                        // same shape, 64 keys per half
   uint8_t* sK = sP + 2 * qterm;                        // [stage][half][128 keys][128 B]
   uint8_t* sV = sK + (size_t)stages * 2 * kHalfBytes;
-  // barriers and flags live in the alignment slack: in front of the aligned area when it is at
-  // least 96 bytes, else in what is then left behind it
-  uint64_t* bars = reinterpret_cast<uint64_t*>((smem - smem_raw >= 128) ? smem_raw : sV + (size_t)stages * 2 * kHalfBytes);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 12);
+  // Barriers, flags and the exchange rows of the softmax pairs (two parities x two halves x NQ
+  // floats) live in what the 1024-byte alignment leaves over: in front of the aligned area when
+  // that holds them, else behind it.  (The window normally starts aligned, so they sit behind.)
+  uint8_t* tail = sV + (size_t)stages * 2 * kHalfBytes;
+  const uint32_t pad = (uint32_t)(smem - smem_raw), need = (uint32_t)kCtlBytes + 16u * (uint32_t)NQ;
+  const uint32_t back = (uint32_t)a.smem_bytes - pad - (uint32_t)(tail - smem);
+  if (pad < need && back < need) {   // cannot happen with the sizes the launcher asks for unless the window starts oddly
+    if (threadIdx.x == 0) atomicOr(a.status, CS_DEV_SMEM);
+    return;
+  }
+  uint64_t* bars = reinterpret_cast<uint64_t*>(pad >= need ? smem_raw : tail);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
   volatile int* s_abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
   volatile int* s_never = reinterpret_cast<volatile int*>(tmem_slot + 2);
   int* s_lmax = reinterpret_cast<int*>(tmem_slot + 3);
+  float* s_xch = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(bars) + kCtlBytes);   // [parity][half][NQ]
   const uint32_t b_kfull = smem_u32(bars), b_vfull = smem_u32(bars + 2), b_kfree = smem_u32(bars + 4),
                  b_vfree = smem_u32(bars + 6), b_qfull = smem_u32(bars + 8), b_sready = smem_u32(bars + 9),
-                 b_pready = smem_u32(bars + 10), b_odone = smem_u32(bars + 11);
+                 b_pready = smem_u32(bars + 10), b_odone = smem_u32(bars + 11), b_pair = smem_u32(bars + 12);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int b = blockIdx.x / a.Hkv, kvh = blockIdx.x % a.Hkv, split = blockIdx.y;
   const int nact = (nq + 31) >> 5;                     // softmax warps that own real rows
   constexpr uint32_t kTmemCols = 256, kOCol = 128;     // S in columns 0..127, O in 128..255
 
-  if (tid == 128) {
+  if (tid == kProdWarp * 32) {
     for (int s = 0; s < 2; ++s) {
       mbar_init(b_kfull + 8 * s, 1); mbar_init(b_vfull + 8 * s, 1);
       mbar_init(b_kfree + 8 * s, 1); mbar_init(b_vfree + 8 * s, 1);
     }
     mbar_init(b_qfull, 1);
     mbar_init(b_sready, 1);
-    mbar_init(b_pready, (uint32_t)nact * 32u);
+    mbar_init(b_pready, (uint32_t)nact * 64u);
     mbar_init(b_odone, 1);
+    for (int w = 0; w < 4; ++w) mbar_init(b_pair + 8 * w, 64);
     *s_abort = 0; *s_never = 0; *s_lmax = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmKV) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmQ) : "memory");
   }
-  if (warp == 5) {
+  if (warp == kMmaWarp) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -232,7 +247,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
   const long long vrow = ((((long long)a.layer * 2 + 1) * a.max_batch + b) * a.Hkv + kvh) * (long long)a.max_seq;
   const int key_first = split * kTileKeys;
   bool early = false;
-  if (warp == 4 && lane == 0 && a.kv_len_early != nullptr) {
+  if (warp == kProdWarp && lane == 0 && a.kv_len_early != nullptr) {
     // a tile of cached keys only: nothing in flight writes it, so it need not wait
     if (key_first + kTileKeys <= min(a.kv_len_early[b], a.max_seq)) {
       early = true;
@@ -247,13 +262,13 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
   }
   asm volatile("griddepcontrol.wait;" ::: "memory");
 
-  if (warp < 4) {
+  if (warp < 8) {
     int lm = 0;
-    for (int r = tid; r < Rcur; r += 128) lm = max(lm, a.row_lim[b * R + r0 + r]);
+    for (int r = tid; r < Rcur; r += 256) lm = max(lm, a.row_lim[b * R + r0 + r]);
     lm = __reduce_max_sync(0xffffffffu, lm);
     if (lane == 0 && lm > 0) atomicMax(s_lmax, lm);
   }
-  if (warp == 4 && lane == 0) {
+  if (warp == kProdWarp && lane == 0) {
     // K first (it comes from HBM and the first product waits for it), then the queries (fresh in
     // L2), V last: it is not needed before the softmax of the tile is done
     const uint32_t dk = smem_u32(sK), dv = smem_u32(sV);
@@ -278,7 +293,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
   const int ntiles = (lmax + kTileKeys - 1) / kTileKeys;
   const int ntl = (ntiles > split) ? (ntiles - split + a.nsplit - 1) / a.nsplit : 0;
 
-  if (warp == 4) {
+  if (warp == kProdWarp) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       int ik = 1, iv = 1;   // K and V tiles requested so far (tile 0 of this slice is already on its way)
@@ -306,7 +321,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
         for (int j = max(0, iv - stages); j < iv; ++j) mbar_wait(b_vfull + 8 * (j % stages), (uint32_t)(j / stages) & 1u, s_never);
       }
     }
-  } else if (warp == 5) {
+  } else if (warp == kMmaWarp) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0 && ntl > 0) {
       const uint32_t idesc1 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
@@ -349,19 +364,33 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
       }
       if (!ok) { *s_abort = 1; atomicOr(a.status, CS_DEV_TIMEOUT); }
     }
-  } else if (warp < nact) {
-    // ------------------------------------------------------------------ softmax + epilogue (thread = query row)
-    const int q = tid;
+  } else if ((warp & 3) < nact) {
+    // ------------------------------------------------------------------ softmax + epilogue (two threads per query row)
+    const int wq = warp & 3, half = warp >> 2;
+    const int q = wq * 32 + lane;
     const bool valid = q < nq;
     const int lim = valid ? a.row_lim[b * R + r0 + q / G] : 0;
-    const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
+    const uint32_t lane_base = tmem_base + ((uint32_t)(wq * 32) << 16);
+    const uint32_t col0 = (uint32_t)half * 64u;        // this thread's keys of a tile and its output dims
+    const uint32_t pairbar = b_pair + 8u * (uint32_t)wq;
     const float sc = a.scale_log2e;
-    float m = -INFINITY, l = 0.f;                      // running max (log2 domain) and sum of this row
+    float m = -INFINITY, l = 0.f;                      // running max (log2 domain, whole row) and sum of this half
     bool have = ntl > 0;
+    uint32_t xuse = 0;                                 // exchanges done so far
+    // hand `mine` to the other thread of the row and return what it handed over
+    auto exchange = [&](float mine, float& theirs) -> bool {
+      float* slot = s_xch + (size_t)(xuse & 1u) * 2 * NQ;
+      if (valid) slot[half * NQ + q] = mine;
+      mbar_arrive(pairbar);
+      const bool ok = mbar_wait(pairbar, xuse & 1u, s_abort);
+      theirs = (ok && valid) ? slot[(half ^ 1) * NQ + q] : mine;
+      ++xuse;
+      return ok;
+    };
     for (int i = 0; i < ntl; ++i) {
       const int s = i % stages;
       const uint32_t ph = (uint32_t)(i / stages) & 1u;
-      const int key0 = (split + i * a.nsplit) * kTileKeys;
+      const int key0 = (split + i * a.nsplit) * kTileKeys + (int)col0;   // first key of this thread's half tile
       // (S of this tile complete also means the previous tile's P V product has retired:
       //  P may be overwritten and O is up to date)
       bool ok = mbar_wait(b_sready, (uint32_t)i & 1u, s_abort);
@@ -369,11 +398,11 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
       if (!ok) { *s_abort = 1; have = false; break; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       float mx = -INFINITY;
-      const bool whole = key0 + kTileKeys <= lim;      // no key of this tile is masked for this row
+      const bool whole = key0 + 64 <= lim;             // no key of this half tile is masked for this row
 #pragma unroll 1
-      for (int c = 0; c < 4; ++c) {
+      for (int c = 0; c < 2; ++c) {
         float v[32];
-        tmem_ld32(lane_base + (uint32_t)(c * 32), v);
+        tmem_ld32(lane_base + col0 + (uint32_t)(c * 32), v);
         if (whole) {
 #pragma unroll
           for (int j = 0; j < 32; ++j) mx = fmaxf(mx, v[j]);
@@ -383,27 +412,31 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
             if (key0 + c * 32 + j < lim) mx = fmaxf(mx, v[j]);
         }
       }
-      mx *= sc;                                        // sc > 0: scaling commutes with the maximum
+      float mx_other;
+      ok = exchange(mx, mx_other);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) { *s_abort = 1; have = false; break; }
+      mx = fmaxf(mx, mx_other) * sc;                   // sc > 0: scaling commutes with the maximum
       const float m_new = fmaxf(m, mx);
       const float corr = (m == -INFINITY) ? 0.f : ex2(m - m_new);
       if (i > 0 && __any_sync(0xffffffffu, m_new > m)) {
 #pragma unroll 1
-        for (int c = 0; c < 8; ++c) {
+        for (int c = 0; c < 4; ++c) {
           float o[16];
-          tmem_ld16(lane_base + kOCol + (uint32_t)(c * 16), o);
+          tmem_ld16(lane_base + kOCol + col0 + (uint32_t)(c * 16), o);
 #pragma unroll
           for (int j = 0; j < 16; ++j) o[j] *= corr;
-          tmem_st16(lane_base + kOCol + (uint32_t)(c * 16), o);
+          tmem_st16(lane_base + kOCol + col0 + (uint32_t)(c * 16), o);
         }
         asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
       }
       l *= corr;
       m = m_new;
-      uint8_t* prow = sP + (size_t)q * 128;
+      uint8_t* prow = sP + (size_t)half * qhalf + (size_t)q * 128;
 #pragma unroll 1
-      for (int c = 0; c < 4; ++c) {
+      for (int c = 0; c < 2; ++c) {
         float v[32];
-        tmem_ld32(lane_base + (uint32_t)(c * 32), v);
+        tmem_ld32(lane_base + col0 + (uint32_t)(c * 32), v);
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
           v[j] = (whole || key0 + c * 32 + j < lim) ? ex2(fmaf(v[j], sc, -m_new)) : 0.f;
@@ -414,17 +447,18 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
           for (int h = 0; h < 4; ++h) {      // 8 keys = one 16-byte chunk of the operand row
             uint4 hi, lo;
             split8(v + 8 * h, hi, lo);
-            const uint32_t off = (uint32_t)(c >> 1) * qhalf + ((((uint32_t)(4 * c + h) & 7u) ^ ((uint32_t)q & 7u)) << 4);
+            const uint32_t off = (((uint32_t)(4 * c + h)) ^ ((uint32_t)q & 7u)) << 4;
             *reinterpret_cast<uint4*>(prow + off) = hi;
             *reinterpret_cast<uint4*>(prow + qterm + off) = lo;
           }
         }
       }
       // keys past the longest row of this sequence hold whatever the cache held: zero their V rows
-      if (key0 + kTileKeys > lmax) {
+      const int tile0 = key0 - (int)col0;
+      if (tile0 + kTileKeys > lmax) {
         if (!mbar_wait(b_vfull + 8 * s, ph, s_abort)) *s_abort = 1;
         uint8_t* vs = sV + (size_t)s * 2 * kHalfBytes;
-        for (int rr = max(lmax - key0, 0) + tid; rr < kTileKeys; rr += nact * 32) {
+        for (int rr = max(lmax - tile0, 0) + half * nact * 32 + q; rr < kTileKeys; rr += nact * 64) {
 #pragma unroll
           for (int c = 0; c < 8; ++c) {
             *reinterpret_cast<uint4*>(vs + (size_t)rr * 128 + c * 16) = make_uint4(0u, 0u, 0u, 0u);
@@ -445,31 +479,38 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const size_t obase = valid ? ((size_t)split * a.rows + (b * R + r0 + q / G)) * a.H + (kvh * G + q % G) : 0;
 #pragma unroll 1
-    for (int c = 0; c < 8; ++c) {
+    for (int c = 0; c < 4; ++c) {
       float o[16];
       if (have) {
-        tmem_ld16(lane_base + kOCol + (uint32_t)(c * 16), o);
+        tmem_ld16(lane_base + kOCol + col0 + (uint32_t)(c * 16), o);
       } else {
 #pragma unroll
         for (int j = 0; j < 16; ++j) o[j] = 0.f;
       }
       if (valid) {
-        float4* dst = reinterpret_cast<float4*>(a.out_o + obase * kDh + c * 16);
+        float4* dst = reinterpret_cast<float4*>(a.out_o + obase * kDh + col0 + c * 16);
 #pragma unroll
         for (int j = 0; j < 4; ++j) dst[j] = make_float4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
       }
     }
-    if (valid) {
+    // the row's sum is the sum of its two halves (both are relative to the same maximum)
+    float l_other = 0.f;
+    if (have) {
+      bool ok = exchange(l, l_other);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) { *s_abort = 1; have = false; }
+    }
+    if (valid && half == 0) {
       constexpr float kLn2 = 0.6931471805599453f;
       a.out_ml[obase * 2] = have ? m * kLn2 : -INFINITY;
-      a.out_ml[obase * 2 + 1] = have ? l : 0.f;
+      a.out_ml[obase * 2 + 1] = have ? l + l_other : 0.f;
     }
     if (*s_abort && lane == 0) atomicOr(a.status, CS_DEV_TIMEOUT);
   }
   // ---------------------------------------------------------------------- teardown
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
-  if (warp == 5) {
+  if (warp == kMmaWarp) {
     if (*s_abort && lane == 0 && ntl > 0) mbar_wait(b_odone, (uint32_t)(ntl - 1) & 1u, s_never);   // MMAs retired (bounded)
     __syncwarp();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -503,14 +544,17 @@ int cs_launch_attention_tc(cs_ctx* ctx, const void* kv_cache, int layer, int B, 
     if (cs_encode_tiled(ctx, &ctx->tmQ, ctx->qbuf, 3, dims, strides, box) != CS_OK) return -1;
     ctx->tmQ_R = Rg;
   }
-  // 1 KB of slack for the 1024-byte alignment; the barriers (96 bytes) fit inside it.  Small
-  // query tiles take one K/V stage and two CTAs per SM - short key slices, twice the CTAs -
-  // larger ones two stages and the whole SM.
+  // 1 KB of slack for the 1024-byte alignment; barriers, flags and the softmax exchange rows
+  // (kCtlBytes + 16 NQ bytes) fit inside it for the small tiles, larger ones get that much more.
+  // Small query tiles take one K/V stage and two CTAs per SM - short key slices, twice the
+  // CTAs - larger ones two stages and the whole SM.
   const size_t ab = (size_t)8 * NQ * 128;                       // Q and P, two terms of two halves each
   const size_t two_per_sm = 113 * 1024, limit = 227 * 1024;
-  const bool small = 1024 + ab + (size_t)4 * kHalfBytes <= two_per_sm;
-  const int stages = small ? 1 : ((1024 + ab + (size_t)2 * 4 * kHalfBytes <= limit) ? 2 : 1);
-  const size_t smem = 1024 + ab + (size_t)stages * 4 * kHalfBytes;
+  const size_t ctl = (size_t)kCtlBytes + 16 * (size_t)NQ;
+  const bool small = 1024 + ab + (size_t)4 * kHalfBytes <= two_per_sm && ctl <= 1024;
+  const size_t extra = small ? 0 : (ctl + 127) / 128 * 128;
+  const int stages = small ? 1 : ((1024 + extra + ab + (size_t)2 * 4 * kHalfBytes <= limit) ? 2 : 1);
+  const size_t smem = 1024 + extra + ab + (size_t)stages * 4 * kHalfBytes;
   int nsplit = (small ? 2 : 1) * ctx->num_sms / (B * c.n_kv_heads * ngroups);
   if (nsplit > ctx->attn_splits) nsplit = ctx->attn_splits;
   if (nsplit < 1) nsplit = 1;
@@ -527,6 +571,7 @@ int cs_launch_attention_tc(cs_ctx* ctx, const void* kv_cache, int layer, int B, 
   a.kv_len_early = ctx->kv_len_early;
   a.layer = layer; a.R = R; a.Rg = Rg; a.G = G; a.H = c.n_heads; a.Hkv = c.n_kv_heads;
   a.max_batch = c.max_batch; a.max_seq = c.max_seq; a.nsplit = nsplit; a.NQ = NQ; a.rows = B * R; a.stages = stages;
+  a.smem_bytes = (int)smem;
   a.scale_log2e = 1.4426950408889634f / sqrtf((float)kDh);
   a.out_o = ctx->attn_o; a.out_ml = ctx->attn_ml; a.status = ctx->d_status;
   if (cs_launch_pdl(k_attn_tc, dim3(B * c.n_kv_heads, nsplit, ngroups), dim3(kThreads), smem, st, ctx->tmKV, ctx->tmQ, a) != cudaSuccess) {

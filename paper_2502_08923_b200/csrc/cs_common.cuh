@@ -17,7 +17,8 @@
 enum : int {
   CS_DEV_CAPACITY = 1,  // KV cache / history row too small for this step
   CS_DEV_BADARG = 2,    // cs_kv_truncate asked to grow
-  CS_DEV_TIMEOUT = 4    // a bounded wait ran out
+  CS_DEV_TIMEOUT = 4,   // a bounded wait ran out
+  CS_DEV_SMEM = 8       // a kernel found its shared-memory window laid out in a way it cannot use
 };
 
 static constexpr int CS_MAX_ROWS = 256;   // rows of one verification block (UMMA N limit)
