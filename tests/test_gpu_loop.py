@@ -153,3 +153,40 @@ def test_wide_blocks_match_the_simulator(k):
         assert st[key] == st_o[key], key
     assert max(s["tau"] for s in steps) > 20          # the wide window is actually used
     ctx.close()
+
+
+def test_real_mode_loop_with_wide_heads_and_caches_of_many_key_tiles():
+    """Real-mode decoding with 128-wide heads (the tensor-core attention kernel) over caches of
+    10-14 key tiles, batch 8: with 9 key slices per (sequence, KV head) several slices walk two
+    tiles, and inside the loop the tiles of cached keys are fetched ahead of the dependency
+    wait.  Every emitted token must be the oracle's greedy choice up to the logit tolerance
+    (losslessness, Sec. 1 / App. B.2), so a wrong attention result cannot hide behind a script."""
+    cfg = inputs.ModelConfig(n_layers=2, d_model=256, n_heads=8, n_kv_heads=4, head_dim=128, d_ffn=512, vocab=512,
+                             rope_theta=500000.0, rms_eps=1e-5)
+    B, k, max_new, max_seq = 8, 10, 16, 1792
+    ctx, model = make_pair(cfg, max_seq, B, k, seed=5, gain_jitter=0.1)
+    rng = np.random.default_rng(5)
+    lens = [1700, 1301, 1536, 1663, 1409, 1280, 1599, 1688]
+    hists = []
+    for n in lens:
+        h = rng.integers(0, cfg.vocab, size=n).astype(np.int32)
+        src = int(rng.integers(0, n // 2))
+        h[n - 40:] = h[src:src + 40]          # the context ends inside a replay of an earlier span
+        hists.append(h)
+    h, n, kvl, st = _run_gpu(ctx, hists, lens, 1728, 3, k, max_new, cs.LATEST)
+    assert st["attempts"] >= B                 # every sequence opened with a match and a 10-token draft
+    tot = O.new_stats()
+    same = True
+    for b in range(B):
+        gen = h[b, lens[b]:n[b]].tolist()
+        assert len(gen) == max_new and kvl[b] == n[b] - 1
+        assert max(greedy_margins(model, cfg, hists[b], gen)) < LOGIT_TOL, b
+        cache = O.KVCache(cfg, 1, max_seq); model.prefill(hists[b].tolist(), cache, 0)
+        got, so = O.decode_loop(model, cache, 0, hists[b].tolist(), 3, k, O.LATEST, max_new)
+        same = same and gen == got
+        for key in ("steps", "attempts", "accepted", "emitted", "no_match"):
+            tot[key] += so[key]
+    if same:
+        for key in ("steps", "attempts", "accepted", "emitted", "no_match"):
+            assert st[key] == tot[key], key
+    ctx.close()
