@@ -37,7 +37,10 @@ Pins (tests/test_oracle_*.py): brute-force enumeration of all matches; closed fo
 re-implemented separately; a Hugging Face Llama forward (library routine) for the
 whole transformer; cache-vs-recompute and block-vs-single-row invariants; RoPE
 relative-position property; real-mode output == plain greedy decoding; scripted-mode
-output == the script and == a model-free integer simulator; a constructed example with
+output == the script and == a model-free integer simulator; the draft-model fallback of
+Sec. 3.3 (decode_loop_drafted) by losslessness, by the closed form "a draft model equal to
+the target has every proposal accepted", by delta = 0 reducing to decode_loop and by its
+rolled-back cache equalling a fresh forward over the accepted tokens; a constructed example with
 the structure of Fig. 2 (gamma=3, 10 copied tokens, accepted prefix + 1 extra token).
 The paper's tables (tokens/s, tau, % copied) depend on trained weights and datasets:
 parity with them is unpinned.
@@ -352,6 +355,75 @@ def decode_loop(model, cache, b, hist, gamma, k, policy, max_new, eos_id=-1, scr
             trace.append({"n": n, "p0": p0, "draft": draft, "argmax": am, "tau": c - 1,
                           "out": list(out)})
     return emitted, st
+
+
+def decode_loop_drafted(target, t_cache, drafter, d_cache, d_len, b, hist, gamma, k, delta, policy,
+                        max_new, eos_id=-1, script=None, trace=None):
+    """CopySpec merged with vanilla speculative decoding (Sec. 3.3; App. B.3 steps 1-4).
+    Every step first looks for a match of the last gamma tokens; with a match the k copied
+    tokens are the draft (step 2).  Without one the smaller draft model proposes delta tokens
+    one at a time at temperature 0 (step 3(a)); the target verifies them in one block exactly
+    like a copied draft (step 3(b)), and the draft model's cache is rolled back to the accepted
+    prefix together with the target's (step 3(c)).
+    `d_cache` holds the draft model's K/V for positions [0, d_len) of `hist`, d_len <= len(hist)-1;
+    copy steps leave it alone, so before it drafts the draft model first runs over the tokens
+    it has not seen.  Readings: the draft model is greedy like the target (the paper evaluates
+    at temperature 0); a drafted block earns the extra guaranteed token too (Sec. 3.2).
+    Returns (emitted tokens, stats, d_len); stats as in decode_loop (attempts / accepted /
+    tau_hist count copy attempts only) plus draft_attempts and draft_accepted."""
+    emitted = []
+    st = new_stats()
+    st["draft_attempts"] = 0
+    st["draft_accepted"] = 0
+    done = False
+    while len(emitted) < max_new and not done:
+        n = len(hist)
+        e = len(emitted)
+        p0 = find_match(np.asarray(hist, dtype=np.int64), n, gamma, policy)
+        drafted = p0 < 0 and delta > 0
+        if drafted:
+            lg = drafter.forward_block(hist[d_len:n], d_len, d_cache, b)     # catch up; last row predicts position n
+            d_len = n
+            draft = [argmax_lowest(lg[-1])]
+            while len(draft) < delta:
+                lg = drafter.forward_block([draft[-1]], d_len, d_cache, b)
+                d_len += 1
+                draft.append(argmax_lowest(lg[0]))
+        else:
+            draft = gather_draft(hist, n, p0, gamma, k)
+        block = [hist[-1]] + draft
+        logits = target.forward_block(block, n - 1, t_cache, b)
+        am = [argmax_lowest(logits[r]) for r in range(len(block))]
+        if script is None:
+            tgt = am
+        else:
+            tgt = [int(script[e + r]) if e + r < max_new else -1 for r in range(len(block))]
+        tau = accept_length(draft, tgt)
+        out = tgt[:tau + 1][:max_new - e]
+        if script is None and eos_id >= 0 and eos_id in out:
+            out = out[:out.index(eos_id) + 1]
+            done = True
+        c = len(out)
+        hist.extend(out)
+        emitted.extend(out)
+        if drafted:
+            # positions n .. n+c-2 hold draft tokens that were accepted; the rest is rolled back
+            d_len = min(d_len, n + c - 1)
+        st["steps"] += 1
+        st["emitted"] += c
+        if p0 >= 0:
+            st["attempts"] += 1
+            st["accepted"] += c - 1
+            st["tau_hist"][min(c - 1, len(st["tau_hist"]) - 1)] += 1
+        else:
+            st["no_match"] += 1
+            if drafted:
+                st["draft_attempts"] += 1
+                st["draft_accepted"] += c - 1
+        if trace is not None:
+            trace.append({"n": n, "p0": p0, "drafted": drafted, "draft": list(draft), "argmax": am,
+                          "tau": c - 1, "out": list(out), "d_len": d_len})
+    return emitted, st, d_len
 
 
 def greedy_decode(model, cache, b, hist, max_new, eos_id=-1):
