@@ -235,6 +235,40 @@ void cs_loop_end(cs_ctx* ctx);
 /* Kernel launches in one step of the loop in progress (nodes of its graph; 0 if none). */
 int cs_loop_launches_per_step(const cs_ctx* ctx);
 
+/* CopySpec merged with vanilla speculative decoding (Sec. 3.3; App. B.3 steps 1-4), for ONE
+ * sequence.  Synchronous.  Every step searches the last gamma tokens; with a match the k
+ * copied tokens are the draft, without one the draft model `drafter` proposes `delta` tokens
+ * greedily, one single-row forward each (step 3(a)).  Either draft is verified by one target
+ * block and the longest agreeing prefix plus one extra token is emitted (step 3(b); Sec. 3.2);
+ * the target's cache and, after a drafted step, the draft model's cache are rolled back to the
+ * accepted prefix (step 3(c)).  Copy steps do not touch the draft model: before it next
+ * drafts it runs over the accepted tokens it has not seen, in blocks of its k_max + 1 rows.
+ *   target, drafter: two contexts (different objects) with the same vocabulary;
+ *            k, delta <= target's k_max.  Neither may have a cs_loop_begin session open
+ *            (the loop buffers of both workspaces serve as scratch).
+ *   hist int32 [stride] device, hist_len int32 [1] device, in/out as in cs_decode_loop.
+ *   kv_target / kv_len_target [1]: the target's cache, kv_len_target = hist_len - 1 on entry.
+ *   kv_drafter / kv_len_drafter [1]: the draft model's cache, holding any prefix
+ *            (0 <= kv_len_drafter <= hist_len - 1) of the same history; on return it holds
+ *            the positions below the returned kv_len_drafter.
+ *   delta = 0: drafter, kv_drafter, kv_len_drafter may be NULL; the loop is then
+ *            cs_decode_loop's, driven from the host.
+ *   script int32 [max_new] device or NULL: scripted-target mode as in cs_decode_loop.
+ *   stats_out host or NULL: attempts / accepted / tau_hist count copy attempts only, no_match
+ *            counts every step without a match.  draft_stats_out host uint64 [2] or NULL:
+ *            steps the draft model drafted, and its proposals that were accepted.
+ * The host reads the match position and the accepted block every step (one or two stream
+ * synchronisations per step).  Requires stride >= hist_len + max_new, target max_seq >=
+ * hist_len + max_new + max(k, delta), drafter max_seq >= hist_len + max_new + delta
+ * (CS_ERR_CAPACITY before anything is launched).  Returns the first error among the host
+ * checks, CUDA and the two device status words. */
+cs_status cs_decode_loop_drafted(cs_ctx* target, cs_ctx* drafter, int32_t* hist, int32_t* hist_len,
+                                 int stride, void* kv_target, int32_t* kv_len_target,
+                                 void* kv_drafter, int32_t* kv_len_drafter, int gamma, int k,
+                                 int delta, cs_match_policy policy, int max_new, int eos_id,
+                                 const int32_t* script, cs_stats* stats_out,
+                                 uint64_t* draft_stats_out, void* stream);
+
 /* Measurement aid (no counterpart in the paper): runs cs_verify_step once with a CUDA event
  * pair around every kernel launch and returns, per kernel family, the summed device time
  * in milliseconds and the number of launches.  Families: 0 = projection GEMMs of the

@@ -48,7 +48,8 @@ class CsStats(C.Structure):
 
 
 EXPORTS = ("cs_workspace_bytes", "cs_create", "cs_destroy", "cs_last_error", "cs_sync_status",
-           "cs_find_match", "cs_verify_step", "cs_kv_truncate", "cs_decode_loop", "cs_prefill", "cs_linear",
+           "cs_find_match", "cs_verify_step", "cs_kv_truncate", "cs_decode_loop", "cs_decode_loop_drafted",
+           "cs_prefill", "cs_linear",
            "cs_loop_begin", "cs_loop_steps", "cs_loop_poll", "cs_loop_end", "cs_profile_verify_step",
            "cs_loop_launches_per_step", "cs_lm_head", "cs_lm_head_static", "cs_gram_index_bytes",
            "cs_gram_index_reset", "cs_gram_index_update", "cs_find_match_indexed", "cs_gram_index_status")
@@ -89,6 +90,9 @@ def load(build_if_missing: bool = True) -> C.CDLL:
     lib.cs_kv_truncate.argtypes = [vp, ip, ip, i, vp]
     lib.cs_decode_loop.restype = i
     lib.cs_decode_loop.argtypes = [vp, ip, ip, i, i, vp, ip, i, i, i, i, i, ip, C.POINTER(CsStats), vp]
+    lib.cs_decode_loop_drafted.restype = i
+    lib.cs_decode_loop_drafted.argtypes = [vp, vp, ip, ip, i, vp, ip, vp, ip, i, i, i, i, i, i, ip,
+                                           C.POINTER(CsStats), C.POINTER(C.c_uint64), vp]
     lib.cs_loop_begin.restype = i
     lib.cs_loop_begin.argtypes = [vp, ip, ip, i, i, vp, ip, i, i, i, i, i, ip, vp]
     lib.cs_loop_steps.restype = i
@@ -334,6 +338,26 @@ class Context:
                                      _i32(script, "script"), C.byref(st), _stream())
         self._check(rc, "cs_decode_loop")
         return st.as_dict()
+
+    def cs_decode_loop_drafted(self, drafter, hist, hist_len, kv_cache, kv_len, kv_drafter, kv_len_drafter, gamma, k,
+                               delta, max_new, policy=LATEST, eos_id=-1, script=None):
+        """The loop merged with a draft model (`self` is the target, `drafter` another Context or
+        None when delta is 0), one sequence: hist [1][stride].  Returns the statistics as a dict
+        with draft_attempts and draft_accepted added."""
+        B, stride = hist.shape
+        if B != 1:
+            raise ValueError("cs_decode_loop_drafted takes one sequence")
+        st = CsStats()
+        ds = (C.c_uint64 * 2)()
+        rc = self.lib.cs_decode_loop_drafted(self.handle, drafter.handle if drafter is not None else None,
+                                             _i32(hist, "hist"), _i32(hist_len, "hist_len"), stride, _ptr(kv_cache),
+                                             _i32(kv_len, "kv_len"), _ptr(kv_drafter) if kv_drafter is not None else None,
+                                             _i32(kv_len_drafter, "kv_len_drafter"), gamma, k, delta, policy, max_new,
+                                             eos_id, _i32(script, "script"), C.byref(st), ds, _stream())
+        self._check(rc, "cs_decode_loop_drafted")
+        out = st.as_dict()
+        out["draft_attempts"], out["draft_accepted"] = int(ds[0]), int(ds[1])
+        return out
 
     def cs_loop_begin(self, hist, hist_len, kv_cache, kv_len, gamma, k, max_new, policy=LATEST, eos_id=-1,
                       script=None):

@@ -60,6 +60,8 @@ def test_context_calls_reject_null():
     assert lib.cs_verify_step(None, None, None, None, 1, 1, None, None, None, None, None, None, None, None) == cs.CS_ERR_ARG
     assert lib.cs_kv_truncate(None, None, None, 1, None) == cs.CS_ERR_ARG
     assert lib.cs_decode_loop(None, None, None, 1, 1, None, None, 3, 10, 0, 1, -1, None, None, None) == cs.CS_ERR_ARG
+    assert lib.cs_decode_loop_drafted(None, None, None, None, 8, None, None, None, None, 3, 10, 3, 0, 1, -1, None, None,
+                                      None, None) == cs.CS_ERR_ARG
     assert lib.cs_prefill(None, None, None, 1, 1, 1, None, None, None) == cs.CS_ERR_ARG
     assert lib.cs_sync_status(None, None) == cs.CS_ERR_ARG
     h = C.c_void_p()
