@@ -507,6 +507,8 @@ def run_workload(args):
         print(json.dumps(line), flush=True)
         ctx.close()
         return 0
+    if name == "drafted_b1_k10":
+        return run_drafted(args, cs, inputs, dev)
     if name == "long_context_b1_k10":
         cases, k = [inputs.long_context_case(100)], 10
     elif name == "long_context_b8_k20":
@@ -582,6 +584,82 @@ def run_workload(args):
     return 0
 
 
+def run_drafted(args, cs, inputs, dev):
+    """CopySpec merged with a draft model (Sec. 3.3) at the 8B shape: a 1B-class draft model
+    (16 layers, d 2048, 32/8 heads of 64, FFN 8192, same vocabulary) proposes delta tokens where
+    the search finds no match.  Scripted target: the stream alternates spans lifted from the
+    4,096-token context with stretches that follow the draft model's own greedy choice three
+    times out of four (built with the draft model on the GPU before the timed runs), so that both
+    kinds of draft are partly accepted.  One line: the merged loop at delta = 3, with delta = 5,
+    copy only (delta = 0, same host-driven loop) and plain decoding beside it."""
+    import torch
+    cfg = inputs.LLAMA8B
+    dcfg = inputs.ModelConfig(n_layers=16, d_model=2048, n_heads=32, n_kv_heads=8, head_dim=64, d_ffn=8192,
+                              vocab=cfg.vocab, rope_theta=500000.0, rms_eps=1e-5)
+    n0, max_new, k = 4096, 768, K_DRAFT
+    stride, max_seq = n0 + max_new + 64, n0 + max_new + k + 64
+    tctx = cs.Context(cfg, inputs.make_weights(cfg, seed=0, device=str(dev)), max_seq=max_seq, max_batch=1, k_max=k)
+    dctx = cs.Context(dcfg, inputs.make_weights(dcfg, seed=1, device=str(dev)), max_seq=max_seq, max_batch=1, k_max=15)
+    g = torch.Generator(device=dev); g.manual_seed(1)
+    kv_t, kv_d = tctx.alloc_kv(), dctx.alloc_kv()
+    for kv, c in ((kv_t, cfg), (kv_d, dcfg)):
+        for layer in range(c.n_layers):
+            kv[layer, :, :, :, :n0 - 1, :] = torch.randn(2, 1, c.n_kv_heads, n0 - 1, c.head_dim, device=dev,
+                                                          generator=g).to(torch.bfloat16)
+    rng = np.random.default_rng(0)
+    context = inputs.zipf_tokens(rng, n0, cfg.vocab, 1.1).astype(np.int32)
+    # ---- the script, built with the draft model itself (single-row greedy steps)
+    kvl = torch.tensor([n0 - 1], dtype=torch.int32, device=dev)
+    last = torch.tensor([int(context[-1])], dtype=torch.int32, device=dev)
+    zero = torch.zeros(1, dtype=torch.int32, device=dev)
+    script = []
+    while len(script) < max_new:
+        if rng.random() < 0.5:
+            src = int(rng.integers(0, n0 - 64))
+            span, follow = [int(t) for t in context[src:src + int(rng.integers(20, 60))]], False
+        else:
+            span, follow = [None] * int(rng.integers(10, 30)), True
+        for t in span:
+            _, ot, _ = dctx.cs_verify_step(last, None, zero, kv_d, kvl)      # caches `last`, predicts the next token
+            if follow:
+                t = int(ot[0, 0]) if rng.random() < 0.75 else int(inputs.zipf_tokens(rng, 1, cfg.vocab, 1.1)[0])
+            script.append(t)
+            last.fill_(t)
+    script = np.asarray(script[:max_new], dtype=np.int32)
+    script_d = torch.from_numpy(script).to(dev)
+    h = np.zeros((1, stride), dtype=np.int32)
+    h[0, :n0] = context
+    res = {}
+    for label, kk, delta in (("copy_and_draft_d3", k, 3), ("copy_and_draft_d5", k, 5), ("copy_only", k, 0), ("plain_decode", 0, 0)):
+        hd = torch.from_numpy(h).to(dev)
+        ld = torch.tensor([n0], dtype=torch.int32, device=dev)
+        kvl_t = torch.tensor([n0 - 1], dtype=torch.int32, device=dev)
+        kvl_d = torch.tensor([n0 - 1], dtype=torch.int32, device=dev)
+        new = max_new if kk else min(max_new, 4 * args.steps)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        st = tctx.cs_decode_loop_drafted(dctx if delta else None, hd, ld, kv_t, kvl_t, kv_d if delta else None,
+                                         kvl_d if delta else None, GAMMA, kk, delta, new, script=script_d)
+        torch.cuda.synchronize()
+        sec = time.perf_counter() - t0
+        if hd[0, n0:n0 + new].cpu().tolist() != script[:new].tolist():
+            raise RuntimeError("the loop did not reproduce the script")
+        res[label] = {"tokens_per_s": st["emitted"] / sec, "ms_per_step": sec / st["steps"] * 1e3, "steps": st["steps"],
+                      "copy_attempts": st["attempts"], "mean_tau_copy": st["accepted"] / max(1, st["attempts"]),
+                      "draft_attempts": st["draft_attempts"],
+                      "mean_tau_draft": st["draft_accepted"] / max(1, st["draft_attempts"])}
+    main_r = res["copy_and_draft_d3"]
+    line = {"metric": METRIC, "value": main_r["tokens_per_s"], "unit": UNIT, "n_gpus": 1, "steps": main_r["steps"],
+            "warmup": 0, "ms_per_step": main_r["ms_per_step"], "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "drafted_b1_k10", "batch": 1, "gamma": GAMMA, "k": k, "delta": 3, "context": n0,
+                       "draft_model": "16L d2048 H32/8 Dh64 F8192 V128256", "timing": "host wall clock around the whole loop "
+                       "(it synchronises every step)", **res,
+                       "speedup_vs_plain_decode": {lab: r["tokens_per_s"] / res["plain_decode"]["tokens_per_s"] for lab, r in res.items()}}}
+    print(json.dumps(line), flush=True)
+    tctx.close(); dctx.close()
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -591,7 +669,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--workload", default="verify",
                     choices=["verify", "verify_plain_decode", "long_context_b1_k10", "long_context_b8_k20", "k_sweep_long_context_b1", "prefill_b1_4096",
-                             "multi_turn_b16_k10", "match_search"],
+                             "multi_turn_b16_k10", "match_search", "drafted_b1_k10"],
                     help="verify = the benchmark; the others are additional single-GPU measurements")
     ap.add_argument("--layers", type=int, default=0,
                     help="profiling aid: keep only this many of the 32 layers (small case for ncu captures; "
