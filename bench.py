@@ -14,7 +14,8 @@ each step accepts a prescribed number of draft tokens).
 
 `value` is emitted tokens per second (accepted draft tokens plus the one guaranteed token
 per step) with everything resident in HBM; `e2e` drives the same steps from pinned host
-buffers through cs_find_match / cs_verify_step with the copies inside the timed region.
+buffers through cs_step_host (one C call per step: copies in, search, verify, copies out,
+host append), all inside the timed region.
 With N > 1 every rank runs an independent replica (the path does not shard).
 `--impl reference` times the CPU oracle, as it stands, on a bounded sample.
 """
@@ -294,38 +295,28 @@ def run_ours(args):
         raise RuntimeError(f"loop ran {steps_run} steps / {emitted} tokens, expected {K} / {expect}")
     ms, value = aggregate_replicas(ms, emitted, world, dev)
 
-    # ---- end to end from pinned host buffers (search + verify per step, host bookkeeping)
+    # ---- end to end from pinned host buffers: one cs_step_host call per step (history, length
+    # and script row host -> device, search + verify, accepted length and tokens device -> host,
+    # the host appends)
     Ke = min(K, 50)
     hist_p = torch.from_numpy(hist_h.copy()).pin_memory()
     len_p = torch.tensor([n0], dtype=torch.int32).pin_memory()
     scr_p = torch.zeros(1, K_DRAFT + 1, dtype=torch.int32).pin_memory()
-    res_p = torch.zeros(1, K_DRAFT + 2, dtype=torch.int32).pin_memory()
+    acc_p = torch.zeros(1, dtype=torch.int32).pin_memory()
+    out_p = torch.zeros(1, K_DRAFT + 1, dtype=torch.int32).pin_memory()
     hist_e = torch.empty_like(hist_d)
     len_e = torch.empty_like(len_d)
-    scr_e = torch.empty(1, K_DRAFT + 1, dtype=torch.int32, device=dev)
-    res_e = torch.empty(1, K_DRAFT + 2, dtype=torch.int32, device=dev)
-    mp = torch.empty(1, dtype=torch.int32, device=dev)
-    dr = torch.empty(1, K_DRAFT, dtype=torch.int32, device=dev)
-    dl = torch.empty(1, dtype=torch.int32, device=dev)
-    am = torch.empty(1, K_DRAFT + 1, dtype=torch.int32, device=dev)
     kvlen_d.fill_(n0 - 1)
-    script_pad = np.concatenate([script, np.full(K_DRAFT + 1, -1, dtype=np.int32)])
-    h2d = hist_p.numel() * 4 + 4 + scr_p.numel() * 4
-    d2h = res_p.numel() * 4
+    script_pad = torch.from_numpy(np.concatenate([script, np.full(K_DRAFT + 1, -1, dtype=np.int32)]))
+    d2h = (acc_p.numel() + out_p.numel()) * 4
+    h2d_total = 0
 
     def host_step(n, e):
-        scr_p[0].copy_(torch.from_numpy(script_pad[e:e + K_DRAFT + 1]))
-        len_p[0] = n
-        hist_e.copy_(hist_p, non_blocking=True)
-        len_e.copy_(len_p, non_blocking=True)
-        scr_e.copy_(scr_p, non_blocking=True)
-        cs.cs_find_match(hist_e, len_e, GAMMA, K_DRAFT, out=(mp, dr, dl))
-        last = hist_e[:, n - 1].contiguous()
-        ctx.cs_verify_step(last, dr, dl, kv, kvlen_d, target_script=scr_e, out=(res_e[0, :1], res_e[:, 1:], am))
-        res_p.copy_(res_e, non_blocking=True)
-        torch.cuda.current_stream().synchronize()
-        tau = int(res_p[0, 0])
-        hist_p[0, n:n + tau + 1] = res_p[0, 1:tau + 2]
+        nonlocal h2d_total
+        scr_p[0].copy_(script_pad[e:e + K_DRAFT + 1])
+        ctx.cs_step_host(hist_p, len_p, hist_e, len_e, kv, kvlen_d, GAMMA, K_DRAFT, acc_p, out_p, script_host=scr_p)
+        h2d_total += n * 4 + 4 + scr_p.numel() * 4
+        tau = int(acc_p[0])
         return n + tau + 1, e + tau + 1
 
     n, e = n0, 0
@@ -334,6 +325,7 @@ def run_ours(args):
     barrier()
     t0 = time.perf_counter()
     e_start = e
+    h2d_total = 0
     for _ in range(Ke):
         n, e = host_step(n, e)
     torch.cuda.synchronize()
@@ -345,8 +337,8 @@ def run_ours(args):
     # ---- roofline of the dominant kernel (the weight-streaming projection GEMM) ---------
     kvlen_d.fill_(n0 - 1)
     last = torch.tensor([int(hist[-1])], dtype=torch.int32, device=dev)
-    dr.copy_(torch.from_numpy(script[None, :K_DRAFT].copy()))
-    dl.fill_(K_DRAFT)
+    dr = torch.from_numpy(script[None, :K_DRAFT].copy()).to(dev)
+    dl = torch.full((1,), K_DRAFT, dtype=torch.int32, device=dev)
     fam_ms, fam_n = None, None
     for _ in range(3):
         kvlen_d.fill_(n0 - 1)
@@ -382,7 +374,7 @@ def run_ours(args):
                            "tokens_per_step": emitted / K, "l2": "inputs larger than L2 (15 GB of weights per step)",
                            "replicas": world, "draft_tokens_accepted_per_s": world * (emitted - K) / (ms * 1e-3)},
                 "clocks": clocks,
-                "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": h2d_total // Ke, "d2h_bytes_per_step": d2h,
                         "steps": Ke, "ms_per_step": e2e_s / Ke * 1e3},
                 "gpu_launches": launches_per_step * K,
                 "roofline": roofline, "cpu_baseline": cpu}

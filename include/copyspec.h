@@ -191,6 +191,29 @@ cs_status cs_verify_step(cs_ctx* ctx, const int32_t* last_tok, const int32_t* dr
                          int32_t* out_tokens, int32_t* argmax_ids, float* logits_dbg,
                          void* stream);
 
+/* One whole step driven from HOST memory (App. B.3 steps 1, 2 and 4; Sec. 3.2), for callers
+ * that keep the token histories on the host.  Synchronous: returns when the step is done.
+ * Copies the accepted tokens (hist_len_host[b] ints per sequence), the lengths and this step's
+ * script rows to the device, runs cs_find_match and cs_verify_step on them, copies the accepted
+ * lengths and the emitted tokens back, and appends the tau + 1 emitted tokens of every sequence
+ * to hist_host (hist_len_host advances; kv_len advances on the device).
+ *   hist_host int32 [B][stride] host (pinned memory makes the copies asynchronous), in/out;
+ *   hist_len_host int32 [B] host, in/out; hist_len_host[b] + k + 1 <= stride (CS_ERR_CAPACITY).
+ *   hist_dev int32 [B][stride], hist_len_dev int32 [B]: device buffers of the caller that the
+ *            call overwrites.  kv_cache / kv_len as in cs_verify_step (kv_len[b] =
+ *            hist_len[b] - 1 on entry).
+ *   script_host int32 [B][k+1] host or NULL: the target tokens of this step's rows
+ *            (scripted-target mode), NULL = real mode.
+ *   accept_len_host int32 [B], out_tokens_host int32 [B][k+1]: host outputs (tau, then the
+ *            tau + 1 emitted tokens; -1 beyond).  A sequence the device skipped for lack of
+ *            cache room has accept_len -1, is left as it was, and cs_sync_status reports it.
+ * The context's loop buffers serve as scratch: not to be mixed with an open cs_loop_begin
+ * session.  Errors: CS_ERR_ARG / CS_ERR_CAPACITY on the host before any copy, CS_ERR_CUDA. */
+cs_status cs_step_host(cs_ctx* ctx, int32_t* hist_host, int32_t* hist_len_host, int B, int stride,
+                       int32_t* hist_dev, int32_t* hist_len_dev, void* kv_cache, int32_t* kv_len,
+                       int gamma, int k, cs_match_policy policy, const int32_t* script_host,
+                       int32_t* accept_len_host, int32_t* out_tokens_host, void* stream);
+
 /* KV truncation to an accepted length (App. B.2; App. B.3 step 2(b)).  Async.
  * kv_len[b] = new_len[b] where 0 <= new_len[b] <= kv_len[b]; otherwise kv_len[b] is
  * left as is and CS_ERR_ARG is recorded in the status word.  The cache is contiguous

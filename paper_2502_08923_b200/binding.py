@@ -48,7 +48,7 @@ class CsStats(C.Structure):
 
 
 EXPORTS = ("cs_workspace_bytes", "cs_create", "cs_destroy", "cs_last_error", "cs_sync_status",
-           "cs_find_match", "cs_verify_step", "cs_kv_truncate", "cs_decode_loop", "cs_decode_loop_drafted",
+           "cs_find_match", "cs_verify_step", "cs_kv_truncate", "cs_decode_loop", "cs_decode_loop_drafted", "cs_step_host",
            "cs_prefill", "cs_linear",
            "cs_loop_begin", "cs_loop_steps", "cs_loop_poll", "cs_loop_end", "cs_profile_verify_step",
            "cs_loop_launches_per_step", "cs_lm_head", "cs_lm_head_static", "cs_gram_index_bytes",
@@ -90,6 +90,8 @@ def load(build_if_missing: bool = True) -> C.CDLL:
     lib.cs_kv_truncate.argtypes = [vp, ip, ip, i, vp]
     lib.cs_decode_loop.restype = i
     lib.cs_decode_loop.argtypes = [vp, ip, ip, i, i, vp, ip, i, i, i, i, i, ip, C.POINTER(CsStats), vp]
+    lib.cs_step_host.restype = i
+    lib.cs_step_host.argtypes = [vp, ip, ip, i, i, ip, ip, vp, ip, i, i, i, ip, ip, ip, vp]
     lib.cs_decode_loop_drafted.restype = i
     lib.cs_decode_loop_drafted.argtypes = [vp, vp, ip, ip, i, vp, ip, vp, ip, i, i, i, i, i, i, ip,
                                            C.POINTER(CsStats), C.POINTER(C.c_uint64), vp]
@@ -123,6 +125,14 @@ def _ptr(t):
         return None
     if not t.is_cuda or not t.is_contiguous():
         raise ValueError("expected a contiguous CUDA tensor")
+    return C.c_void_p(t.data_ptr())
+
+
+def _host_i32(t, name):
+    if t is None:
+        return None
+    if t.is_cuda or not t.is_contiguous() or t.dtype != torch.int32:
+        raise ValueError(f"{name} must be a contiguous int32 host tensor")
     return C.c_void_p(t.data_ptr())
 
 
@@ -316,6 +326,18 @@ class Context:
                                      _i32(ot, "out_tokens"), _i32(am, "argmax_ids"), _ptr(logits_dbg), _stream())
         self._check(rc, "cs_verify_step")
         return al, ot, am
+
+    def cs_step_host(self, hist_host, hist_len_host, hist_dev, hist_len_dev, kv_cache, kv_len, gamma, k,
+                     accept_len_host, out_tokens_host, policy=LATEST, script_host=None):
+        """One step from host (CPU, ideally pinned) int32 tensors; hist_host / hist_len_host advance in
+        place, accept_len_host [B] and out_tokens_host [B][k+1] receive the step's result."""
+        B, stride = hist_host.shape
+        rc = self.lib.cs_step_host(self.handle, _host_i32(hist_host, "hist_host"), _host_i32(hist_len_host, "hist_len_host"),
+                                   B, stride, _i32(hist_dev, "hist_dev"), _i32(hist_len_dev, "hist_len_dev"),
+                                   _ptr(kv_cache), _i32(kv_len, "kv_len"), gamma, k, policy,
+                                   _host_i32(script_host, "script_host"), _host_i32(accept_len_host, "accept_len_host"),
+                                   _host_i32(out_tokens_host, "out_tokens_host"), _stream())
+        self._check(rc, "cs_step_host")
 
     def cs_kv_truncate(self, kv_len, new_len):
         rc = self.lib.cs_kv_truncate(self.handle, _i32(kv_len, "kv_len"), _i32(new_len, "new_len"),

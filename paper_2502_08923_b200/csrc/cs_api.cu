@@ -404,6 +404,53 @@ cs_status cs_verify_step(cs_ctx* ctx, const int32_t* last_tok, const int32_t* dr
   return CS_OK;
 }
 
+cs_status cs_step_host(cs_ctx* ctx, int32_t* hist_host, int32_t* hist_len_host, int B, int stride,
+                       int32_t* hist_dev, int32_t* hist_len_dev, void* kv_cache, int32_t* kv_len, int gamma, int k,
+                       cs_match_policy policy, const int32_t* script_host, int32_t* accept_len_host,
+                       int32_t* out_tokens_host, void* stream) {
+  if (ctx == nullptr) return CS_ERR_ARG;
+  if (B < 1 || B > ctx->cfg.max_batch || k < 0 || k > ctx->cfg.k_max || gamma < 1 || stride < 1)
+    return fail(ctx, CS_ERR_ARG, "B, k, gamma or stride out of range");
+  if (hist_host == nullptr || hist_len_host == nullptr || hist_dev == nullptr || hist_len_dev == nullptr ||
+      kv_cache == nullptr || kv_len == nullptr || accept_len_host == nullptr || out_tokens_host == nullptr)
+    return fail(ctx, CS_ERR_ARG, "NULL argument");
+  for (int b = 0; b < B; ++b)
+    if (hist_len_host[b] < 1 || hist_len_host[b] + k + 1 > stride)
+      return fail(ctx, CS_ERR_CAPACITY, "history row too short for one more block");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // ---- host -> device: the accepted tokens of every sequence, the lengths, this step's script rows
+  for (int b = 0; b < B; ++b)
+    CS_CUDA_OK(ctx, cudaMemcpyAsync(hist_dev + (size_t)b * stride, hist_host + (size_t)b * stride,
+                                    (size_t)hist_len_host[b] * 4, cudaMemcpyHostToDevice, st));
+  CS_CUDA_OK(ctx, cudaMemcpyAsync(hist_len_dev, hist_len_host, (size_t)B * 4, cudaMemcpyHostToDevice, st));
+  const int32_t* script_dev = nullptr;
+  if (script_host != nullptr) {
+    CS_CUDA_OK(ctx, cudaMemcpyAsync(ctx->loop_emitted, script_host, (size_t)B * (k + 1) * 4, cudaMemcpyHostToDevice, st));
+    script_dev = ctx->loop_emitted;
+  }
+  // ---- App. B.3 step 1 (search, gather), step 2 (verify, accept, truncate)
+  cs_status s = cs_launch_find_match(hist_dev, hist_len_dev, B, stride, gamma, k, (int)policy, ctx->loop_mpos,
+                                     ctx->loop_draft, ctx->loop_dlen, ctx->loop_last, nullptr, st);
+  if (s != CS_OK) return fail(ctx, s, "match kernel launch failed");
+  cs_launch_block_setup(ctx, ctx->loop_last, ctx->loop_draft, ctx->loop_dlen, kv_len, nullptr, B, k, st);
+  s = enqueue_forward(ctx, B, k + 1, kv_cache, true, nullptr, st);
+  if (s != CS_OK) return s;
+  cs_launch_accept(ctx, B, k, ctx->loop_draft, ctx->loop_dlen, script_dev, k + 1, nullptr, k + 1, ctx->loop_accept,
+                   ctx->loop_out, ctx->loop_argmax, kv_len, 1, st);
+  // ---- device -> host, then step 4 on the host: append what was emitted
+  CS_CUDA_OK(ctx, cudaMemcpyAsync(accept_len_host, ctx->loop_accept, (size_t)B * 4, cudaMemcpyDeviceToHost, st));
+  CS_CUDA_OK(ctx, cudaMemcpyAsync(out_tokens_host, ctx->loop_out, (size_t)B * (k + 1) * 4, cudaMemcpyDeviceToHost, st));
+  CS_CUDA_OK(ctx, cudaStreamSynchronize(st));
+  for (int b = 0; b < B; ++b) {
+    const int tau = accept_len_host[b];
+    if (tau < 0 || tau > k) continue;                  // the device skipped this sequence (status word)
+    const int n = hist_len_host[b];
+    for (int i = 0; i <= tau; ++i) hist_host[(size_t)b * stride + n + i] = out_tokens_host[(size_t)b * (k + 1) + i];
+    hist_len_host[b] = n + tau + 1;
+  }
+  return CS_OK;
+}
+
 cs_status cs_kv_truncate(cs_ctx* ctx, int32_t* kv_len, const int32_t* new_len, int B, void* stream) {
   if (ctx == nullptr) return CS_ERR_ARG;
   if (B < 0 || kv_len == nullptr || new_len == nullptr) return fail(ctx, CS_ERR_ARG, "bad argument");

@@ -62,6 +62,7 @@ def test_context_calls_reject_null():
     assert lib.cs_decode_loop(None, None, None, 1, 1, None, None, 3, 10, 0, 1, -1, None, None, None) == cs.CS_ERR_ARG
     assert lib.cs_decode_loop_drafted(None, None, None, None, 8, None, None, None, None, 3, 10, 3, 0, 1, -1, None, None,
                                       None, None) == cs.CS_ERR_ARG
+    assert lib.cs_step_host(None, None, None, 1, 8, None, None, None, None, 3, 1, 0, None, None, None, None) == cs.CS_ERR_ARG
     assert lib.cs_prefill(None, None, None, 1, 1, 1, None, None, None) == cs.CS_ERR_ARG
     assert lib.cs_sync_status(None, None) == cs.CS_ERR_ARG
     h = C.c_void_p()

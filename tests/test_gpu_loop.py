@@ -190,3 +190,62 @@ def test_real_mode_loop_with_wide_heads_and_caches_of_many_key_tiles():
         for key in ("steps", "attempts", "accepted", "emitted", "no_match"):
             assert st[key] == tot[key], key
     ctx.close()
+
+
+def test_steps_driven_from_host_memory():
+    """cs_step_host: histories kept on the host, one call per step.  Scripted mode against the
+    model-free simulator (two sequences of different lengths), then real mode against the
+    oracle's greedy choice."""
+    cfg = inputs.TINY
+    ctx, model = make_pair(cfg, 1024, 2, 10)
+    rng = np.random.default_rng(11)
+    ctxt, _ = inputs.tiny_context(seed=1)
+    lens = [512, 300]
+    max_new, stride, k = 80, 640, 10
+    scripts = [inputs.copy_script(rng, ctxt[:n], max_new, 0.6, 5, 30, cfg.vocab, zipf_s=None) for n in lens]
+
+    def prefilled():
+        h = np.zeros((2, stride), dtype=np.int32)
+        for b, n in enumerate(lens):
+            h[b, :n] = ctxt[:n]
+        kv = ctx.alloc_kv()
+        kvl = torch.zeros(2, dtype=torch.int32, device="cuda")
+        ctx.cs_prefill(i32(h), i32(lens), max(lens), kv, kvl)
+        return torch.from_numpy(h).pin_memory(), torch.tensor(lens, dtype=torch.int32).pin_memory(), kv, kvl
+
+    hist_h, len_h, kv, kvl = prefilled()
+    hist_d, len_d = torch.empty(2, stride, dtype=torch.int32, device="cuda"), torch.empty(2, dtype=torch.int32, device="cuda")
+    acc, out = torch.zeros(2, dtype=torch.int32).pin_memory(), torch.zeros(2, k + 1, dtype=torch.int32).pin_memory()
+    scr = torch.zeros(2, k + 1, dtype=torch.int32).pin_memory()
+    pads = [np.concatenate([s, np.full(k + 1, -1, dtype=np.int32)]) for s in scripts]
+    sims = [O.scripted_simulator(ctxt[:n], s, 3, k, O.LATEST, max_new + k + 1)[0] for n, s in zip(lens, pads)]
+    for step in range(6):
+        e = [int(len_h[b]) - lens[b] for b in range(2)]
+        assert max(e) + k + 1 <= max_new          # every row of the block still has a script entry
+        for b in range(2):
+            scr[b] = torch.from_numpy(pads[b][e[b]:e[b] + k + 1])
+        ctx.cs_step_host(hist_h, len_h, hist_d, len_d, kv, kvl, 3, k, acc, out, script_host=scr)
+        for b in range(2):
+            rec = sims[b][step]
+            assert int(acc[b]) == rec["tau"] and out[b, :rec["tau"] + 1].tolist() == rec["out"], (step, b)
+            assert int(len_h[b]) == rec["n"] + rec["tau"] + 1
+    assert ctx.cs_sync_status() == 0
+    assert kvl.cpu().tolist() == [int(len_h[b]) - 1 for b in range(2)]
+    for b in range(2):
+        n = int(len_h[b])
+        assert hist_h[b, lens[b]:n].tolist() == scripts[b][:n - lens[b]].tolist()
+
+    # real mode: every emitted token is the oracle's greedy choice up to the logit tolerance
+    hist_h, len_h, kv, kvl = prefilled()
+    for _ in range(8):
+        ctx.cs_step_host(hist_h, len_h, hist_d, len_d, kv, kvl, 3, k, acc, out)
+    assert ctx.cs_sync_status() == 0
+    for b in range(2):
+        gen = hist_h[b, lens[b]:int(len_h[b])].tolist()
+        assert len(gen) >= 8 and max(greedy_margins(model, cfg, ctxt[:lens[b]], gen)) < LOGIT_TOL
+    # a history row without room for one more block is refused on the host, nothing changes
+    len_h[0] = stride - 5
+    with pytest.raises(cs.CsError):
+        ctx.cs_step_host(hist_h, len_h, hist_d, len_d, kv, kvl, 3, k, acc, out)
+    assert int(len_h[0]) == stride - 5
+    ctx.close()
