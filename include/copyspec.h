@@ -207,8 +207,10 @@ cs_status cs_verify_step(cs_ctx* ctx, const int32_t* last_tok, const int32_t* dr
  *   accept_len_host int32 [B], out_tokens_host int32 [B][k+1]: host outputs (tau, then the
  *            tau + 1 emitted tokens; -1 beyond).  A sequence the device skipped for lack of
  *            cache room has accept_len -1, is left as it was, and cs_sync_status reports it.
- * The context's loop buffers serve as scratch: not to be mixed with an open cs_loop_begin
- * session.  Errors: CS_ERR_ARG / CS_ERR_CAPACITY on the host before any copy, CS_ERR_CUDA. */
+ * The kernels of the step are replayed as a CUDA graph that the context keeps while B, k, gamma,
+ * the policy, the mode and the device buffers stay the same (first call and every change: one
+ * capture).  The context's loop buffers serve as scratch: not to be mixed with an open
+ * cs_loop_begin session.  Errors: CS_ERR_ARG / CS_ERR_CAPACITY on the host before any copy, CS_ERR_CUDA. */
 cs_status cs_step_host(cs_ctx* ctx, int32_t* hist_host, int32_t* hist_len_host, int B, int stride,
                        int32_t* hist_dev, int32_t* hist_len_dev, void* kv_cache, int32_t* kv_len,
                        int gamma, int k, cs_match_policy policy, const int32_t* script_host,

@@ -356,6 +356,8 @@ void cs_destroy(cs_ctx* ctx) {
   if (ctx == nullptr) return;
   cs_loop_end(ctx);
   if (ctx->cap_stream) cudaStreamDestroy(ctx->cap_stream);
+  if (ctx->host_step.exec) cudaGraphExecDestroy(ctx->host_step.exec);
+  if (ctx->host_step.graph) cudaGraphDestroy(ctx->host_step.graph);
   delete[] ctx->layers;
   delete ctx;
 }
@@ -428,15 +430,56 @@ cs_status cs_step_host(cs_ctx* ctx, int32_t* hist_host, int32_t* hist_len_host, 
     CS_CUDA_OK(ctx, cudaMemcpyAsync(ctx->loop_emitted, script_host, (size_t)B * (k + 1) * 4, cudaMemcpyHostToDevice, st));
     script_dev = ctx->loop_emitted;
   }
-  // ---- App. B.3 step 1 (search, gather), step 2 (verify, accept, truncate)
-  cs_status s = cs_launch_find_match(hist_dev, hist_len_dev, B, stride, gamma, k, (int)policy, ctx->loop_mpos,
-                                     ctx->loop_draft, ctx->loop_dlen, ctx->loop_last, nullptr, st);
-  if (s != CS_OK) return fail(ctx, s, "match kernel launch failed");
-  cs_launch_block_setup(ctx, ctx->loop_last, ctx->loop_draft, ctx->loop_dlen, kv_len, nullptr, B, k, st);
-  s = enqueue_forward(ctx, B, k + 1, kv_cache, true, nullptr, st);
-  if (s != CS_OK) return s;
-  cs_launch_accept(ctx, B, k, ctx->loop_draft, ctx->loop_dlen, script_dev, k + 1, nullptr, k + 1, ctx->loop_accept,
-                   ctx->loop_out, ctx->loop_argmax, kv_len, 1, st);
+  // ---- App. B.3 step 1 (search, gather), step 2 (verify, accept, truncate): the kernels of one
+  // step, replayed as a graph while the launch shape and the buffers stay the same
+  // (CS_NO_GRAPH=1 enqueues them one by one)
+  HostStepGraph& G = ctx->host_step;
+  const char* env = getenv("CS_NO_GRAPH");
+  const bool use_graph = !(env != nullptr && env[0] == '1');
+  const bool same = G.exec != nullptr && G.hist_dev == hist_dev && G.hist_len_dev == hist_len_dev &&
+                    G.kv_cache == kv_cache && G.kv_len == kv_len && G.B == B && G.stride == stride &&
+                    G.gamma == gamma && G.k == k && G.policy == (int)policy && G.scripted == (script_dev != nullptr);
+  auto enqueue = [&](cudaStream_t q) -> cs_status {
+    cs_status r = cs_launch_find_match(hist_dev, hist_len_dev, B, stride, gamma, k, (int)policy, ctx->loop_mpos,
+                                       ctx->loop_draft, ctx->loop_dlen, ctx->loop_last, nullptr, q);
+    if (r != CS_OK) return fail(ctx, r, "match kernel launch failed");
+    cs_launch_block_setup(ctx, ctx->loop_last, ctx->loop_draft, ctx->loop_dlen, kv_len, nullptr, B, k, q);
+    // the search opens the step stream-ordered and every call ends synchronised, so the cached
+    // rows and kv_len are settled while the forward runs
+    ctx->kv_len_early = kv_len;
+    r = enqueue_forward(ctx, B, k + 1, kv_cache, true, nullptr, q);
+    ctx->kv_len_early = nullptr;
+    if (r != CS_OK) return r;
+    cs_launch_accept(ctx, B, k, ctx->loop_draft, ctx->loop_dlen, script_dev, k + 1, nullptr, k + 1, ctx->loop_accept,
+                     ctx->loop_out, ctx->loop_argmax, kv_len, 1, q);
+    return CS_OK;
+  };
+  cs_status s = CS_OK;
+  if (!use_graph) {
+    s = enqueue(st);
+    if (s != CS_OK) return s;
+  } else {
+    if (!same) {
+      if (G.exec) cudaGraphExecDestroy(G.exec);
+      if (G.graph) cudaGraphDestroy(G.graph);
+      G = HostStepGraph{};
+      s = ensure_act_maps(ctx, cs_ceil_div(B * (k + 1), 16) * 16);   // host work that must precede capture
+      if (s != CS_OK) return s;
+      CS_CUDA_OK(ctx, cudaStreamBeginCapture(ctx->cap_stream, cudaStreamCaptureModeRelaxed));
+      s = enqueue(ctx->cap_stream);
+      cudaError_t e = cudaStreamEndCapture(ctx->cap_stream, &G.graph);
+      if (s == CS_OK && e == cudaSuccess) e = cudaGraphInstantiate(&G.exec, G.graph, 0);
+      if (s != CS_OK || e != cudaSuccess) {
+        if (G.graph) cudaGraphDestroy(G.graph);
+        G = HostStepGraph{};
+        if (s != CS_OK) return s;
+        CS_CUDA_OK(ctx, e);
+      }
+      G.hist_dev = hist_dev; G.hist_len_dev = hist_len_dev; G.kv_cache = kv_cache; G.kv_len = kv_len;
+      G.B = B; G.stride = stride; G.gamma = gamma; G.k = k; G.policy = (int)policy; G.scripted = script_dev != nullptr;
+    }
+    CS_CUDA_OK(ctx, cudaGraphLaunch(G.exec, st));
+  }
   // ---- device -> host, then step 4 on the host: append what was emitted
   CS_CUDA_OK(ctx, cudaMemcpyAsync(accept_len_host, ctx->loop_accept, (size_t)B * 4, cudaMemcpyDeviceToHost, st));
   CS_CUDA_OK(ctx, cudaMemcpyAsync(out_tokens_host, ctx->loop_out, (size_t)B * (k + 1) * 4, cudaMemcpyDeviceToHost, st));

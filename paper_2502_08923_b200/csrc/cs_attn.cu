@@ -257,10 +257,9 @@ int launch(cs_ctx* ctx, const void* kv_cache, int layer, int B, int R, cudaStrea
   if (nsplit > ctx->attn_splits) nsplit = ctx->attn_splits;
   if (nsplit < 1) nsplit = 1;
   const size_t smem = (size_t)2 * kStages * kKeys * (DH + 8) * 2;
-  static bool set = false;
-  if (!set) {
+  if (!(ctx->attn_mma_attr_set & (1u << (DH / 32)))) {
     cudaFuncSetAttribute(k_attn_mma<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    set = true;
+    ctx->attn_mma_attr_set |= 1u << (DH / 32);
   }
   const float scale_log2e = 1.4426950408889634f / sqrtf((float)DH);
   cs_launch_pdl(k_attn_mma<DH>, dim3(B * c.n_kv_heads, nsplit, rgs), dim3(kThreads), smem, st, ctx->qbuf,

@@ -558,13 +558,12 @@ int cs_launch_attention_tc(cs_ctx* ctx, const void* kv_cache, int layer, int B, 
   int nsplit = (small ? 2 : 1) * ctx->num_sms / (B * c.n_kv_heads * ngroups);
   if (nsplit > ctx->attn_splits) nsplit = ctx->attn_splits;
   if (nsplit < 1) nsplit = 1;
-  static size_t smem_set = 0;
-  if (smem > smem_set) {
+  if (smem > ctx->attn_tc_smem_set) {
     if (cudaFuncSetAttribute(k_attn_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
       snprintf(ctx->err, sizeof(ctx->err), "attention needs %zu bytes of shared memory", smem);
       return -1;
     }
-    smem_set = smem;
+    ctx->attn_tc_smem_set = smem;
   }
   AttnArgs a;
   a.row_lim = ctx->row_lim;

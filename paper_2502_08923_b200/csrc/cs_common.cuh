@@ -53,6 +53,15 @@ struct LoopState {
   cudaGraphExec_t exec;
 };
 
+// cs_step_host keeps the graph of its last launch shape: the kernels of one step between the
+// host -> device and device -> host copies
+struct HostStepGraph {
+  const void *hist_dev, *hist_len_dev, *kv_cache, *kv_len;
+  int B, stride, gamma, k, policy, scripted;
+  cudaGraph_t graph;
+  cudaGraphExec_t exec;
+};
+
 // event brackets around kernel families (cs_profile_verify_step)
 static constexpr int CS_PROF_MAX = 2048;
 static constexpr int CS_PROF_FAMILIES = 4;
@@ -126,10 +135,16 @@ struct cs_ctx {
   // ordinary stream-ordered launch (the generation loop); NULL elsewhere.  The attention
   // kernel may then fetch tiles of cached keys before it waits for the preceding kernel.
   const int* kv_len_early;
+  // shared-memory opt-ins already made for this context's device (per context, not per
+  // process: another context may live on another GPU)
+  bool gemm_attr_set;
+  unsigned attn_mma_attr_set;   // bit DH/32 per head size
+  size_t attn_tc_smem_set;
   int attn_force;            // 0 = choose by shape, 1 = mma.sync kernel, 2 = tcgen05 kernel
   int tune_smem_kb;          // > 0: shared memory budget of a GEMM CTA (CS_TUNE_SMEM_KB, read at creation)
 
   LoopState loop;
+  HostStepGraph host_step;
   Prof* prof;   // non-NULL only inside cs_profile_verify_step
 
   char err[256];

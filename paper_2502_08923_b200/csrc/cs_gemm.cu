@@ -749,10 +749,9 @@ cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX,
   }
   a.stages = stages;
   const size_t smem = (size_t)fixed + (size_t)stages * stage_bytes;
-  static bool attr_set = false;
-  if (!attr_set) {
+  if (!ctx->gemm_attr_set) {
     CS_CUDA_OK(ctx, cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-    attr_set = true;
+    ctx->gemm_attr_set = true;
   }
   cudaLaunchConfig_t lc = {};
   lc.gridDim = dim3(tiles, a.splits, 1);
