@@ -356,6 +356,10 @@ void cs_destroy(cs_ctx* ctx) {
   if (ctx == nullptr) return;
   cs_loop_end(ctx);
   if (ctx->cap_stream) cudaStreamDestroy(ctx->cap_stream);
+  for (int i = 0; i < CS_VERIFY_GRAPHS; ++i) {
+    if (ctx->verify_graphs[i].exec) cudaGraphExecDestroy(ctx->verify_graphs[i].exec);
+    if (ctx->verify_graphs[i].graph) cudaGraphDestroy(ctx->verify_graphs[i].graph);
+  }
   if (ctx->host_step.exec) cudaGraphExecDestroy(ctx->host_step.exec);
   if (ctx->host_step.graph) cudaGraphDestroy(ctx->host_step.graph);
   delete[] ctx->layers;
@@ -405,6 +409,60 @@ cs_status cs_verify_step(cs_ctx* ctx, const int32_t* last_tok, const int32_t* dr
   CS_CUDA_OK(ctx, cudaGetLastError());
   return CS_OK;
 }
+
+}  // extern "C"
+
+cs_status cs_verify_step_cached(cs_ctx* ctx, const int32_t* last_tok, const int32_t* draft, const int32_t* draft_len,
+                                int B, int k, void* kv_cache, int32_t* kv_len, const int32_t* target_script,
+                                int32_t* accept_len, int32_t* out_tokens, int32_t* argmax_ids, cudaStream_t st) {
+  const char* env = getenv("CS_NO_GRAPH");
+  if (env != nullptr && env[0] == '1')
+    return cs_verify_step(ctx, last_tok, draft, draft_len, B, k, kv_cache, kv_len, target_script, accept_len,
+                          out_tokens, argmax_ids, nullptr, st);
+  if (ctx == nullptr) return CS_ERR_ARG;
+  if (B < 1 || B > ctx->cfg.max_batch || k < 0 || k > ctx->cfg.k_max) return fail(ctx, CS_ERR_ARG, "B or k out of range");
+  if (last_tok == nullptr || draft_len == nullptr || (draft == nullptr && k > 0) || kv_cache == nullptr ||
+      kv_len == nullptr || accept_len == nullptr || out_tokens == nullptr || argmax_ids == nullptr)
+    return fail(ctx, CS_ERR_ARG, "NULL argument");
+  const void* key[9] = {last_tok, draft, draft_len, kv_cache, kv_len, target_script, accept_len, out_tokens, argmax_ids};
+  VerifyGraph* g = nullptr;
+  for (int i = 0; i < CS_VERIFY_GRAPHS && g == nullptr; ++i) {
+    VerifyGraph& c = ctx->verify_graphs[i];
+    if (c.exec != nullptr && c.B == B && c.k == k && memcmp(c.key, key, sizeof(key)) == 0) g = &c;
+  }
+  if (g == nullptr) {
+    g = &ctx->verify_graphs[ctx->verify_graph_next];
+    ctx->verify_graph_next = (ctx->verify_graph_next + 1) % CS_VERIFY_GRAPHS;
+    if (g->exec) cudaGraphExecDestroy(g->exec);
+    if (g->graph) cudaGraphDestroy(g->graph);
+    *g = VerifyGraph{};
+    cs_status s = ensure_act_maps(ctx, cs_ceil_div(B * (k + 1), 16) * 16);   // host work that must precede capture
+    if (s != CS_OK) return s;
+    CS_CUDA_OK(ctx, cudaStreamBeginCapture(ctx->cap_stream, cudaStreamCaptureModeRelaxed));
+    cs_launch_block_setup(ctx, last_tok, draft, draft_len, kv_len, nullptr, B, k, ctx->cap_stream);
+    ctx->kv_len_early = kv_len;      // nothing before the acceptance kernel changes it
+    s = enqueue_forward(ctx, B, k + 1, kv_cache, true, nullptr, ctx->cap_stream);
+    ctx->kv_len_early = nullptr;
+    if (s == CS_OK)
+      cs_launch_accept(ctx, B, k, draft, draft_len, target_script, k + 1, nullptr, k + 1, accept_len, out_tokens,
+                       argmax_ids, kv_len, 1, ctx->cap_stream);
+    cudaError_t e = cudaStreamEndCapture(ctx->cap_stream, &g->graph);
+    if (s == CS_OK && e == cudaSuccess) e = cudaGraphInstantiate(&g->exec, g->graph, 0);
+    if (s != CS_OK || e != cudaSuccess) {
+      if (g->graph) cudaGraphDestroy(g->graph);
+      *g = VerifyGraph{};
+      if (s != CS_OK) return s;
+      CS_CUDA_OK(ctx, e);
+    }
+    memcpy(g->key, key, sizeof(key));
+    g->B = B;
+    g->k = k;
+  }
+  CS_CUDA_OK(ctx, cudaGraphLaunch(g->exec, st));
+  return CS_OK;
+}
+
+extern "C" {
 
 cs_status cs_step_host(cs_ctx* ctx, int32_t* hist_host, int32_t* hist_len_host, int B, int stride,
                        int32_t* hist_dev, int32_t* hist_len_dev, void* kv_cache, int32_t* kv_len, int gamma, int k,

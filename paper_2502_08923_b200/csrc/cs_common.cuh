@@ -62,6 +62,15 @@ struct HostStepGraph {
   cudaGraphExec_t exec;
 };
 
+// cs_verify_step_cached keeps the graphs of its last few launch shapes
+struct VerifyGraph {
+  const void* key[9];   // last_tok, draft, draft_len, kv_cache, kv_len, script, accept_len, out_tokens, argmax_ids
+  int B, k;
+  cudaGraph_t graph;
+  cudaGraphExec_t exec;
+};
+static constexpr int CS_VERIFY_GRAPHS = 8;
+
 // event brackets around kernel families (cs_profile_verify_step)
 static constexpr int CS_PROF_MAX = 2048;
 static constexpr int CS_PROF_FAMILIES = 4;
@@ -145,6 +154,8 @@ struct cs_ctx {
 
   LoopState loop;
   HostStepGraph host_step;
+  VerifyGraph verify_graphs[CS_VERIFY_GRAPHS];
+  int verify_graph_next;
   Prof* prof;   // non-NULL only inside cs_profile_verify_step
 
   char err[256];
@@ -244,6 +255,13 @@ void cs_launch_block_setup(cs_ctx* ctx, const int32_t* last_tok, const int32_t* 
 void cs_launch_prefill_setup(cs_ctx* ctx, const int32_t* hist, const int32_t* hist_len, int B,
                              int stride, int start, int R, cudaStream_t st);
 void cs_launch_embed_rmsnorm(cs_ctx* ctx, const __nv_bfloat16* gain, int rows, cudaStream_t st);
+// cs_verify_step replayed from a graph kept per launch shape (all pointers and B, k equal):
+// for host-ordered loops that call it with a few fixed sets of buffers.  The launch is one
+// stream-ordered unit, so the attention kernel may fetch cached tiles early.
+cs_status cs_verify_step_cached(cs_ctx* ctx, const int32_t* last_tok, const int32_t* draft, const int32_t* draft_len,
+                                int B, int k, void* kv_cache, int32_t* kv_len, const int32_t* target_script,
+                                int32_t* accept_len, int32_t* out_tokens, int32_t* argmax_ids, cudaStream_t st);
+
 void cs_launch_attention(cs_ctx* ctx, const void* kv_cache, int layer, int B, int R,
                          cudaStream_t st);
 void cs_launch_attn_merge(cs_ctx* ctx, int nsplit, int rows, cudaStream_t st);

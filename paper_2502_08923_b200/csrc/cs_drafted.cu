@@ -13,8 +13,10 @@
 //
 // The host reads the match position and the accepted block back every step, so this loop
 // synchronises once or twice per step; the device-resident loop without a draft model is
-// cs_decode_loop.  Scratch: the loop buffers of the two contexts' workspaces (CS_MAX_ROWS
-// ints each), so neither context may have a cs_loop_begin session open.
+// cs_decode_loop.  Every forward is replayed from a graph kept per launch shape (the target's
+// block, the draft model's catch-up block, its single-row steps).  Scratch: the loop buffers
+// of the two contexts' workspaces (CS_MAX_ROWS ints each), so neither context may have a
+// cs_loop_begin session open.
 #include <algorithm>
 #include <cstring>
 #include <vector>
@@ -105,27 +107,34 @@ extern "C" cs_status cs_decode_loop_drafted(cs_ctx* target, cs_ctx* drafter, int
       int32_t* d_accept = drafter->loop_accept;
       int32_t* d_out = drafter->loop_out;
       int32_t* d_argmax = drafter->loop_argmax;
+      // (fixed buffers and a fixed block height of kd + 1 rows, rows past the block's tokens dead,
+      //  so that every block replays the same graph)
+      int32_t* d_last = drafter->loop_last + 1;
       int r = 0;
       while (d_len < n) {
         r = std::min(n - d_len, kd + 1);
         const int dl = r - 1;
-        if (dl > 0) DR_CUDA(cudaMemcpyAsync(d_draft, hist + d_len + 1, (size_t)dl * 4, cudaMemcpyDeviceToDevice, st));
-        // script row: the dl draft tokens, then a value that is never looked at by this loop
-        DR_CUDA(cudaMemsetAsync(d_script, 0xFF, (size_t)r * 4, st));
-        if (dl > 0) DR_CUDA(cudaMemcpyAsync(d_script, hist + d_len + 1, (size_t)dl * 4, cudaMemcpyDeviceToDevice, st));
+        DR_CUDA(cudaMemcpyAsync(d_last, hist + d_len, sizeof(int), cudaMemcpyDeviceToDevice, st));
+        // script row: the dl draft tokens, then values that are never looked at by this loop
+        DR_CUDA(cudaMemsetAsync(d_script, 0xFF, (size_t)(kd + 1) * 4, st));
+        if (dl > 0) {
+          DR_CUDA(cudaMemcpyAsync(d_draft, hist + d_len + 1, (size_t)dl * 4, cudaMemcpyDeviceToDevice, st));
+          DR_CUDA(cudaMemcpyAsync(d_script, hist + d_len + 1, (size_t)dl * 4, cudaMemcpyDeviceToDevice, st));
+        }
         DR_CUDA(cudaMemcpyAsync(d_dlen, &dl, sizeof(int), cudaMemcpyHostToDevice, st));
-        DR_OK(cs_verify_step(drafter, hist + d_len, d_draft, d_dlen, 1, dl, kv_drafter, kv_len_drafter, d_script,
-                             d_accept, d_out, d_argmax, nullptr, st));
+        DR_OK(cs_verify_step_cached(drafter, d_last, d_draft, d_dlen, 1, kd, kv_drafter, kv_len_drafter, d_script,
+                                    d_accept, d_out, d_argmax, st));
         d_len += r;
       }
       DR_CUDA(cudaMemcpyAsync(t_draft, d_argmax + (r - 1), sizeof(int), cudaMemcpyDeviceToDevice, st));
       // the remaining delta - 1 proposals, one single-row greedy step each; the new token is
       // written straight into the target's draft row
+      int32_t* d_zero = drafter->loop_last + 2;
       const int zero = 0;
-      DR_CUDA(cudaMemcpyAsync(d_dlen, &zero, sizeof(int), cudaMemcpyHostToDevice, st));
+      DR_CUDA(cudaMemcpyAsync(d_zero, &zero, sizeof(int), cudaMemcpyHostToDevice, st));
       for (int i = 1; i < delta; ++i) {
-        DR_OK(cs_verify_step(drafter, t_draft + (i - 1), d_draft, d_dlen, 1, 0, kv_drafter, kv_len_drafter, nullptr,
-                             d_accept, t_draft + i, d_argmax, nullptr, st));
+        DR_OK(cs_verify_step_cached(drafter, t_draft + (i - 1), nullptr, d_zero, 1, 0, kv_drafter, kv_len_drafter, nullptr,
+                                    d_accept, t_draft + i, d_argmax, st));
         d_len += 1;
       }
       DR_CUDA(cudaMemcpyAsync(t_dlen, &delta, sizeof(int), cudaMemcpyHostToDevice, st));
@@ -138,8 +147,10 @@ extern "C" cs_status cs_decode_loop_drafted(cs_ctx* target, cs_ctx* drafter, int
       DR_CUDA(cudaMemcpyAsync(t_script, script + emitted, (size_t)have * 4, cudaMemcpyDeviceToDevice, st));
       script_row = t_script;
     }
-    DR_OK(cs_verify_step(target, hist + (n - 1), t_draft, t_dlen, 1, kt, kv_target, kv_len_target, script_row,
-                         t_accept, t_out, t_argmax, nullptr, st));
+    int32_t* t_last = target->loop_last + 1;
+    DR_CUDA(cudaMemcpyAsync(t_last, hist + (n - 1), sizeof(int), cudaMemcpyDeviceToDevice, st));
+    DR_OK(cs_verify_step_cached(target, t_last, t_draft, t_dlen, 1, kt, kv_target, kv_len_target, script_row,
+                                t_accept, t_out, t_argmax, st));
     int tau = -1;
     DR_CUDA(cudaMemcpyAsync(&tau, t_accept, sizeof(int), cudaMemcpyDeviceToHost, st));
     DR_CUDA(cudaMemcpyAsync(out_h.data(), t_out, (size_t)(kt + 1) * 4, cudaMemcpyDeviceToHost, st));
