@@ -130,7 +130,10 @@ def test_a_draft_model_equal_to_the_target_has_every_proposal_accepted():
     tctx.close(); dctx.close()
 
 
-def test_scripted_mode_mixes_copy_steps_and_drafted_steps():
+@pytest.mark.parametrize("no_graph", [False, True])
+def test_scripted_mode_mixes_copy_steps_and_drafted_steps(no_graph, monkeypatch):
+    if no_graph:      # the forwards enqueued kernel by kernel instead of replayed from their graphs
+        monkeypatch.setenv("CS_NO_GRAPH", "1")
     max_new, cap, stride = 120, 384, 320
     tctx, tm = make_pair(TARGET, cap, 1, 10, seed=3)
     dctx, dm = make_pair(SMALL, cap, 1, 3, seed=13)
