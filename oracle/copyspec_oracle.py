@@ -28,9 +28,6 @@ nearest-even bf16 when they are stored in the cache.  Nothing else is rounded: a
 the residual stream, norms, RoPE, softmax and all accumulation are wide (fp64 here; the
 CUDA path carries activations as two bf16 terms, i.e. fp32-equivalent operands, and
 accumulates in fp32).  `contract=False` stores K/V unrounded too: the plain fp64 definition.
-`bf16_operands=True` additionally rounds every contraction's activation operand to a single
-bf16 term; it is kept to show how large that rounding noise would be (about 0.05 in the logits
-per layer at the 8B shape, 0.2 after 32 layers - ten times the logit tolerance).
 
 Pins (tests/test_oracle_*.py): brute-force enumeration of all matches; closed forms
 (constant, increasing and periodic histories); the paper's hash-map dictionary method
@@ -201,11 +198,10 @@ class KVCache:
 class Model:
     """Decoder-only target model evaluated block-wise against a KV cache."""
 
-    def __init__(self, cfg, weights, contract=True, bf16_operands=False, cache_weights=True):
+    def __init__(self, cfg, weights, contract=True, cache_weights=True):
         self.cfg = cfg
         self.w = weights
         self.contract = contract
-        self.bf16_operands = bf16_operands
         self._cache = {} if cache_weights else None
 
     # weights are converted to fp64 on use (and kept, for small models)
@@ -219,15 +215,12 @@ class Model:
             self._cache[key] = a
         return a
 
-    def _opnd(self, x):
-        return round_bf16(x) if self.bf16_operands else x
-
     def _store(self, x):
         return round_bf16(x) if self.contract else x
 
     def _mm(self, x, layer, name):
         """x [R][in] times W[out][in]^T (W holds bf16 values)."""
-        return self._opnd(x) @ self._w(layer, name).T
+        return x @ self._w(layer, name).T
 
     def embed(self, tokens):
         return self._w(None, "embed")[np.asarray(tokens, dtype=np.int64)]
@@ -250,7 +243,7 @@ class Model:
             q = qkv[:, :H * Dh].reshape(R, H, Dh)
             kk = qkv[:, H * Dh:(H + Hkv) * Dh].reshape(R, Hkv, Dh)
             vv = qkv[:, (H + Hkv) * Dh:].reshape(R, Hkv, Dh)
-            q = self._opnd(rope(q, pos, cfg.rope_theta))
+            q = rope(q, pos, cfg.rope_theta)
             kk = self._store(rope(kk, pos, cfg.rope_theta))
             vv = self._store(vv)
             cache.a[l, 0, b, :, pos0:pos0 + R, :] = kk.transpose(1, 0, 2)
@@ -266,7 +259,6 @@ class Model:
                 s = s - s.max(axis=-1, keepdims=True)
                 p = np.exp(s)
                 p = p / p.sum(axis=-1, keepdims=True)
-                p = self._opnd(p)
                 o[:, hd, :] = p @ V
             x = x + self._mm(o.reshape(R, H * Dh), l, "wo")
             xn = rmsnorm(x, self._w(l, "ffn_norm"), cfg.rms_eps)
