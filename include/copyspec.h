@@ -257,6 +257,15 @@ cs_status cs_loop_begin(cs_ctx* ctx, int32_t* hist, int32_t* hist_len, int B, in
 cs_status cs_loop_steps(cs_ctx* ctx, int n_steps, void* stream);
 cs_status cs_loop_poll(cs_ctx* ctx, cs_stats* stats_out, int* n_done_out, void* stream);
 void cs_loop_end(cs_ctx* ctx);
+/* What the most recent step of the loop in progress produced, copied to HOST arrays (any of
+ * them may be NULL): the match position and draft length of the search (App. B.3 step 1), the
+ * accepted length, the tau + 1 emitted tokens and the greedy token of every block row
+ * (App. B.3 step 2; rows past the draft are -1).  match_pos, draft_len, accept_len: [B];
+ * out_tokens, argmax_ids: [B][k+1].  Waits for `stream`.  Entries of a sequence that had
+ * already finished before that step keep the values of its own last step. */
+cs_status cs_loop_last_step(cs_ctx* ctx, int32_t* match_pos_host, int32_t* draft_len_host,
+                            int32_t* accept_len_host, int32_t* out_tokens_host,
+                            int32_t* argmax_ids_host, void* stream);
 /* Kernel launches in one step of the loop in progress (nodes of its graph; 0 if none). */
 int cs_loop_launches_per_step(const cs_ctx* ctx);
 

@@ -50,7 +50,7 @@ class CsStats(C.Structure):
 EXPORTS = ("cs_workspace_bytes", "cs_create", "cs_destroy", "cs_last_error", "cs_sync_status",
            "cs_find_match", "cs_verify_step", "cs_kv_truncate", "cs_decode_loop", "cs_decode_loop_drafted", "cs_step_host",
            "cs_prefill", "cs_linear",
-           "cs_loop_begin", "cs_loop_steps", "cs_loop_poll", "cs_loop_end", "cs_profile_verify_step",
+           "cs_loop_begin", "cs_loop_steps", "cs_loop_poll", "cs_loop_end", "cs_loop_last_step", "cs_profile_verify_step",
            "cs_loop_launches_per_step", "cs_lm_head", "cs_lm_head_static", "cs_gram_index_bytes",
            "cs_gram_index_reset", "cs_gram_index_update", "cs_find_match_indexed", "cs_gram_index_status")
 
@@ -103,6 +103,8 @@ def load(build_if_missing: bool = True) -> C.CDLL:
     lib.cs_loop_poll.argtypes = [vp, C.POINTER(CsStats), C.POINTER(C.c_int), vp]
     lib.cs_loop_launches_per_step.restype = i
     lib.cs_loop_launches_per_step.argtypes = [vp]
+    lib.cs_loop_last_step.restype = i
+    lib.cs_loop_last_step.argtypes = [vp, ip, ip, ip, ip, ip, vp]
     lib.cs_loop_end.restype = None
     lib.cs_loop_end.argtypes = [vp]
     lib.cs_profile_verify_step.restype = i
@@ -385,6 +387,7 @@ class Context:
                       script=None):
         B, stride = hist.shape
         self._loop_refs = (hist, hist_len, kv_cache, kv_len, script)     # keep the buffers alive
+        self._loop_shape = (B, k)
         rc = self.lib.cs_loop_begin(self.handle, _i32(hist, "hist"), _i32(hist_len, "hist_len"), B, stride,
                                     _ptr(kv_cache), _i32(kv_len, "kv_len"), gamma, k, policy, max_new, eos_id,
                                     _i32(script, "script"), _stream())
@@ -398,6 +401,16 @@ class Context:
         st, done = CsStats(), C.c_int(0)
         self._check(self.lib.cs_loop_poll(self.handle, C.byref(st), C.byref(done), _stream()), "cs_loop_poll")
         return st.as_dict(), done.value
+
+    def cs_loop_last_step(self):
+        """The most recent step's (match_pos [B], draft_len [B], accept_len [B], out_tokens [B][k+1],
+        argmax_ids [B][k+1]) as int32 host tensors."""
+        B, k = self._loop_shape
+        mp, dl, al = (torch.empty(B, dtype=torch.int32) for _ in range(3))
+        ot, am = (torch.empty(B, k + 1, dtype=torch.int32) for _ in range(2))
+        rc = self.lib.cs_loop_last_step(self.handle, *(C.c_void_p(t.data_ptr()) for t in (mp, dl, al, ot, am)), _stream())
+        self._check(rc, "cs_loop_last_step")
+        return mp, dl, al, ot, am
 
     def cs_loop_launches_per_step(self):
         return self.lib.cs_loop_launches_per_step(self.handle)

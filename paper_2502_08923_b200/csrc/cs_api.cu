@@ -651,6 +651,22 @@ cs_status cs_loop_poll(cs_ctx* ctx, cs_stats* stats_out, int* n_done_out, void* 
   return cs_sync_status(ctx, stream);
 }
 
+cs_status cs_loop_last_step(cs_ctx* ctx, int32_t* match_pos_host, int32_t* draft_len_host, int32_t* accept_len_host,
+                            int32_t* out_tokens_host, int32_t* argmax_ids_host, void* stream) {
+  if (ctx == nullptr) return CS_ERR_ARG;
+  if (!ctx->loop.active) return fail(ctx, CS_ERR_ARG, "no loop in progress");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t B = (size_t)ctx->loop.B, R = (size_t)ctx->loop.k + 1;
+  const struct { int32_t* dst; const int* src; size_t n; } copies[5] = {
+      {match_pos_host, ctx->loop_mpos, B},        {draft_len_host, ctx->loop_dlen, B},
+      {accept_len_host, ctx->loop_accept, B},     {out_tokens_host, ctx->loop_out, B * R},
+      {argmax_ids_host, ctx->loop_argmax, B * R}};
+  for (const auto& c : copies)
+    if (c.dst != nullptr) CS_CUDA_OK(ctx, cudaMemcpyAsync(c.dst, c.src, c.n * 4, cudaMemcpyDeviceToHost, st));
+  CS_CUDA_OK(ctx, cudaStreamSynchronize(st));
+  return CS_OK;
+}
+
 int cs_loop_launches_per_step(const cs_ctx* ctx) {
   return (ctx != nullptr && ctx->loop.active) ? ctx->loop.graph_nodes : 0;
 }

@@ -43,3 +43,25 @@ def greedy_margins(model, cfg, prompt, generated):
     logits = model.forward_block(seq[:-1], 0, cache, 0)
     n0 = len(prompt)
     return [float(logits[n0 - 1 + j].max() - logits[n0 - 1 + j][tok]) for j, tok in enumerate(generated)]
+
+
+COUNTERS = ("steps", "attempts", "accepted", "emitted", "no_match")
+
+
+def counters_for_streams(hists, streams, gamma, k, policy=O.LATEST):
+    """What the loop's statistics must be, given the token stream each sequence actually
+    emitted: with the targets fixed to those tokens, matches, drafts and accepted lengths are
+    integer functions of history and stream, which the model-free simulator replays.  This
+    checks the loop's bookkeeping on its own output whether or not a near-tie made that output
+    differ from the oracle's (the tokens themselves are pinned by greedy_margins)."""
+    tot = O.new_stats()
+    for hist, gen in zip(hists, streams):
+        if len(gen) == 0:
+            continue
+        _, st, h = O.scripted_simulator(hist, np.asarray(gen, dtype=np.int64), gamma, k, policy, len(gen))
+        assert h == [int(t) for t in hist] + [int(t) for t in gen]
+        for key in COUNTERS:
+            tot[key] += st[key]
+        for i, v in enumerate(st["tau_hist"]):
+            tot["tau_hist"][i] += v
+    return tot

@@ -7,7 +7,7 @@ import torch
 
 from oracle import copyspec_oracle as O
 from paper_2502_08923_b200 import binding as cs, inputs
-from helpers import LOGIT_TOL, greedy_margins, i32, make_pair
+from helpers import LOGIT_TOL, counters_for_streams, greedy_margins, i32, make_pair
 
 pytestmark = pytest.mark.gpu
 
@@ -95,12 +95,20 @@ def test_real_mode_with_a_draft_model(delta):
     assert st["steps"] == st["attempts"] + st["no_match"] and st["draft_attempts"] == st["no_match"] > 0
     assert st["emitted"] == max_new == st["steps"] + st["accepted"] + st["draft_accepted"]
     h_o, got, st_o, d_len, tc, dc, trace = _oracle_run(tm, dm, hist, cap, 3, 10, delta, max_new)
-    if gen != got:
-        pytest.skip("near-tie: the continuation legitimately differs from the oracle's")
-    for key in KEYS:
-        assert st[key] == st_o[key], key
-    assert kvl_d == d_len
-    assert _cache_close(kv_t, tc, n - 1) and _cache_close(kv_d, dc, d_len)
+    # The target's cache is that of the accepted tokens whatever the draft model proposed.
+    t_ref = O.KVCache(TARGET, 1, cap)
+    tm.forward_block([int(t) for t in h[:n - 1]], 0, t_ref, 0)
+    assert _cache_close(kv_t, t_ref, n - 1)
+    # Which steps drafted and how much of each proposal survived depends on the draft model's own
+    # greedy choices, so the step counters are compared where the two runs took the same path: the
+    # streams agree (they do unless a near-tie of the target flipped a token, which the margin
+    # check above bounds) and so does the number of drafted steps.
+    if gen == got and st["draft_attempts"] == st_o["draft_attempts"]:
+        for key in KEYS:
+            assert st[key] == st_o[key], key
+        assert kvl_d == d_len and _cache_close(kv_d, dc, d_len)
+    else:
+        assert gen == got or max(greedy_margins(tm, TARGET, hist, gen)) < LOGIT_TOL
     tctx.close(); dctx.close()
 
 
@@ -170,9 +178,10 @@ def test_delta_zero_needs_no_draft_model_and_eos_stops_the_loop():
     assert gen[-1] == eos and eos not in gen[:-1] and kvl_t == n - 1 and st["draft_attempts"] == 0
     c1 = O.KVCache(TARGET, 1, cap); tm.prefill(hist, c1, 0)
     got, st_o = O.decode_loop(tm, c1, 0, list(hist), 3, 10, O.LATEST, max_new, eos_id=eos)
-    if gen == got:
-        for key in ("steps", "attempts", "accepted", "emitted", "no_match"):
-            assert st[key] == st_o[key], key
+    want = counters_for_streams([hist], [gen], 3, 10)      # the loop's bookkeeping on the stream it emitted
+    for key in ("steps", "attempts", "accepted", "emitted", "no_match"):
+        assert st[key] == want[key], key
+    assert gen != got or all(st[key] == st_o[key] for key in ("steps", "attempts", "accepted", "emitted", "no_match"))
     tctx.close()
 
 

@@ -67,9 +67,12 @@ def test_one_verify_step_logits_against_oracle_at_full_size(big):
     err = float(np.abs(got - lg).max())
     assert err <= LOGIT_TOL, err
     assert not argmax_consistent(lg, am[0].cpu().tolist())
-    # greedy acceptance from those ids
-    tau = O.accept_length(draft, [int(np.argmax(lg[r])) for r in range(K + 1)])
-    assert int(al[0]) == tau or argmax_consistent(lg, am[0].cpu().tolist()) == []
+    # greedy acceptance follows the ids the step reported (they may differ from the oracle's only
+    # inside its margin, checked above; where they agree this is the oracle's accepted length)
+    ids = am[0].cpu().tolist()
+    assert int(al[0]) == O.accept_length(draft, ids)
+    assert ot[0].cpu().tolist() == ids[:int(al[0]) + 1] + [-1] * (K - int(al[0]))
+    assert int(kvl[0]) == n0 - 1 + int(al[0]) + 1
     # the block's K/V rows landed in the cache within bf16 resolution
     new = kv_run[:, :, 0, :, n0 - 1:n0 + K, :].float().cpu().numpy()
     want = cache.a[:, :, 0, :, n0 - 1:n0 + K, :]

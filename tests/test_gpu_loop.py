@@ -6,7 +6,7 @@ import torch
 
 from oracle import copyspec_oracle as O
 from paper_2502_08923_b200 import binding as cs, inputs
-from helpers import LOGIT_TOL, greedy_margins, i32, make_pair
+from helpers import COUNTERS, LOGIT_TOL, counters_for_streams, greedy_margins, i32, make_pair
 
 pytestmark = pytest.mark.gpu
 
@@ -61,11 +61,14 @@ def test_tiny_config_real_mode_is_greedy_decoding():
     gpu_tokens = h[0, 512:n[0]].tolist()
     # every emitted token is the oracle's greedy choice, or within the logit tolerance of it
     assert max(greedy_margins(model, cfg, ctxt, gpu_tokens)) < LOGIT_TOL
-    if gpu_tokens != got_o:
-        pytest.skip("near-tie: the continuation legitimately differs from the oracle's")
     assert n[0] == 512 + max_new and kvl[0] == n[0] - 1
-    for key in ("steps", "attempts", "accepted", "emitted", "no_match"):
-        assert st[key] == st_o[key], key
+    # the statistics are those of a loop whose targets are the emitted tokens (and the oracle
+    # loop's own when the streams agree, which they do unless a near-tie flipped a token)
+    want = counters_for_streams([ctxt], [gpu_tokens], 3, 10)
+    for key in COUNTERS:
+        assert st[key] == want[key], key
+    assert st["tau_hist"][:11] == want["tau_hist"][:11]
+    assert gpu_tokens != got_o or all(st[key] == st_o[key] for key in COUNTERS)
     # plain decoding from the same kernels (k = 0) gives the same tokens
     h0, n0, _, st0 = _run_gpu(ctx, [ctxt], [512], 1024, 3, 0, max_new, cs.LATEST)
     assert h0[0, 512:n0[0]].tolist() == gpu_tokens and st0["steps"] == max_new and st0["accepted"] == 0
@@ -85,23 +88,20 @@ def test_batch_of_sequences_with_eos_and_different_lengths():
     ref0 = O.greedy_decode(model, c0, 0, hists[0].tolist(), max_new)
     eos = ref0[max_new // 2]
     h, n, kvl, st = _run_gpu(ctx, hists, lens, 128, 3, k, max_new, cs.LATEST, eos_id=eos)
-    tot = O.new_stats()
-    same = True
+    gens, stopped = [], 0
     for b in range(B):
-        cache = O.KVCache(cfg, 1, 256); model.prefill(hists[b].tolist(), cache, 0)
-        ho = hists[b].tolist()
-        got, so = O.decode_loop(model, cache, 0, ho, 3, k, O.LATEST, max_new, eos_id=eos)
         gen = h[b, lens[b]:n[b]].tolist()
         assert kvl[b] == n[b] - 1
         assert max(greedy_margins(model, cfg, hists[b], gen)) < LOGIT_TOL, b
         assert len(gen) == max_new or gen[-1] == eos       # stops at max_new or at the first EOS
         assert eos not in gen[:-1]
-        same = same and gen == got
-        for key in ("steps", "attempts", "accepted", "emitted", "no_match"):
-            tot[key] += so[key]
-    if same:     # identical token streams must give identical counters
-        for key in ("steps", "attempts", "accepted", "emitted", "no_match"):
-            assert st[key] == tot[key], key
+        stopped += len(gen) < max_new
+        gens.append(gen)
+    assert stopped >= 1                                    # the EOS rule was exercised
+    want = counters_for_streams(hists, gens, 3, k)        # per sequence, on the stream it emitted
+    for key in COUNTERS:
+        assert st[key] == want[key], key
+    assert st["tau_hist"][:k + 1] == want["tau_hist"][:k + 1]
     assert st["emitted"] == int(sum(n[b] - lens[b] for b in range(B)))
     ctx.close()
 
@@ -175,20 +175,16 @@ def test_real_mode_loop_with_wide_heads_and_caches_of_many_key_tiles():
         hists.append(h)
     h, n, kvl, st = _run_gpu(ctx, hists, lens, 1728, 3, k, max_new, cs.LATEST)
     assert st["attempts"] >= B                 # every sequence opened with a match and a 10-token draft
-    tot = O.new_stats()
-    same = True
+    gens = []
     for b in range(B):
         gen = h[b, lens[b]:n[b]].tolist()
         assert len(gen) == max_new and kvl[b] == n[b] - 1
         assert max(greedy_margins(model, cfg, hists[b], gen)) < LOGIT_TOL, b
-        cache = O.KVCache(cfg, 1, max_seq); model.prefill(hists[b].tolist(), cache, 0)
-        got, so = O.decode_loop(model, cache, 0, hists[b].tolist(), 3, k, O.LATEST, max_new)
-        same = same and gen == got
-        for key in ("steps", "attempts", "accepted", "emitted", "no_match"):
-            tot[key] += so[key]
-    if same:
-        for key in ("steps", "attempts", "accepted", "emitted", "no_match"):
-            assert st[key] == tot[key], key
+        gens.append(gen)
+    want = counters_for_streams(hists, gens, 3, k)
+    for key in COUNTERS:
+        assert st[key] == want[key], key
+    assert st["tau_hist"][:k + 1] == want["tau_hist"][:k + 1]
     ctx.close()
 
 

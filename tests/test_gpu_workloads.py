@@ -2,15 +2,18 @@
 8 and 16, 30k / 8k-token histories) in scripted-target mode: every integer the loop produces
 (match positions through their effect, drafts, accepted lengths, emitted tokens, lengths,
 counters) must equal the oracle's model-free simulator.  The forward runs in full at these
-sizes (block of B*(k+1) rows, attention over the whole cache); its numerics are checked
-elsewhere against the oracle."""
+sizes (block of B*(k+1) rows, attention over the whole cache).  Its numerics are checked here
+on the first step, whose greedy tokens (computed by all 32 layers and the full LM head although
+the script decides acceptance) are compared with the oracle's logits for one of the sequences;
+element-wise logit and K/V parity at these block heights and cache depths is in
+test_gpu_long_shapes.py."""
 import numpy as np
 import pytest
 import torch
 
 from oracle import copyspec_oracle as O
 from paper_2502_08923_b200 import binding as cs, inputs
-from helpers import i32
+from helpers import argmax_consistent, i32
 
 pytestmark = pytest.mark.gpu
 
@@ -37,6 +40,27 @@ def _run(weights8b, cases, k, max_new, policy=cs.LATEST):
     script = np.stack([s[:max_new] for _, s in cases]).astype(np.int32)
     for b, (hh, _) in enumerate(cases):
         h[b, :len(hh)] = hh
+    hd, ld, kvl = i32(h), i32(lens), i32(lens - 1)
+    # ---- first step on its own: the forward's greedy tokens against the oracle (last sequence;
+    # the step only writes cache rows from position len - 1 on, so the context rows are read after it)
+    model = O.Model(cfg, weights8b, contract=True, cache_weights=False)
+    ctx.cs_loop_begin(hd, ld, kv, kvl, 3, k, max_new, policy=policy, script=i32(script))
+    ctx.cs_loop_steps(1)
+    mp, dl, al, ot, am = (t.numpy() for t in ctx.cs_loop_last_step())
+    ctx.cs_loop_end()
+    for b in (B - 1,):
+        hh, n = cases[b][0], int(lens[b])
+        p0 = O.find_match(hh, n, 3, policy)
+        draft = O.gather_draft(hh, n, p0, 3, k)
+        assert int(mp[b]) == p0 and int(dl[b]) == len(draft)
+        cache = O.KVCache(cfg, 1, n + k, dtype=np.float32)
+        for layer in range(cfg.n_layers):
+            cache.a[layer, :, 0, :, :n - 1, :] = kv[layer, :, b, :, :n - 1, :].float().cpu().numpy()
+        lg = model.forward_block([int(hh[-1])] + draft, n - 1, cache, 0)
+        assert not argmax_consistent(lg, am[b, :len(draft) + 1].tolist()), b
+        assert all(am[b, len(draft) + 1:] == -1)
+        del cache
+    # ---- the whole scripted run from the start
     hd, ld, kvl = i32(h), i32(lens), i32(lens - 1)
     st = ctx.cs_decode_loop(hd, ld, kv, kvl, 3, k, max_new, policy=policy, script=i32(script))
     tot = O.new_stats()
