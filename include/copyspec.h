@@ -45,8 +45,20 @@
  * State kept between steps of the loop: hist_len[b] = n counts every accepted token
  * including the last one; kv_len[b] = n - 1.
  *
- * Precision: weights, GEMM activation operands and the KV cache are bf16; accumulation,
- * the residual stream, norms, RoPE and softmax are fp32.
+ * Precision: weights and the KV cache are bf16.  Every activation that enters a tensor-core
+ * product (normed activations, rotated queries, softmax weights, attention output, SwiGLU
+ * output) is carried as TWO bf16 terms, value = hi + lo, and multiplied twice against the same
+ * weight / K / V tile, so activation operands are fp32-equivalent; accumulation, the residual
+ * stream, norms, RoPE and softmax are fp32.  Only K/V rows are rounded (to nearest-even bf16)
+ * when they are stored in the cache.
+ *
+ * Environment, read once by cs_create (measurement and test switches; not needed in use):
+ *   CS_NO_GRAPH=1          steps are enqueued kernel by kernel instead of replayed from a
+ *                          captured CUDA graph (cs_loop_*, cs_step_host, cs_decode_loop_drafted);
+ *   CS_ATTN_KERNEL=tc|mma  forces the tcgen05 or the mma.sync attention kernel (default: by
+ *                          head size);
+ *   CS_WAIT_LIMIT_US=n     time limit of the kernels' bounded waits in microseconds (default
+ *                          2,000,000), see cs_debug_drop_tile.
  */
 #ifndef COPYSPEC_H
 #define COPYSPEC_H
@@ -121,7 +133,8 @@ cs_status cs_create(cs_ctx** out, const cs_model_config* cfg, const cs_weights* 
                     void* workspace, size_t workspace_bytes);
 void cs_destroy(cs_ctx* ctx);
 
-/* Text of the last host-side error of this context (static string if ctx is NULL). */
+/* Text of the last host-side error of this context.  With ctx == NULL: the text of the last
+ * failed cs_create of this thread (cs_create has no context to leave it in), or "". */
 const char* cs_last_error(const cs_ctx* ctx);
 
 /* Waits for `stream`, then returns and clears the device status word of the context:
@@ -166,6 +179,19 @@ cs_status cs_find_match_indexed(const void* index, int B, int capacity_tokens, c
                                 int32_t* draft_len, void* stream);
 cs_status cs_gram_index_status(const void* index, int B, int capacity_tokens, void* stream);
 
+/* Makes the generation loop of this context (cs_decode_loop, cs_loop_*) search through a
+ * gamma-gram index instead of scanning the history (Sec. 3.1; App. B.3 step 1 and step 2(d)):
+ * cs_loop_begin empties the index and builds it from the histories, every step looks the last
+ * gamma tokens up and, after the append, inserts the grams that have become admissible.
+ * Results are those of the scan, bit for bit; the cost no longer grows with the history, which
+ * pays beyond roughly 100k tokens per sequence.  `index` is a caller-allocated DEVICE buffer of
+ * cs_gram_index_bytes(B, capacity_tokens) bytes for the B the loop will run with;
+ * capacity_tokens must be at least the loop's `stride` (CS_ERR_CAPACITY from cs_loop_begin
+ * otherwise).  A table that overflows all the same is reported as CS_ERR_CAPACITY by
+ * cs_loop_poll / cs_decode_loop.  index == NULL goes back to the scan.  Not while a loop is
+ * in progress. */
+cs_status cs_set_match_index(cs_ctx* ctx, void* index, int capacity_tokens);
+
 /* One verification forward plus acceptance (Sec. 3.2; App. B.2; App. B.3 step 2). Async.
  * Evaluates the block [last_tok[b], draft[b][0 .. draft_len[b])] of every sequence at
  * positions kv_len[b].. in one forward, appends the block's K/V rows to the cache,
@@ -207,6 +233,12 @@ cs_status cs_verify_step(cs_ctx* ctx, const int32_t* last_tok, const int32_t* dr
  *   accept_len_host int32 [B], out_tokens_host int32 [B][k+1]: host outputs (tau, then the
  *            tau + 1 emitted tokens; -1 beyond).  A sequence the device skipped for lack of
  *            cache room has accept_len -1, is left as it was, and cs_sync_status reports it.
+ * Only what the device does not have yet crosses the bus: the call remembers how many tokens
+ * of each row it has uploaded to hist_dev, and while the same hist_host / hist_dev pair comes
+ * back with every row exactly as long as the previous call left it, it uploads just the tokens
+ * that call appended.  Anything else (other buffers, B, stride, a length the call did not
+ * produce) uploads the rows in full.  A caller that rewrites tokens below hist_len_host[b] in
+ * place without changing the length must call cs_step_host_reset first.
  * The kernels of the step are replayed as a CUDA graph that the context keeps while B, k, gamma,
  * the policy, the mode and the device buffers stay the same (first call and every change: one
  * capture).  The context's loop buffers serve as scratch: not to be mixed with an open
@@ -215,6 +247,9 @@ cs_status cs_step_host(cs_ctx* ctx, int32_t* hist_host, int32_t* hist_len_host, 
                        int32_t* hist_dev, int32_t* hist_len_dev, void* kv_cache, int32_t* kv_len,
                        int gamma, int k, cs_match_policy policy, const int32_t* script_host,
                        int32_t* accept_len_host, int32_t* out_tokens_host, void* stream);
+
+/* Forget what cs_step_host has uploaded: its next call uploads the histories in full. */
+void cs_step_host_reset(cs_ctx* ctx);
 
 /* KV truncation to an accepted length (App. B.2; App. B.3 step 2(b)).  Async.
  * kv_len[b] = new_len[b] where 0 <= new_len[b] <= kv_len[b]; otherwise kv_len[b] is
@@ -233,9 +268,12 @@ cs_status cs_kv_truncate(cs_ctx* ctx, int32_t* kv_len, const int32_t* new_len, i
  * script[b][emitted_b + r]; the emitted stream then equals the script.  k = 0 gives
  * plain one-token decoding from the same kernels.
  *   stats_out: host pointer or NULL.  stride >= hist_len[b] + max_new and
- *   max_seq >= hist_len[b] + max_new + k are required (checked on the device:
- *   CS_ERR_CAPACITY, that sequence stops).
- * Returns the first error among the host checks, CUDA and the device status word. */
+ *   max_seq >= hist_len[b] + max_new + k are required, and kv_len[b] == hist_len[b] - 1
+ *   (checked on the device: CS_ERR_CAPACITY / CS_ERR_ARG).  A sequence that fails these
+ *   checks is left unmodified and counts as finished; the others run to their end, and the
+ *   call then returns that error.
+ * Returns the first error among the host checks, CUDA and the device status word; a CUDA
+ * error or a bounded wait that ran out ends the loop at once. */
 cs_status cs_decode_loop(cs_ctx* ctx, int32_t* hist, int32_t* hist_len, int B, int stride,
                          void* kv_cache, int32_t* kv_len, int gamma, int k,
                          cs_match_policy policy, int max_new, int eos_id,
@@ -303,17 +341,21 @@ cs_status cs_decode_loop_drafted(cs_ctx* target, cs_ctx* drafter, int32_t* hist,
                                  const int32_t* script, cs_stats* stats_out,
                                  uint64_t* draft_stats_out, void* stream);
 
-/* Measurement aid (no counterpart in the paper): runs cs_verify_step once with a CUDA event
- * pair around every kernel launch and returns, per kernel family, the summed device time
- * in milliseconds and the number of launches.  Families: 0 = projection GEMMs of the
- * layers, 1 = attention, 2 = LM-head GEMM with fused argmax, 3 = element-wise kernels
- * (embedding, norms, RoPE/KV append, SwiGLU).  family_ms and family_launches are host
- * arrays of 4.  Synchronous. */
-cs_status cs_profile_verify_step(cs_ctx* ctx, const int32_t* last_tok, const int32_t* draft,
-                                 const int32_t* draft_len, int B, int k, void* kv_cache,
-                                 int32_t* kv_len, const int32_t* target_script,
-                                 int32_t* accept_len, int32_t* out_tokens, int32_t* argmax_ids,
-                                 float* family_ms, int* family_launches, void* stream);
+/* Measurement aid (no counterpart in the paper): a timeline of the step's kernels taken inside
+ * the running pipeline.  `stamps` is a caller-allocated DEVICE array of `capacity` 64-bit slots
+ * (zero it once); NULL or capacity 0 switches the aid off.  While it is set, stamped launch i
+ * of every step the context enqueues or captures afterwards - the projection GEMMs, the
+ * attention and merge kernels, the LM-head GEMM, embedding + first norm, acceptance, commit -
+ * has each of its CTAs leave the nanosecond time (%globaltimer) at which it finished in
+ * stamps[i], largest wins, so stamps[i] - stamps[i-1] is what kernel i added to the pipelined
+ * step (the search and block set-up are not stamped: they count towards the embedding's
+ * slot).  Set it before cs_loop_begin / the first cs_step_host; it cannot change while a loop
+ * is in progress.  cs_stamp_layout returns the number of slots one step uses and writes the
+ * kernel family of each slot to the HOST array `family` (0 = layer projection GEMM,
+ * 1 = attention, 2 = LM-head GEMM with fused argmax, 3 = merge of the attention's key slices,
+ * 4 = everything else).  Costs one atomic per CTA while set, nothing otherwise. */
+cs_status cs_set_stamps(cs_ctx* ctx, unsigned long long* stamps, int capacity);
+int cs_stamp_layout(const cs_ctx* ctx, int* family, int capacity);
 
 /* Helper off the hot path: computes the KV cache of positions [0, hist_len[b] - 1) by
  * running the forward over the history in blocks with every row forced (no LM head, no
@@ -328,6 +370,14 @@ cs_status cs_prefill(cs_ctx* ctx, const int32_t* hist, const int32_t* hist_len, 
  * ceil(rows/16)*16 rows.  Async. */
 cs_status cs_linear(cs_ctx* ctx, const void* X, const void* W, int rows, int N, int K,
                     float* Y, void* stream);
+
+/* Test hook for the bounded waits (no counterpart in the paper): the next cs_linear / GEMM
+ * launch of this context leaves out the loads of 64-wide K block `k_block` of every CTA, so the
+ * consumer's wait for that block runs out after the context's wait limit (CS_WAIT_LIMIT_US),
+ * the CTA drains its other copies, frees its tensor memory and returns, and cs_sync_status
+ * reports CS_ERR_TIMEOUT.  Nothing faults and the context stays usable.  Meant for
+ * non-clustered launches (a GEMM small enough to run without split-K).  k_block < 0 clears it. */
+cs_status cs_debug_drop_tile(cs_ctx* ctx, int k_block);
 
 /* The LM-head stage of the verification forward on its own (Sec. 3.2; App. B.2: greedy
  * token at temperature 0): ids[r] = the lowest token id with the largest logit of
@@ -350,14 +400,17 @@ cs_status cs_lm_head(cs_ctx* ctx, const void* X, int rows, int32_t* ids, float* 
  * that loads the library holds until the process exits.  It calls no allocating routine.
  *
  *   X bf16 [rows][d_model] (readable for ceil(rows/16)*16 rows), W bf16 [vocab][d_model]
- *   (the LM head, 16-byte aligned), ids int32 [rows]: the lowest token id with the largest
- *   logit of X[r] . W^T.  d_model a multiple of 8.  Async on `stream`.
+ *   (the LM head), both 16-byte aligned; ids int32 [rows]: the lowest token id with the
+ *   largest logit of X[r] . W^T.  d_model a multiple of 8.  Async on `stream`.
  *   Limits: rows <= 64 and vocab <= 131072; anything larger returns CS_ERR_LIMIT and does
- *   nothing.  Other errors: CS_ERR_ARG, CS_ERR_CUDA.  A row whose GEMM gave up on a bounded
- *   wait gets id -2.
+ *   nothing.  Other errors, all found before anything is enqueued: CS_ERR_ARG (NULL, sizes,
+ *   alignment), CS_ERR_CUDA (no device address for the array, or the driver cannot encode
+ *   the operand maps).  A row whose GEMM gave up on a bounded wait gets id -2.
  *
  * The first call on a device looks up the array's device address (and raises the kernel's
- * shared-memory limit); make that first call outside any stream capture.  All calls share
+ * shared-memory limit); make that first call outside any stream capture, and from one thread
+ * (two threads making the first call on the same device at once would both do the set-up).
+ * All calls share
  * the one array, which keeps the previous call's contents (only its status word is cleared
  * per call): two calls that overlap on the GPU - different streams, or threads - race on it
  * and give wrong tokens.  Keep calls on one stream, or order them yourself. */

@@ -15,6 +15,7 @@ CS_OK = 0
 CS_ERR_ARG, CS_ERR_SHAPE, CS_ERR_CAPACITY, CS_ERR_CUDA, CS_ERR_TIMEOUT, CS_ERR_UNSUPPORTED = -1, -2, -3, -4, -5, -6
 CS_ERR_LIMIT = -7
 LATEST, FIRST = 0, 1
+STAMP_FAMILIES = ("gemm", "attention", "lm_head", "merge", "other")
 TAU_HIST = 65
 
 _STATUS = {0: "CS_OK", -1: "CS_ERR_ARG", -2: "CS_ERR_SHAPE", -3: "CS_ERR_CAPACITY", -4: "CS_ERR_CUDA",
@@ -49,8 +50,8 @@ class CsStats(C.Structure):
 
 EXPORTS = ("cs_workspace_bytes", "cs_create", "cs_destroy", "cs_last_error", "cs_sync_status",
            "cs_find_match", "cs_verify_step", "cs_kv_truncate", "cs_decode_loop", "cs_decode_loop_drafted", "cs_step_host",
-           "cs_prefill", "cs_linear",
-           "cs_loop_begin", "cs_loop_steps", "cs_loop_poll", "cs_loop_end", "cs_loop_last_step", "cs_profile_verify_step",
+           "cs_prefill", "cs_linear", "cs_step_host_reset", "cs_debug_drop_tile",
+           "cs_loop_begin", "cs_loop_steps", "cs_loop_poll", "cs_loop_end", "cs_loop_last_step", "cs_set_stamps", "cs_stamp_layout", "cs_set_match_index",
            "cs_loop_launches_per_step", "cs_lm_head", "cs_lm_head_static", "cs_gram_index_bytes",
            "cs_gram_index_reset", "cs_gram_index_update", "cs_find_match_indexed", "cs_gram_index_status")
 
@@ -107,15 +108,22 @@ def load(build_if_missing: bool = True) -> C.CDLL:
     lib.cs_loop_last_step.argtypes = [vp, ip, ip, ip, ip, ip, vp]
     lib.cs_loop_end.restype = None
     lib.cs_loop_end.argtypes = [vp]
-    lib.cs_profile_verify_step.restype = i
-    lib.cs_profile_verify_step.argtypes = [vp, ip, ip, ip, i, i, vp, ip, ip, ip, ip, ip, C.POINTER(C.c_float),
-                                           C.POINTER(C.c_int), vp]
+    lib.cs_set_match_index.restype = i
+    lib.cs_set_match_index.argtypes = [vp, vp, i]
+    lib.cs_set_stamps.restype = i
+    lib.cs_set_stamps.argtypes = [vp, vp, i]
+    lib.cs_stamp_layout.restype = i
+    lib.cs_stamp_layout.argtypes = [vp, C.POINTER(C.c_int), i]
     lib.cs_prefill.restype = i
     lib.cs_prefill.argtypes = [vp, ip, ip, i, i, i, vp, ip, vp]
     lib.cs_lm_head.restype = i
     lib.cs_lm_head.argtypes = [vp, vp, i, ip, vp, vp]
     lib.cs_lm_head_static.restype = i
     lib.cs_lm_head_static.argtypes = [vp, vp, i, i, i, ip, vp]
+    lib.cs_step_host_reset.restype = None
+    lib.cs_step_host_reset.argtypes = [vp]
+    lib.cs_debug_drop_tile.restype = i
+    lib.cs_debug_drop_tile.argtypes = [vp, i]
     lib.cs_linear.restype = i
     lib.cs_linear.argtypes = [vp, vp, vp, i, i, i, vp, vp]
     _lib = lib
@@ -341,6 +349,12 @@ class Context:
                                    _host_i32(out_tokens_host, "out_tokens_host"), _stream())
         self._check(rc, "cs_step_host")
 
+    def cs_step_host_reset(self):
+        self.lib.cs_step_host_reset(self.handle)
+
+    def cs_debug_drop_tile(self, k_block):
+        self._check(self.lib.cs_debug_drop_tile(self.handle, k_block), "cs_debug_drop_tile")
+
     def cs_kv_truncate(self, kv_len, new_len):
         rc = self.lib.cs_kv_truncate(self.handle, _i32(kv_len, "kv_len"), _i32(new_len, "new_len"),
                                      kv_len.shape[0], _stream())
@@ -419,24 +433,27 @@ class Context:
         self.lib.cs_loop_end(self.handle)
         self._loop_refs = None
 
-    def cs_profile_verify_step(self, last_tok, draft, draft_len, kv_cache, kv_len, target_script=None):
-        """cs_verify_step with event brackets; returns ({family: ms}, {family: launches})."""
-        B = last_tok.shape[0]
-        k = draft.shape[1] if draft is not None and draft.dim() == 2 else 0
-        dev = last_tok.device
-        al = torch.empty(B, dtype=torch.int32, device=dev)
-        ot = torch.empty(B, k + 1, dtype=torch.int32, device=dev)
-        am = torch.empty(B, k + 1, dtype=torch.int32, device=dev)
-        ms, n = (C.c_float * 4)(), (C.c_int * 4)()
-        rc = self.lib.cs_profile_verify_step(self.handle, _i32(last_tok, "last_tok"),
-                                             C.c_void_p(draft.data_ptr()) if k > 0 else None,
-                                             _i32(draft_len, "draft_len"), B, k, _ptr(kv_cache),
-                                             _i32(kv_len, "kv_len"), _i32(target_script, "target_script"),
-                                             _i32(al, "accept_len"), _i32(ot, "out_tokens"), _i32(am, "argmax_ids"),
-                                             ms, n, _stream())
-        self._check(rc, "cs_profile_verify_step")
-        names = ("gemm", "attention", "lm_head", "elementwise")
-        return dict(zip(names, list(ms))), dict(zip(names, list(n)))
+    def cs_set_match_index(self, index):
+        """The loop searches through `index` (a GramIndex sized for the loop's batch and stride) or,
+        with None, scans."""
+        self._match_index = index
+        if index is None:
+            rc = self.lib.cs_set_match_index(self.handle, None, 0)
+        else:
+            rc = self.lib.cs_set_match_index(self.handle, index._p(), index.cap)
+        self._check(rc, "cs_set_match_index")
+
+    def cs_set_stamps(self, stamps):
+        """Step timeline on (`stamps`: zeroed int64 CUDA tensor, one slot per stamped launch) or off (None)."""
+        self._stamps = stamps
+        n = 0 if stamps is None else stamps.numel()
+        self._check(self.lib.cs_set_stamps(self.handle, _ptr(stamps), n), "cs_set_stamps")
+
+    def cs_stamp_layout(self):
+        """Kernel family of every slot one step uses (see STAMP_FAMILIES)."""
+        fam = (C.c_int * 4096)()
+        n = self.lib.cs_stamp_layout(self.handle, fam, 4096)
+        return [STAMP_FAMILIES[f] for f in list(fam)[:n]]
 
     def cs_lm_head(self, X, rows=None, logits_dbg=None):
         """Greedy token ids of bf16 rows X[rows][d_model] under the model's LM head."""

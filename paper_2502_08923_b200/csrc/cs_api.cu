@@ -81,6 +81,9 @@ WsLayout ws_layout(const cs_model_config* c) {
   return L;
 }
 
+// cs_create has no context to leave an error text in: the last failure of this thread is kept here
+thread_local char g_create_err[256] = "";
+
 cs_status fail(cs_ctx* ctx, cs_status s, const char* msg) {
   if (ctx) snprintf(ctx->err, sizeof(ctx->err), "%s", msg);
   return s;
@@ -98,21 +101,6 @@ cs_status ensure_act_maps(cs_ctx* ctx, int n_tok) {
   return CS_OK;
 }
 
-void prof_begin(cs_ctx* ctx, int fam, cudaStream_t st) {
-  Prof* p = ctx->prof;
-  if (p == nullptr || p->n >= CS_PROF_MAX) return;
-  cudaEventCreate(&p->ev[2 * p->n]);
-  cudaEventCreate(&p->ev[2 * p->n + 1]);
-  p->fam[p->n] = fam;
-  cudaEventRecord(p->ev[2 * p->n], st);
-}
-void prof_end(cs_ctx* ctx, cudaStream_t st) {
-  Prof* p = ctx->prof;
-  if (p == nullptr || p->n >= CS_PROF_MAX) return;
-  cudaEventRecord(p->ev[2 * p->n + 1], st);
-  p->n += 1;
-}
-
 // The forward of Sec. 3.2 over the rows prepared by a *_setup kernel: B sequences of R
 // rows each.  With `with_lm` the LM head leaves per-tile (max, id) pairs for k_accept.
 cs_status enqueue_forward(cs_ctx* ctx, int B, int R, void* kv_cache, bool with_lm, float* logits,
@@ -128,21 +116,14 @@ cs_status enqueue_forward(cs_ctx* ctx, int B, int R, void* kv_cache, bool with_l
   for (int l = 0; l < c.n_layers; ++l) {
     const LayerPlan& L = ctx->layers[l];
     if (l == 0) {
-      prof_begin(ctx, CS_FAM_ELEMENTWISE, st);
       cs_launch_embed_rmsnorm(ctx, L.attn_norm, rows, st);
-      prof_end(ctx, st);
     }
-    prof_begin(ctx, CS_FAM_GEMM, st);
     const QkvEpi qe = {ctx->rope_cs, ctx->row_pos, ctx->row_write, ctx->qbuf, static_cast<__nv_bfloat16*>(kv_cache),
                        R, l, c.n_heads, c.n_kv_heads, c.head_dim, c.max_batch, c.max_seq};
     s = cs_launch_gemm(ctx, &L.qkv, &ctx->tmXn, CS_MAX_ROWS, rows, CS_EPI_QKV, nullptr, nullptr, nullptr, 0, &qe,
                        &take_norm, st);
-    prof_end(ctx, st);
     if (s != CS_OK) return s;
-    prof_begin(ctx, CS_FAM_ATTENTION, st);
     cs_launch_attention(ctx, kv_cache, l, B, R, st);
-    prof_end(ctx, st);
-    prof_begin(ctx, CS_FAM_GEMM, st);
     NormFuse give = {};
     give.gain_out = L.ffn_norm;
     give.xn_out = ctx->xn;
@@ -150,7 +131,6 @@ cs_status enqueue_forward(cs_ctx* ctx, int B, int R, void* kv_cache, bool with_l
     give.slot_stride = ctx->ssq_stride;
     s = cs_launch_gemm(ctx, &L.o, &ctx->tmAttn, CS_MAX_ROWS, rows, CS_EPI_RESIDUAL, ctx->x, nullptr, nullptr, 0, nullptr,
                        &give, st);
-    prof_end(ctx, st);
     if (s != CS_OK) return s;
     take_norm = NormFuse{};
     take_norm.ssq_in = ctx->ssq;
@@ -162,18 +142,14 @@ cs_status enqueue_forward(cs_ctx* ctx, int B, int R, void* kv_cache, bool with_l
     take_norm.slot_stride = ctx->ssq_stride;
     take_norm.inv_d = 1.f / (float)c.d_model;
     take_norm.eps = c.rms_eps;
-    prof_begin(ctx, CS_FAM_GEMM, st);
     s = cs_launch_gemm(ctx, &L.gate_up, &ctx->tmXn, CS_MAX_ROWS, rows, CS_EPI_SWIGLU, nullptr, ctx->act,
                        ctx->act + (size_t)CS_MAX_ROWS * c.d_ffn, c.d_ffn, nullptr, &take_norm, st);
-    prof_end(ctx, st);
     if (s != CS_OK) return s;
     // the norm after this layer: the next layer's, or the final one before the LM head
     const __nv_bfloat16* next_gain = (l + 1 < c.n_layers) ? ctx->layers[l + 1].attn_norm : (with_lm ? ctx->final_norm : nullptr);
     give.gain_out = next_gain;
-    prof_begin(ctx, CS_FAM_GEMM, st);
     s = cs_launch_gemm(ctx, &L.down, &ctx->tmAct, CS_MAX_ROWS, rows, CS_EPI_RESIDUAL, ctx->x, nullptr, nullptr, 0, nullptr,
                        &give, st);
-    prof_end(ctx, st);
     if (s != CS_OK) return s;
     {
       int sp, kbs;
@@ -182,10 +158,8 @@ cs_status enqueue_forward(cs_ctx* ctx, int B, int R, void* kv_cache, bool with_l
     }
   }
   if (with_lm) {
-    prof_begin(ctx, CS_FAM_LMHEAD, st);
     s = cs_launch_gemm(ctx, &ctx->lm, &ctx->tmXn, CS_MAX_ROWS, rows, CS_EPI_ARGMAX, logits, nullptr, nullptr, 0, nullptr,
                        &take_norm, st);
-    prof_end(ctx, st);
     if (s != CS_OK) return s;
   }
   CS_CUDA_OK(ctx, cudaGetLastError());
@@ -195,8 +169,14 @@ cs_status enqueue_forward(cs_ctx* ctx, int B, int R, void* kv_cache, bool with_l
 // One iteration of the generation loop (App. B.3 steps 1, 2, 4) on device-resident state.
 cs_status enqueue_loop_step(cs_ctx* ctx, cudaStream_t st) {
   const LoopState& L = ctx->loop;
-  cs_status r = cs_launch_find_match(L.hist, L.hist_len, L.B, L.stride, L.gamma, L.k, L.policy, ctx->loop_mpos,
-                                     ctx->loop_draft, ctx->loop_dlen, ctx->loop_last, ctx->loop_done, st);
+  ctx->stamp_n = 0;
+  // App. B.3 step 1: the scan, or the lookup in the gamma-gram index (Sec. 3.1) - same outputs
+  cs_status r = L.use_index
+                    ? cs_launch_gram_lookup(ctx->match_index, L.B, ctx->match_index_cap, L.hist, L.hist_len, L.stride, L.gamma,
+                                            L.k, L.policy, ctx->loop_mpos, ctx->loop_draft, ctx->loop_dlen, ctx->loop_last,
+                                            ctx->loop_done, st)
+                    : cs_launch_find_match(L.hist, L.hist_len, L.B, L.stride, L.gamma, L.k, L.policy, ctx->loop_mpos,
+                                           ctx->loop_draft, ctx->loop_dlen, ctx->loop_last, ctx->loop_done, st);
   if (r != CS_OK) return fail(ctx, r, "match kernel launch failed");
   cs_launch_block_setup(ctx, ctx->loop_last, ctx->loop_draft, ctx->loop_dlen, L.kv_len, ctx->loop_done, L.B, L.k, st);
   // the step opened with a stream-ordered launch and nothing before k_loop_commit changes kv_len
@@ -208,6 +188,12 @@ cs_status enqueue_loop_step(cs_ctx* ctx, cudaStream_t st) {
                    ctx->loop_accept, ctx->loop_out, ctx->loop_argmax, L.kv_len, 0, st);
   cs_launch_loop_commit(ctx, L.hist, L.hist_len, L.B, L.stride, L.kv_len, L.k, L.max_new, L.eos_id,
                         L.script != nullptr, st);
+  if (L.use_index) {
+    // App. B.3 step 2(d): the grams that the appended tokens made admissible enter the index
+    r = cs_launch_gram_update(ctx->match_index, L.B, ctx->match_index_cap, L.hist, L.hist_len, L.stride, L.gamma, 1,
+                              ctx->d_status, st);
+    if (r != CS_OK) return fail(ctx, r, "index update launch failed");
+  }
   CS_CUDA_OK(ctx, cudaGetLastError());
   return CS_OK;
 }
@@ -229,34 +215,43 @@ size_t cs_workspace_bytes(const cs_model_config* cfg) {
   return ws_layout(cfg).total;
 }
 
-const char* cs_last_error(const cs_ctx* ctx) { return ctx ? ctx->err : "no context"; }
+const char* cs_last_error(const cs_ctx* ctx) { return ctx ? ctx->err : g_create_err; }
 
 cs_status cs_create(cs_ctx** out, const cs_model_config* cfg, const cs_weights* w, void* workspace,
                     size_t workspace_bytes) {
-  if (out == nullptr) return CS_ERR_ARG;
+  auto create_fail = [](cs_status st, const char* msg) {
+    snprintf(g_create_err, sizeof(g_create_err), "cs_create: %s", msg);
+    return st;
+  };
+  if (out == nullptr) return create_fail(CS_ERR_ARG, "NULL output pointer");
   *out = nullptr;
-  if (cfg == nullptr || w == nullptr || workspace == nullptr) return CS_ERR_ARG;
-  if (!config_ok(cfg)) return CS_ERR_SHAPE;
+  if (cfg == nullptr || w == nullptr || workspace == nullptr) return create_fail(CS_ERR_ARG, "NULL argument");
+  if (!config_ok(cfg)) return create_fail(CS_ERR_SHAPE, "model configuration outside what the kernels support");
   if (w->embed == nullptr || w->lm_head == nullptr || w->final_norm == nullptr || w->attn_norm == nullptr ||
       w->wqkv == nullptr || w->wo == nullptr || w->ffn_norm == nullptr || w->w_gate_up == nullptr ||
       w->w_down == nullptr)
-    return CS_ERR_ARG;
+    return create_fail(CS_ERR_ARG, "NULL weight pointer");
   const WsLayout L = ws_layout(cfg);
-  if (workspace_bytes < L.total) return CS_ERR_CAPACITY;
-  if (reinterpret_cast<uintptr_t>(workspace) & 1023) return CS_ERR_ARG;
+  if (workspace_bytes < L.total) return create_fail(CS_ERR_CAPACITY, "workspace smaller than cs_workspace_bytes");
+  if (reinterpret_cast<uintptr_t>(workspace) & 1023) return create_fail(CS_ERR_ARG, "workspace not 1024-byte aligned");
 
   cs_ctx* ctx = new (std::nothrow) cs_ctx();
-  if (ctx == nullptr) return CS_ERR_ARG;
+  if (ctx == nullptr) return create_fail(CS_ERR_ARG, "out of host memory");
   memset(static_cast<void*>(ctx), 0, sizeof(*ctx));
   ctx->cfg = *cfg;
   ctx->max_rows = cfg->max_batch * (cfg->k_max + 1);
   ctx->rows_pad = CS_MAX_ROWS;
   ctx->attn_splits = L.attn_splits;
   {
-    const char* kb = getenv("CS_TUNE_SMEM_KB");
-    ctx->tune_smem_kb = (kb != nullptr) ? atoi(kb) : 0;
+    // the environment switches of the library, all read here and nowhere else
     const char* k = getenv("CS_ATTN_KERNEL");
     ctx->attn_force = (k == nullptr) ? 0 : (strcmp(k, "mma") == 0 ? 1 : (strcmp(k, "tc") == 0 ? 2 : 0));
+    const char* ng = getenv("CS_NO_GRAPH");
+    ctx->no_graph = ng != nullptr && ng[0] == '1';
+    const char* wl = getenv("CS_WAIT_LIMIT_US");
+    const long long us = (wl != nullptr) ? atoll(wl) : 0;
+    ctx->wait_limit_ns = (us > 0) ? (unsigned long long)us * 1000ull : 2000000000ull;
+    ctx->debug_drop_kb = -1;
   }
   ctx->qkv_elems = L.qkv_elems;
   ctx->layers = new (std::nothrow) LayerPlan[cfg->n_layers];
@@ -267,16 +262,17 @@ cs_status cs_create(cs_ctx** out, const cs_model_config* cfg, const cs_weights* 
   do {                                                                                         \
     cudaError_t e__ = (call);                                                                  \
     if (e__ != cudaSuccess) {                                                                  \
-      fprintf(stderr, "cs_create: %s: %s\n", #call, cudaGetErrorString(e__));                  \
+      snprintf(g_create_err, sizeof(g_create_err), "cs_create: %s: %s", #call, cudaGetErrorString(e__)); \
       cs_destroy(ctx);                                                                         \
       return CS_ERR_CUDA;                                                                      \
     }                                                                                          \
   } while (0)
-  if (ctx->layers == nullptr) { cs_destroy(ctx); return CS_ERR_ARG; }
+  if (ctx->layers == nullptr) { cs_destroy(ctx); return create_fail(CS_ERR_ARG, "out of host memory"); }
   CREATE_OK(cudaGetDevice(&dev));
   CREATE_OK(cudaGetDeviceProperties(&prop, dev));
   if (prop.major != 10) {
-    fprintf(stderr, "cs_create: this library is built for sm_100a only (device is sm_%d%d)\n", prop.major, prop.minor);
+    snprintf(g_create_err, sizeof(g_create_err), "cs_create: this library is built for sm_100a only (device is sm_%d%d)",
+             prop.major, prop.minor);
     cs_destroy(ctx);
     return CS_ERR_UNSUPPORTED;
   }
@@ -343,7 +339,7 @@ cs_status cs_create(cs_ctx** out, const cs_model_config* cfg, const cs_weights* 
   }
   if (s == CS_OK) s = cs_gemm_plan(ctx, &ctx->lm, w->lm_head, cfg->vocab, d, false);
   if (s != CS_OK) {
-    fprintf(stderr, "cs_create: %s\n", ctx->err);
+    snprintf(g_create_err, sizeof(g_create_err), "cs_create: %.200s", ctx->err[0] ? ctx->err : "NULL layer weight pointer");
     cs_destroy(ctx);
     return s;
   }
@@ -401,6 +397,7 @@ cs_status cs_verify_step(cs_ctx* ctx, const int32_t* last_tok, const int32_t* dr
       kv_len == nullptr || accept_len == nullptr || out_tokens == nullptr || argmax_ids == nullptr)
     return fail(ctx, CS_ERR_ARG, "NULL argument");
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  ctx->stamp_n = 0;
   cs_launch_block_setup(ctx, last_tok, draft, draft_len, kv_len, nullptr, B, k, st);
   cs_status s = enqueue_forward(ctx, B, k + 1, kv_cache, true, logits_dbg, st);
   if (s != CS_OK) return s;
@@ -415,11 +412,10 @@ cs_status cs_verify_step(cs_ctx* ctx, const int32_t* last_tok, const int32_t* dr
 cs_status cs_verify_step_cached(cs_ctx* ctx, const int32_t* last_tok, const int32_t* draft, const int32_t* draft_len,
                                 int B, int k, void* kv_cache, int32_t* kv_len, const int32_t* target_script,
                                 int32_t* accept_len, int32_t* out_tokens, int32_t* argmax_ids, cudaStream_t st) {
-  const char* env = getenv("CS_NO_GRAPH");
-  if (env != nullptr && env[0] == '1')
+  if (ctx == nullptr) return CS_ERR_ARG;
+  if (ctx->no_graph)
     return cs_verify_step(ctx, last_tok, draft, draft_len, B, k, kv_cache, kv_len, target_script, accept_len,
                           out_tokens, argmax_ids, nullptr, st);
-  if (ctx == nullptr) return CS_ERR_ARG;
   if (B < 1 || B > ctx->cfg.max_batch || k < 0 || k > ctx->cfg.k_max) return fail(ctx, CS_ERR_ARG, "B or k out of range");
   if (last_tok == nullptr || draft_len == nullptr || (draft == nullptr && k > 0) || kv_cache == nullptr ||
       kv_len == nullptr || accept_len == nullptr || out_tokens == nullptr || argmax_ids == nullptr)
@@ -439,6 +435,7 @@ cs_status cs_verify_step_cached(cs_ctx* ctx, const int32_t* last_tok, const int3
     cs_status s = ensure_act_maps(ctx, cs_ceil_div(B * (k + 1), 16) * 16);   // host work that must precede capture
     if (s != CS_OK) return s;
     CS_CUDA_OK(ctx, cudaStreamBeginCapture(ctx->cap_stream, cudaStreamCaptureModeRelaxed));
+    ctx->stamp_n = 0;
     cs_launch_block_setup(ctx, last_tok, draft, draft_len, kv_len, nullptr, B, k, ctx->cap_stream);
     ctx->kv_len_early = kv_len;      // nothing before the acceptance kernel changes it
     s = enqueue_forward(ctx, B, k + 1, kv_cache, true, nullptr, ctx->cap_stream);
@@ -469,8 +466,9 @@ cs_status cs_step_host(cs_ctx* ctx, int32_t* hist_host, int32_t* hist_len_host, 
                        cs_match_policy policy, const int32_t* script_host, int32_t* accept_len_host,
                        int32_t* out_tokens_host, void* stream) {
   if (ctx == nullptr) return CS_ERR_ARG;
-  if (B < 1 || B > ctx->cfg.max_batch || k < 0 || k > ctx->cfg.k_max || gamma < 1 || stride < 1)
+  if (B < 1 || B > ctx->cfg.max_batch || k < 0 || k > ctx->cfg.k_max || gamma < 1 || gamma > CS_MAX_GAMMA || stride < 1)
     return fail(ctx, CS_ERR_ARG, "B, k, gamma or stride out of range");
+  if (policy != CS_MATCH_LATEST && policy != CS_MATCH_FIRST) return fail(ctx, CS_ERR_ARG, "bad policy");
   if (hist_host == nullptr || hist_len_host == nullptr || hist_dev == nullptr || hist_len_dev == nullptr ||
       kv_cache == nullptr || kv_len == nullptr || accept_len_host == nullptr || out_tokens_host == nullptr)
     return fail(ctx, CS_ERR_ARG, "NULL argument");
@@ -478,10 +476,20 @@ cs_status cs_step_host(cs_ctx* ctx, int32_t* hist_host, int32_t* hist_len_host, 
     if (hist_len_host[b] < 1 || hist_len_host[b] + k + 1 > stride)
       return fail(ctx, CS_ERR_CAPACITY, "history row too short for one more block");
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  // ---- host -> device: the accepted tokens of every sequence, the lengths, this step's script rows
-  for (int b = 0; b < B; ++b)
-    CS_CUDA_OK(ctx, cudaMemcpyAsync(hist_dev + (size_t)b * stride, hist_host + (size_t)b * stride,
-                                    (size_t)hist_len_host[b] * 4, cudaMemcpyHostToDevice, st));
+  // ---- host -> device: the tokens the device copy of each history lacks (everything on the first
+  // call with these buffers, afterwards what the previous call appended), the lengths, this step's
+  // script rows
+  HostStepGraph& G = ctx->host_step;
+  const bool known = G.up_host == hist_host && G.up_dev == hist_dev && G.up_B == B && G.up_stride == stride;
+  for (int b = 0; b < B; ++b) {
+    const int n = hist_len_host[b];
+    const int have = (known && G.host_len[b] == n && G.uploaded[b] <= n) ? G.uploaded[b] : 0;
+    if (n > have)
+      CS_CUDA_OK(ctx, cudaMemcpyAsync(hist_dev + (size_t)b * stride + have, hist_host + (size_t)b * stride + have,
+                                      (size_t)(n - have) * 4, cudaMemcpyHostToDevice, st));
+    G.uploaded[b] = n;
+  }
+  G.up_host = hist_host; G.up_dev = hist_dev; G.up_B = B; G.up_stride = stride;
   CS_CUDA_OK(ctx, cudaMemcpyAsync(hist_len_dev, hist_len_host, (size_t)B * 4, cudaMemcpyHostToDevice, st));
   const int32_t* script_dev = nullptr;
   if (script_host != nullptr) {
@@ -491,13 +499,12 @@ cs_status cs_step_host(cs_ctx* ctx, int32_t* hist_host, int32_t* hist_len_host, 
   // ---- App. B.3 step 1 (search, gather), step 2 (verify, accept, truncate): the kernels of one
   // step, replayed as a graph while the launch shape and the buffers stay the same
   // (CS_NO_GRAPH=1 enqueues them one by one)
-  HostStepGraph& G = ctx->host_step;
-  const char* env = getenv("CS_NO_GRAPH");
-  const bool use_graph = !(env != nullptr && env[0] == '1');
+  const bool use_graph = !ctx->no_graph;
   const bool same = G.exec != nullptr && G.hist_dev == hist_dev && G.hist_len_dev == hist_len_dev &&
                     G.kv_cache == kv_cache && G.kv_len == kv_len && G.B == B && G.stride == stride &&
                     G.gamma == gamma && G.k == k && G.policy == (int)policy && G.scripted == (script_dev != nullptr);
   auto enqueue = [&](cudaStream_t q) -> cs_status {
+    ctx->stamp_n = 0;
     cs_status r = cs_launch_find_match(hist_dev, hist_len_dev, B, stride, gamma, k, (int)policy, ctx->loop_mpos,
                                        ctx->loop_draft, ctx->loop_dlen, ctx->loop_last, nullptr, q);
     if (r != CS_OK) return fail(ctx, r, "match kernel launch failed");
@@ -520,7 +527,7 @@ cs_status cs_step_host(cs_ctx* ctx, int32_t* hist_host, int32_t* hist_len_host, 
     if (!same) {
       if (G.exec) cudaGraphExecDestroy(G.exec);
       if (G.graph) cudaGraphDestroy(G.graph);
-      G = HostStepGraph{};
+      G.exec = nullptr; G.graph = nullptr;
       s = ensure_act_maps(ctx, cs_ceil_div(B * (k + 1), 16) * 16);   // host work that must precede capture
       if (s != CS_OK) return s;
       CS_CUDA_OK(ctx, cudaStreamBeginCapture(ctx->cap_stream, cudaStreamCaptureModeRelaxed));
@@ -529,7 +536,7 @@ cs_status cs_step_host(cs_ctx* ctx, int32_t* hist_host, int32_t* hist_len_host, 
       if (s == CS_OK && e == cudaSuccess) e = cudaGraphInstantiate(&G.exec, G.graph, 0);
       if (s != CS_OK || e != cudaSuccess) {
         if (G.graph) cudaGraphDestroy(G.graph);
-        G = HostStepGraph{};
+        G.exec = nullptr; G.graph = nullptr;
         if (s != CS_OK) return s;
         CS_CUDA_OK(ctx, e);
       }
@@ -549,6 +556,17 @@ cs_status cs_step_host(cs_ctx* ctx, int32_t* hist_host, int32_t* hist_len_host, 
     for (int i = 0; i <= tau; ++i) hist_host[(size_t)b * stride + n + i] = out_tokens_host[(size_t)b * (k + 1) + i];
     hist_len_host[b] = n + tau + 1;
   }
+  for (int b = 0; b < B; ++b) G.host_len[b] = hist_len_host[b];
+  return CS_OK;
+}
+
+void cs_step_host_reset(cs_ctx* ctx) {
+  if (ctx != nullptr) ctx->host_step.up_host = nullptr;
+}
+
+cs_status cs_debug_drop_tile(cs_ctx* ctx, int k_block) {
+  if (ctx == nullptr) return CS_ERR_ARG;
+  ctx->debug_drop_kb = k_block < 0 ? -1 : k_block;
   return CS_OK;
 }
 
@@ -573,6 +591,7 @@ cs_status cs_prefill(cs_ctx* ctx, const int32_t* hist, const int32_t* hist_len, 
   const int total = max_len - 1;   // positions whose K/V are cached
   for (int start = 0; start < total; start += R) {
     const int r = (total - start < R) ? total - start : R;
+    ctx->stamp_n = 0;
     cs_launch_prefill_setup(ctx, hist, hist_len, B, stride, start, r, st);
     cs_status s = enqueue_forward(ctx, B, r, kv_cache, false, nullptr, st);
     if (s != CS_OK) return s;
@@ -598,8 +617,15 @@ cs_status cs_loop_begin(cs_ctx* ctx, int32_t* hist, int32_t* hist_len, int B, in
   LoopState& L = ctx->loop;
   L.hist = hist; L.hist_len = hist_len; L.B = B; L.stride = stride; L.kv_cache = kv_cache; L.kv_len = kv_len;
   L.gamma = gamma; L.k = k; L.policy = (int)policy; L.max_new = max_new; L.eos_id = eos_id; L.script = script;
-  const char* env = getenv("CS_NO_GRAPH");
-  L.use_graph = !(env != nullptr && env[0] == '1');
+  L.use_graph = !ctx->no_graph;
+  L.use_index = ctx->match_index != nullptr;
+  if (L.use_index) {
+    if (ctx->match_index_cap < stride) return fail(ctx, CS_ERR_CAPACITY, "the gamma-gram index is sized for fewer tokens than a history row holds");
+    // built afresh from the histories as they stand
+    cs_status r = cs_gram_index_reset(ctx->match_index, B, ctx->match_index_cap, st);
+    if (r == CS_OK) r = cs_launch_gram_update(ctx->match_index, B, ctx->match_index_cap, hist, hist_len, stride, gamma, 64, ctx->d_status, st);
+    if (r != CS_OK) return fail(ctx, r, "index build failed");
+  }
 
   cs_launch_loop_init(ctx, hist_len, kv_len, B, stride, max_new, k, st);
   CS_CUDA_OK(ctx, cudaGetLastError());
@@ -687,46 +713,64 @@ cs_status cs_decode_loop(cs_ctx* ctx, int32_t* hist, int32_t* hist_len, int B, i
                               script, stream);
   if (s != CS_OK) return s;
   // every live sequence emits at least one token per step, so max_new steps always suffice
+  // A status that concerns single sequences (no room, inconsistent lengths: those sequences
+  // were marked finished and left alone) is remembered while the others run on; a CUDA error or
+  // a wait that ran out ends the loop.
   const int poll = 4;
   int steps = 0, done = 0;
-  while (s == CS_OK) {
+  cs_status first = CS_OK;
+  char first_msg[sizeof(ctx->err)] = "";
+  while (true) {
     const int nrun = (max_new - steps < poll) ? max_new - steps : poll;
     if (nrun > 0) s = cs_loop_steps(ctx, nrun, stream);
     steps += nrun;
     if (s != CS_OK) break;
     s = cs_loop_poll(ctx, stats_out, &done, stream);
-    if (done >= B || steps >= max_new) break;
+    if (s == CS_ERR_CAPACITY || s == CS_ERR_ARG) {
+      if (first == CS_OK) { first = s; snprintf(first_msg, sizeof(first_msg), "%s", ctx->err); }
+      s = CS_OK;
+    }
+    if (s != CS_OK || done >= B || steps >= max_new) break;
   }
   cs_loop_end(ctx);
+  if (s == CS_OK && first != CS_OK) {
+    snprintf(ctx->err, sizeof(ctx->err), "%s", first_msg);
+    s = first;
+  }
   return s;
 }
 
-cs_status cs_profile_verify_step(cs_ctx* ctx, const int32_t* last_tok, const int32_t* draft,
-                                 const int32_t* draft_len, int B, int k, void* kv_cache, int32_t* kv_len,
-                                 const int32_t* target_script, int32_t* accept_len, int32_t* out_tokens,
-                                 int32_t* argmax_ids, float* family_ms, int* family_launches, void* stream) {
-  if (ctx == nullptr || family_ms == nullptr || family_launches == nullptr) return CS_ERR_ARG;
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
-  Prof prof;
-  memset(&prof, 0, sizeof(prof));
-  ctx->prof = &prof;
-  cs_status s = cs_verify_step(ctx, last_tok, draft, draft_len, B, k, kv_cache, kv_len, target_script, accept_len,
-                               out_tokens, argmax_ids, nullptr, stream);
-  ctx->prof = nullptr;
-  cudaError_t e = cudaStreamSynchronize(st);
-  for (int f = 0; f < CS_PROF_FAMILIES; ++f) { family_ms[f] = 0.f; family_launches[f] = 0; }
-  for (int i = 0; i < prof.n; ++i) {
-    float ms = 0.f;
-    if (e == cudaSuccess && s == CS_OK && cudaEventElapsedTime(&ms, prof.ev[2 * i], prof.ev[2 * i + 1]) == cudaSuccess) {
-      family_ms[prof.fam[i]] += ms;
-      family_launches[prof.fam[i]] += 1;
-    }
-    cudaEventDestroy(prof.ev[2 * i]);
-    cudaEventDestroy(prof.ev[2 * i + 1]);
-  }
-  if (s != CS_OK) return s;
-  CS_CUDA_OK(ctx, e);
+cs_status cs_set_match_index(cs_ctx* ctx, void* index, int capacity_tokens) {
+  if (ctx == nullptr || (index != nullptr && capacity_tokens < 1)) return CS_ERR_ARG;
+  if (ctx->loop.active) return fail(ctx, CS_ERR_ARG, "the search method cannot change while a loop is in progress");
+  ctx->match_index = index;
+  ctx->match_index_cap = index != nullptr ? capacity_tokens : 0;
   return CS_OK;
+}
+
+cs_status cs_set_stamps(cs_ctx* ctx, unsigned long long* stamps, int capacity) {
+  if (ctx == nullptr || capacity < 0) return CS_ERR_ARG;
+  if (ctx->loop.active) return fail(ctx, CS_ERR_ARG, "stamps cannot change while a loop is in progress (its graph holds the slots)");
+  ctx->stamp_buf = (capacity > 0) ? stamps : nullptr;
+  ctx->stamp_cap = (stamps != nullptr) ? capacity : 0;
+  ctx->stamp_n = 0;
+  // graphs captured earlier hold the old slots
+  for (int i = 0; i < CS_VERIFY_GRAPHS; ++i) {
+    if (ctx->verify_graphs[i].exec) cudaGraphExecDestroy(ctx->verify_graphs[i].exec);
+    if (ctx->verify_graphs[i].graph) cudaGraphDestroy(ctx->verify_graphs[i].graph);
+    ctx->verify_graphs[i] = VerifyGraph{};
+  }
+  if (ctx->host_step.exec) cudaGraphExecDestroy(ctx->host_step.exec);
+  if (ctx->host_step.graph) cudaGraphDestroy(ctx->host_step.graph);
+  ctx->host_step.exec = nullptr;
+  ctx->host_step.graph = nullptr;
+  return CS_OK;
+}
+
+int cs_stamp_layout(const cs_ctx* ctx, int* family, int capacity) {
+  if (ctx == nullptr) return 0;
+  for (int i = 0; i < ctx->stamp_n && i < capacity && family != nullptr; ++i) family[i] = ctx->stamp_fam[i];
+  return ctx->stamp_n;
 }
 
 cs_status cs_linear(cs_ctx* ctx, const void* X, const void* W, int rows, int N, int K, float* Y, void* stream) {

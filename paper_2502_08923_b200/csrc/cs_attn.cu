@@ -57,7 +57,8 @@ template <int DH>
 __global__ void __launch_bounds__(kThreads)
 k_attn_mma(const __nv_bfloat16* __restrict__ qbuf, const __nv_bfloat16* __restrict__ kv,
            const int* __restrict__ row_lim, int layer, int R, int H, int Hkv, int max_batch, int max_seq,
-           int nsplit, float scale_log2e, float* __restrict__ out_o, float* __restrict__ out_ml, int rows) {
+           int nsplit, float scale_log2e, float* __restrict__ out_o, float* __restrict__ out_ml, int rows,
+           unsigned long long* stamp) {
   CS_PDL_PROLOGUE();
   constexpr int STRIDE = DH + 8;          // bf16 elements per shared-memory row
   constexpr int KSTEPS = DH / 16;         // MMA k-steps of the QK^T product
@@ -245,6 +246,10 @@ k_attn_mma(const __nv_bfloat16* __restrict__ qbuf, const __nv_bfloat16* __restri
       *reinterpret_cast<float2*>(out_o + base * DH + nd * 8 + 2 * t) = make_float2(o[nd][2], o[nd][3]);
     if (t == 0) { out_ml[base * 2] = m_hi * kLn2; out_ml[base * 2 + 1] = l_hi; }
   }
+  if (stamp != nullptr) {
+    __syncthreads();
+    if (threadIdx.x == 0) cs_stamp_end(stamp);
+  }
 }
 
 template <int DH>
@@ -264,7 +269,8 @@ int launch(cs_ctx* ctx, const void* kv_cache, int layer, int B, int R, cudaStrea
   const float scale_log2e = 1.4426950408889634f / sqrtf((float)DH);
   cs_launch_pdl(k_attn_mma<DH>, dim3(B * c.n_kv_heads, nsplit, rgs), dim3(kThreads), smem, st, ctx->qbuf,
                 static_cast<const __nv_bfloat16*>(kv_cache), ctx->row_lim, layer, R, c.n_heads, c.n_kv_heads,
-                c.max_batch, c.max_seq, nsplit, scale_log2e, ctx->attn_o, ctx->attn_ml, B * R);
+                c.max_batch, c.max_seq, nsplit, scale_log2e, ctx->attn_o, ctx->attn_ml, B * R,
+                cs_next_stamp(ctx, CS_FAM_ATTENTION));
   return nsplit;
 }
 

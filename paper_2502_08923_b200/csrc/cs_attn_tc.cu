@@ -21,7 +21,7 @@
 // tile's K lands during the softmax and its V during the next score product.  When the caller
 // vouches for the cached lengths (kv_len_early), a slice whose first tile lies wholly below
 // the cached length requests that tile before it waits for the preceding kernel: those rows
-// were written by earlier steps.  Every wait is bounded (2 s): on expiry the CTA flags
+// were written by earlier steps.  Every wait is bounded (2 s by default): on expiry the CTA flags
 // CS_DEV_TIMEOUT, drains its copies, frees its TMEM and returns.
 #include <stdlib.h>
 
@@ -36,7 +36,6 @@ constexpr int kTileKeys = 128;
 constexpr int kDh = 128;
 constexpr int kHalfBytes = kTileKeys * 128;          // one [128 keys x 64 dims] half tile
 constexpr int kNQMax = 128;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 struct AttnArgs {
   const int* row_lim;
@@ -47,6 +46,8 @@ struct AttnArgs {
   float* out_o;
   float* out_ml;
   int* status;
+  unsigned long long wait_ns;   // limit of every bounded wait
+  unsigned long long* stamp;    // step timeline slot of this launch, or NULL
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -71,7 +72,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                       unsigned long long limit_ns) {
   unsigned long long t0 = 0;
   for (uint32_t it = 0;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
@@ -79,7 +81,7 @@ __device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile i
       if (*abort_flag) return false;
       const unsigned long long now = globaltimer_ns();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > kWaitLimitNs) return false;
+      else if (now - t0 > limit_ns) return false;
     }
   }
 }
@@ -303,12 +305,12 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
         const uint32_t ph = (uint32_t)(i / stages) & 1u;
         const int key0 = (split + i * a.nsplit) * kTileKeys;
         const uint32_t dk = smem_u32(sK + (size_t)s * 2 * kHalfBytes), dv = smem_u32(sV + (size_t)s * 2 * kHalfBytes);
-        if (!mbar_wait(b_kfree + 8 * s, ph ^ 1u, s_abort)) { ok = false; break; }
+        if (!mbar_wait(b_kfree + 8 * s, ph ^ 1u, s_abort, a.wait_ns)) { ok = false; break; }
         mbar_expect_tx(b_kfull + 8 * s, 2u * kHalfBytes);
         tma_load_2d(dk, &tmKV, b_kfull + 8 * s, 0, (int)(krow + key0));
         tma_load_2d(dk + kHalfBytes, &tmKV, b_kfull + 8 * s, 64, (int)(krow + key0));
         ik = i + 1;
-        if (!mbar_wait(b_vfree + 8 * s, ph ^ 1u, s_abort)) { ok = false; break; }
+        if (!mbar_wait(b_vfree + 8 * s, ph ^ 1u, s_abort, a.wait_ns)) { ok = false; break; }
         mbar_expect_tx(b_vfull + 8 * s, 2u * kHalfBytes);
         tma_load_2d(dv, &tmKV, b_vfull + 8 * s, 0, (int)(vrow + key0));
         tma_load_2d(dv + kHalfBytes, &tmKV, b_vfull + 8 * s, 64, (int)(vrow + key0));
@@ -316,9 +318,9 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
       }
       if (!ok) { *s_abort = 1; atomicOr(a.status, CS_DEV_TIMEOUT); }
       if (*s_abort || ntl == 0) {   // let the copies land before the shared memory goes away
-        mbar_wait(b_qfull, 0, s_never);
-        for (int j = max(0, ik - stages); j < ik; ++j) mbar_wait(b_kfull + 8 * (j % stages), (uint32_t)(j / stages) & 1u, s_never);
-        for (int j = max(0, iv - stages); j < iv; ++j) mbar_wait(b_vfull + 8 * (j % stages), (uint32_t)(j / stages) & 1u, s_never);
+        mbar_wait(b_qfull, 0, s_never, a.wait_ns);
+        for (int j = max(0, ik - stages); j < ik; ++j) mbar_wait(b_kfull + 8 * (j % stages), (uint32_t)(j / stages) & 1u, s_never, a.wait_ns);
+        for (int j = max(0, iv - stages); j < iv; ++j) mbar_wait(b_vfull + 8 * (j % stages), (uint32_t)(j / stages) & 1u, s_never, a.wait_ns);
       }
     }
   } else if (warp == kMmaWarp) {
@@ -330,7 +332,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
       // S of tile i: issued behind the P V product of tile i - 1, so one commit covers both
       auto issue_scores = [&](int i) -> bool {
         const int s = i % stages;
-        if (!mbar_wait(b_kfull + 8 * s, (uint32_t)(i / stages) & 1u, s_abort)) return false;
+        if (!mbar_wait(b_kfull + 8 * s, (uint32_t)(i / stages) & 1u, s_abort, a.wait_ns)) return false;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t ak = smem_u32(sK + (size_t)s * 2 * kHalfBytes);
 #pragma unroll
@@ -345,11 +347,11 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
         umma_commit(b_sready);
         return true;
       };
-      bool ok = mbar_wait(b_qfull, 0, s_abort) && issue_scores(0);
+      bool ok = mbar_wait(b_qfull, 0, s_abort, a.wait_ns) && issue_scores(0);
       for (int i = 0; i < ntl && ok; ++i) {
         const int s = i % stages;
         const uint32_t ph = (uint32_t)(i / stages) & 1u;
-        if (!mbar_wait(b_pready, (uint32_t)i & 1u, s_abort) || !mbar_wait(b_vfull + 8 * s, ph, s_abort)) { ok = false; break; }
+        if (!mbar_wait(b_pready, (uint32_t)i & 1u, s_abort, a.wait_ns) || !mbar_wait(b_vfull + 8 * s, ph, s_abort, a.wait_ns)) { ok = false; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t av = smem_u32(sV + (size_t)s * 2 * kHalfBytes);
 #pragma unroll
@@ -382,7 +384,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
       float* slot = s_xch + (size_t)(xuse & 1u) * 2 * NQ;
       if (valid) slot[half * NQ + q] = mine;
       mbar_arrive(pairbar);
-      const bool ok = mbar_wait(pairbar, xuse & 1u, s_abort);
+      const bool ok = mbar_wait(pairbar, xuse & 1u, s_abort, a.wait_ns);
       theirs = (ok && valid) ? slot[(half ^ 1) * NQ + q] : mine;
       ++xuse;
       return ok;
@@ -393,7 +395,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
       const int key0 = (split + i * a.nsplit) * kTileKeys + (int)col0;   // first key of this thread's half tile
       // (S of this tile complete also means the previous tile's P V product has retired:
       //  P may be overwritten and O is up to date)
-      bool ok = mbar_wait(b_sready, (uint32_t)i & 1u, s_abort);
+      bool ok = mbar_wait(b_sready, (uint32_t)i & 1u, s_abort, a.wait_ns);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) { *s_abort = 1; have = false; break; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -456,7 +458,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
       // keys past the longest row of this sequence hold whatever the cache held: zero their V rows
       const int tile0 = key0 - (int)col0;
       if (tile0 + kTileKeys > lmax) {
-        if (!mbar_wait(b_vfull + 8 * s, ph, s_abort)) *s_abort = 1;
+        if (!mbar_wait(b_vfull + 8 * s, ph, s_abort, a.wait_ns)) *s_abort = 1;
         uint8_t* vs = sV + (size_t)s * 2 * kHalfBytes;
         for (int rr = max(lmax - tile0, 0) + half * nact * 32 + q; rr < kTileKeys; rr += nact * 64) {
 #pragma unroll
@@ -472,7 +474,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
     }
     // ---- un-normalised result of this key slice
     if (have) {
-      bool ok = mbar_wait(b_odone, (uint32_t)(ntl - 1) & 1u, s_abort);
+      bool ok = mbar_wait(b_odone, (uint32_t)(ntl - 1) & 1u, s_abort, a.wait_ns);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) { *s_abort = 1; have = false; }
     }
@@ -510,8 +512,9 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
   // ---------------------------------------------------------------------- teardown
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
+  if (tid == 0) cs_stamp_end(a.stamp);
   if (warp == kMmaWarp) {
-    if (*s_abort && lane == 0 && ntl > 0) mbar_wait(b_odone, (uint32_t)(ntl - 1) & 1u, s_never);   // MMAs retired (bounded)
+    if (*s_abort && lane == 0 && ntl > 0) mbar_wait(b_odone, (uint32_t)(ntl - 1) & 1u, s_never, a.wait_ns);   // MMAs retired (bounded)
     __syncwarp();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
@@ -573,6 +576,8 @@ int cs_launch_attention_tc(cs_ctx* ctx, const void* kv_cache, int layer, int B, 
   a.smem_bytes = (int)smem;
   a.scale_log2e = 1.4426950408889634f / sqrtf((float)kDh);
   a.out_o = ctx->attn_o; a.out_ml = ctx->attn_ml; a.status = ctx->d_status;
+  a.wait_ns = ctx->wait_limit_ns;
+  a.stamp = cs_next_stamp(ctx, CS_FAM_ATTENTION);
   if (cs_launch_pdl(k_attn_tc, dim3(B * c.n_kv_heads, nsplit, ngroups), dim3(kThreads), smem, st, ctx->tmKV, ctx->tmQ, a) != cudaSuccess) {
     snprintf(ctx->err, sizeof(ctx->err), "attention launch failed");
     return -1;

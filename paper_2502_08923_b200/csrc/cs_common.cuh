@@ -44,6 +44,7 @@ struct LayerPlan {
 // device-resident generation loop between cs_loop_begin and cs_loop_end
 struct LoopState {
   bool active, use_graph;
+  bool use_index;    // the search is the gamma-gram index's lookup instead of the scan
   int32_t *hist, *hist_len, *kv_len;
   const int32_t* script;
   void* kv_cache;
@@ -60,6 +61,11 @@ struct HostStepGraph {
   int B, stride, gamma, k, policy, scripted;
   cudaGraph_t graph;
   cudaGraphExec_t exec;
+  // what the device copy of the histories holds: rows [0, uploaded[b]) of up_host -> up_dev
+  const void *up_host, *up_dev;
+  int up_B, up_stride;
+  int uploaded[CS_MAX_ROWS];    // tokens of row b on the device
+  int host_len[CS_MAX_ROWS];    // hist_len_host[b] as the previous call left it
 };
 
 // cs_verify_step_cached keeps the graphs of its last few launch shapes
@@ -71,15 +77,12 @@ struct VerifyGraph {
 };
 static constexpr int CS_VERIFY_GRAPHS = 8;
 
-// event brackets around kernel families (cs_profile_verify_step)
-static constexpr int CS_PROF_MAX = 2048;
-static constexpr int CS_PROF_FAMILIES = 4;
-enum : int { CS_FAM_GEMM = 0, CS_FAM_ATTENTION = 1, CS_FAM_LMHEAD = 2, CS_FAM_ELEMENTWISE = 3 };
-struct Prof {
-  cudaEvent_t ev[2 * CS_PROF_MAX];
-  int fam[CS_PROF_MAX];
-  int n;
-};
+// Step timeline (cs_set_stamps): every stamped launch of a step owns one 64-bit slot of a
+// caller-provided device buffer, into which each of its CTAs leaves the time at which it
+// finished (largest wins).  Kernel i's share of the pipelined step is then
+// end[i] - end[i - 1], measured inside the running pipeline with no event between launches.
+static constexpr int CS_STAMP_MAX = 4096;
+enum : int { CS_FAM_GEMM = 0, CS_FAM_ATTENTION = 1, CS_FAM_LMHEAD = 2, CS_FAM_MERGE = 3, CS_FAM_OTHER = 4 };
 
 struct cs_ctx {
   cs_model_config cfg;
@@ -150,13 +153,20 @@ struct cs_ctx {
   unsigned attn_mma_attr_set;   // bit DH/32 per head size
   size_t attn_tc_smem_set;
   int attn_force;            // 0 = choose by shape, 1 = mma.sync kernel, 2 = tcgen05 kernel
-  int tune_smem_kb;          // > 0: shared memory budget of a GEMM CTA (CS_TUNE_SMEM_KB, read at creation)
+  bool no_graph;             // CS_NO_GRAPH=1 at creation: steps are enqueued kernel by kernel
+  unsigned long long wait_limit_ns;   // limit of the kernels' bounded waits (CS_WAIT_LIMIT_US at creation; 2 s)
+  int debug_drop_kb;         // test hook: the next GEMM launch leaves out this K block's loads (-1 = none)
+
+  void* match_index;         // cs_set_match_index: the loop searches through this gamma-gram index (NULL = scan)
+  int match_index_cap;
 
   LoopState loop;
   HostStepGraph host_step;
   VerifyGraph verify_graphs[CS_VERIFY_GRAPHS];
   int verify_graph_next;
-  Prof* prof;   // non-NULL only inside cs_profile_verify_step
+  unsigned long long* stamp_buf;   // device, caller-owned; NULL = no stamps
+  int stamp_cap, stamp_n;          // slots available / handed out for the step being enqueued
+  unsigned char stamp_fam[CS_STAMP_MAX];
 
   char err[256];
 };
@@ -172,6 +182,23 @@ struct cs_ctx {
   } while (0)
 
 static inline int cs_ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// slot of the next stamped launch of the step being enqueued (NULL when stamps are off)
+static inline unsigned long long* cs_next_stamp(cs_ctx* ctx, int family) {
+  if (ctx->stamp_buf == nullptr || ctx->stamp_n >= ctx->stamp_cap || ctx->stamp_n >= CS_STAMP_MAX) return nullptr;
+  ctx->stamp_fam[ctx->stamp_n] = (unsigned char)family;
+  return ctx->stamp_buf + ctx->stamp_n++;
+}
+#ifdef __CUDACC__
+// called by one thread of a CTA once the CTA's work is done
+__device__ __forceinline__ void cs_stamp_end(unsigned long long* slot) {
+  if (slot != nullptr) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    atomicMax(slot, t);
+  }
+}
+#endif
 
 // GEMM epilogues
 enum : int { CS_EPI_STORE = 0, CS_EPI_ARGMAX = 1, CS_EPI_RESIDUAL = 2, CS_EPI_SWIGLU = 3, CS_EPI_QKV = 4 };
@@ -237,6 +264,13 @@ cs_status cs_launch_find_match(const int32_t* hist, const int32_t* hist_len, int
                                int gamma, int k, int policy, int32_t* match_pos, int32_t* draft,
                                int32_t* draft_len, int32_t* last_tok, const int32_t* skip,
                                cudaStream_t st);
+// cs_index.cu
+cs_status cs_launch_gram_lookup(const void* index, int B, int capacity_tokens, const int32_t* hist, const int32_t* hist_len,
+                                int stride, int gamma, int k, int policy, int32_t* match_pos, int32_t* draft,
+                                int32_t* draft_len, int32_t* last_tok, const int32_t* skip, cudaStream_t st);
+// inserts the grams that became admissible; overflow is flagged in `status` (NULL = the index's own word)
+cs_status cs_launch_gram_update(void* index, int B, int capacity_tokens, const int32_t* hist, const int32_t* hist_len,
+                                int stride, int gamma, int max_chunks, int* status, cudaStream_t st);
 // cs_gemm.cu
 cs_status cs_gemm_plan(cs_ctx* ctx, GemmPlan* g, const void* w, int N, int K, bool allow_split);
 void cs_gemm_splits(const cs_ctx* ctx, const GemmPlan* g, int rows, int* splits, int* kb_per_split);

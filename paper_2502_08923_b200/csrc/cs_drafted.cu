@@ -128,13 +128,18 @@ extern "C" cs_status cs_decode_loop_drafted(cs_ctx* target, cs_ctx* drafter, int
       }
       DR_CUDA(cudaMemcpyAsync(t_draft, d_argmax + (r - 1), sizeof(int), cudaMemcpyDeviceToDevice, st));
       // the remaining delta - 1 proposals, one single-row greedy step each; the new token is
-      // written straight into the target's draft row
+      // copied into the target's draft row
+      // (through one fixed input slot and one fixed output slot, so that all of them replay the same graph)
       int32_t* d_zero = drafter->loop_last + 2;
+      int32_t* d_in = drafter->loop_mpos;
+      int32_t* d_tok = drafter->loop_mpos + 1;
       const int zero = 0;
       DR_CUDA(cudaMemcpyAsync(d_zero, &zero, sizeof(int), cudaMemcpyHostToDevice, st));
       for (int i = 1; i < delta; ++i) {
-        DR_OK(cs_verify_step_cached(drafter, t_draft + (i - 1), nullptr, d_zero, 1, 0, kv_drafter, kv_len_drafter, nullptr,
-                                    d_accept, t_draft + i, d_argmax, st));
+        DR_CUDA(cudaMemcpyAsync(d_in, t_draft + (i - 1), sizeof(int), cudaMemcpyDeviceToDevice, st));
+        DR_OK(cs_verify_step_cached(drafter, d_in, nullptr, d_zero, 1, 0, kv_drafter, kv_len_drafter, nullptr,
+                                    d_accept, d_tok, d_argmax, st));
+        DR_CUDA(cudaMemcpyAsync(t_draft + i, d_tok, sizeof(int), cudaMemcpyDeviceToDevice, st));
         d_len += 1;
       }
       DR_CUDA(cudaMemcpyAsync(t_dlen, &delta, sizeof(int), cudaMemcpyHostToDevice, st));

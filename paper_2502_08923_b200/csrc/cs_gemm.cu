@@ -44,7 +44,7 @@ namespace {
 
 constexpr int kThreads = 192;          // warps 0-3 epilogue, warp 4 TMA producer, warp 5 MMA
 constexpr int kTileABytes = CS_GEMM_BM * CS_GEMM_BK * 2;   // 16 KB
-constexpr unsigned long long kWaitLimitNs = 2000000000ull; // 2 s
+constexpr unsigned long long kWaitLimitNs = 2000000000ull; // default limit of every wait: 2 s
 
 struct GemmArgs {
   int rows, n_tok, N, K;
@@ -60,6 +60,10 @@ struct GemmArgs {
   int* tile_idx;
   int tile_stride;
   int* status;
+  unsigned long long wait_ns;   // limit of every bounded wait
+  int smem_bytes;               // dynamic shared memory of the launch
+  int drop_kb;                  // test hook: the producer leaves out this K block's loads (-1 = none)
+  unsigned long long* stamp;    // step timeline slot of this launch, or NULL
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -88,8 +92,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait.  Returns false when another role of this CTA gave up or 2 s passed.
-__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+// Bounded wait.  Returns false when another role of this CTA gave up or `limit_ns` passed.
+__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                       unsigned long long limit_ns) {
   unsigned long long t0 = 0;
   for (uint32_t it = 0;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
@@ -97,7 +102,7 @@ __device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile i
       if (*abort_flag) return false;
       const unsigned long long now = globaltimer_ns();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > kWaitLimitNs) return false;
+      else if (now - t0 > limit_ns) return false;
     }
   }
 }
@@ -200,6 +205,11 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
   int* red_idx = reinterpret_cast<int*>(red_val + 4 * a.n_tok);
   float* rstd_s = reinterpret_cast<float*>(red_idx + 4 * a.n_tok);   // [n_tok] (folded RMSNorm)
   float* dump = reinterpret_cast<float*>(smem);                   // [n_tok][128] fp32, reuses the operand ring
+  // the launcher sizes the window for exactly this layout; a mismatch is reported, not written through
+  if ((size_t)(reinterpret_cast<uint8_t*>(rstd_s + a.n_tok) - smem_raw) > (size_t)a.smem_bytes) {
+    if (threadIdx.x == 0) atomicOr(a.status, CS_DEV_SMEM);
+    return;
+  }
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tile = blockIdx.x;
@@ -243,12 +253,14 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
       // weights depend on nothing: fill the ring with them before waiting for the predecessor
       const int npre = min(nkb, a.stages);
       for (int i = 0; i < npre; ++i) {
+        if (i == a.drop_kb) continue;   // (test hook: this stage never fills, the consumer's wait runs out)
         mbar_expect_tx(bar_full + 8 * i, (uint32_t)stage_bytes);
         tma_load_2d(smem_u32(smem + (size_t)i * stage_bytes), &tmW, bar_full + 8 * i, (kb0 + i) * CS_GEMM_BK, n0);
       }
       asm volatile("griddepcontrol.wait;" ::: "memory");
       for (int i = 0; i < npre; ++i)
       {
+        if (i == a.drop_kb) continue;
         const uint32_t sx = smem_u32(smem + (size_t)i * stage_bytes) + kTileABytes;
         tma_load_2d(sx, &tmX, bar_full + 8 * i, (kb0 + i) * CS_GEMM_BK, 0);
         if (two) tma_load_2d(sx + xtile, &tmX, bar_full + 8 * i, (kb0 + i) * CS_GEMM_BK, a.lo_row);
@@ -257,8 +269,9 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
       for (; i < nkb; ++i) {
         const int s = i % a.stages;
         const uint32_t ph = (uint32_t)(i / a.stages) & 1u;
-        if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, s_abort)) { ok = false; break; }
+        if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, s_abort, a.wait_ns)) { ok = false; break; }
         const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
+        if (i == a.drop_kb) continue;
         mbar_expect_tx(bar_full + 8 * s, (uint32_t)stage_bytes);
         tma_load_2d(sa, &tmW, bar_full + 8 * s, (kb0 + i) * CS_GEMM_BK, n0);
         tma_load_2d(sa + kTileABytes, &tmX, bar_full + 8 * s, (kb0 + i) * CS_GEMM_BK, 0);
@@ -271,7 +284,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
       if (*s_abort) {
         // copies still in flight must land before this CTA's shared memory is reused or released
         for (int j = max(0, i - a.stages); j < i; ++j)
-          mbar_wait(bar_full + 8 * (j % a.stages), (uint32_t)(j / a.stages) & 1u, s_never);
+          if (j != a.drop_kb) mbar_wait(bar_full + 8 * (j % a.stages), (uint32_t)(j / a.stages) & 1u, s_never, a.wait_ns);
       }
     }
   } else if (warp == 5) {
@@ -283,7 +296,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
       for (int i = 0; i < nkb; ++i) {
         const int s = i % a.stages;
         const uint32_t ph = (uint32_t)(i / a.stages) & 1u;
-        if (!mbar_wait(bar_full + 8 * s, ph, s_abort)) { ok = false; break; }
+        if (!mbar_wait(bar_full + 8 * s, ph, s_abort, a.wait_ns)) { ok = false; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
         const uint64_t da = umma_desc(sa), db = umma_desc(sa + kTileABytes),
@@ -317,7 +330,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
       }
       asm volatile("bar.sync 1, 128;" ::: "memory");
     }
-    if (nkb > 0) ok = mbar_wait(bar_acc, 0, s_abort);
+    if (nkb > 0) ok = mbar_wait(bar_acc, 0, s_abort, a.wait_ns);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     ok = __all_sync(0xffffffffu, ok) && (*s_abort == 0);
     if (!ok && lane == 0) atomicOr(a.status, CS_DEV_TIMEOUT);
@@ -576,8 +589,9 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
   // ---------------------------------------------------------------- teardown
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
+  if (threadIdx.x == 0) cs_stamp_end(a.stamp);
   if (warp == 5) {
-    if (*s_abort && lane == 0 && nkb > 0) mbar_wait(bar_acc, 0, s_never);  // MMAs retired
+    if (*s_abort && lane == 0 && nkb > 0) mbar_wait(bar_acc, 0, s_never, a.wait_ns);  // MMAs retired
     __syncwarp();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols)
@@ -675,7 +689,6 @@ cs_status cs_gemm_plan(cs_ctx* ctx, GemmPlan* g, const void* w, int N, int K, bo
     const long cost = (long)cs_ceil_div(tiles * s, avail) * (cs_ceil_div(kb, s) + 2);
     if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = s; }
   }
-  if (allow_split && getenv("CS_TUNE_SPLITS")) best = max(1, min(CS_MAX_SPLITS, min(kb, atoi(getenv("CS_TUNE_SPLITS")))));
   g->kb_per_split = cs_ceil_div(kb, best);
   g->splits = cs_ceil_div(kb, g->kb_per_split);
   return encode_2d(ctx, &g->tmW, w, N, K, CS_GEMM_BM, true);
@@ -729,6 +742,8 @@ cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX,
   a.tile_stride = ctx->rows_pad;
   a.status = ctx->d_status;
   const int stage_bytes = kTileABytes + (lo_row >= 0 ? 2 : 1) * a.n_tok * 128;
+  // behind the ring: 2 * stages + 1 barriers, the TMEM slot and flags, the ARGMAX scratch and 1/rms
+  // (the stage count is capped at 8 below, so 17 barriers is the most the kernel places)
   const int fixed = 1024 /*alignment slack*/ + (2 * 8 + 1) * 8 + 16 + 9 * a.n_tok * 4;
   // Two CTAs per SM wherever two stages fit into half an SM: the grids (224-240 CTAs) are
   // sized for the 296 slots that gives, and a one-CTA-per-SM launch would run them in two
@@ -740,7 +755,6 @@ cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX,
     stages = (two >= 2 && park_fits) ? two : (220 * 1024 - fixed) / stage_bytes;
   }
   if (stages > 8) stages = 8;
-  if (ctx->tune_smem_kb > 0) stages = min(12, (ctx->tune_smem_kb * 1024 - fixed) / stage_bytes);
   // the parked tile ([n_tok][128] fp32) reuses the ring
   // (a GEMM that feeds a norm keeps [n_tok][32] more floats behind it)
   if (stages < 2 || (size_t)stages * stage_bytes < (size_t)a.n_tok * (CS_GEMM_BM + 32) * 4) {
@@ -749,6 +763,15 @@ cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX,
   }
   a.stages = stages;
   const size_t smem = (size_t)fixed + (size_t)stages * stage_bytes;
+  a.smem_bytes = (int)smem;
+  a.wait_ns = ctx->wait_limit_ns;
+  a.stamp = cs_next_stamp(ctx, mode == CS_EPI_ARGMAX ? CS_FAM_LMHEAD : CS_FAM_GEMM);
+  a.drop_kb = ctx->debug_drop_kb;
+  ctx->debug_drop_kb = -1;            // the hook covers one launch
+  if (a.drop_kb >= 0 && a.splits > 1) {
+    snprintf(ctx->err, sizeof(ctx->err), "the dropped-tile test hook is for launches without split-K");
+    return CS_ERR_UNSUPPORTED;
+  }
   if (!ctx->gemm_attr_set) {
     CS_CUDA_OK(ctx, cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
     ctx->gemm_attr_set = true;
@@ -849,6 +872,7 @@ extern "C" cs_status cs_lm_head_static(const void* X, const void* W, int rows, i
                                        int32_t* ids, void* stream) {
   if (X == nullptr || W == nullptr || ids == nullptr || rows < 1 || vocab < 1 || d_model < 8 || (d_model % 8))
     return CS_ERR_ARG;
+  if (((reinterpret_cast<uintptr_t>(X) | reinterpret_cast<uintptr_t>(W)) & 15) != 0) return CS_ERR_ARG;
   const int tiles = cs_ceil_div(vocab, CS_GEMM_BM);
   if (rows > kStaticMaxRows || tiles > kStaticMaxTiles) return CS_ERR_LIMIT;
   void* scratch = nullptr;
@@ -858,18 +882,19 @@ extern "C" cs_status cs_lm_head_static(const void* X, const void* W, int rows, i
   float* tile_max = static_cast<float*>(scratch);
   int* tile_idx = reinterpret_cast<int*>(static_cast<unsigned char*>(scratch) + kStaticMaxBytes);
   int* status = reinterpret_cast<int*>(static_cast<unsigned char*>(scratch) + 2 * kStaticMaxBytes);
-  // the array keeps whatever the last call left: the status word is the only part that is
-  // read before it is written, so it is the only part cleared
-  if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return CS_ERR_CUDA;
 
+  // host work that can fail comes first, so that a failed call has enqueued nothing
   cs_ctx err_sink;                      // only its error string is touched by the encoder
   err_sink.err[0] = 0;
   CUtensorMap tmW, tmX;
   GemmArgs a;
   a.rows = rows;
   a.n_tok = cs_ceil_div(rows, 16) * 16;
-  if ((s = encode_2d(&err_sink, &tmW, W, vocab, d_model, CS_GEMM_BM, true)) != CS_OK) return s;
-  if ((s = encode_2d(&err_sink, &tmX, X, a.n_tok, d_model, a.n_tok, false)) != CS_OK) return s;
+  if (encode_2d(&err_sink, &tmW, W, vocab, d_model, CS_GEMM_BM, true) != CS_OK) return CS_ERR_CUDA;
+  if (encode_2d(&err_sink, &tmX, X, a.n_tok, d_model, a.n_tok, false) != CS_OK) return CS_ERR_CUDA;
+  // the array keeps whatever the last call left: the status word is the only part that is
+  // read before it is written, so it is the only part cleared
+  if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return CS_ERR_CUDA;
   a.N = vocab;
   a.K = d_model;
   a.num_kb = cs_ceil_div(d_model, CS_GEMM_BK);
@@ -888,14 +913,17 @@ extern "C" cs_status cs_lm_head_static(const void* X, const void* W, int rows, i
   a.status = status;
   const int stage_bytes = kTileABytes + a.n_tok * 128;
   const int fixed = 1024 + (2 * 8 + 1) * 8 + 16 + 9 * a.n_tok * 4;
-  int stages = (100 * 1024 - fixed) / stage_bytes;
+  int stages = (100 * 1024 - fixed) / stage_bytes;   // at least 4 for rows <= 64
   if (stages > 8) stages = 8;
-  if (stages < 2) return CS_ERR_UNSUPPORTED;
   a.stages = stages;
+  a.smem_bytes = fixed + stages * stage_bytes;
+  a.wait_ns = kWaitLimitNs;
+  a.drop_kb = -1;
+  a.stamp = nullptr;
   cudaLaunchConfig_t lc = {};
   lc.gridDim = dim3(tiles, 1, 1);
   lc.blockDim = dim3(kThreads, 1, 1);
-  lc.dynamicSmemBytes = (size_t)fixed + (size_t)stages * stage_bytes;
+  lc.dynamicSmemBytes = (size_t)a.smem_bytes;
   lc.stream = st;
   cudaLaunchAttribute at[1];
   at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;

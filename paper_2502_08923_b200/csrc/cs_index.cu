@@ -76,16 +76,18 @@ __global__ void k_gram_commit(const int* __restrict__ hist_len, int stride, int 
 // Look the last gamma tokens up and gather the draft (same outputs as the scan).
 __global__ void k_gram_lookup(const int2* __restrict__ table, unsigned slots, const int* __restrict__ hist,
                               const int* __restrict__ hist_len, int stride, int gamma, int k, int policy,
-                              int* __restrict__ match_pos, int* __restrict__ draft, int* __restrict__ draft_len) {
+                              int* __restrict__ match_pos, int* __restrict__ draft, int* __restrict__ draft_len,
+                              int* __restrict__ last_tok, const int* __restrict__ skip) {
   const int b = blockIdx.x;
   const int* h = hist + (size_t)b * stride;
   const int2* T = table + (size_t)b * slots;
   int n = hist_len[b];
   n = n > stride ? stride : (n < 0 ? 0 : n);
+  const bool dead = (skip != nullptr && skip[b] != 0);   // a finished sequence of the loop: no match, no draft
   __shared__ int s_p0;
   if (threadIdx.x == 0) {
     int p0 = -1;
-    if (n >= 2 * gamma) {
+    if (n >= 2 * gamma && !dead) {
       const int* key = h + n - gamma;
       unsigned s = gram_hash(key, gamma) & (slots - 1);
       for (unsigned probe = 0; probe < slots; ++probe, s = (s + 1) & (slots - 1)) {
@@ -105,11 +107,36 @@ __global__ void k_gram_lookup(const int2* __restrict__ table, unsigned slots, co
   if (threadIdx.x == 0) {
     match_pos[b] = p0;
     draft_len[b] = len;
+    if (last_tok != nullptr) last_tok[b] = (n > 0) ? h[n - 1] : 0;
   }
   for (int i = threadIdx.x; i < k; i += blockDim.x) draft[(size_t)b * k + i] = (i < len) ? h[start + i] : -1;
 }
 
 }  // namespace
+
+// The loop's use of the index (App. B.3 step 1 by lookup, step 2(d) by insertion): same outputs as
+// the scan's launcher; table overflow goes to `status` (the context's status word).
+cs_status cs_launch_gram_lookup(const void* index, int B, int capacity_tokens, const int32_t* hist, const int32_t* hist_len,
+                                int stride, int gamma, int k, int policy, int32_t* match_pos, int32_t* draft,
+                                int32_t* draft_len, int32_t* last_tok, const int32_t* skip, cudaStream_t st) {
+  if (gamma < 1 || gamma > CS_MAX_GAMMA || (policy != CS_MATCH_LATEST && policy != CS_MATCH_FIRST) || k < 0 || B < 1)
+    return CS_ERR_ARG;
+  k_gram_lookup<<<B, 128, 0, st>>>(static_cast<const int2*>(index), idx_slots(capacity_tokens), hist, hist_len, stride, gamma, k,
+                                   policy, match_pos, draft, draft_len, last_tok, skip);
+  return cudaGetLastError() == cudaSuccess ? CS_OK : CS_ERR_CUDA;
+}
+
+cs_status cs_launch_gram_update(void* index, int B, int capacity_tokens, const int32_t* hist, const int32_t* hist_len,
+                                int stride, int gamma, int max_chunks, int* status, cudaStream_t st) {
+  const unsigned slots = idx_slots(capacity_tokens);
+  int* ilen = reinterpret_cast<int*>(static_cast<char*>(index) + (size_t)B * slots * sizeof(int2));
+  int chunks = cs_ceil_div(stride, kIdxThreads);
+  chunks = chunks < 1 ? 1 : (chunks > max_chunks ? max_chunks : chunks);
+  k_gram_insert<<<dim3(chunks, B), kIdxThreads, 0, st>>>(static_cast<int2*>(index), slots, hist, hist_len, stride, gamma, ilen,
+                                                        status != nullptr ? status : ilen + B);
+  k_gram_commit<<<cs_ceil_div(B, 128), 128, 0, st>>>(hist_len, stride, gamma, B, ilen);
+  return cudaGetLastError() == cudaSuccess ? CS_OK : CS_ERR_CUDA;
+}
 
 extern "C" size_t cs_gram_index_bytes(int B, int capacity_tokens) {
   if (B < 1 || capacity_tokens < 1) return 0;
@@ -135,16 +162,8 @@ extern "C" cs_status cs_gram_index_update(void* index, int B, int capacity_token
   if (index == nullptr || hist == nullptr || hist_len == nullptr || B < 1 || B > 65535 || capacity_tokens < 1 || stride < 0)
     return CS_ERR_ARG;
   if (gamma < 1 || gamma > CS_MAX_GAMMA) return CS_ERR_ARG;
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const unsigned slots = idx_slots(capacity_tokens);
-  int* ilen = idx_len_ptr(index, B, capacity_tokens);
-  int* status = ilen + B;
-  int chunks = cs_ceil_div(stride, kIdxThreads);
-  chunks = chunks < 1 ? 1 : (chunks > 64 ? 64 : chunks);
-  k_gram_insert<<<dim3(chunks, B), kIdxThreads, 0, st>>>(static_cast<int2*>(index), slots, hist, hist_len, stride, gamma, ilen,
-                                                        status);
-  k_gram_commit<<<cs_ceil_div(B, 128), 128, 0, st>>>(hist_len, stride, gamma, B, ilen);
-  return cudaGetLastError() == cudaSuccess ? CS_OK : CS_ERR_CUDA;
+  return cs_launch_gram_update(index, B, capacity_tokens, hist, hist_len, stride, gamma, 64, nullptr,
+                               static_cast<cudaStream_t>(stream));
 }
 
 extern "C" cs_status cs_find_match_indexed(const void* index, int B, int capacity_tokens, const int32_t* hist,
@@ -155,10 +174,8 @@ extern "C" cs_status cs_find_match_indexed(const void* index, int B, int capacit
     return CS_ERR_ARG;
   if (gamma < 1 || gamma > CS_MAX_GAMMA) return CS_ERR_ARG;
   if (policy != CS_MATCH_LATEST && policy != CS_MATCH_FIRST) return CS_ERR_ARG;
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
-  k_gram_lookup<<<B, 128, 0, st>>>(static_cast<const int2*>(index), idx_slots(capacity_tokens), hist, hist_len, stride, gamma, k,
-                                   (int)policy, match_pos, draft, draft_len);
-  return cudaGetLastError() == cudaSuccess ? CS_OK : CS_ERR_CUDA;
+  return cs_launch_gram_lookup(index, B, capacity_tokens, hist, hist_len, stride, gamma, k, (int)policy, match_pos, draft,
+                               draft_len, nullptr, nullptr, static_cast<cudaStream_t>(stream));
 }
 
 // 0 if every insertion so far found a slot, CS_ERR_CAPACITY otherwise; synchronises the stream.

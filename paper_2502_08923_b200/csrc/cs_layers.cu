@@ -1,7 +1,9 @@
-// Everything of the verification forward that is not a weight GEMM (Sec. 3.2; App. B.2):
-// block assembly, embedding, RMSNorm with the split-K reduction and residual add folded
-// in, RoPE + KV append, causal block attention over the KV cache, SwiGLU, the final
-// argmax / prefix acceptance, KV truncation and the loop's commit step.
+// The small kernels around the GEMMs and the attention of the verification forward
+// (Sec. 3.2; App. B.2): block assembly (rows, positions, rotary table), embedding lookup with
+// the first RMSNorm, the merge of the attention's key slices, the reduction of the LM-head
+// tile maxima with prefix acceptance, KV truncation, and the loop's init and commit steps.
+// RoPE, the K/V append, SwiGLU, the residual adds and every later RMSNorm live in the GEMM
+// epilogues (cs_gemm.cu); attention is in cs_attn_tc.cu and cs_attn.cu.
 #include <math.h>
 
 #include "cs_common.cuh"
@@ -94,7 +96,7 @@ constexpr int kNormThreads = 1024;
 __global__ void __launch_bounds__(kNormThreads)
 k_embed_rmsnorm(const __nv_bfloat16* __restrict__ E, const int* __restrict__ row_tok, float* __restrict__ x, int d,
                 const __nv_bfloat16* __restrict__ gain, float eps, __nv_bfloat16* __restrict__ xn,
-                __nv_bfloat16* __restrict__ xn_lo) {
+                __nv_bfloat16* __restrict__ xn_lo, unsigned long long* stamp) {
   CS_PDL_PROLOGUE();
   const int row = blockIdx.x;
   const __nv_bfloat16* er = E + (size_t)row_tok[row] * d;
@@ -150,11 +152,16 @@ k_embed_rmsnorm(const __nv_bfloat16* __restrict__ E, const int* __restrict__ row
   }
   for (int i = 4 * kNormThreads * 4 + threadIdx.x * 4; i < d; i += kNormThreads * 4)
     emit(i, *reinterpret_cast<const float4*>(xr + i));
+  if (stamp != nullptr) {
+    __syncthreads();
+    if (threadIdx.x == 0) cs_stamp_end(stamp);
+  }
 }
 
 // Combine the key slices: o = sum_s o_s e^(m_s - M) / sum_s l_s e^(m_s - M).
 __global__ void k_attn_merge(const float* __restrict__ in_o, const float* __restrict__ in_ml, int nsplit,
-                             int rows, int H, int Dh, __nv_bfloat16* __restrict__ attn_out) {
+                             int rows, int H, int Dh, __nv_bfloat16* __restrict__ attn_out,
+                             unsigned long long* stamp) {
   CS_PDL_PROLOGUE();
   const int row = blockIdx.x, h = blockIdx.y, dd = threadIdx.x;
   const int lane = threadIdx.x & 31;
@@ -193,6 +200,10 @@ __global__ void k_attn_merge(const float* __restrict__ in_o, const float* __rest
   const __nv_bfloat16 hi = __float2bfloat16_rn(acc);
   attn_out[((size_t)row * H + h) * Dh + dd] = hi;
   attn_out[((size_t)(CS_MAX_ROWS + row) * H + h) * Dh + dd] = __float2bfloat16_rn(acc - __bfloat162float(hi));
+  if (stamp != nullptr) {
+    __syncthreads();
+    if (threadIdx.x == 0) cs_stamp_end(stamp);
+  }
 }
 
 // ------------------------------------------------------------------ acceptance
@@ -205,7 +216,7 @@ k_accept(const float* __restrict__ tile_max, const int* __restrict__ tile_idx, i
          const int* __restrict__ seq_ok, const int* __restrict__ script, int script_stride,
          const int* __restrict__ script_off, int script_limit, int* __restrict__ accept_len,
          int* __restrict__ out_tokens, int* __restrict__ argmax_ids, int* __restrict__ kv_len,
-         int update_kv) {
+         int update_kv, unsigned long long* stamp) {
   CS_PDL_PROLOGUE();
   const int b = blockIdx.x, R = k + 1;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
@@ -256,6 +267,7 @@ k_accept(const float* __restrict__ tile_max, const int* __restrict__ tile_idx, i
     if (!ok) {
       accept_len[b] = -1;
       for (int r = 0; r < R; ++r) out_tokens[(size_t)b * R + r] = -1;
+      cs_stamp_end(stamp);
       return;
     }
     const int off = (script != nullptr && script_off != nullptr) ? script_off[b] : 0;
@@ -273,6 +285,7 @@ k_accept(const float* __restrict__ tile_max, const int* __restrict__ tile_idx, i
     }
     accept_len[b] = tau;
     if (update_kv) kv_len[b] += tau + 1;
+    cs_stamp_end(stamp);
   }
 }
 
@@ -350,9 +363,11 @@ __global__ void k_loop_init(const int* hist_len, const int* kv_len, int B, int s
 // EOS in real mode, advance the lengths (the KV truncation of App. B.2) and count.
 __global__ void k_loop_commit(int* hist, int* hist_len, int B, int stride, int* kv_len, int k, int max_new,
                               int eos_id, int scripted, const int* accept, const int* out, const int* mpos,
-                              int* emitted, int* done, int max_batch, unsigned long long* stats) {
+                              int* emitted, int* done, int max_batch, unsigned long long* stats,
+                              unsigned long long* stamp) {
   CS_PDL_PROLOGUE();
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b == 0) cs_stamp_end(stamp);   // (the kernel is a few dozen instructions: its start stands for its end)
   if (b >= B || done[b]) return;
   cs_stats* st = reinterpret_cast<cs_stats*>(stats);
   const int tau = accept[b];
@@ -410,13 +425,14 @@ void cs_launch_prefill_setup(cs_ctx* ctx, const int32_t* hist, const int32_t* hi
 
 void cs_launch_embed_rmsnorm(cs_ctx* ctx, const __nv_bfloat16* gain, int rows, cudaStream_t st) {
   cs_launch_pdl(k_embed_rmsnorm, dim3(rows), dim3(kNormThreads), 0, st, ctx->embed, ctx->row_tok, ctx->x, ctx->cfg.d_model, gain,
-                ctx->cfg.rms_eps, ctx->xn, ctx->xn + (size_t)CS_MAX_ROWS * ctx->cfg.d_model);
+                ctx->cfg.rms_eps, ctx->xn, ctx->xn + (size_t)CS_MAX_ROWS * ctx->cfg.d_model,
+                cs_next_stamp(ctx, CS_FAM_OTHER));
 }
 
 void cs_launch_attn_merge(cs_ctx* ctx, int nsplit, int rows, cudaStream_t st) {
   const cs_model_config& c = ctx->cfg;
   cs_launch_pdl(k_attn_merge, dim3(rows, c.n_heads), dim3(c.head_dim), 0, st, ctx->attn_o, ctx->attn_ml, nsplit, rows,
-                c.n_heads, c.head_dim, ctx->attn_out);
+                c.n_heads, c.head_dim, ctx->attn_out, cs_next_stamp(ctx, CS_FAM_MERGE));
 }
 
 void cs_launch_accept(cs_ctx* ctx, int B, int k, const int32_t* draft, const int32_t* draft_len,
@@ -425,7 +441,8 @@ void cs_launch_accept(cs_ctx* ctx, int B, int k, const int32_t* draft, const int
                       int update_kv, cudaStream_t st) {
   cs_launch_pdl(k_accept, dim3(B), dim3(512), 0, st, ctx->tile_max, ctx->tile_idx,
                 cs_ceil_div(ctx->cfg.vocab, CS_GEMM_BM), ctx->rows_pad, k, draft, draft_len, ctx->seq_ok, script,
-                script_stride, script_off, script_limit, accept_len, out_tokens, argmax_ids, kv_len, update_kv);
+                script_stride, script_off, script_limit, accept_len, out_tokens, argmax_ids, kv_len, update_kv,
+                cs_next_stamp(ctx, CS_FAM_OTHER));
 }
 
 void cs_launch_tile_reduce(cs_ctx* ctx, int rows, int32_t* ids, cudaStream_t st) {
@@ -451,5 +468,5 @@ void cs_launch_loop_commit(cs_ctx* ctx, int32_t* hist, int32_t* hist_len, int B,
                            int k, int max_new, int eos_id, int scripted, cudaStream_t st) {
   cs_launch_pdl(k_loop_commit, dim3(cs_ceil_div(B, 128)), dim3(128), 0, st, hist, hist_len, B, stride, kv_len, k,
                 max_new, eos_id, scripted, ctx->loop_accept, ctx->loop_out, ctx->loop_mpos, ctx->loop_emitted,
-                ctx->loop_done, ctx->cfg.max_batch, ctx->loop_stats);
+                ctx->loop_done, ctx->cfg.max_batch, ctx->loop_stats, cs_next_stamp(ctx, CS_FAM_OTHER));
 }

@@ -117,6 +117,9 @@ cs_status cs_launch_find_match(const int32_t* hist, const int32_t* hist_len, int
                                int gamma, int k, int policy, int32_t* match_pos, int32_t* draft,
                                int32_t* draft_len, int32_t* last_tok, const int32_t* skip,
                                cudaStream_t st) {
+  // no entry point reaches the kernel with a key longer than its compare loop or an unknown policy
+  if (gamma < 1 || gamma > CS_MAX_GAMMA || (policy != CS_MATCH_LATEST && policy != CS_MATCH_FIRST) || k < 0 || B < 0)
+    return CS_ERR_ARG;
   if (B == 0) return CS_OK;
   // 4096 candidates per CTA keep every thread at >= 4 vector iterations on long
   // histories; short ones use a single CTA per sequence

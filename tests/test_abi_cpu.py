@@ -67,5 +67,11 @@ def test_context_calls_reject_null():
     assert lib.cs_sync_status(None, None) == cs.CS_ERR_ARG
     h = C.c_void_p()
     assert lib.cs_create(C.byref(h), None, None, None, 0) == cs.CS_ERR_ARG
-    assert lib.cs_last_error(None) == b"no context"
+    assert lib.cs_last_error(None) == b"cs_create: NULL argument"     # cs_create leaves its text with the thread
+    bad = _cfg(inputs.TINY); bad.head_dim = 48
+    assert lib.cs_create(C.byref(h), C.byref(bad), C.byref(cs.CsWeights()), C.c_void_p(1024), 0) == cs.CS_ERR_SHAPE
+    assert b"configuration" in lib.cs_last_error(None)
+    assert lib.cs_loop_last_step(None, None, None, None, None, None, None) == cs.CS_ERR_ARG
+    assert lib.cs_debug_drop_tile(None, 0) == cs.CS_ERR_ARG
+    lib.cs_step_host_reset(None)
     lib.cs_destroy(None)

@@ -135,6 +135,33 @@ def test_loop_capacity_is_reported():
     ctx.close()
 
 
+def test_a_sequence_without_room_does_not_stop_the_others():
+    """Batch of two: the second history leaves no room for max_new more tokens.  The loop reports
+    CS_ERR_CAPACITY, leaves that sequence untouched and still runs the first one to its end."""
+    cfg = inputs.TINY
+    ctx, _ = make_pair(cfg, 1024, 2, 10)
+    ctxt, _ = inputs.tiny_context(seed=1)
+    max_new, stride = 120, 600
+    lens = [400, 512]                      # 512 + 120 > 600
+    script = inputs.copy_script(np.random.default_rng(3), ctxt[:400], max_new, 0.6, 5, 30, cfg.vocab, zipf_s=None)
+    h = np.zeros((2, stride), dtype=np.int32)
+    for b, n in enumerate(lens):
+        h[b, :n] = ctxt[:n]
+    hd, ld = i32(h), i32(lens)
+    kv = ctx.alloc_kv()
+    kvl = torch.zeros(2, dtype=torch.int32, device="cuda")
+    ctx.cs_prefill(hd, ld, 512, kv, kvl)
+    with pytest.raises(cs.CsError) as err:
+        ctx.cs_decode_loop(hd, ld, kv, kvl, 3, 10, max_new, script=i32(np.stack([script, script])))
+    assert err.value.code == cs.CS_ERR_CAPACITY
+    _, _, h_sim = O.scripted_simulator(ctxt[:400], script, 3, 10, O.LATEST, max_new)
+    assert ld.cpu().tolist() == [400 + max_new, 512] and kvl.cpu().tolist() == [400 + max_new - 1, 511]
+    assert hd[0, :400 + max_new].cpu().tolist() == h_sim
+    assert hd[1].cpu().tolist() == h[1].tolist()
+    assert ctx.cs_sync_status() == 0       # the status was reported once and cleared
+    ctx.close()
+
+
 @pytest.mark.parametrize("k", [50, 100])
 def test_wide_blocks_match_the_simulator(k):
     """Copy windows of 50 and 100 tokens (the sweep of Sec. 4 / App. B.1): blocks of 51 and 101
@@ -239,6 +266,18 @@ def test_steps_driven_from_host_memory():
     for b in range(2):
         gen = hist_h[b, lens[b]:int(len_h[b])].tolist()
         assert len(gen) >= 8 and max(greedy_margins(model, cfg, ctxt[:lens[b]], gen)) < LOGIT_TOL
+    # a caller that rewrote a row in place says so; the next call uploads the rows in full again
+    ctx.cs_step_host_reset()
+    before = [int(len_h[b]) for b in range(2)]
+    ctx.cs_step_host(hist_h, len_h, hist_d, len_d, kv, kvl, 3, k, acc, out)
+    for b in range(2):
+        assert int(len_h[b]) == before[b] + int(acc[b]) + 1
+        assert hist_d[b, :before[b]].cpu().tolist() == hist_h[b, :before[b]].tolist()
+    # a key longer than the search kernel compares, or an unknown policy, is refused on the host
+    for bad in (dict(gamma=9), dict(gamma=3, policy=7)):
+        with pytest.raises(cs.CsError) as err:
+            ctx.cs_step_host(hist_h, len_h, hist_d, len_d, kv, kvl, bad["gamma"], k, acc, out, policy=bad.get("policy", cs.LATEST))
+        assert err.value.code == cs.CS_ERR_ARG
     # a history row without room for one more block is refused on the host, nothing changes
     len_h[0] = stride - 5
     with pytest.raises(cs.CsError):
