@@ -107,6 +107,9 @@ cs_status enqueue_forward(cs_ctx* ctx, int B, int R, void* kv_cache, bool with_l
                           cudaStream_t st) {
   const cs_model_config& c = ctx->cfg;
   const int rows = B * R;
+  // second bf16 term of every activation operand (row offset in the operand maps), or -1 when the
+  // caller settles for the leading term
+  const int lo_row = ctx->one_term ? -1 : CS_MAX_ROWS;
   cs_status s = ensure_act_maps(ctx, cs_ceil_div(rows, 16) * 16);
   if (s != CS_OK) return s;
   // Only the first RMSNorm runs as a kernel.  Every later one is folded into the GEMMs around
@@ -120,7 +123,7 @@ cs_status enqueue_forward(cs_ctx* ctx, int B, int R, void* kv_cache, bool with_l
     }
     const QkvEpi qe = {ctx->rope_cs, ctx->row_pos, ctx->row_write, ctx->qbuf, static_cast<__nv_bfloat16*>(kv_cache),
                        R, l, c.n_heads, c.n_kv_heads, c.head_dim, c.max_batch, c.max_seq};
-    s = cs_launch_gemm(ctx, &L.qkv, &ctx->tmXn, CS_MAX_ROWS, rows, CS_EPI_QKV, nullptr, nullptr, nullptr, 0, &qe,
+    s = cs_launch_gemm(ctx, &L.qkv, &ctx->tmXn, lo_row, rows, CS_EPI_QKV, nullptr, nullptr, nullptr, 0, &qe,
                        &take_norm, st);
     if (s != CS_OK) return s;
     cs_launch_attention(ctx, kv_cache, l, B, R, st);
@@ -129,36 +132,36 @@ cs_status enqueue_forward(cs_ctx* ctx, int B, int R, void* kv_cache, bool with_l
     give.xn_out = ctx->xn;
     give.ssq_out = ctx->ssq;
     give.slot_stride = ctx->ssq_stride;
-    s = cs_launch_gemm(ctx, &L.o, &ctx->tmAttn, CS_MAX_ROWS, rows, CS_EPI_RESIDUAL, ctx->x, nullptr, nullptr, 0, nullptr,
+    s = cs_launch_gemm(ctx, &L.o, &ctx->tmAttn, lo_row, rows, CS_EPI_RESIDUAL, ctx->x, nullptr, nullptr, 0, nullptr,
                        &give, st);
     if (s != CS_OK) return s;
     take_norm = NormFuse{};
     take_norm.ssq_in = ctx->ssq;
     {
-      int sp, kbs;
-      cs_gemm_splits(ctx, &L.o, rows, &sp, &kbs);
-      take_norm.slots_in = cs_ceil_div(L.o.N, CS_GEMM_BM) * sp;
+      GemmShape sh;
+      if (cs_gemm_shape(ctx, &L.o, rows, lo_row >= 0, &sh) != CS_OK) return fail(ctx, CS_ERR_UNSUPPORTED, "no launch shape for the attention-output GEMM");
+      take_norm.slots_in = cs_ceil_div(L.o.N, CS_GEMM_BM) * sh.splits;
     }
     take_norm.slot_stride = ctx->ssq_stride;
     take_norm.inv_d = 1.f / (float)c.d_model;
     take_norm.eps = c.rms_eps;
-    s = cs_launch_gemm(ctx, &L.gate_up, &ctx->tmXn, CS_MAX_ROWS, rows, CS_EPI_SWIGLU, nullptr, ctx->act,
+    s = cs_launch_gemm(ctx, &L.gate_up, &ctx->tmXn, lo_row, rows, CS_EPI_SWIGLU, nullptr, ctx->act,
                        ctx->act + (size_t)CS_MAX_ROWS * c.d_ffn, c.d_ffn, nullptr, &take_norm, st);
     if (s != CS_OK) return s;
     // the norm after this layer: the next layer's, or the final one before the LM head
     const __nv_bfloat16* next_gain = (l + 1 < c.n_layers) ? ctx->layers[l + 1].attn_norm : (with_lm ? ctx->final_norm : nullptr);
     give.gain_out = next_gain;
-    s = cs_launch_gemm(ctx, &L.down, &ctx->tmAct, CS_MAX_ROWS, rows, CS_EPI_RESIDUAL, ctx->x, nullptr, nullptr, 0, nullptr,
+    s = cs_launch_gemm(ctx, &L.down, &ctx->tmAct, lo_row, rows, CS_EPI_RESIDUAL, ctx->x, nullptr, nullptr, 0, nullptr,
                        &give, st);
     if (s != CS_OK) return s;
     {
-      int sp, kbs;
-      cs_gemm_splits(ctx, &L.down, rows, &sp, &kbs);
-      take_norm.slots_in = cs_ceil_div(L.down.N, CS_GEMM_BM) * sp;
+      GemmShape sh;
+      if (cs_gemm_shape(ctx, &L.down, rows, lo_row >= 0, &sh) != CS_OK) return fail(ctx, CS_ERR_UNSUPPORTED, "no launch shape for the down GEMM");
+      take_norm.slots_in = cs_ceil_div(L.down.N, CS_GEMM_BM) * sh.splits;
     }
   }
   if (with_lm) {
-    s = cs_launch_gemm(ctx, &ctx->lm, &ctx->tmXn, CS_MAX_ROWS, rows, CS_EPI_ARGMAX, logits, nullptr, nullptr, 0, nullptr,
+    s = cs_launch_gemm(ctx, &ctx->lm, &ctx->tmXn, lo_row, rows, CS_EPI_ARGMAX, logits, nullptr, nullptr, 0, nullptr,
                        &take_norm, st);
     if (s != CS_OK) return s;
   }
@@ -594,8 +597,9 @@ cs_status cs_prefill(cs_ctx* ctx, const int32_t* hist, const int32_t* hist_len, 
     ctx->stamp_n = 0;
     cs_launch_prefill_setup(ctx, hist, hist_len, B, stride, start, r, st);
     cs_status s = enqueue_forward(ctx, B, r, kv_cache, false, nullptr, st);
-    if (s != CS_OK) return s;
+    if (s != CS_OK) { ctx->one_term = false; return s; }
   }
+  ctx->one_term = false;
   if (total <= 0) cs_launch_prefill_setup(ctx, hist, hist_len, B, stride, 0, 1, st);   // sets seq_ok
   cs_launch_prefill_finish(ctx, hist_len, kv_len, B, st);
   CS_CUDA_OK(ctx, cudaGetLastError());

@@ -34,6 +34,14 @@ struct GemmPlan {
   int N, K;
   int splits;           // split-K factor
   int kb_per_split;     // 64-wide K blocks per split
+  bool allow_split;
+};
+
+// how one GEMM is launched for a given block height
+struct GemmShape {
+  int n_tok;            // token rows rounded up to 16 (UMMA N)
+  int mt;               // 128-feature sub-tiles per CTA
+  int splits, kb_per_split, stages, stage_bytes, smem;
 };
 
 struct LayerPlan {
@@ -153,6 +161,7 @@ struct cs_ctx {
   unsigned attn_mma_attr_set;   // bit DH/32 per head size
   size_t attn_tc_smem_set;
   int attn_force;            // 0 = choose by shape, 1 = mma.sync kernel, 2 = tcgen05 kernel
+  bool one_term;             // the forward being enqueued feeds its GEMMs the leading bf16 term only
   bool no_graph;             // CS_NO_GRAPH=1 at creation: steps are enqueued kernel by kernel
   unsigned long long wait_limit_ns;   // limit of the kernels' bounded waits (CS_WAIT_LIMIT_US at creation; 2 s)
   int debug_drop_kb;         // test hook: the next GEMM launch leaves out this K block's loads (-1 = none)
@@ -273,7 +282,7 @@ cs_status cs_launch_gram_update(void* index, int B, int capacity_tokens, const i
                                 int stride, int gamma, int max_chunks, int* status, cudaStream_t st);
 // cs_gemm.cu
 cs_status cs_gemm_plan(cs_ctx* ctx, GemmPlan* g, const void* w, int N, int K, bool allow_split);
-void cs_gemm_splits(const cs_ctx* ctx, const GemmPlan* g, int rows, int* splits, int* kb_per_split);
+cs_status cs_gemm_shape(const cs_ctx* ctx, const GemmPlan* g, int rows, bool two_terms, GemmShape* out);
 cs_status cs_make_act_map(cs_ctx* ctx, CUtensorMap* tm, const void* base, int rows_total, int K,
                           int box_rows);
 // mode = CS_EPI_*: `out` is the fp32 destination (STORE, RESIDUAL) or the optional logits dump

@@ -187,6 +187,9 @@ __device__ __forceinline__ void keep_alive(const float4& p, const float4& q) {
   asm volatile("" ::"f"(p.x), "f"(p.y), "f"(p.z), "f"(p.w), "f"(q.x), "f"(q.y), "f"(q.z), "f"(q.w) : "memory");
 }
 
+// MT = 128-feature sub-tiles per CTA (compile-time, so that the one-tile kernel of the short blocks
+// carries no loop overhead in its issue paths: its ring is latency-bound)
+template <int MT>
 __global__ void __launch_bounds__(kThreads, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, GemmArgs a) {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -195,7 +198,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
   uint8_t* smem = smem_raw + (((raw + 1023u) & ~1023u) - raw);   // operand tiles need 1024-byte alignment
   const int xtile = a.n_tok * 128;                 // one activation tile
   const bool two = a.lo_row >= 0;                   // activations come as two bf16 terms
-  const int stage_bytes = kTileABytes + (two ? 2 : 1) * xtile;
+  const int wbytes = MT * kTileABytes;            // the CTA's weight sub-tiles of one K block
+  const int stage_bytes = wbytes + (two ? 2 : 1) * xtile;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)a.stages * stage_bytes);
   // bars[0..stages) = tile landed, bars[stages..2*stages) = tile consumed, bars[2*stages] = accumulator done
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * a.stages + 1);
@@ -212,14 +216,14 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
   }
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int tile = blockIdx.x;
+  const int cta_tile = blockIdx.x;
   const int split = (a.splits > 1) ? (int)cluster_rank() : 0;
-  const int n0 = tile * CS_GEMM_BM;
+  const int cta_n0 = cta_tile * MT * CS_GEMM_BM;
   const int kb0 = split * a.kb_per_split;
   const int kb1 = min(a.num_kb, kb0 + a.kb_per_split);
   const int nkb = max(0, kb1 - kb0);
   uint32_t tmem_cols = 32;
-  while ((int)tmem_cols < a.n_tok) tmem_cols <<= 1;
+  while ((int)tmem_cols < MT * a.n_tok) tmem_cols <<= 1;   // one accumulator of n_tok columns per sub-tile
 
   const uint32_t bar_full = smem_u32(bars), bar_empty = smem_u32(bars + a.stages),
                  bar_acc = smem_u32(bars + 2 * a.stages);
@@ -255,13 +259,16 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
       for (int i = 0; i < npre; ++i) {
         if (i == a.drop_kb) continue;   // (test hook: this stage never fills, the consumer's wait runs out)
         mbar_expect_tx(bar_full + 8 * i, (uint32_t)stage_bytes);
-        tma_load_2d(smem_u32(smem + (size_t)i * stage_bytes), &tmW, bar_full + 8 * i, (kb0 + i) * CS_GEMM_BK, n0);
+#pragma unroll
+        for (int m = 0; m < MT; ++m)
+          tma_load_2d(smem_u32(smem + (size_t)i * stage_bytes) + m * kTileABytes, &tmW, bar_full + 8 * i,
+                      (kb0 + i) * CS_GEMM_BK, cta_n0 + m * CS_GEMM_BM);
       }
       asm volatile("griddepcontrol.wait;" ::: "memory");
       for (int i = 0; i < npre; ++i)
       {
         if (i == a.drop_kb) continue;
-        const uint32_t sx = smem_u32(smem + (size_t)i * stage_bytes) + kTileABytes;
+        const uint32_t sx = smem_u32(smem + (size_t)i * stage_bytes) + wbytes;
         tma_load_2d(sx, &tmX, bar_full + 8 * i, (kb0 + i) * CS_GEMM_BK, 0);
         if (two) tma_load_2d(sx + xtile, &tmX, bar_full + 8 * i, (kb0 + i) * CS_GEMM_BK, a.lo_row);
       }
@@ -273,9 +280,11 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
         const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
         if (i == a.drop_kb) continue;
         mbar_expect_tx(bar_full + 8 * s, (uint32_t)stage_bytes);
-        tma_load_2d(sa, &tmW, bar_full + 8 * s, (kb0 + i) * CS_GEMM_BK, n0);
-        tma_load_2d(sa + kTileABytes, &tmX, bar_full + 8 * s, (kb0 + i) * CS_GEMM_BK, 0);
-        if (two) tma_load_2d(sa + kTileABytes + xtile, &tmX, bar_full + 8 * s, (kb0 + i) * CS_GEMM_BK, a.lo_row);
+#pragma unroll
+        for (int m = 0; m < MT; ++m)
+          tma_load_2d(sa + m * kTileABytes, &tmW, bar_full + 8 * s, (kb0 + i) * CS_GEMM_BK, cta_n0 + m * CS_GEMM_BM);
+        tma_load_2d(sa + wbytes, &tmX, bar_full + 8 * s, (kb0 + i) * CS_GEMM_BK, 0);
+        if (two) tma_load_2d(sa + wbytes + xtile, &tmX, bar_full + 8 * s, (kb0 + i) * CS_GEMM_BK, a.lo_row);
       }
       if (!ok) {
         *s_abort = 1;
@@ -299,12 +308,16 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
         if (!mbar_wait(bar_full + 8 * s, ph, s_abort, a.wait_ns)) { ok = false; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
-        const uint64_t da = umma_desc(sa), db = umma_desc(sa + kTileABytes),
-                       dl = umma_desc(sa + kTileABytes + xtile);
+        const uint64_t db = umma_desc(sa + wbytes), dl = umma_desc(sa + wbytes + xtile);
 #pragma unroll
-        for (int kk = 0; kk < CS_GEMM_BK / 16; ++kk) {   // 16 K-elements = 32 bytes per instruction
-          umma_bf16(tmem_base, da + 2 * kk, db + 2 * kk, idesc, (i > 0 || kk > 0) ? 1u : 0u);
-          if (two) umma_bf16(tmem_base, da + 2 * kk, dl + 2 * kk, idesc, 1u);   // x = hi + lo
+        for (int m = 0; m < MT; ++m) {                   // every sub-tile against the same activation tile
+          const uint64_t da = umma_desc(sa + m * kTileABytes);
+          const uint32_t acc = tmem_base + (uint32_t)(m * a.n_tok);
+#pragma unroll
+          for (int kk = 0; kk < CS_GEMM_BK / 16; ++kk) {   // 16 K-elements = 32 bytes per instruction
+            umma_bf16(acc, da + 2 * kk, db + 2 * kk, idesc, (i > 0 || kk > 0) ? 1u : 0u);
+            if (two) umma_bf16(acc, da + 2 * kk, dl + 2 * kk, idesc, 1u);   // x = hi + lo
+          }
         }
         umma_commit(bar_empty + 8 * s);
       }
@@ -315,11 +328,9 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
       umma_commit(bar_acc);
     }
   } else {
-    // ------------------------------------------------------------- accumulator read-out (warps 0-3)
-    const int feat = n0 + warp * 32 + lane;
+    // ------------------------------------------------------------- epilogue warps 0-3: wait for the accumulators
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    const bool scaled = a.nf.ssq_in != nullptr;
-    if (scaled) {
+    if (a.nf.ssq_in != nullptr) {
       // 1/rms of every token row while the main loop runs: slots summed in a fixed order
       for (int tok = warp; tok < a.rows; tok += 4) {
         float ss = 0.f;
@@ -334,10 +345,24 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     ok = __all_sync(0xffffffffu, ok) && (*s_abort == 0);
     if (!ok && lane == 0) atomicOr(a.status, CS_DEV_TIMEOUT);
+  }
+  if (warp >= 4) asm volatile("griddepcontrol.wait;" ::: "memory");
+
+  // One pass per 128-feature sub-tile: read its accumulator out, then (all but ARGMAX) the split-K
+  // reduction and the epilogue.  Every CTA of a cluster takes the same number of passes.
+#pragma unroll 1
+  for (int m = 0; m < MT; ++m) {
+  const int tile = cta_tile * MT + m;
+  const int n0 = cta_n0 + m * CS_GEMM_BM;
+  if (n0 >= a.N) break;
+  if (warp < 4) {
+    // ------------------------------------------------------------- accumulator read-out (warps 0-3)
+    const int feat = n0 + warp * 32 + lane;
+    const bool scaled = a.nf.ssq_in != nullptr;
     for (int c0 = 0; c0 < a.n_tok && c0 < a.rows; c0 += 16) {
       uint32_t v[16];
       if (nkb > 0 && ok) {
-        tmem_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
+        tmem_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(m * a.n_tok + c0), v);
       } else {
 #pragma unroll
         for (int j = 0; j < 16; ++j) v[j] = 0u;
@@ -384,9 +409,9 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
           a.tile_idx[(size_t)tile * a.tile_stride + tok] = idx;
         }
       }
+      if (MT > 1) asm volatile("bar.sync 1, 128;" ::: "memory");   // the scratch rows are reused by the next pass
     }
   }
-  if (warp >= 4) asm volatile("griddepcontrol.wait;" ::: "memory");
 
   // ---------------------------------------------------------------- split-K reduction + epilogue
   if (a.mode != CS_EPI_ARGMAX) {
@@ -583,9 +608,12 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
     }
     if (a.splits > 1) {
       if (!arrived) cluster_arrive();
-      cluster_wait();                              // nobody leaves while a peer still reads its tile
+      cluster_wait();                              // nobody leaves (or parks its next tile) while a peer still reads this one
+    } else if (MT > 1) {
+      __syncthreads();                             // the parked tile is read out before the next one is parked
     }
   }
+  }   // sub-tile passes
   // ---------------------------------------------------------------- teardown
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
@@ -675,6 +703,7 @@ cs_status cs_gemm_plan(cs_ctx* ctx, GemmPlan* g, const void* w, int N, int K, bo
   g->W = static_cast<const __nv_bfloat16*>(w);
   g->N = N;
   g->K = K;
+  g->allow_split = allow_split;
   const int tiles = cs_ceil_div(N, CS_GEMM_BM), kb = cs_ceil_div(K, CS_GEMM_BK);
   // two CTAs fit on an SM; clustered launches are planned for 85 % of those slots, because
   // a cluster must find all its CTAs free inside one GPC and a grid that needs every slot
@@ -694,18 +723,75 @@ cs_status cs_gemm_plan(cs_ctx* ctx, GemmPlan* g, const void* w, int N, int K, bo
   return encode_2d(ctx, &g->tmW, w, N, K, CS_GEMM_BM, true);
 }
 
-// Split-K factor and K blocks per split for a block of `rows` token rows.  The plan's factor is
-// made for two CTAs per SM; blocks too tall for that run one CTA per SM, and their grid is kept
-// within one wave where the tile count allows it.
-void cs_gemm_splits(const cs_ctx* ctx, const GemmPlan* g, int rows, int* splits, int* kb_per_split) {
-  const int n_tok = cs_ceil_div(rows, 16) * 16;
+// Launch shape of one GEMM for a block of `rows` token rows.
+//  - Short blocks (two CTAs fit on an SM): one 128-feature tile per CTA and the plan's split-K
+//    factor, made for two CTAs per SM - the HBM-bound regime of 11-row blocks.
+//  - Tall blocks (one CTA per SM): every CTA re-reads its K range of the activations from L2,
+//    which at 100+ rows is several times the weight bytes, so a CTA takes 2 or 4 sub-tiles that
+//    share each activation tile (one TMEM accumulator each), and the split-K factor is chosen
+//    for whole waves of one CTA per SM.  Candidates are ranked by a cost model calibrated on
+//    measurements (K blocks per CTA times the cost of one, plus the epilogue, times waves).
+cs_status cs_gemm_shape(const cs_ctx* ctx, const GemmPlan* g, int rows, bool two_terms, GemmShape* out) {
+  GemmShape sh = {};
+  sh.n_tok = cs_ceil_div(rows, 16) * 16;
+  const int terms = two_terms ? 2 : 1;
+  const int xbytes = terms * sh.n_tok * 128;
   const int tiles = cs_ceil_div(g->N, CS_GEMM_BM), kb = cs_ceil_div(g->K, CS_GEMM_BK);
-  int s = g->splits;
-  const int stage_bytes = CS_GEMM_BM * CS_GEMM_BK * 2 + 2 * n_tok * 128;
-  const bool one_per_sm = (113 * 1024 - 2048) / stage_bytes < 2;
-  if (one_per_sm && s > 1 && tiles * s > ctx->num_sms) s = max(1, ctx->num_sms / tiles);
-  *kb_per_split = cs_ceil_div(kb, s);
-  *splits = cs_ceil_div(kb, *kb_per_split);
+  // behind the ring: up to 2 * 8 + 1 barriers, the TMEM slot and flags, the ARGMAX scratch and 1/rms
+  const int fixed = 1024 /*alignment slack*/ + (2 * 8 + 1) * 8 + 16 + 9 * sh.n_tok * 4;
+  const size_t park = (size_t)sh.n_tok * (CS_GEMM_BM + 32) * 4;   // parked tile + sums of squares reuse the ring
+  const int sb1 = kTileABytes + xbytes;
+  // Two CTAs per SM wherever two stages fit into half an SM: the grids (224-240 CTAs) are
+  // sized for the 296 slots that gives.  Only blocks too tall for that take the whole SM.
+  int stages = (100 * 1024 - fixed) / sb1;
+  bool tall = false;
+  if (stages < 4) {
+    const int two = (113 * 1024 - fixed) / sb1;
+    if (two >= 2 && (size_t)two * sb1 >= park) stages = two;
+    else tall = true;
+  }
+  if (!tall) {
+    sh.mt = 1;
+    sh.stages = stages > 8 ? 8 : stages;
+    sh.splits = g->splits;
+    sh.kb_per_split = g->kb_per_split;
+    sh.stage_bytes = sb1;
+  } else {
+    long best = -1;
+    for (int mt = 1; mt <= 4; mt *= 2) {
+      if (mt * sh.n_tok > 512 || (mt > 1 && mt > tiles)) continue;
+      const int sb = mt * kTileABytes + xbytes;
+      int st = (220 * 1024 - fixed) / sb;
+      if (st > 8) st = 8;
+      if (st < 2 || (size_t)st * sb < park) continue;
+      const int ctas = cs_ceil_div(tiles, mt);
+      // Cycles of one K block, calibrated on 176-row blocks: the mt * terms * 4 MMAs take n_tok / 2
+      // cycles each; a stage comes back L cycles after it was handed to the producer (about 2,100
+      // for a 61 KB stage, 3,300 for a 77 KB one), and with `st` stages in flight a K block costs
+      // (L + mma) / st unless the tensor pipe is the slower.  The epilogue (accumulator read-out,
+      // split-K reduction over the cluster, stores) costs about 4,000 + 145 n_tok cycles per sub-tile.
+      const long mma = (long)mt * terms * 4 * (sh.n_tok / 2);
+      const long lat = 2120 + (long)((sb - 62464) * 0.072);
+      const long turn = ((lat > 1000 ? lat : 1000) + mma) / st;
+      const long per_kb = mma > turn ? mma : turn;
+      const long epi = (long)mt * (4000 + 145L * sh.n_tok);
+      const int smax = g->allow_split ? max(1, min(CS_MAX_SPLITS, kb / 4)) : 1;
+      for (int sp = 1; sp <= smax; ++sp) {
+        const int kps = cs_ceil_div(kb, sp), spl = cs_ceil_div(kb, kps);
+        const long waves = cs_ceil_div(ctas * spl, ctx->num_sms);
+        const long cost = waves * ((long)kps * per_kb + epi);
+        if (best < 0 || cost < best) {
+          best = cost;
+          sh.mt = mt; sh.stages = st; sh.splits = spl; sh.kb_per_split = kps; sh.stage_bytes = sb;
+        }
+      }
+    }
+    if (best < 0) return CS_ERR_UNSUPPORTED;
+  }
+  if (sh.stages < 2 || (size_t)sh.stages * sh.stage_bytes < park) return CS_ERR_UNSUPPORTED;
+  sh.smem = fixed + sh.stages * sh.stage_bytes;
+  *out = sh;
+  return CS_OK;
 }
 
 cs_status cs_make_act_map(cs_ctx* ctx, CUtensorMap* tm, const void* base, int rows_total, int K,
@@ -716,14 +802,20 @@ cs_status cs_make_act_map(cs_ctx* ctx, CUtensorMap* tm, const void* base, int ro
 cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX, int lo_row, int rows, int mode,
                          float* out, __nv_bfloat16* act, __nv_bfloat16* act_lo, int F, const QkvEpi* q,
                          const NormFuse* nf, cudaStream_t st) {
-  const int tiles = cs_ceil_div(g->N, CS_GEMM_BM);
+  GemmShape sh;
+  if (cs_gemm_shape(ctx, g, rows, lo_row >= 0, &sh) != CS_OK) {
+    snprintf(ctx->err, sizeof(ctx->err), "no GEMM launch shape fits shared memory for %d rows", rows);
+    return CS_ERR_UNSUPPORTED;
+  }
+  const int tiles = cs_ceil_div(cs_ceil_div(g->N, CS_GEMM_BM), sh.mt);   // CTAs along the features
   GemmArgs a;
   a.rows = rows;
-  a.n_tok = cs_ceil_div(rows, 16) * 16;
+  a.n_tok = sh.n_tok;
   a.N = g->N;
   a.K = g->K;
   a.num_kb = cs_ceil_div(g->K, CS_GEMM_BK);
-  cs_gemm_splits(ctx, g, rows, &a.splits, &a.kb_per_split);
+  a.splits = sh.splits;
+  a.kb_per_split = sh.kb_per_split;
   a.mode = mode;
   a.out = out;
   a.act = act;
@@ -741,29 +833,9 @@ cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX,
   a.tile_idx = ctx->tile_idx;
   a.tile_stride = ctx->rows_pad;
   a.status = ctx->d_status;
-  const int stage_bytes = kTileABytes + (lo_row >= 0 ? 2 : 1) * a.n_tok * 128;
-  // behind the ring: 2 * stages + 1 barriers, the TMEM slot and flags, the ARGMAX scratch and 1/rms
-  // (the stage count is capped at 8 below, so 17 barriers is the most the kernel places)
-  const int fixed = 1024 /*alignment slack*/ + (2 * 8 + 1) * 8 + 16 + 9 * a.n_tok * 4;
-  // Two CTAs per SM wherever two stages fit into half an SM: the grids (224-240 CTAs) are
-  // sized for the 296 slots that gives, and a one-CTA-per-SM launch would run them in two
-  // waves.  Only blocks too tall for that take the whole SM.
-  int stages = (100 * 1024 - fixed) / stage_bytes;
-  if (stages < 4) {
-    const int two = (113 * 1024 - fixed) / stage_bytes;
-    const bool park_fits = (size_t)two * stage_bytes >= (size_t)a.n_tok * (CS_GEMM_BM + 32) * 4;
-    stages = (two >= 2 && park_fits) ? two : (220 * 1024 - fixed) / stage_bytes;
-  }
-  if (stages > 8) stages = 8;
-  // the parked tile ([n_tok][128] fp32) reuses the ring
-  // (a GEMM that feeds a norm keeps [n_tok][32] more floats behind it)
-  if (stages < 2 || (size_t)stages * stage_bytes < (size_t)a.n_tok * (CS_GEMM_BM + 32) * 4) {
-    snprintf(ctx->err, sizeof(ctx->err), "GEMM stage of %d bytes does not fit shared memory", stage_bytes);
-    return CS_ERR_UNSUPPORTED;
-  }
-  a.stages = stages;
-  const size_t smem = (size_t)fixed + (size_t)stages * stage_bytes;
-  a.smem_bytes = (int)smem;
+  a.stages = sh.stages;
+  const size_t smem = (size_t)sh.smem;
+  a.smem_bytes = sh.smem;
   a.wait_ns = ctx->wait_limit_ns;
   a.stamp = cs_next_stamp(ctx, mode == CS_EPI_ARGMAX ? CS_FAM_LMHEAD : CS_FAM_GEMM);
   a.drop_kb = ctx->debug_drop_kb;
@@ -772,8 +844,12 @@ cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX,
     snprintf(ctx->err, sizeof(ctx->err), "the dropped-tile test hook is for launches without split-K");
     return CS_ERR_UNSUPPORTED;
   }
+  void (*kernel)(const CUtensorMap, const CUtensorMap, GemmArgs) =
+      sh.mt == 4 ? k_gemm_tc<4> : (sh.mt == 2 ? k_gemm_tc<2> : k_gemm_tc<1>);
   if (!ctx->gemm_attr_set) {
-    CS_CUDA_OK(ctx, cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+    CS_CUDA_OK(ctx, cudaFuncSetAttribute(k_gemm_tc<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+    CS_CUDA_OK(ctx, cudaFuncSetAttribute(k_gemm_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+    CS_CUDA_OK(ctx, cudaFuncSetAttribute(k_gemm_tc<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
     ctx->gemm_attr_set = true;
   }
   cudaLaunchConfig_t lc = {};
@@ -795,7 +871,7 @@ cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX,
   }
   lc.attrs = at;
   lc.numAttrs = na;
-  CS_CUDA_OK(ctx, cudaLaunchKernelEx(&lc, k_gemm_tc, g->tmW, *tmX, a));
+  CS_CUDA_OK(ctx, cudaLaunchKernelEx(&lc, kernel, g->tmW, *tmX, a));
   return CS_OK;
 }
 
@@ -829,7 +905,7 @@ cs_status static_scratch(void** out) {
   if (g_lm_scratch_dev[dev] == nullptr) {
     void* p = nullptr;
     if (cudaGetSymbolAddress(&p, g_lm_scratch) != cudaSuccess || p == nullptr) return CS_ERR_CUDA;
-    if (cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+    if (cudaFuncSetAttribute(k_gemm_tc<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
       return CS_ERR_CUDA;
     g_lm_scratch_dev[dev] = p;
   }
@@ -930,7 +1006,7 @@ extern "C" cs_status cs_lm_head_static(const void* X, const void* W, int rows, i
   at[0].val.programmaticStreamSerializationAllowed = 1;
   lc.attrs = at;
   lc.numAttrs = 1;
-  if (cudaLaunchKernelEx(&lc, k_gemm_tc, tmW, tmX, a) != cudaSuccess) return CS_ERR_CUDA;
+  if (cudaLaunchKernelEx(&lc, k_gemm_tc<1>, tmW, tmX, a) != cudaSuccess) return CS_ERR_CUDA;
   if (cs_launch_pdl(k_tile_reduce_static, dim3(rows), dim3(128), 0, st, (const float*)tile_max,
                     (const int*)tile_idx, tiles, kStaticMaxRows, (const int*)status, ids) != cudaSuccess)
     return CS_ERR_CUDA;

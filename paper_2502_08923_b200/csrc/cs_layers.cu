@@ -221,47 +221,30 @@ k_accept(const float* __restrict__ tile_max, const int* __restrict__ tile_idx, i
   const int b = blockIdx.x, R = k + 1;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
   __shared__ int s_arg[CS_MAX_ROWS];
-  __shared__ float s_val[32][16];
-  __shared__ int s_idx[32][16];
   int dl = draft_len[b];
   dl = dl < 0 ? 0 : (dl > k ? k : dl);
   const bool ok = seq_ok[b] != 0;
-  // Greedy token of every live row: the whole block scans the tile maxima of 16 rows at a time
-  // (one or two independent loads per thread and row), then one warp per row finishes.
-  for (int r0 = 0; r0 < R; r0 += 16) {
-    for (int rr = 0; rr < 16; ++rr) {
-      const int r = r0 + rr;
-      float val = -INFINITY;
-      int idx = INT32_MAX;
-      if (ok && r <= dl && r < R) {
-        const int row = b * R + r;
-        for (int t = threadIdx.x; t < tiles; t += blockDim.x) {
-          const float v = tile_max[(size_t)t * tile_stride + row];
-          const int id = tile_idx[(size_t)t * tile_stride + row];
-          if (v > val || (v == val && id < idx)) { val = v; idx = id; }
-        }
-        for (int off = 16; off > 0; off >>= 1) {
-          const float ov = __shfl_xor_sync(0xffffffffu, val, off);
-          const int oi = __shfl_xor_sync(0xffffffffu, idx, off);
-          if (ov > val || (ov == val && oi < idx)) { val = ov; idx = oi; }
-        }
+  // Greedy token of every live row: one warp per row, its lanes striding over the tile maxima (all
+  // of a lane's loads are independent, so their latencies overlap), then a shuffle reduction.
+  for (int r = warp; r < R; r += nwarps) {
+    float val = -INFINITY;
+    int idx = INT32_MAX;
+    if (ok && r <= dl) {
+      const int row = b * R + r;
+      for (int t = lane; t < tiles; t += 32) {
+        const float v = tile_max[(size_t)t * tile_stride + row];
+        const int id = tile_idx[(size_t)t * tile_stride + row];
+        if (v > val || (v == val && id < idx)) { val = v; idx = id; }
       }
-      if (lane == 0) { s_val[warp][rr] = val; s_idx[warp][rr] = idx; }
-    }
-    __syncthreads();
-    if (warp < 16 && r0 + warp < R) {
-      const int r = r0 + warp;
-      float val = (lane < nwarps) ? s_val[lane][warp] : -INFINITY;
-      int idx = (lane < nwarps) ? s_idx[lane][warp] : INT32_MAX;
       for (int off = 16; off > 0; off >>= 1) {
         const float ov = __shfl_xor_sync(0xffffffffu, val, off);
         const int oi = __shfl_xor_sync(0xffffffffu, idx, off);
         if (ov > val || (ov == val && oi < idx)) { val = ov; idx = oi; }
       }
-      if (lane == 0) s_arg[r] = (ok && r <= dl && idx != INT32_MAX) ? idx : -1;
     }
-    __syncthreads();
+    if (lane == 0) s_arg[r] = (ok && r <= dl && idx != INT32_MAX) ? idx : -1;
   }
+  __syncthreads();
   for (int r = threadIdx.x; r < R; r += blockDim.x) argmax_ids[(size_t)b * R + r] = s_arg[r];
   if (threadIdx.x == 0) {
     if (!ok) {
