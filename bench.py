@@ -607,7 +607,7 @@ def run_workload(args):
                            "gbs_cold": 64 * 32768 * 4 / us / 1e3, **out}}
         print(json.dumps(line), flush=True)
         return 0
-    cfg = inputs.LLAMA8B
+    cfg = inputs.LLAMA8B if args.layers <= 0 else inputs.sliced(inputs.LLAMA8B, args.layers)   # --layers: small case for ncu captures
     if name == "prefill_b1_4096":
         # context ingestion through cs_prefill (chunks of 256 block rows through the same kernels)
         n_ctx = 4096

@@ -344,12 +344,12 @@ cs_status cs_decode_loop_drafted(cs_ctx* target, cs_ctx* drafter, int32_t* hist,
 /* Measurement aid (no counterpart in the paper): a timeline of the step's kernels taken inside
  * the running pipeline.  `stamps` is a caller-allocated DEVICE array of `capacity` 64-bit slots
  * (zero it once); NULL or capacity 0 switches the aid off.  While it is set, stamped launch i
- * of every step the context enqueues or captures afterwards - the projection GEMMs, the
- * attention and merge kernels, the LM-head GEMM, embedding + first norm, acceptance, commit -
- * has each of its CTAs leave the nanosecond time (%globaltimer) at which it finished in
- * stamps[i], largest wins, so stamps[i] - stamps[i-1] is what kernel i added to the pipelined
- * step (the search and block set-up are not stamped: they count towards the embedding's
- * slot).  Set it before cs_loop_begin / the first cs_step_host; it cannot change while a loop
+ * of every step the context enqueues or captures afterwards - search (the scan), block set-up,
+ * embedding + first norm, the projection GEMMs, the attention and merge kernels, the LM-head
+ * GEMM, acceptance, commit - has each of its CTAs leave the nanosecond time (%globaltimer) at
+ * which it finished in stamps[i], largest wins, so stamps[i] - stamps[i-1] is what kernel i added
+ * to the pipelined step (the index kernels of cs_set_match_index are not stamped: they count
+ * towards the slot that follows).  Set it before cs_loop_begin / the first cs_step_host; it cannot change while a loop
  * is in progress.  cs_stamp_layout returns the number of slots one step uses and writes the
  * kernel family of each slot to the HOST array `family` (0 = layer projection GEMM,
  * 1 = attention, 2 = LM-head GEMM with fused argmax, 3 = merge of the attention's key slices,

@@ -179,7 +179,8 @@ cs_status enqueue_loop_step(cs_ctx* ctx, cudaStream_t st) {
                                             L.k, L.policy, ctx->loop_mpos, ctx->loop_draft, ctx->loop_dlen, ctx->loop_last,
                                             ctx->loop_done, st)
                     : cs_launch_find_match(L.hist, L.hist_len, L.B, L.stride, L.gamma, L.k, L.policy, ctx->loop_mpos,
-                                           ctx->loop_draft, ctx->loop_dlen, ctx->loop_last, ctx->loop_done, st);
+                                           ctx->loop_draft, ctx->loop_dlen, ctx->loop_last, ctx->loop_done, st,
+                                           cs_next_stamp(ctx, CS_FAM_OTHER));
   if (r != CS_OK) return fail(ctx, r, "match kernel launch failed");
   cs_launch_block_setup(ctx, ctx->loop_last, ctx->loop_draft, ctx->loop_dlen, L.kv_len, ctx->loop_done, L.B, L.k, st);
   // the step opened with a stream-ordered launch and nothing before k_loop_commit changes kv_len
@@ -648,6 +649,14 @@ cs_status cs_loop_begin(cs_ctx* ctx, int32_t* hist, int32_t* hist_len, int B, in
     if (e != cudaSuccess) { cs_loop_end(ctx); CS_CUDA_OK(ctx, e); }
     size_t nodes = 0;
     if (cudaGraphGetNodes(L.graph, nullptr, &nodes) == cudaSuccess) L.graph_nodes = (int)nodes;
+    // the same step CS_LOOP_UNROLL times over in one graph, for runs of several steps
+    CS_CUDA_OK(ctx, cudaStreamBeginCapture(ctx->cap_stream, cudaStreamCaptureModeRelaxed));
+    for (int i = 0; i < CS_LOOP_UNROLL && s == CS_OK; ++i) s = enqueue_loop_step(ctx, ctx->cap_stream);
+    e = cudaStreamEndCapture(ctx->cap_stream, &L.graph_n);
+    if (s != CS_OK) { cs_loop_end(ctx); return s; }
+    if (e != cudaSuccess) { cs_loop_end(ctx); CS_CUDA_OK(ctx, e); }
+    e = cudaGraphInstantiate(&L.exec_n, L.graph_n, 0);
+    if (e != cudaSuccess) { cs_loop_end(ctx); CS_CUDA_OK(ctx, e); }
   }
   L.active = true;
   return CS_OK;
@@ -659,6 +668,11 @@ cs_status cs_loop_steps(cs_ctx* ctx, int n_steps, void* stream) {
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   for (int i = 0; i < n_steps; ++i) {
     if (ctx->loop.use_graph) {
+      if (n_steps - i >= CS_LOOP_UNROLL && ctx->loop.exec_n != nullptr) {
+        CS_CUDA_OK(ctx, cudaGraphLaunch(ctx->loop.exec_n, st));
+        i += CS_LOOP_UNROLL - 1;
+        continue;
+      }
       CS_CUDA_OK(ctx, cudaGraphLaunch(ctx->loop.exec, st));
     } else {
       cs_status s = enqueue_loop_step(ctx, st);
@@ -705,8 +719,12 @@ void cs_loop_end(cs_ctx* ctx) {
   if (ctx == nullptr) return;
   if (ctx->loop.exec) cudaGraphExecDestroy(ctx->loop.exec);
   if (ctx->loop.graph) cudaGraphDestroy(ctx->loop.graph);
+  if (ctx->loop.exec_n) cudaGraphExecDestroy(ctx->loop.exec_n);
+  if (ctx->loop.graph_n) cudaGraphDestroy(ctx->loop.graph_n);
   ctx->loop.exec = nullptr;
   ctx->loop.graph = nullptr;
+  ctx->loop.exec_n = nullptr;
+  ctx->loop.graph_n = nullptr;
   ctx->loop.active = false;
 }
 

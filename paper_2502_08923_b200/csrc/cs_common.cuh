@@ -60,7 +60,11 @@ struct LoopState {
   int graph_nodes;   // kernel launches in one step
   cudaGraph_t graph;
   cudaGraphExec_t exec;
+  // several steps in one graph: consecutive graph launches leave a gap of some 10 us between them
+  cudaGraph_t graph_n;
+  cudaGraphExec_t exec_n;
 };
+static constexpr int CS_LOOP_UNROLL = 4;   // steps per launch of graph_n
 
 // cs_step_host keeps the graph of its last launch shape: the kernels of one step between the
 // host -> device and device -> host copies
@@ -121,7 +125,7 @@ struct cs_ctx {
   int ssq_stride;
   float* rope_cs;            // cos/sin of this block [rows][Dh/2][2]
   double* inv_freq;          // theta^(-2i/Dh) [Dh/2]
-  float* tile_max;           // LM-head tile maxima [tiles][rows_pad]
+  float* tile_max;           // LM-head tile maxima [rows_pad][tiles]
   int* tile_idx;             // and their token ids
   int* row_tok;              // token id per row [rows_pad]
   int* row_pos;              // absolute position per row
@@ -272,7 +276,7 @@ static inline int cs_max_splits(int tiles, int kb) {
 cs_status cs_launch_find_match(const int32_t* hist, const int32_t* hist_len, int B, int stride,
                                int gamma, int k, int policy, int32_t* match_pos, int32_t* draft,
                                int32_t* draft_len, int32_t* last_tok, const int32_t* skip,
-                               cudaStream_t st);
+                               cudaStream_t st, unsigned long long* stamp = nullptr);
 // cs_index.cu
 cs_status cs_launch_gram_lookup(const void* index, int B, int capacity_tokens, const int32_t* hist, const int32_t* hist_len,
                                 int stride, int gamma, int k, int policy, int32_t* match_pos, int32_t* draft,

@@ -56,7 +56,7 @@ struct GemmArgs {
   int F;
   QkvEpi q;              // QKV: where the rotated queries and the new K/V rows go
   NormFuse nf;           // RMSNorm folded into this GEMM's read-out (consumer) or residual update (producer)
-  float* tile_max;       // ARGMAX: [tiles][tile_stride]
+  float* tile_max;       // ARGMAX: [rows][tile_stride] (a row's tile maxima are contiguous: the reduction reads them coalesced)
   int* tile_idx;
   int tile_stride;
   int* status;
@@ -405,8 +405,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
             const int oi = red_idx[w * a.n_tok + tok];
             if (ov > val || (ov == val && oi < idx)) { val = ov; idx = oi; }
           }
-          a.tile_max[(size_t)tile * a.tile_stride + tok] = val;
-          a.tile_idx[(size_t)tile * a.tile_stride + tok] = idx;
+          a.tile_max[(size_t)tok * a.tile_stride + tile] = val;
+          a.tile_idx[(size_t)tok * a.tile_stride + tile] = idx;
         }
       }
       if (MT > 1) asm volatile("bar.sync 1, 128;" ::: "memory");   // the scratch rows are reused by the next pass
@@ -831,7 +831,7 @@ cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX,
   }
   a.tile_max = ctx->tile_max;
   a.tile_idx = ctx->tile_idx;
-  a.tile_stride = ctx->rows_pad;
+  a.tile_stride = cs_ceil_div(g->N, CS_GEMM_BM);
   a.status = ctx->d_status;
   a.stages = sh.stages;
   const size_t smem = (size_t)sh.smem;
@@ -922,8 +922,8 @@ k_tile_reduce_static(const float* __restrict__ tile_max, const int* __restrict__
   float val = -INFINITY;
   int idx = INT32_MAX;
   for (int t = threadIdx.x; t < tiles; t += 128) {
-    const float v = tile_max[(size_t)t * tile_stride + row];
-    const int id = tile_idx[(size_t)t * tile_stride + row];
+    const float v = tile_max[(size_t)row * tile_stride + t];
+    const int id = tile_idx[(size_t)row * tile_stride + t];
     if (v > val || (v == val && id < idx)) { val = v; idx = id; }
   }
   __shared__ float sv[4];
@@ -985,7 +985,7 @@ extern "C" cs_status cs_lm_head_static(const void* X, const void* W, int rows, i
   a.nf = NormFuse{};
   a.tile_max = tile_max;
   a.tile_idx = tile_idx;
-  a.tile_stride = kStaticMaxRows;
+  a.tile_stride = kStaticMaxTiles;
   a.status = status;
   const int stage_bytes = kTileABytes + a.n_tok * 128;
   const int fixed = 1024 + (2 * 8 + 1) * 8 + 16 + 9 * a.n_tok * 4;
@@ -1008,7 +1008,7 @@ extern "C" cs_status cs_lm_head_static(const void* X, const void* W, int rows, i
   lc.numAttrs = 1;
   if (cudaLaunchKernelEx(&lc, k_gemm_tc<1>, tmW, tmX, a) != cudaSuccess) return CS_ERR_CUDA;
   if (cs_launch_pdl(k_tile_reduce_static, dim3(rows), dim3(128), 0, st, (const float*)tile_max,
-                    (const int*)tile_idx, tiles, kStaticMaxRows, (const int*)status, ids) != cudaSuccess)
+                    (const int*)tile_idx, tiles, kStaticMaxTiles, (const int*)status, ids) != cudaSuccess)
     return CS_ERR_CUDA;
   return CS_OK;
 }

@@ -18,7 +18,8 @@ __global__ void k_block_setup(const int* __restrict__ last_tok, const int* __res
                               const int* __restrict__ draft_len, const int* __restrict__ kv_len,
                               const int* __restrict__ skip, int B, int k, int max_seq, int vocab,
                               int half, const double* __restrict__ inv_freq, int* row_tok, int* row_pos,
-                              int* row_lim, int* row_write, int* seq_ok, float* rope_cs, int* status) {
+                              int* row_lim, int* row_write, int* seq_ok, float* rope_cs, int* status,
+                              unsigned long long* stamp) {
   CS_PDL_PROLOGUE();
   const int R = k + 1, rows = B * R;
   for (int row = threadIdx.x; row < rows; row += blockDim.x) {
@@ -50,6 +51,10 @@ __global__ void k_block_setup(const int* __restrict__ last_tok, const int* __res
     sincos(ang, &s, &c);
     rope_cs[2 * i] = (float)c;
     rope_cs[2 * i + 1] = (float)s;
+  }
+  if (stamp != nullptr) {
+    __syncthreads();
+    if (threadIdx.x == 0) cs_stamp_end(stamp);
   }
 }
 
@@ -232,8 +237,8 @@ k_accept(const float* __restrict__ tile_max, const int* __restrict__ tile_idx, i
     if (ok && r <= dl) {
       const int row = b * R + r;
       for (int t = lane; t < tiles; t += 32) {
-        const float v = tile_max[(size_t)t * tile_stride + row];
-        const int id = tile_idx[(size_t)t * tile_stride + row];
+        const float v = tile_max[(size_t)row * tile_stride + t];
+        const int id = tile_idx[(size_t)row * tile_stride + t];
         if (v > val || (v == val && id < idx)) { val = v; idx = id; }
       }
       for (int off = 16; off > 0; off >>= 1) {
@@ -281,8 +286,8 @@ k_tile_reduce(const float* __restrict__ tile_max, const int* __restrict__ tile_i
   float val = -INFINITY;
   int idx = INT32_MAX;
   for (int t = threadIdx.x; t < tiles; t += 128) {
-    const float v = tile_max[(size_t)t * tile_stride + row];
-    const int id = tile_idx[(size_t)t * tile_stride + row];
+    const float v = tile_max[(size_t)row * tile_stride + t];
+    const int id = tile_idx[(size_t)row * tile_stride + t];
     if (v > val || (v == val && id < idx)) { val = v; idx = id; }
   }
   __shared__ float sv[4];
@@ -395,7 +400,7 @@ void cs_launch_block_setup(cs_ctx* ctx, const int32_t* last_tok, const int32_t* 
   const cs_model_config& c = ctx->cfg;
   cs_launch_pdl(k_block_setup, dim3(1), dim3(256), 0, st, last_tok, draft, draft_len, kv_len, skip, B, k, c.max_seq,
                 c.vocab, c.head_dim / 2, ctx->inv_freq, ctx->row_tok, ctx->row_pos, ctx->row_lim, ctx->row_write,
-                ctx->seq_ok, ctx->rope_cs, ctx->d_status);
+                ctx->seq_ok, ctx->rope_cs, ctx->d_status, cs_next_stamp(ctx, CS_FAM_OTHER));
 }
 
 void cs_launch_prefill_setup(cs_ctx* ctx, const int32_t* hist, const int32_t* hist_len, int B, int stride,
@@ -423,14 +428,14 @@ void cs_launch_accept(cs_ctx* ctx, int B, int k, const int32_t* draft, const int
                       int32_t* accept_len, int32_t* out_tokens, int32_t* argmax_ids, int32_t* kv_len,
                       int update_kv, cudaStream_t st) {
   cs_launch_pdl(k_accept, dim3(B), dim3(512), 0, st, ctx->tile_max, ctx->tile_idx,
-                cs_ceil_div(ctx->cfg.vocab, CS_GEMM_BM), ctx->rows_pad, k, draft, draft_len, ctx->seq_ok, script,
+                cs_ceil_div(ctx->cfg.vocab, CS_GEMM_BM), cs_ceil_div(ctx->cfg.vocab, CS_GEMM_BM), k, draft, draft_len, ctx->seq_ok, script,
                 script_stride, script_off, script_limit, accept_len, out_tokens, argmax_ids, kv_len, update_kv,
                 cs_next_stamp(ctx, CS_FAM_OTHER));
 }
 
 void cs_launch_tile_reduce(cs_ctx* ctx, int rows, int32_t* ids, cudaStream_t st) {
   cs_launch_pdl(k_tile_reduce, dim3(rows), dim3(128), 0, st, ctx->tile_max, ctx->tile_idx,
-                cs_ceil_div(ctx->cfg.vocab, CS_GEMM_BM), ctx->rows_pad, ids);
+                cs_ceil_div(ctx->cfg.vocab, CS_GEMM_BM), cs_ceil_div(ctx->cfg.vocab, CS_GEMM_BM), ids);
 }
 
 void cs_launch_truncate(cs_ctx* ctx, int32_t* kv_len, const int32_t* new_len, int B, cudaStream_t st) {

@@ -25,7 +25,7 @@ __global__ void __launch_bounds__(kThreads)
 k_find_match(const int* __restrict__ hist, const int* __restrict__ hist_len, int stride, int gamma,
              int k, int policy, int* __restrict__ match_pos, int* __restrict__ draft,
              int* __restrict__ draft_len, int* __restrict__ last_tok,
-             const int* __restrict__ skip) {
+             const int* __restrict__ skip, unsigned long long* stamp) {
   CS_PDL_PROLOGUE();
   cg::cluster_group cluster = cg::this_cluster();
   const int b = blockIdx.y;
@@ -109,6 +109,10 @@ k_find_match(const int* __restrict__ hist, const int* __restrict__ hist_len, int
     if (last_tok != nullptr) last_tok[b] = (n > 0) ? h[n - 1] : 0;
   }
   for (int i = tid; i < k; i += kThreads) draft[(size_t)b * k + i] = (i < len) ? h[start + i] : -1;
+  if (stamp != nullptr) {
+    __syncthreads();
+    if (tid == 0) cs_stamp_end(stamp);
+  }
 }
 
 }  // namespace
@@ -116,7 +120,7 @@ k_find_match(const int* __restrict__ hist, const int* __restrict__ hist_len, int
 cs_status cs_launch_find_match(const int32_t* hist, const int32_t* hist_len, int B, int stride,
                                int gamma, int k, int policy, int32_t* match_pos, int32_t* draft,
                                int32_t* draft_len, int32_t* last_tok, const int32_t* skip,
-                               cudaStream_t st) {
+                               cudaStream_t st, unsigned long long* stamp) {
   // no entry point reaches the kernel with a key longer than its compare loop or an unknown policy
   if (gamma < 1 || gamma > CS_MAX_GAMMA || (policy != CS_MATCH_LATEST && policy != CS_MATCH_FIRST) || k < 0 || B < 0)
     return CS_ERR_ARG;
@@ -145,6 +149,6 @@ cs_status cs_launch_find_match(const int32_t* hist, const int32_t* hist_len, int
   lc.numAttrs = 1;
   cudaError_t e = cudaLaunchKernelEx(&lc, k_find_match, (const int*)hist, (const int*)hist_len,
                                      stride, gamma, k, policy, (int*)match_pos, (int*)draft,
-                                     (int*)draft_len, (int*)last_tok, (const int*)skip);
+                                     (int*)draft_len, (int*)last_tok, (const int*)skip, stamp);
   return e == cudaSuccess ? CS_OK : CS_ERR_CUDA;
 }

@@ -126,7 +126,7 @@ def test_step_timeline_stamps():
     hd, ld = begin(stamps)
     fams = ctx.cs_stamp_layout()
     L = cfg.n_layers
-    assert fams == ["other"] + ["gemm", "attention", "merge", "gemm", "gemm", "gemm"] * L + ["lm_head", "other", "other"]
+    assert fams == ["other"] * 3 + ["gemm", "attention", "merge", "gemm", "gemm", "gemm"] * L + ["lm_head", "other", "other"]
     ctx.cs_loop_steps(1)
     torch.cuda.synchronize()
     first = stamps[:len(fams)].cpu().numpy()
