@@ -55,8 +55,10 @@
  * Environment, read once by cs_create (measurement and test switches; not needed in use):
  *   CS_NO_GRAPH=1          steps are enqueued kernel by kernel instead of replayed from a
  *                          captured CUDA graph (cs_loop_*, cs_step_host, cs_decode_loop_drafted);
- *   CS_ATTN_KERNEL=tc|mma  forces the tcgen05 or the mma.sync attention kernel (default: by
- *                          head size);
+ *   CS_ATTN_KERNEL=tc|tcw|mma  forces one attention kernel: tcgen05 with the query rows as the
+ *                          M dimension (tc), tcgen05 with the keys and head dims as M (tcw), or
+ *                          mma.sync (mma).  Default: by head size, and between the two tcgen05
+ *                          kernels by how many key tiles a CTA would walk (tcw from three on);
  *   CS_WAIT_LIMIT_US=n     time limit of the kernels' bounded waits in microseconds (default
  *                          2,000,000), see cs_debug_drop_tile.
  */

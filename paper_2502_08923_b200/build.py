@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcopyspec.so")
-SOURCES = ["cs_match.cu", "cs_index.cu", "cs_gemm.cu", "cs_layers.cu", "cs_attn.cu", "cs_attn_tc.cu", "cs_api.cu", "cs_drafted.cu"]
+SOURCES = ["cs_match.cu", "cs_index.cu", "cs_gemm.cu", "cs_layers.cu", "cs_attn.cu", "cs_attn_tc.cu", "cs_attn_tcw.cu", "cs_api.cu", "cs_drafted.cu"]
 
 
 def _newer_than_lib() -> bool:

@@ -249,7 +249,7 @@ cs_status cs_create(cs_ctx** out, const cs_model_config* cfg, const cs_weights* 
   {
     // the environment switches of the library, all read here and nowhere else
     const char* k = getenv("CS_ATTN_KERNEL");
-    ctx->attn_force = (k == nullptr) ? 0 : (strcmp(k, "mma") == 0 ? 1 : (strcmp(k, "tc") == 0 ? 2 : 0));
+    ctx->attn_force = (k == nullptr) ? 0 : (strcmp(k, "mma") == 0 ? 1 : (strcmp(k, "tc") == 0 ? 2 : (strcmp(k, "tcw") == 0 ? 3 : 0)));
     const char* ng = getenv("CS_NO_GRAPH");
     ctx->no_graph = ng != nullptr && ng[0] == '1';
     const char* wl = getenv("CS_WAIT_LIMIT_US");

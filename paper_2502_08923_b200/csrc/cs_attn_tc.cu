@@ -523,6 +523,21 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUte
 
 }  // namespace
 
+// Key tiles a CTA of this kernel walks at most for a block of B x R rows (same launch arithmetic as
+// below): the dispatcher hands longer walks to the kernel with keys and head dims as M.
+int cs_attention_tc_tiles_per_cta(const cs_ctx* ctx, int B, int R) {
+  const cs_model_config& c = ctx->cfg;
+  const int G = c.n_heads / c.n_kv_heads;
+  if (c.head_dim != kDh || G > kNQMax || R < 1) return 0;
+  const int ngroups = cs_ceil_div(G * R, kNQMax), Rg = cs_ceil_div(R, ngroups);
+  const int NQ = (G * Rg + 15) / 16 * 16;
+  const bool small = 1024 + (size_t)8 * NQ * 128 + (size_t)4 * kHalfBytes <= (size_t)113 * 1024 && (size_t)kCtlBytes + 16 * (size_t)NQ <= 1024;
+  int nsplit = (small ? 2 : 1) * ctx->num_sms / (B * c.n_kv_heads * ngroups);
+  if (nsplit > ctx->attn_splits) nsplit = ctx->attn_splits;
+  if (nsplit < 1) nsplit = 1;
+  return cs_ceil_div(cs_ceil_div(c.max_seq, kTileKeys), nsplit);
+}
+
 int cs_launch_attention_tc(cs_ctx* ctx, const void* kv_cache, int layer, int B, int R, cudaStream_t st) {
   const cs_model_config& c = ctx->cfg;
   const int G = c.n_heads / c.n_kv_heads;

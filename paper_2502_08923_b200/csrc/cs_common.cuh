@@ -163,8 +163,8 @@ struct cs_ctx {
   // process: another context may live on another GPU)
   bool gemm_attr_set;
   unsigned attn_mma_attr_set;   // bit DH/32 per head size
-  size_t attn_tc_smem_set;
-  int attn_force;            // 0 = choose by shape, 1 = mma.sync kernel, 2 = tcgen05 kernel
+  size_t attn_tc_smem_set, attn_tcw_smem_set;
+  int attn_force;            // 0 = choose by shape, 1 = mma.sync kernel, 2 = tcgen05 kernel (query rows as M), 3 = tcgen05 kernel (keys as M)
   bool one_term;             // the forward being enqueued feeds its GEMMs the leading bf16 term only
   bool no_graph;             // CS_NO_GRAPH=1 at creation: steps are enqueued kernel by kernel
   unsigned long long wait_limit_ns;   // limit of the kernels' bounded waits (CS_WAIT_LIMIT_US at creation; 2 s)
@@ -315,6 +315,10 @@ void cs_launch_attn_merge(cs_ctx* ctx, int nsplit, int rows, cudaStream_t st);
 // tcgen05 path (head_dim 128, at most 128 query heads per KV head); returns the number of key
 // slices written, 0 when the shape is not covered, -1 on a host error (ctx->err set)
 int cs_launch_attention_tc(cs_ctx* ctx, const void* kv_cache, int layer, int B, int R, cudaStream_t st);
+// the same contract, keys and head dims as the M dimension (long key ranges); `probe` only answers
+// how many key tiles a CTA of the query-rows-as-M kernel would walk at most
+int cs_launch_attention_tcw(cs_ctx* ctx, const void* kv_cache, int layer, int B, int R, cudaStream_t st);
+int cs_attention_tc_tiles_per_cta(const cs_ctx* ctx, int B, int R);
 // bf16 tensor map of rank <= 5, 128-byte swizzle; dims/box innermost first, strides for dims 1..
 cs_status cs_encode_tiled(cs_ctx* ctx, CUtensorMap* tm, const void* base, int rank, const unsigned long long* dims,
                           const unsigned long long* strides_bytes, const unsigned* box);

@@ -80,14 +80,14 @@ def test_one_verify_step_logits_against_oracle_at_full_size(big):
 
 
 def test_both_attention_kernels_agree_at_full_size(big, monkeypatch):
-    """The library picks the attention kernel by block shape; here both are forced in turn on
-    the same 11-row block (44 query rows per KV head, 4,096 cached keys).  The default one is
-    pinned to the oracle by the test above, so agreement pins the other one too."""
+    """The library picks the attention kernel by head size and key range; here all three are forced
+    in turn on the same 11-row block (44 query rows per KV head, 4,096 cached keys).  The default
+    one is pinned to the oracle by the test above, so agreement pins the others too."""
     cfg, w, ctx, kv, hist, script, taus = big
     n0 = len(hist)
     draft = O.gather_draft(hist, n0, O.find_match(hist, n0, GAMMA, O.LATEST), GAMMA, K)
     out = {}
-    for kern in ("mma", "tc"):
+    for kern in ("mma", "tc", "tcw"):
         monkeypatch.setenv("CS_ATTN_KERNEL", kern)
         c2 = cs.Context(cfg, w, max_seq=kv.shape[4], max_batch=1, k_max=K)
         kv_run = kv.clone()
@@ -97,6 +97,7 @@ def test_both_attention_kernels_agree_at_full_size(big, monkeypatch):
         assert c2.cs_sync_status() == 0
         out[kern] = (logits[0].cpu().numpy(), kv_run[:, :, 0, :, n0 - 1:n0 + K, :].float().cpu().numpy())
         c2.close()
-    assert float(np.abs(out["mma"][0] - out["tc"][0]).max()) <= LOGIT_TOL / 4
-    # stored K/V rows: at most a bf16 rounding flip apart
-    assert float(np.abs(out["mma"][1] - out["tc"][1]).max()) <= 2e-2 * max(1.0, float(np.abs(out["mma"][1]).max()))
+    for other in ("mma", "tcw"):
+        assert float(np.abs(out[other][0] - out["tc"][0]).max()) <= LOGIT_TOL / 4, other
+        # stored K/V rows: at most a bf16 rounding flip apart
+        assert float(np.abs(out[other][1] - out["tc"][1]).max()) <= 2e-2 * max(1.0, float(np.abs(out["tc"][1]).max())), other

@@ -2,8 +2,10 @@
 long-context and multi-turn workloads: a 2-layer slice of the 8B-class shape (d 4096, 32 / 8
 heads of 128, FFN 14,336; a 4,096-row head keeps the oracle quick) over synthetic caches of
 30,720 and 8,192 keys, plus small-width models that put every launch variant of the tcgen05
-attention kernel (up to 48, 49-96, 97-128 padded query rows, and blocks cut into row groups)
-on key slices of at least five tiles per CTA.  Logits, greedy tokens, acceptance and the
+attention kernels (up to 48, 49-96, 97-128 padded query rows, and blocks cut into row groups)
+on key slices of at least five tiles per CTA; every case runs once with the kernel the library
+picks for such key ranges (keys and head dims as the M dimension) and once with the other one
+forced (query rows as M).  Logits, greedy tokens, acceptance and the
 block's K/V rows are compared with the oracle element by element.  The second layer's K/V rows
 and the logits depend on the first layer's attention output, so a wrong key tile, ring slot or
 mask anywhere in the slice fails them."""
@@ -22,6 +24,15 @@ SLICE8B = inputs.ModelConfig(n_layers=2, d_model=4096, n_heads=32, n_kv_heads=8,
                              vocab=4096, rope_theta=500000.0, rms_eps=1e-5)
 NARROW = inputs.ModelConfig(n_layers=2, d_model=512, n_heads=8, n_kv_heads=4, head_dim=128, d_ffn=1024,
                             vocab=1024, rope_theta=500000.0, rms_eps=1e-5)
+
+
+@pytest.fixture(autouse=True, params=["default", "tc"])
+def attention_kernel(request, monkeypatch):
+    """Every case runs with the attention kernel the library picks for its key range (keys and head
+    dims as M at these depths) and with the query-rows-as-M kernel forced."""
+    if request.param != "default":
+        monkeypatch.setenv("CS_ATTN_KERNEL", request.param)
+    return request.param
 
 
 @pytest.fixture(scope="module")
