@@ -162,6 +162,7 @@ struct cs_ctx {
   // shared-memory opt-ins already made for this context's device (per context, not per
   // process: another context may live on another GPU)
   bool gemm_attr_set;
+  int tall_clusters[3][CS_MAX_SPLITS + 1];   // clusters of a tall GEMM launch that can run at once, by sub-tile count and cluster size (0 = not asked yet)
   unsigned attn_mma_attr_set;   // bit DH/32 per head size
   size_t attn_tc_smem_set, attn_tcw_smem_set;
   int attn_force;            // 0 = choose by shape, 1 = mma.sync kernel, 2 = tcgen05 kernel (query rows as M), 3 = tcgen05 kernel (keys as M)

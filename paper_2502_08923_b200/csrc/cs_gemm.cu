@@ -331,13 +331,23 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
     // ------------------------------------------------------------- epilogue warps 0-3: wait for the accumulators
     asm volatile("griddepcontrol.wait;" ::: "memory");
     if (a.nf.ssq_in != nullptr) {
-      // 1/rms of every token row while the main loop runs: slots summed in a fixed order
-      for (int tok = warp; tok < a.rows; tok += 4) {
-        float ss = 0.f;
-        for (int sl = lane; sl < a.nf.slots_in; sl += 32) ss += a.nf.ssq_in[(size_t)tok * a.nf.slot_stride + sl];
+      // 1/rms of every token row while the main loop runs: slots summed in a fixed order.  Eight
+      // rows at a time, so that a tall block's loads overlap instead of queueing row after row.
+      for (int tok0 = warp * 8; tok0 < a.rows; tok0 += 32) {
+        float ss[8];
 #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
-        if (lane == 0) rstd_s[tok] = rsqrtf(ss * a.nf.inv_d + a.nf.eps);
+        for (int r = 0; r < 8; ++r) ss[r] = 0.f;
+        for (int sl = lane; sl < a.nf.slots_in; sl += 32) {
+#pragma unroll
+          for (int r = 0; r < 8; ++r)
+            if (tok0 + r < a.rows) ss[r] += a.nf.ssq_in[(size_t)(tok0 + r) * a.nf.slot_stride + sl];
+        }
+#pragma unroll
+        for (int r = 0; r < 8; ++r) {
+#pragma unroll
+          for (int off = 16; off > 0; off >>= 1) ss[r] += __shfl_xor_sync(0xffffffffu, ss[r], off);
+          if (lane == 0 && tok0 + r < a.rows) rstd_s[tok0 + r] = rsqrtf(ss[r] * a.nf.inv_d + a.nf.eps);
+        }
       }
       asm volatile("bar.sync 1, 128;" ::: "memory");
     }
@@ -723,6 +733,41 @@ cs_status cs_gemm_plan(cs_ctx* ctx, GemmPlan* g, const void* w, int N, int K, bo
   return encode_2d(ctx, &g->tmW, w, N, K, CS_GEMM_BM, true);
 }
 
+static cs_status ensure_gemm_attrs(cs_ctx* ctx) {
+  if (!ctx->gemm_attr_set) {
+    CS_CUDA_OK(ctx, cudaFuncSetAttribute(k_gemm_tc<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+    CS_CUDA_OK(ctx, cudaFuncSetAttribute(k_gemm_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+    CS_CUDA_OK(ctx, cudaFuncSetAttribute(k_gemm_tc<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+    ctx->gemm_attr_set = true;
+  }
+  return CS_OK;
+}
+
+// How many clusters of `spl` one-CTA-per-SM CTAs the device runs at once.  A cluster has to find
+// all its CTAs inside one GPC, so this can be well below SMs / spl: 48 clusters of 3 do not fit
+// on 148 SMs, and a launch that needs them takes two waves.  Asked of the runtime once per shape.
+static int tall_clusters_at_once(const cs_ctx* cctx, int mt, int spl, int smem) {
+  cs_ctx* ctx = const_cast<cs_ctx*>(cctx);
+  if (spl <= 1) return ctx->num_sms;
+  int& slot = ctx->tall_clusters[mt == 4 ? 2 : (mt == 2 ? 1 : 0)][spl];
+  if (slot == 0) {
+    int n = 0;
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3(ctx->num_sms, spl, 1);
+    lc.blockDim = dim3(kThreads, 1, 1);
+    lc.dynamicSmemBytes = (size_t)smem;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 1; at[0].val.clusterDim.y = spl; at[0].val.clusterDim.z = 1;
+    lc.attrs = at;
+    lc.numAttrs = 1;
+    void (*kernel)(const CUtensorMap, const CUtensorMap, GemmArgs) = mt == 4 ? k_gemm_tc<4> : (mt == 2 ? k_gemm_tc<2> : k_gemm_tc<1>);
+    if (ensure_gemm_attrs(ctx) == CS_OK && cudaOccupancyMaxActiveClusters(&n, kernel, &lc) == cudaSuccess && n > 0) slot = n;
+    else { (void)cudaGetLastError(); slot = max(1, ctx->num_sms * 85 / 100 / spl); }   // no answer: the planner's allowance
+  }
+  return slot;
+}
+
 // Launch shape of one GEMM for a block of `rows` token rows.
 //  - Short blocks (two CTAs fit on an SM): one 128-feature tile per CTA and the plan's split-K
 //    factor, made for two CTAs per SM - the HBM-bound regime of 11-row blocks.
@@ -778,7 +823,7 @@ cs_status cs_gemm_shape(const cs_ctx* ctx, const GemmPlan* g, int rows, bool two
       const int smax = g->allow_split ? max(1, min(CS_MAX_SPLITS, kb / 4)) : 1;
       for (int sp = 1; sp <= smax; ++sp) {
         const int kps = cs_ceil_div(kb, sp), spl = cs_ceil_div(kb, kps);
-        const long waves = cs_ceil_div(ctas * spl, ctx->num_sms);
+        const long waves = cs_ceil_div(ctas, tall_clusters_at_once(ctx, mt, spl, fixed + st * sb));
         const long cost = waves * ((long)kps * per_kb + epi);
         if (best < 0 || cost < best) {
           best = cost;
@@ -846,11 +891,9 @@ cs_status cs_launch_gemm(cs_ctx* ctx, const GemmPlan* g, const CUtensorMap* tmX,
   }
   void (*kernel)(const CUtensorMap, const CUtensorMap, GemmArgs) =
       sh.mt == 4 ? k_gemm_tc<4> : (sh.mt == 2 ? k_gemm_tc<2> : k_gemm_tc<1>);
-  if (!ctx->gemm_attr_set) {
-    CS_CUDA_OK(ctx, cudaFuncSetAttribute(k_gemm_tc<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-    CS_CUDA_OK(ctx, cudaFuncSetAttribute(k_gemm_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-    CS_CUDA_OK(ctx, cudaFuncSetAttribute(k_gemm_tc<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-    ctx->gemm_attr_set = true;
+  {
+    const cs_status as = ensure_gemm_attrs(ctx);
+    if (as != CS_OK) return as;
   }
   cudaLaunchConfig_t lc = {};
   lc.gridDim = dim3(tiles, a.splits, 1);

@@ -163,7 +163,9 @@ k_embed_rmsnorm(const __nv_bfloat16* __restrict__ E, const int* __restrict__ row
   }
 }
 
-// Combine the key slices: o = sum_s o_s e^(m_s - M) / sum_s l_s e^(m_s - M).
+// Combine the key slices: o = sum_s o_s e^(m_s - M) / sum_s l_s e^(m_s - M).  NS = an upper
+// bound of the slice count known at compile time, so the loads and the sum are unrolled to it.
+template <int NS>
 __global__ void k_attn_merge(const float* __restrict__ in_o, const float* __restrict__ in_ml, int nsplit,
                              int rows, int H, int Dh, __nv_bfloat16* __restrict__ attn_out,
                              unsigned long long* stamp) {
@@ -171,13 +173,13 @@ __global__ void k_attn_merge(const float* __restrict__ in_o, const float* __rest
   const int row = blockIdx.x, h = blockIdx.y, dd = threadIdx.x;
   const int lane = threadIdx.x & 31;
   // all partial outputs of this (row, head, dim) are requested at once, so their latencies
-  // overlap each other and the weight computation below (at most 64 key slices)
-  float v[64];
+  // overlap each other and the weight computation below
+  float v[NS];
   {
     const size_t stride = (size_t)rows * H * Dh;
     const float* src = in_o + ((size_t)row * H + h) * Dh + dd;
 #pragma unroll
-    for (int s = 0; s < 64; ++s) v[s] = (s < nsplit) ? src[(size_t)s * stride] : 0.f;
+    for (int s = 0; s < NS; ++s) v[s] = (s < nsplit) ? src[(size_t)s * stride] : 0.f;
   }
   // every warp works out the slice weights e^(m_s - M) / L itself: lane s owns slices s, s+32
   float m0 = -INFINITY, l0 = 0.f, m1 = -INFINITY, l1 = 0.f;
@@ -185,7 +187,7 @@ __global__ void k_attn_merge(const float* __restrict__ in_o, const float* __rest
     const size_t base = ((size_t)lane * rows + row) * H + h;
     m0 = in_ml[base * 2]; l0 = in_ml[base * 2 + 1];
   }
-  if (lane + 32 < nsplit) {
+  if (NS > 32 && lane + 32 < nsplit) {
     const size_t base = ((size_t)(lane + 32) * rows + row) * H + h;
     m1 = in_ml[base * 2]; l1 = in_ml[base * 2 + 1];
   }
@@ -198,7 +200,7 @@ __global__ void k_attn_merge(const float* __restrict__ in_o, const float* __rest
   w0 *= inv; w1 *= inv;
   float acc = 0.f;
 #pragma unroll
-  for (int s = 0; s < 64; ++s) {
+  for (int s = 0; s < NS; ++s) {
     const float w = __shfl_sync(0xffffffffu, s < 32 ? w0 : w1, s & 31);
     acc = fmaf(v[s], w, acc);
   }
@@ -419,7 +421,10 @@ void cs_launch_embed_rmsnorm(cs_ctx* ctx, const __nv_bfloat16* gain, int rows, c
 
 void cs_launch_attn_merge(cs_ctx* ctx, int nsplit, int rows, cudaStream_t st) {
   const cs_model_config& c = ctx->cfg;
-  cs_launch_pdl(k_attn_merge, dim3(rows, c.n_heads), dim3(c.head_dim), 0, st, ctx->attn_o, ctx->attn_ml, nsplit, rows,
+  auto kernel = nsplit <= 1 ? k_attn_merge<1> : nsplit <= 2 ? k_attn_merge<2> : nsplit <= 4 ? k_attn_merge<4>
+              : nsplit <= 8 ? k_attn_merge<8> : nsplit <= 16 ? k_attn_merge<16> : nsplit <= 32 ? k_attn_merge<32>
+              : nsplit <= 48 ? k_attn_merge<48> : k_attn_merge<64>;
+  cs_launch_pdl(kernel, dim3(rows, c.n_heads), dim3(c.head_dim), 0, st, ctx->attn_o, ctx->attn_ml, nsplit, rows,
                 c.n_heads, c.head_dim, ctx->attn_out, cs_next_stamp(ctx, CS_FAM_MERGE));
 }
 
