@@ -132,14 +132,16 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
 }
 // eight accumulator columns of this thread's lane (no wait: several loads share one wait)
 __device__ __forceinline__ void tmem_ld8_nowait(uint32_t taddr, float* v) {
-  uint32_t r[8];
   asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7])
                : "r"(taddr));
-#pragma unroll
-  for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// The loaded registers are only valid after the wait, which the compiler cannot know: this empty
+// statement, placed behind the wait, redefines them, so no use of theirs is scheduled ahead of it.
+__device__ __forceinline__ void tmem_landed8(float* v) {
+  asm volatile("" : "+f"(v[0]), "+f"(v[1]), "+f"(v[2]), "+f"(v[3]), "+f"(v[4]), "+f"(v[5]), "+f"(v[6]), "+f"(v[7])::"memory");
+}
 __device__ __forceinline__ void tmem_st8(uint32_t taddr, const float* v) {
   asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
                ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
@@ -234,7 +236,7 @@ k_attn_tcw(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUt
   }
   const uint32_t b_kfull = smem_u32(bars), b_kfree = smem_u32(bars + 2), b_vfull = smem_u32(bars + 4),
                  b_vfree = smem_u32(bars + 6), b_qfull = smem_u32(bars + 8), b_sready = smem_u32(bars + 9),
-                 b_pready = smem_u32(bars + 11), b_odone = smem_u32(bars + 12);   // b_odone: two barriers, by tile parity
+                 b_pready = smem_u32(bars + 14), b_odone = smem_u32(bars + 12);   // b_pready (bars 14, 15) and b_odone: two barriers each, by tile parity
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int b = blockIdx.x / a.Hkv, kvh = blockIdx.x % a.Hkv, split = blockIdx.y;
@@ -252,7 +254,7 @@ k_attn_tcw(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUt
       mbar_init(b_sready + 8 * s, 1);
     }
     mbar_init(b_qfull, 1);
-    mbar_init(b_pready, 256);
+    mbar_init(b_pready, 256); mbar_init(b_pready + 8, 256);
     mbar_init(b_odone, 1); mbar_init(b_odone + 8, 1);
     *s_abort = 0; *s_never = 0; *s_lmax = 0; *s_limmin = 0x7fffffff;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -393,10 +395,12 @@ k_attn_tcw(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUt
       for (int i = 0; i < ntl && ok; ++i) {
         // the scores of the next tile go first: they run during this tile's softmax.  (Its S^T buffer
         // was last read by the softmax of tile i - 1, which had finished before P^T of tile i - 1 was
-        // signalled.)
+        // signalled.)  A column group whose tiles are quick - all its rows masked - can therefore be
+        // a tile ahead of the other one, which is why "P^T written" has a barrier per tile parity: it
+        // cannot be two ahead, because the scores of tile i + 2 are only issued after P^T of tile i.
         if (i + 1 < ntl && !issue_scores(i + 1)) { ok = false; break; }
         const int s = i % vstages;
-        if (!mbar_wait(b_pready, (uint32_t)i & 1u, s_abort, a.wait_ns) ||
+        if (!mbar_wait(b_pready + 8 * (i & 1), (uint32_t)(i >> 1) & 1u, s_abort, a.wait_ns) ||
             !mbar_wait(b_vfull + 8 * s, (uint32_t)(i / vstages) & 1u, s_abort, a.wait_ns)) { ok = false; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t av = smem_u32(sV + (size_t)s * 2 * kHalfBytes);
@@ -457,11 +461,17 @@ k_attn_tcw(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUt
             float w[8];
             tmem_ld8_nowait(s_addr + (uint32_t)NQ + 8 * c, w);
             tmem_ld_wait();
+            tmem_landed8(w);
+            tmem_landed8(v + 8 * c);                     // (requested before w: landed as well)
 #pragma unroll
             for (int j = 0; j < 8; ++j) v[8 * c + j] += w[j];
           }
+      } else {
+        tmem_ld_wait();
+#pragma unroll
+        for (int c = 0; c < kCols / 8; ++c)
+          if (c < nch) tmem_landed8(v + 8 * c);
       }
-      tmem_ld_wait();
       if (!whole) {
 #pragma unroll
         for (int c = 0; c < kCols / 8; ++c)
@@ -488,7 +498,9 @@ k_attn_tcw(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUt
       if (i >= a.pbufs)
         ok = mbar_wait(b_odone + 8 * ((i - a.pbufs) & 1), (uint32_t)((i - a.pbufs) >> 1) & 1u, s_abort, a.wait_ns) && ok;
       const bool bad = !ok || *s_abort != 0;
-      if (group_any(1 + half, exceed || bad)) {
+      const bool moved = group_any(1 + half, exceed || bad);
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");   // (the waits above order the reads of O^T below)
+      if (moved) {
         // ---- the rare path: the true maxima of the tile, new reference points where needed
         if (!group_all(1 + half, !bad)) { *s_abort = 1; have = false; break; }   // the same decision in every thread of the group
         float* red_w = s_red + (sp * 8 + warp) * kCols;
@@ -549,6 +561,7 @@ k_attn_tcw(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUt
                   float o[8];
                   tmem_ld8_nowait(lane_base + ocol + (uint32_t)(t * NQ + q0 + 8 * c), o);
                   tmem_ld_wait();
+                  tmem_landed8(o);
 #pragma unroll
                   for (int j = 0; j < 8; ++j) o[j] *= cr[j];
                   tmem_st8(lane_base + ocol + (uint32_t)(t * NQ + q0 + 8 * c), o);
@@ -611,7 +624,7 @@ k_attn_tcw(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUt
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      mbar_arrive(b_pready);
+      mbar_arrive(b_pready + 8 * sp);
     }
     // ---- un-normalised result of this key slice
     if (have) {
@@ -630,6 +643,8 @@ k_attn_tcw(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUt
           tmem_ld8_nowait(lane_base + ocol + (uint32_t)(q0 + 8 * c), o);
           tmem_ld8_nowait(lane_base + ocol + (uint32_t)(NQ + q0 + 8 * c), w);
           tmem_ld_wait();
+          tmem_landed8(o);
+          tmem_landed8(w);
 #pragma unroll
           for (int j = 0; j < 8; ++j) o[j] += w[j];
         } else {

@@ -144,6 +144,8 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
         "=r"(v[15])
       : "r"(taddr));
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+  // the registers are valid only from here on: an empty statement that redefines them keeps their uses behind the wait
+  asm volatile("" : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]), "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15]) :: "memory");
 }
 // the two halves of the cluster barrier; like every barrier they count whole warps, so each
 // warp executes each half exactly once, with all its lanes converged
@@ -563,47 +565,70 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
         const bool feeds_norm = a.mode == CS_EPI_RESIDUAL && a.nf.gain_out != nullptr;
         float* part = dump + a.n_tok * CS_GEMM_BM;   // [rows][32] sums of squares, behind the parked tile
         const int total = per_tok * a.rows, iters = (total + 127) >> 7;
-        for (int it = 0; it < iters; ++it) {
-          const int idx = e + (it << 7);
-          const bool act = idx < total;
-          const int idc = act ? idx : 0;
-          const int f = f_lo + 4 * (idc % per_tok), tok = idc / per_tok;
-          float4 y = make_float4(0.f, 0.f, 0.f, 0.f);
-          if (a.splits > 1) {
-            if (act) y = sum_over_ranks(dump_addr + 4u * (uint32_t)(tok * CS_GEMM_BM + f), a.splits);
-            if (it == iters - 1) { keep_alive(y, y); cluster_arrive(); arrived = true; }
-          } else if (act) {
-            y = *reinterpret_cast<const float4*>(dump + tok * CS_GEMM_BM + f);
+        const bool vec_n = (a.N & 3) == 0;
+        // Two items per turn: the remote reads and the residual reads of both are requested before
+        // either is finished, so a tall block's dozen turns per thread overlap pairwise (128 threads
+        // on an otherwise idle SM have nothing else to hide those latencies behind).
+        for (int it = 0; it < iters; it += 2) {
+          int idx[2], f[2], tok[2];
+          bool act[2], vec[2];
+          float4 y[2], x[2];
+#pragma unroll
+          for (int u = 0; u < 2; ++u) {
+            idx[u] = e + ((it + u) << 7);
+            act[u] = it + u < iters && idx[u] < total;
+            const int idc = act[u] ? idx[u] : 0;
+            f[u] = f_lo + 4 * (idc % per_tok);
+            tok[u] = idc / per_tok;
+            vec[u] = vec_n && n0 + f[u] + 3 < a.N;
+            y[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+            x[u] = y[u];
           }
-          if (!act) continue;
-          if (feeds_norm) part[tok * 32 + idx % per_tok] = 0.f;
-          const float yv[4] = {y.x, y.y, y.z, y.w};
-          float* dst = a.out + (size_t)tok * a.N + n0 + f;
-          if (n0 + f + 3 < a.N && (a.N & 3) == 0) {
-            float4 o = y;
-            if (a.mode == CS_EPI_RESIDUAL) {
-              const float4 x = (it == 0) ? x_pre : *reinterpret_cast<const float4*>(dst);
-              o.x += x.x; o.y += x.y; o.z += x.z; o.w += x.w;
-            }
-            *reinterpret_cast<float4*>(dst) = o;
-            if (feeds_norm) {
-              const uint2 gw = *reinterpret_cast<const uint2*>(a.nf.gain_out + n0 + f);
-              const float2 g01 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&gw.x));
-              const float2 g23 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&gw.y));
-              const float w0 = o.x * g01.x, w1 = o.y * g01.y, w2 = o.z * g23.x, w3 = o.w * g23.y;
-              __nv_bfloat162 h[2], l[2];
-              h[0] = __floats2bfloat162_rn(w0, w1); h[1] = __floats2bfloat162_rn(w2, w3);
-              const float2 h0 = __bfloat1622float2(h[0]), h1 = __bfloat1622float2(h[1]);
-              l[0] = __floats2bfloat162_rn(w0 - h0.x, w1 - h0.y); l[1] = __floats2bfloat162_rn(w2 - h1.x, w3 - h1.y);
-              __nv_bfloat16* xo = a.nf.xn_out + (size_t)tok * a.N + n0 + f;
-              *reinterpret_cast<uint2*>(xo) = *reinterpret_cast<const uint2*>(h);
-              *reinterpret_cast<uint2*>(xo + (size_t)CS_MAX_ROWS * a.N) = *reinterpret_cast<const uint2*>(l);
-              part[tok * 32 + idx % per_tok] = (o.x * o.x + o.y * o.y) + (o.z * o.z + o.w * o.w);
-            }
+          if (a.splits > 1) {
+#pragma unroll
+            for (int u = 0; u < 2; ++u)
+              if (act[u]) y[u] = sum_over_ranks(dump_addr + 4u * (uint32_t)(tok[u] * CS_GEMM_BM + f[u]), a.splits);
           } else {
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
-              if (n0 + f + i < a.N) dst[i] = (a.mode == CS_EPI_RESIDUAL) ? dst[i] + yv[i] : yv[i];
+            for (int u = 0; u < 2; ++u)
+              if (act[u]) y[u] = *reinterpret_cast<const float4*>(dump + tok[u] * CS_GEMM_BM + f[u]);
+          }
+          if (a.mode == CS_EPI_RESIDUAL) {
+#pragma unroll
+            for (int u = 0; u < 2; ++u)
+              if (act[u] && vec[u])
+                x[u] = (it + u == 0) ? x_pre : *reinterpret_cast<const float4*>(a.out + (size_t)tok[u] * a.N + n0 + f[u]);
+          }
+          if (a.splits > 1 && it + 2 >= iters) { keep_alive(y[0], y[1]); cluster_arrive(); arrived = true; }
+#pragma unroll
+          for (int u = 0; u < 2; ++u) {
+            if (!act[u]) continue;
+            if (feeds_norm) part[tok[u] * 32 + idx[u] % per_tok] = 0.f;
+            float* dst = a.out + (size_t)tok[u] * a.N + n0 + f[u];
+            if (vec[u]) {
+              float4 o = y[u];
+              o.x += x[u].x; o.y += x[u].y; o.z += x[u].z; o.w += x[u].w;   // (x stays 0 unless this is a residual update)
+              *reinterpret_cast<float4*>(dst) = o;
+              if (feeds_norm) {
+                const uint2 gw = *reinterpret_cast<const uint2*>(a.nf.gain_out + n0 + f[u]);
+                const float2 g01 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&gw.x));
+                const float2 g23 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&gw.y));
+                const float w0 = o.x * g01.x, w1 = o.y * g01.y, w2 = o.z * g23.x, w3 = o.w * g23.y;
+                __nv_bfloat162 h[2], l[2];
+                h[0] = __floats2bfloat162_rn(w0, w1); h[1] = __floats2bfloat162_rn(w2, w3);
+                const float2 h0 = __bfloat1622float2(h[0]), h1 = __bfloat1622float2(h[1]);
+                l[0] = __floats2bfloat162_rn(w0 - h0.x, w1 - h0.y); l[1] = __floats2bfloat162_rn(w2 - h1.x, w3 - h1.y);
+                __nv_bfloat16* xo = a.nf.xn_out + (size_t)tok[u] * a.N + n0 + f[u];
+                *reinterpret_cast<uint2*>(xo) = *reinterpret_cast<const uint2*>(h);
+                *reinterpret_cast<uint2*>(xo + (size_t)CS_MAX_ROWS * a.N) = *reinterpret_cast<const uint2*>(l);
+                part[tok[u] * 32 + idx[u] % per_tok] = (o.x * o.x + o.y * o.y) + (o.z * o.z + o.w * o.w);
+              }
+            } else {
+              const float yv[4] = {y[u].x, y[u].y, y[u].z, y[u].w};
+#pragma unroll
+              for (int i = 0; i < 4; ++i)
+                if (n0 + f[u] + i < a.N) dst[i] = (a.mode == CS_EPI_RESIDUAL) ? dst[i] + yv[i] : yv[i];
+            }
           }
         }
         if (feeds_norm) {

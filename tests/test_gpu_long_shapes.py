@@ -196,6 +196,18 @@ def test_attention_variants_over_many_key_tiles(narrow, B, k, kv_max, label):
     run_verify(NARROW, w_gpu, model, B, k, kv_lens, draft_lens, seed=B * 1000 + k)
 
 
+@pytest.mark.parametrize("seed", [31, 32, 33])
+def test_one_column_group_fully_masked(narrow, seed):
+    """Short drafts in most sequences: the upper half of the query columns of their CTAs is masked
+    throughout, so that half of the softmax threads finishes its tiles much sooner than the half that
+    works out maxima - the two halves must still hand every tile over together."""
+    _, w_gpu, model = narrow
+    rng = np.random.default_rng(seed)
+    kv_lens = [3100] + [int(x) for x in rng.integers(2200, 3101, size=15)]
+    draft_lens = [10] + [int(x) for x in rng.integers(0, 4, size=15)]
+    run_verify(NARROW, w_gpu, model, 16, 10, kv_lens, draft_lens, seed=seed)
+
+
 def test_attention_variants_inside_the_loop(narrow):
     """The same variants with the step graph and the early tile requests of the loop."""
     _, w_gpu, model = narrow
