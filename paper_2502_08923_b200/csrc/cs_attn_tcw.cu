@@ -43,14 +43,15 @@
 
 namespace {
 
-constexpr int kThreads = 352;   // warps 0-7 softmax/epilogue, warp 8 K/Q producer, warp 9 MMA, warp 10 V producer
-constexpr int kProdWarp = 8, kMmaWarp = 9, kVProdWarp = 10;   // (a warp of its own each: a lane that sleeps in a
+constexpr int kSoftWarps = 12, kSoftThreads = kSoftWarps * 32;   // three column groups of four warps (one per TMEM lane quarter)
+constexpr int kThreads = 480;   // warps 0-11 softmax/epilogue, warp 12 K/Q producer, warp 13 MMA, warp 14 V producer
+constexpr int kProdWarp = 12, kMmaWarp = 13, kVProdWarp = 14;   // (a warp of its own each: a lane that sleeps in a
                                                               //  barrier wait would hold up the other lanes of its warp)
 constexpr int kTileKeys = 128;
 constexpr int kDh = 128;
 constexpr int kHalfBytes = kTileKeys * 128;          // one [128 keys x 64 dims] half tile (also one P^T atom)
 constexpr int kNQMax = 96;                           // query rows per CTA
-constexpr int kCols = kNQMax / 2;                    // query columns per softmax thread, at most
+constexpr int kCols = kNQMax / 3;                    // query columns per softmax thread, at most
 constexpr int kCtlBytes = 192;                       // 16 mbarriers + TMEM slot + flags
 
 struct AttnArgs {
@@ -186,7 +187,7 @@ __device__ __forceinline__ void split8(const float* p, uint4& hi, uint4& lo) {
   hi = make_uint4(h[0], h[1], h[2], h[3]);
   lo = make_uint4(l[0], l[1], l[2], l[3]);
 }
-// barrier of one half of the softmax threads (128 threads, ids 1 and 2) that also ANDs a predicate:
+// barrier of one column group of the softmax threads (128 threads, ids 1 to 3) that also ANDs a predicate:
 // every thread learns whether all of them are still fine, so they leave their loops together
 __device__ __forceinline__ bool group_all(int id, bool pred) {
   uint32_t out;
@@ -228,9 +229,9 @@ k_attn_tcw(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUt
   int* s_lmax = reinterpret_cast<int*>(tmem_slot + 3);
   int* s_limmin = reinterpret_cast<int*>(tmem_slot + 4);     // fewest keys any live query row of the group attends to
   int* s_lim = reinterpret_cast<int*>(ctl + kCtlBytes);                 // [NQ] keys each query row attends to
-  float* s_priv = reinterpret_cast<float*>(s_lim + kNQMax);             // [8 warps][3][kCols] each warp's copy of its columns' reference points
-  float* s_red = reinterpret_cast<float*>(s_priv + 8 * 3 * kCols);      // [2][8 warps][kCols] per-warp column maxima / sums, by tile parity
-  if ((size_t)(reinterpret_cast<uint8_t*>(s_red + 2 * 8 * kCols) - smem_raw) > (size_t)a.smem_bytes) {
+  float* s_priv = reinterpret_cast<float*>(s_lim + kNQMax);             // [12 warps][3][kCols] each warp's copy of its columns' reference points
+  float* s_red = reinterpret_cast<float*>(s_priv + kSoftWarps * 3 * kCols);   // [2][12 warps][kCols] per-warp column maxima / sums, by tile parity
+  if ((size_t)(reinterpret_cast<uint8_t*>(s_red + 2 * kSoftWarps * kCols) - smem_raw) > (size_t)a.smem_bytes) {
     if (threadIdx.x == 0) atomicOr(a.status, CS_DEV_SMEM);   // the launcher sizes the window for exactly this layout
     return;
   }
@@ -254,7 +255,7 @@ k_attn_tcw(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUt
       mbar_init(b_sready + 8 * s, 1);
     }
     mbar_init(b_qfull, 1);
-    mbar_init(b_pready, 256); mbar_init(b_pready + 8, 256);
+    mbar_init(b_pready, kSoftThreads); mbar_init(b_pready + 8, kSoftThreads);
     mbar_init(b_odone, 1); mbar_init(b_odone + 8, 1);
     *s_abort = 0; *s_never = 0; *s_lmax = 0; *s_limmin = 0x7fffffff;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -301,9 +302,9 @@ k_attn_tcw(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUt
   }
   asm volatile("griddepcontrol.wait;" ::: "memory");
 
-  if (warp < 8) {
+  if (warp < kSoftWarps) {
     int lm = 0, ln = 0x7fffffff;
-    for (int r = tid; r < Rcur; r += 256) {
+    for (int r = tid; r < Rcur; r += kSoftThreads) {
       const int v = a.row_lim[b * R + r0 + r];
       lm = max(lm, v);
       ln = min(ln, v);
@@ -312,7 +313,7 @@ k_attn_tcw(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUt
     ln = __reduce_min_sync(0xffffffffu, ln);
     if (lane == 0 && lm > 0) atomicMax(s_lmax, lm);
     if (lane == 0) atomicMin(s_limmin, ln);
-    for (int q = tid; q < NQ; q += 256) {
+    for (int q = tid; q < NQ; q += kSoftThreads) {
       s_lim[q] = (q < nq) ? a.row_lim[b * R + r0 + q / G] : 0;
     }
   }
@@ -416,10 +417,10 @@ k_attn_tcw(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUt
   } else {
     // ------------------------------------------------------------------ softmax + epilogue
     // thread = one TMEM lane (a key of the tile for S^T, a head dim for O^T) and half of the columns
-    const int wq = warp & 3, half = warp >> 2;
+    const int wq = warp & 3, grp = warp >> 2;
     const int row = wq * 32 + lane;                    // TMEM lane of this thread
-    const int ncol = NQ >> 1, nch = ncol >> 3;         // this thread's columns, in chunks of 8
-    const int q0 = half * ncol;
+    const int ncol = NQ / 3, nch = ncol >> 3;          // this thread's columns (8, 16, 24 or 32), in chunks of 8
+    const int q0 = grp * ncol;
     const uint32_t lane_base = tmem_base + ((uint32_t)(wq * 32) << 16);
     const float sc = a.scale_log2e;
     float lsum[kCols];                                 // this key lane's share of every column's sum
@@ -498,30 +499,24 @@ k_attn_tcw(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUt
       if (i >= a.pbufs)
         ok = mbar_wait(b_odone + 8 * ((i - a.pbufs) & 1), (uint32_t)((i - a.pbufs) >> 1) & 1u, s_abort, a.wait_ns) && ok;
       const bool bad = !ok || *s_abort != 0;
-      const bool moved = group_any(1 + half, exceed || bad);
+      const bool moved = group_any(1 + grp, exceed || bad);
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");   // (the waits above order the reads of O^T below)
       if (moved) {
         // ---- the rare path: the true maxima of the tile, new reference points where needed
-        if (!group_all(1 + half, !bad)) { *s_abort = 1; have = false; break; }   // the same decision in every thread of the group
-        float* red_w = s_red + (sp * 8 + warp) * kCols;
+        if (!group_all(1 + grp, !bad)) { *s_abort = 1; have = false; break; }   // the same decision in every thread of the group
+        float* red_w = s_red + (sp * kSoftWarps + warp) * kCols;
         {
           float x[32];
 #pragma unroll
           for (int j = 0; j < 32; ++j) x[j] = (j < ncol) ? v[j] : -INFINITY;
           const float r = warp_max32(x, lane);
           if (lane < ncol) red_w[lane] = r;
-          if (nch > 4) {                                 // columns 32 .. 47
-#pragma unroll
-            for (int j = 0; j < 32; ++j) x[j] = (j + 32 < kCols && j + 32 < ncol) ? v[(j + 32 < kCols) ? j + 32 : 0] : -INFINITY;
-            const float r1 = warp_max32(x, lane);
-            if (lane + 32 < ncol) red_w[32 + lane] = r1;
-          }
         }
-        group_all(1 + half, true);
-        const float* red = s_red + (sp * 8 + half * 4) * kCols;
-        // lane j works columns j and j + 32 out; the other lanes get the factors by shuffle
-        float mnA = -INFINITY, crA = 1.f, mnB = -INFINITY, crB = 1.f;
-        bool mvA = false, mvB = false;
+        group_all(1 + grp, true);
+        const float* red = s_red + (sp * kSoftWarps + grp * 4) * kCols;
+        // lane j works column j out; the other lanes get the factors by shuffle
+        float mnA = -INFINITY, crA = 1.f;
+        bool mvA = false;
         if (lane < ncol && q0 + lane < nq) {
           const float t = fmaxf(fmaxf(red[lane], red[kCols + lane]), fmaxf(red[2 * kCols + lane], red[3 * kCols + lane])) * sc;
           const float mo = w_mo[lane];                   // (sc > 0: scaling commutes with the maximum)
@@ -529,25 +524,17 @@ k_attn_tcw(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUt
           mnA = mvA ? t : mo;
           crA = mvA ? ((mo == -INFINITY) ? 0.f : ex2(mo - t)) : 1.f;
         }
-        if (nch > 4 && lane + 32 < ncol && q0 + lane + 32 < nq) {
-          const int col = lane + 32;
-          const float t = fmaxf(fmaxf(red[col], red[kCols + col]), fmaxf(red[2 * kCols + col], red[3 * kCols + col])) * sc;
-          const float mo = w_mo[col];
-          mvB = (mo == -INFINITY) ? (t > mo) : (t > mo + 8.f);
-          mnB = mvB ? t : mo;
-          crB = mvB ? ((mo == -INFINITY) ? 0.f : ex2(mo - t)) : 1.f;
-        }
-        const unsigned grewA = __ballot_sync(0xffffffffu, mvA), grewB = __ballot_sync(0xffffffffu, mvB);
+        const unsigned grewA = __ballot_sync(0xffffffffu, mvA);
         bool prev_done = a.pbufs == 1;                   // is the P V product of tile i - 1 known to have retired?
 #pragma unroll
         for (int c = 0; c < kCols / 8; ++c) {
           if (c < nch) {
-            const bool grew = (((c < 4 ? grewA : grewB) >> ((8 * c) & 31)) & 0xffu) != 0;   // the same in every thread of the group
+            const bool grew = ((grewA >> (8 * c)) & 0xffu) != 0;   // the same in every thread of the group
             if (grew) {
               float cr[8];
 #pragma unroll
               for (int j = 0; j < 8; ++j) {
-                cr[j] = __shfl_sync(0xffffffffu, c < 4 ? crA : crB, (8 * c + j) & 31);
+                cr[j] = __shfl_sync(0xffffffffu, crA, 8 * c + j);
                 lsum[8 * c + j] *= cr[j];
               }
               if (i > 0) {
@@ -575,11 +562,6 @@ k_attn_tcw(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUt
           w_mo[lane] = mnA;
           w_thr[lane] = (mnA + 8.f) / sc;
           w_nme[lane] = (mnA == -INFINITY) ? -INFINITY : -mnA;
-        }
-        if (nch > 4 && lane + 32 < ncol && q0 + lane + 32 < nq) {
-          w_mo[lane + 32] = mnB;
-          w_thr[lane + 32] = (mnB + 8.f) / sc;
-          w_nme[lane + 32] = (mnB == -INFINITY) ? -INFINITY : -mnB;
         }
         __syncwarp();
       }
@@ -614,7 +596,7 @@ k_attn_tcw(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUt
         const int s = i % vstages;
         if (!mbar_wait(b_vfull + 8 * s, (uint32_t)(i / vstages) & 1u, s_abort, a.wait_ns)) *s_abort = 1;
         uint8_t* vs = sV + (size_t)s * 2 * kHalfBytes;
-        for (int rr = max(lmax - tile0, 0) + (warp * 32 + lane); rr < kTileKeys; rr += 256) {
+        for (int rr = max(lmax - tile0, 0) + (warp * 32 + lane); rr < kTileKeys; rr += kSoftThreads) {
 #pragma unroll
           for (int c = 0; c < 8; ++c) {
             *reinterpret_cast<uint4*>(vs + (size_t)rr * 128 + c * 16) = make_uint4(0u, 0u, 0u, 0u);
@@ -629,7 +611,7 @@ k_attn_tcw(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUt
     // ---- un-normalised result of this key slice
     if (have) {
       bool ok = mbar_wait(b_odone + 8 * ((ntl - 1) & 1), (uint32_t)((ntl - 1) >> 1) & 1u, s_abort, a.wait_ns);
-      ok = group_all(1 + half, ok && *s_abort == 0);
+      ok = group_all(1 + grp, ok && *s_abort == 0);
       if (!ok) { *s_abort = 1; have = false; }
     }
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -675,10 +657,10 @@ k_attn_tcw(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUt
         }
       }
     }
-    group_all(1 + half, true);
+    group_all(1 + grp, true);
     if (wq == 0) {
-      const float* red = s_red + (half * 4) * kCols;
-      const float* m_fin = w_mo;                       // (warp 4 * half: its own copy)
+      const float* red = s_red + (grp * 4) * kCols;
+      const float* m_fin = w_mo;                       // (warp 4 * grp: its own copy)
       constexpr float kLn2 = 0.6931471805599453f;
       for (int col = lane; col < ncol; col += 32) {
         const int q = q0 + col;
@@ -714,7 +696,7 @@ int cs_launch_attention_tcw(cs_ctx* ctx, const void* kv_cache, int layer, int B,
   const int ngroups = cs_ceil_div(G * R, kNQMax), Rg = cs_ceil_div(R, ngroups);
   if (G * Rg > kNQMax) return 0;
   const int nq = G * Rg;
-  const int NQ = (nq + 15) / 16 * 16;
+  const int NQ = (nq + 23) / 24 * 24;                  // three column groups of whole 8-column chunks
   if (ctx->tmKV_base != kv_cache) {
     const unsigned long long rows = (unsigned long long)c.n_layers * 2 * c.max_batch * c.n_kv_heads * c.max_seq;
     if (rows > 0x7fffffffull) return 0;
@@ -735,7 +717,7 @@ int cs_launch_attention_tcw(cs_ctx* ctx, const void* kv_cache, int layer, int B,
   const size_t natoms = (size_t)(2 * NQ + 63) / 64;
   const size_t base = 1024 + (size_t)4 * NQ * 128 + (size_t)2 * 2 * kHalfBytes;
   const size_t pbuf = natoms * kHalfBytes, vstage = (size_t)2 * kHalfBytes;
-  const size_t ctl = (size_t)kCtlBytes + kNQMax * 4 + 8 * 3 * kCols * 4 + 2 * 8 * kCols * 4;
+  const size_t ctl = (size_t)kCtlBytes + kNQMax * 4 + kSoftWarps * 3 * kCols * 4 + 2 * kSoftWarps * kCols * 4;
   const size_t limit = 227 * 1024;
   // in order of what it buys: a second P^T buffer (the softmax no longer waits for the previous
   // tile's P V product), then a second V stage
