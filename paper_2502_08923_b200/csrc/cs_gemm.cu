@@ -34,6 +34,7 @@
 #include <stdlib.h>
 
 #include <algorithm>
+#include <type_traits>
 
 #include "cs_common.cuh"
 
@@ -566,15 +567,18 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
         float* part = dump + a.n_tok * CS_GEMM_BM;   // [rows][32] sums of squares, behind the parked tile
         const int total = per_tok * a.rows, iters = (total + 127) >> 7;
         const bool vec_n = (a.N & 3) == 0;
-        // Two items per turn: the remote reads and the residual reads of both are requested before
-        // either is finished, so a tall block's dozen turns per thread overlap pairwise (128 threads
-        // on an otherwise idle SM have nothing else to hide those latencies behind).
-        for (int it = 0; it < iters; it += 2) {
-          int idx[2], f[2], tok[2];
-          bool act[2], vec[2];
-          float4 y[2], x[2];
+        // Tall blocks take two items per turn: the remote reads and the residual reads of both are
+        // requested before either is finished, so a dozen turns per thread overlap pairwise (128
+        // threads on an otherwise idle SM have nothing else to hide those latencies behind).  Short
+        // blocks have one turn and take it without the second item's bookkeeping.
+        auto turns = [&](auto per_turn) {
+        constexpr int NU = decltype(per_turn)::value;
+        for (int it = 0; it < iters; it += NU) {
+          int idx[NU], f[NU], tok[NU];
+          bool act[NU], vec[NU];
+          float4 y[NU], x[NU];
 #pragma unroll
-          for (int u = 0; u < 2; ++u) {
+          for (int u = 0; u < NU; ++u) {
             idx[u] = e + ((it + u) << 7);
             act[u] = it + u < iters && idx[u] < total;
             const int idc = act[u] ? idx[u] : 0;
@@ -586,22 +590,22 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
           }
           if (a.splits > 1) {
 #pragma unroll
-            for (int u = 0; u < 2; ++u)
+            for (int u = 0; u < NU; ++u)
               if (act[u]) y[u] = sum_over_ranks(dump_addr + 4u * (uint32_t)(tok[u] * CS_GEMM_BM + f[u]), a.splits);
           } else {
 #pragma unroll
-            for (int u = 0; u < 2; ++u)
+            for (int u = 0; u < NU; ++u)
               if (act[u]) y[u] = *reinterpret_cast<const float4*>(dump + tok[u] * CS_GEMM_BM + f[u]);
           }
           if (a.mode == CS_EPI_RESIDUAL) {
 #pragma unroll
-            for (int u = 0; u < 2; ++u)
+            for (int u = 0; u < NU; ++u)
               if (act[u] && vec[u])
                 x[u] = (it + u == 0) ? x_pre : *reinterpret_cast<const float4*>(a.out + (size_t)tok[u] * a.N + n0 + f[u]);
           }
-          if (a.splits > 1 && it + 2 >= iters) { keep_alive(y[0], y[1]); cluster_arrive(); arrived = true; }
+          if (a.splits > 1 && it + NU >= iters) { keep_alive(y[0], y[NU - 1]); cluster_arrive(); arrived = true; }
 #pragma unroll
-          for (int u = 0; u < 2; ++u) {
+          for (int u = 0; u < NU; ++u) {
             if (!act[u]) continue;
             if (feeds_norm) part[tok[u] * 32 + idx[u] % per_tok] = 0.f;
             float* dst = a.out + (size_t)tok[u] * a.N + n0 + f[u];
@@ -631,6 +635,9 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
             }
           }
         }
+        };
+        if (iters > 1) turns(std::integral_constant<int, 2>{});
+        else turns(std::integral_constant<int, 1>{});
         if (feeds_norm) {
           asm volatile("bar.sync 1, 128;" ::: "memory");
           for (int tok = e; tok < a.rows; tok += 128) {
