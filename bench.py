@@ -637,6 +637,8 @@ def run_workload(args):
         return 0
     if name == "drafted_b1_k10":
         return run_drafted(args, cs, inputs, dev)
+    if name == "step_timeline":
+        return run_step_timeline(args, cs, inputs, dev, cfg)
     if name == "long_context_b1_k10":
         cases, k = [inputs.long_context_case(100)], 10
     elif name == "long_context_b8_k20":
@@ -709,6 +711,72 @@ def run_workload(args):
         line["config"]["speedup_by_k"] = {str(kk): res[kk]["tokens_per_s"] / res[0]["tokens_per_s"] for kk in res}
     print(json.dumps(line), flush=True)
     ctx.close()
+    return 0
+
+
+def run_step_timeline(args, cs, inputs, dev, cfg):
+    """Per-kernel timeline of a loop step (cs_set_stamps: every launch leaves the time at which its last
+    CTA finished; a kernel's share = its end minus its predecessor's end inside the replayed step
+    graph, mean over --steps steps), for any batch, window and cache depth of the 8B shape (use
+    --layers for a slice).  The script replays a span of the context, so every step accepts k tokens."""
+    import torch
+    B, k, S, W = args.batch, args.k, args.steps, args.warmup
+    max_new = (W + S + 2) * (k + 1)
+    n0 = args.kv + 1
+    stride = (n0 + max_new + 67) // 4 * 4
+    max_seq = n0 + max_new + k + 64
+    weights = inputs.make_weights(cfg, seed=0, device=str(dev))
+    ctx = cs.Context(cfg, weights, max_seq=max_seq, max_batch=B, k_max=k)
+    kv = inputs.synthetic_kv(cfg, B, max_seq, n0 - 1, seed=1, device=str(dev))
+    rng = np.random.default_rng(0)
+    h = np.zeros((B, stride), dtype=np.int32)
+    scripts = []
+    for b in range(B):
+        hh = rng.integers(0, cfg.vocab, size=n0).astype(np.int32)
+        src = 100 + 37 * b
+        hh[n0 - GAMMA:] = hh[src:src + GAMMA]
+        h[b, :n0] = hh
+        scripts.append(hh[src + GAMMA: src + GAMMA + max_new])
+    hd = torch.from_numpy(h).to(dev)
+    ld = torch.full((B,), n0, dtype=torch.int32, device=dev)
+    kvl = torch.full((B,), n0 - 1, dtype=torch.int32, device=dev)
+    stamps = torch.zeros(4096, dtype=torch.int64, device=dev)
+    ctx.cs_set_stamps(stamps)
+    ctx.cs_loop_begin(hd, ld, kv, kvl, GAMMA, k, max_new, script=torch.from_numpy(np.stack(scripts).astype(np.int32)).to(dev))
+    fams = ctx.cs_stamp_layout()
+    nst = len(fams)
+    rows = torch.zeros(S + 1, nst, dtype=torch.int64).pin_memory()
+    ctx.cs_loop_steps(W)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(S + 1):
+        ctx.cs_loop_steps(1)
+        rows[i].copy_(stamps[:nst], non_blocking=True)
+    e1.record()
+    torch.cuda.synchronize()
+    st, _ = ctx.cs_loop_poll()
+    ctx.cs_loop_end()
+    ctx.close()
+    ends = rows.numpy().astype(np.float64)
+    iv = np.zeros(nst)
+    for i in range(1, S + 1):
+        for j in range(nst):
+            iv[j] += (ends[i, j] - (ends[i, j - 1] if j else ends[i - 1, nst - 1])) / S / 1e3
+    # launches of a step: search, set-up, embedding, then per layer QKV, attention, merge, O, gate/up, down, then LM head, acceptance, commit
+    per_layer = (nst - 6) // cfg.n_layers
+    if per_layer != 6:
+        raise RuntimeError(f"unexpected launch layout: {nst} launches for {cfg.n_layers} layers")
+    lay = iv[3:3 + 6 * cfg.n_layers].reshape(cfg.n_layers, 6)
+    names = ["qkv", "attention", "merge", "o", "gate_up", "down"]
+    line = {"metric": "step timeline", "value": float(iv.sum()), "unit": "us", "higher_is_better": False, "n_gpus": 1,
+            "steps": S, "warmup": W, "ms_per_step": e0.elapsed_time(e1) / (S + 1), "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "step_timeline", "batch": B, "k": k, "kv": args.kv, "layers": cfg.n_layers,
+                       "layer_us": float(lay.sum(1).mean()),
+                       "per_layer_us": {n: float(lay[:, i].mean()) for i, n in enumerate(names)},
+                       "search_us": float(iv[0]), "setup_us": float(iv[1]), "embed_us": float(iv[2]),
+                       "lm_head_us": float(iv[-3]), "accept_us": float(iv[-2]), "commit_us": float(iv[-1]),
+                       "emitted_per_step": st["emitted"] / max(1, st["steps"])}}
+    print(json.dumps(line), flush=True)
     return 0
 
 
@@ -800,8 +868,11 @@ def main():
                     help="profiling aid: leave out plain decoding and the match-search part (fewer launches under ncu)")
     ap.add_argument("--workload", default="verify",
                     choices=["verify", "verify_plain_decode", "long_context_b1_k10", "long_context_b8_k20", "k_sweep_long_context_b1", "prefill_b1_4096",
-                             "multi_turn_b16_k10", "match_search", "drafted_b1_k10"],
+                             "multi_turn_b16_k10", "match_search", "drafted_b1_k10", "step_timeline"],
                     help="verify = the benchmark; the others are additional single-GPU measurements")
+    ap.add_argument("--batch", type=int, default=1, help="step_timeline: sequences")
+    ap.add_argument("--k", type=int, default=K_DRAFT, help="step_timeline: copied tokens per step")
+    ap.add_argument("--kv", type=int, default=KV_START, help="step_timeline: cached tokens per sequence")
     ap.add_argument("--layers", type=int, default=0,
                     help="profiling aid: keep only this many of the 32 layers (small case for ncu captures; "
                          "not the benchmark workload)")
