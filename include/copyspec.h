@@ -58,7 +58,8 @@
  *   CS_ATTN_KERNEL=tc|tcw|mma  forces one attention kernel: tcgen05 with the query rows as the
  *                          M dimension (tc), tcgen05 with the keys and head dims as M (tcw), or
  *                          mma.sync (mma).  Default: by head size, and between the two tcgen05
- *                          kernels by how many key tiles a CTA would walk (tcw from three on);
+ *                          kernels by how many key tiles a CTA would walk (tcw from three on,
+ *                          unless the block fills the 128 query rows of a tc CTA anyway);
  *   CS_WAIT_LIMIT_US=n     time limit of the kernels' bounded waits in microseconds (default
  *                          2,000,000), see cs_debug_drop_tile.
  */

@@ -276,16 +276,20 @@ int launch(cs_ctx* ctx, const void* kv_cache, int layer, int B, int R, cudaStrea
 
 }  // namespace
 
+int cs_attention_tc_group_rows(const cs_ctx* ctx, int R);   // cs_attn_tc.cu
+
 void cs_launch_attention(cs_ctx* ctx, const void* kv_cache, int layer, int B, int R, cudaStream_t st) {
   // head_dim 128 runs on the tcgen05 kernels: the one with the query rows as M while a CTA walks
   // at most two key tiles (a 4k context at batch 1: a latency chain, one tile on each of two CTAs
-  // per SM), the one with keys and head dims as M beyond that (its MMAs only cover the real query
-  // rows).  The register-resident mma.sync kernel takes the other head sizes.
+  // per SM) or when the block fills its 128 M rows anyway (256-row prefill chunks: measured 102 vs
+  // 132 us per layer over 3,840 keys); the one with keys and head dims as M otherwise (its MMAs only
+  // cover the real query rows).  The register-resident mma.sync kernel takes the other head sizes.
   // CS_ATTN_KERNEL=tc|tcw|mma, read when the context is created, forces one of them (tests run
   // them on the same inputs).
   int nsplit = 0;
   if (ctx->attn_force != 1) {
-    const bool wide = ctx->attn_force == 3 || (ctx->attn_force == 0 && cs_attention_tc_tiles_per_cta(ctx, B, R) > 2);
+    const bool wide = ctx->attn_force == 3 || (ctx->attn_force == 0 && cs_attention_tc_tiles_per_cta(ctx, B, R) > 2 &&
+                                               cs_attention_tc_group_rows(ctx, R) < 112);
     if (wide) nsplit = cs_launch_attention_tcw(ctx, kv_cache, layer, B, R, st);
     if (nsplit == 0) nsplit = cs_launch_attention_tc(ctx, kv_cache, layer, B, R, st);
   }

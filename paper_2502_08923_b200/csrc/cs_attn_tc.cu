@@ -541,6 +541,15 @@ int cs_attention_tc_tiles_per_cta(const cs_ctx* ctx, int B, int R) {
   return cs_ceil_div(cs_ceil_div(c.max_seq, kTileKeys), nsplit);
 }
 
+// Query rows per KV head that one CTA of this kernel holds for a block of R rows (of its 128 M rows).
+int cs_attention_tc_group_rows(const cs_ctx* ctx, int R) {
+  const cs_model_config& c = ctx->cfg;
+  const int G = c.n_heads / c.n_kv_heads;
+  if (c.head_dim != kDh || G > kNQMax || R < 1) return 0;
+  const int ngroups = cs_ceil_div(G * R, kNQMax);
+  return G * cs_ceil_div(R, ngroups);
+}
+
 int cs_launch_attention_tc(cs_ctx* ctx, const void* kv_cache, int layer, int B, int R, cudaStream_t st) {
   const cs_model_config& c = ctx->cfg;
   const int G = c.n_heads / c.n_kv_heads;
