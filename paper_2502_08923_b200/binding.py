@@ -48,6 +48,7 @@ class CsStats(C.Structure):
                 "emitted": self.emitted, "no_match": self.no_match, "tau_hist": list(self.tau_hist)}
 
 
+WORKSPACE_GUARD, GUARD_BYTE = 4096, 0xA5   # guard bands around a Context's workspace
 EXPORTS = ("cs_workspace_bytes", "cs_create", "cs_destroy", "cs_last_error", "cs_sync_status",
            "cs_find_match", "cs_verify_step", "cs_kv_truncate", "cs_decode_loop", "cs_decode_loop_drafted", "cs_step_host",
            "cs_prefill", "cs_linear", "cs_step_host_reset", "cs_debug_drop_tile",
@@ -264,9 +265,12 @@ class Context:
         if nbytes == 0:
             raise CsError(CS_ERR_SHAPE, "cs_workspace_bytes", "unsupported configuration")
         self.workspace_bytes = nbytes
-        raw = torch.empty(nbytes + 1024, dtype=torch.uint8, device="cuda")
-        off = (-raw.data_ptr()) % 1024
-        self._raw = raw
+        # the workspace sits between two guard bands of a fixed byte pattern (workspace_guards_intact)
+        raw = torch.empty(nbytes + 1024 + 2 * WORKSPACE_GUARD, dtype=torch.uint8, device="cuda")
+        off = WORKSPACE_GUARD + (-(raw.data_ptr() + WORKSPACE_GUARD)) % 1024
+        raw[:off].fill_(GUARD_BYTE)
+        raw[off + nbytes:].fill_(GUARD_BYTE)
+        self._raw, self._ws_off = raw, off
         self.weights = weights          # keeps the tensors alive
         L = cfg.n_layers
         self._arrs = {}
@@ -292,6 +296,13 @@ class Context:
                            C.c_void_p(raw.data_ptr() + off), nbytes)
         if rc != CS_OK:
             raise CsError(rc, "cs_create")
+
+    def workspace_guards_intact(self) -> bool:
+        """True while nothing has written into the guard bands on either side of the workspace
+        (synchronises the device)."""
+        torch.cuda.synchronize()
+        lo, hi = self._raw[:self._ws_off], self._raw[self._ws_off + self.workspace_bytes:]
+        return bool((lo == GUARD_BYTE).all().item() and (hi == GUARD_BYTE).all().item())
 
     def close(self):
         if getattr(self, "handle", None):

@@ -65,3 +65,34 @@ def counters_for_streams(hists, streams, gamma, k, policy=O.LATEST):
         for i, v in enumerate(st["tau_hist"]):
             tot["tau_hist"][i] += v
     return tot
+
+
+# ------------------------------------------------------------------ write canaries around a KV cache
+GUARD = 1 << 16     # bf16 elements on either side of the cache
+PATTERN = -1232.0   # exactly representable in bf16
+
+
+def guarded_kv(cfg, B, max_seq, fill_len, seed, device="cuda"):
+    """(whole buffer, cache view inside it): the cache holds N(0,1) up to fill_len and a pattern behind
+    it, the guard bands hold the pattern."""
+    n = cfg.n_layers * 2 * B * cfg.n_kv_heads * max_seq * cfg.head_dim
+    buf = torch.full((n + 2 * GUARD,), PATTERN, dtype=torch.bfloat16, device=device)
+    kv = buf[GUARD:GUARD + n].view(cfg.n_layers, 2, B, cfg.n_kv_heads, max_seq, cfg.head_dim)
+    kv[:, :, :, :, :fill_len, :] = inputs.synthetic_kv(cfg, B, max_seq, fill_len, seed=seed, device=device)[:, :, :, :, :fill_len, :]
+    return buf, kv
+
+
+def assert_only_rows_written(buf, kv, before, written):
+    """`written[b]` = (first, count): the only positions of sequence b that may differ from `before`."""
+    assert torch.all(buf[:GUARD] == PATTERN) and torch.all(buf[-GUARD:] == PATTERN), "guard band of the cache overwritten"
+    same = (kv == before)
+    for b, (first, count) in enumerate(written):
+        same[:, :, b, :, first:first + count, :] = True
+    bad = torch.nonzero(~same)
+    assert bad.numel() == 0, f"cache written outside the block's rows, first at (layer, k/v, seq, head, pos, dim) = {bad[0].tolist()}"
+    for b, (first, count) in enumerate(written):
+        if count:
+            rows = kv[:, :, b, :, first:first + count, :]
+            assert torch.isfinite(rows.float()).all() and not torch.all(rows == PATTERN), b
+
+

@@ -47,3 +47,28 @@ def test_shapes_of_the_named_configurations():
     assert torch.equal(p[0:64], w[0:64]) and torch.equal(p[64:128], w[100:164])
     assert torch.equal(p[128:164], w[64:100]) and torch.equal(p[192:228], w[164:200])
     assert p[164:192].abs().sum() == 0 and p[228:].abs().sum() == 0
+
+
+# ------------------------------------------------------------------ the write-canary checker itself
+def test_canary_checker_catches_stray_writes():
+    """The checker of the GPU canary tests, tried on CPU tensors with planted stray writes: one
+    position behind the block, one in front of it, one in another sequence, one in a guard band."""
+    import pytest
+    import torch
+    from helpers import PATTERN, assert_only_rows_written, guarded_kv
+    cfg = inputs.TINY
+    B, max_seq, kv_len, rows = 2, 40, 17, 5
+    buf, kv = guarded_kv(cfg, B, max_seq, kv_len, seed=1, device="cpu")
+    before = kv.clone()
+    kv[:, :, 0, :, kv_len:kv_len + rows, :] = 0.5                      # what a step may write
+    assert_only_rows_written(buf, kv, before, [(kv_len, rows), (kv_len, 0)])
+    for where in [(0, 0, 0, 0, kv_len + rows, 0), (1, 1, 0, 0, kv_len - 1, 3), (0, 1, 1, 0, kv_len, 0)]:
+        bad = kv.clone()
+        bad[where] = 7.0
+        with pytest.raises(AssertionError):
+            assert_only_rows_written(buf, bad, before, [(kv_len, rows), (kv_len, 0)])
+    buf2 = buf.clone()
+    buf2[5] = 0.0
+    with pytest.raises(AssertionError):
+        assert_only_rows_written(buf2, kv, before, [(kv_len, rows), (kv_len, 0)])
+    assert float(torch.tensor(PATTERN, dtype=torch.bfloat16)) == PATTERN
