@@ -16,20 +16,23 @@
 // 2 NQ rows, [P_hi^T | P_lo^T] as one of 2 NQ columns - and one instruction per 16 K-elements
 // does the work of two; the two halves of the accumulator are added where it is read (S^T keeps
 // one NQ-wide accumulator and two instructions when TMEM has no room for 2 NQ columns twice).
-// TMEM lane = key (S^T) or head dim (O^T), column = query row.  Softmax: thread t of a lane
-// quarter owns key t of the tile and half of the query columns (warps w and w + 4 share the
-// lanes).  Each column has a running reference point m for its exponentials, which follows the
-// column's true maximum only from afar: it moves when a score exceeds it by more than 2^8.
-// Softmax does not depend on the reference point, and weights up to 2^8 are as exact in two
-// bf16 terms as weights up to 1.  So on most tiles a thread only compares its scores with the
-// columns' thresholds and the threads of a column group vote (one predicate-reducing barrier);
-// the true maxima (a butterfly of 31 shuffles per warp plus a four-entry combine through shared
-// memory), the correction of the sums and the rescaling of O^T in TMEM happen only on the few
-// tiles where a reference point moves.  Each thread keeps its own share of every column's sum;
+// TMEM lane = key (S^T) or head dim (O^T), column = query row.  Softmax: twelve warps in three
+// column groups; thread t of a lane quarter owns key t of the tile and a third of the query
+// columns (warps w, w + 4 and w + 8 share the lanes).  Each column has a running reference point
+// m for its exponentials, which follows the column's true maximum only from afar: it moves when
+// a score exceeds it by more than 2^8.  Softmax does not depend on the reference point, and
+// weights up to 2^8 are as exact in two bf16 terms as weights up to 1.  So on most tiles a
+// thread only compares its scores with the columns' thresholds and the threads of a column
+// group vote (one predicate-reducing barrier); the true maxima (a butterfly of 31 shuffles per
+// warp plus a four-entry combine through shared memory), the correction of the sums and the
+// rescaling of O^T in TMEM happen only on the few tiles where a reference point moves.  The
+// weights pass works on column pairs with the packed fp32 instructions (fma / add / sub .f32x2).
+// Each thread keeps its own share of every column's sum;
 // the shares are added up once at the end.  P^T is written as one swizzled 16-byte chunk per 8
 // columns into the row of the thread's key, which is exactly the MN-major operand layout, so
 // nothing is transposed.  S^T is double-buffered in TMEM: the score product of tile i+1 runs
-// during the softmax of tile i.  K tiles move through a two-stage TMA ring and V tiles through a
+// during the softmax of tile i.  Blocks of up to 48 query rows have room for four S^T buffers:
+// their softmax takes the key tiles two at a time (one wait, one vote, two sets of weights).  K tiles move through a two-stage TMA ring and V tiles through a
 // one- or two-stage ring, each fed by its own producer thread, so K runs a tile ahead.  Each CTA
 // writes its un-normalised (O, m, sum); k_attn_merge combines the key slices.  When the caller
 // vouches for the cached lengths (kv_len_early), tiles that lie wholly below the cached length
@@ -156,6 +159,32 @@ __device__ __forceinline__ float ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// Two fp32 values in one 64-bit register and the packed fp32 arithmetic of this architecture
+// (fma / add / sub on both halves in one instruction): the weights pass works on column pairs.
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) {
+  f32x2 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 r, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(r));
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+  f32x2 d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+  f32x2 d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) {
+  f32x2 d;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
 // Maximum over the 32 lanes of each of 32 per-lane values with 31 shuffles (instead of five per
 // value): every step halves the values a lane is responsible for - it keeps one half of its array,
 // combined with what its partner sends of the same half - so that lane L ends up with the
@@ -172,20 +201,6 @@ __device__ __forceinline__ float warp_max32(float (&x)[32], int lane) {
     }
   }
   return x[0];
-}
-// eight values as eight leading bf16 terms and the eight bf16 terms of what that rounding lost
-__device__ __forceinline__ void split8(const float* p, uint4& hi, uint4& lo) {
-  uint32_t h[4], l[4];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const __nv_bfloat162 a = __floats2bfloat162_rn(p[2 * i], p[2 * i + 1]);
-    const float2 af = __bfloat1622float2(a);
-    const __nv_bfloat162 b = __floats2bfloat162_rn(p[2 * i] - af.x, p[2 * i + 1] - af.y);
-    h[i] = *reinterpret_cast<const uint32_t*>(&a);
-    l[i] = *reinterpret_cast<const uint32_t*>(&b);
-  }
-  hi = make_uint4(h[0], h[1], h[2], h[3]);
-  lo = make_uint4(l[0], l[1], l[2], l[3]);
 }
 // barrier of one column group of the softmax threads (128 threads, ids 1 to 3) that also ANDs a predicate:
 // every thread learns whether all of them are still fine, so they leave their loops together
@@ -205,6 +220,9 @@ __device__ __forceinline__ bool group_any(int id, bool pred) {
   return out != 0;
 }
 
+// KC = query columns per softmax thread at most (register arrays), NSB = S^T buffers in TMEM: 2, or 4
+// for blocks of up to 48 query rows, whose softmax then takes the key tiles two at a time.
+template <int KC, int NSB>
 __global__ void __launch_bounds__(kThreads, 1)
 k_attn_tcw(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUtensorMap tmQ, AttnArgs a) {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -223,7 +241,7 @@ k_attn_tcw(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUt
   uint8_t* sV = sK + 2 * 2 * kHalfBytes;               // [vstages][half][128 keys][128 B]
   uint8_t* ctl = sV + (size_t)vstages * 2 * kHalfBytes;
   uint64_t* bars = reinterpret_cast<uint64_t*>(ctl);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 20);
   volatile int* s_abort = reinterpret_cast<volatile int*>(tmem_slot + 1);
   volatile int* s_never = reinterpret_cast<volatile int*>(tmem_slot + 2);
   int* s_lmax = reinterpret_cast<int*>(tmem_slot + 3);
@@ -236,7 +254,7 @@ k_attn_tcw(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUt
     return;
   }
   const uint32_t b_kfull = smem_u32(bars), b_kfree = smem_u32(bars + 2), b_vfull = smem_u32(bars + 4),
-                 b_vfree = smem_u32(bars + 6), b_qfull = smem_u32(bars + 8), b_sready = smem_u32(bars + 9),
+                 b_vfree = smem_u32(bars + 6), b_qfull = smem_u32(bars + 8), b_sready = smem_u32(bars + 16),   // b_sready: one per S^T buffer (bars 16-19)
                  b_pready = smem_u32(bars + 14), b_odone = smem_u32(bars + 12);   // b_pready (bars 14, 15) and b_odone: two barriers each, by tile parity
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -244,7 +262,7 @@ k_attn_tcw(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUt
   // TMEM columns: S^T of even tiles, S^T of odd tiles (each NQ wide, or 2 NQ when the two query terms
   // are kept apart), then O^T, 2 NQ wide: the leading and the trailing weight terms' shares
   const uint32_t cstride = (uint32_t)(((a.qstack ? 2 * NQ : NQ) + 31) & ~31);
-  const uint32_t ocol = 2 * cstride;
+  const uint32_t ocol = NSB * cstride;
   uint32_t tmem_cols = 32;
   while (tmem_cols < ocol + (uint32_t)((2 * NQ + 31) & ~31)) tmem_cols <<= 1;
 
@@ -252,8 +270,8 @@ k_attn_tcw(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUt
     for (int s = 0; s < 2; ++s) {
       mbar_init(b_kfull + 8 * s, 1); mbar_init(b_kfree + 8 * s, 1);
       mbar_init(b_vfull + 8 * s, 1); mbar_init(b_vfree + 8 * s, 1);
-      mbar_init(b_sready + 8 * s, 1);
     }
+    for (int s = 0; s < NSB; ++s) mbar_init(b_sready + 8 * s, 1);
     mbar_init(b_qfull, 1);
     mbar_init(b_pready, kSoftThreads); mbar_init(b_pready + 8, kSoftThreads);
     mbar_init(b_odone, 1); mbar_init(b_odone + 8, 1);
@@ -366,11 +384,11 @@ k_attn_tcw(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUt
       const uint32_t idesc_o = idesc(2 * NQ) | (1u << 15) | (1u << 16);   // A (= V) and B (= P^T) are MN-major
       const uint32_t aq = smem_u32(sQ), ap = smem_u32(sP);
       auto issue_scores = [&](int i) -> bool {
-        const int s = i & 1;
+        const int s = i & 1, sb = i & (NSB - 1);           // K stage, S^T buffer
         if (!mbar_wait(b_kfull + 8 * s, (uint32_t)(i >> 1) & 1u, s_abort, a.wait_ns)) return false;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t ak = smem_u32(sK + (size_t)s * 2 * kHalfBytes);
-        const uint32_t acc = tmem_base + (uint32_t)s * cstride;
+        const uint32_t acc = tmem_base + (uint32_t)sb * cstride;
         if (a.qstack) {
 #pragma unroll
           for (int dh = 0; dh < 2; ++dh)
@@ -389,17 +407,21 @@ k_attn_tcw(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUt
                           idesc_s, (term | dh | kk) ? 1u : 0u);
         }
         umma_commit(b_kfree + 8 * s);
-        umma_commit(b_sready + 8 * s);
+        umma_commit(b_sready + 8 * sb);
         return true;
       };
-      bool ok = mbar_wait(b_qfull, 0, s_abort, a.wait_ns) && issue_scores(0);
+      bool ok = mbar_wait(b_qfull, 0, s_abort, a.wait_ns);
+      int qk = 0;                                          // score products issued so far
       for (int i = 0; i < ntl && ok; ++i) {
-        // the scores of the next tile go first: they run during this tile's softmax.  (Its S^T buffer
-        // was last read by the softmax of tile i - 1, which had finished before P^T of tile i - 1 was
-        // signalled.)  A column group whose tiles are quick - all its rows masked - can therefore be
-        // a tile ahead of the other one, which is why "P^T written" has a barrier per tile parity: it
-        // cannot be two ahead, because the scores of tile i + 2 are only issued after P^T of tile i.
-        if (i + 1 < ntl && !issue_scores(i + 1)) { ok = false; break; }
+        // The scores of the next tiles go first: they run during this tile's softmax.  The S^T buffer
+        // of tile t was last read by the softmax of tile t - NSB, which had finished before P^T of
+        // that tile was signalled - and this thread has waited for the P^T of every tile before i.
+        // A column group whose tiles are quick - all its rows masked - can therefore be a tile ahead
+        // of the others, which is why "P^T written" has a barrier per tile parity: it cannot be two
+        // ahead, because the scores of tile i + 2 are only issued after P^T of tile i (with four
+        // buffers the softmax hands tiles over in pairs, odd after even, so parity still tells them apart).
+        while (qk < ntl && qk < i + NSB && ok) { ok = issue_scores(qk); ++qk; }
+        if (!ok) break;
         const int s = i % vstages;
         if (!mbar_wait(b_pready + 8 * (i & 1), (uint32_t)(i >> 1) & 1u, s_abort, a.wait_ns) ||
             !mbar_wait(b_vfull + 8 * s, (uint32_t)(i / vstages) & 1u, s_abort, a.wait_ns)) { ok = false; break; }
@@ -423,9 +445,10 @@ k_attn_tcw(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUt
     const int q0 = grp * ncol;
     const uint32_t lane_base = tmem_base + ((uint32_t)(wq * 32) << 16);
     const float sc = a.scale_log2e;
-    float lsum[kCols];                                 // this key lane's share of every column's sum
+    f32x2 lsum[KC / 2];                             // this key lane's share of every column's sum, two columns per register pair
 #pragma unroll
-    for (int j = 0; j < kCols; ++j) lsum[j] = 0.f;
+    for (int j = 0; j < KC / 2; ++j) lsum[j] = pack2(0.f, 0.f);
+    const f32x2 sc2 = pack2(sc, sc);
     // This warp's own copy of its columns' running reference points (every warp of the group works
     // out the same values): the reference m (log2 domain), the raw score above which it has to
     // move, (m + 8) / scale, and -m for the exponent.  A column that has seen no key yet holds
@@ -442,22 +465,20 @@ k_attn_tcw(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUt
     __syncwarp();
     bool have = ntl > 0;
     const int limmin = *s_limmin;
-    for (int i = 0; i < ntl; ++i) {
-      const int sp = i & 1;
-      const int tile0 = (split + i * a.nsplit) * kTileKeys;
-      const int key = tile0 + row;                       // the key of this lane
-      const bool whole = tile0 + kTileKeys <= limmin;    // no live query row masks a key of this tile
-      bool ok = mbar_wait(b_sready + 8 * sp, (uint32_t)(i >> 1) & 1u, s_abort, a.wait_ns);
+    // ---- the pieces of one tile's softmax
+    // this key's scores of this thread's columns (masked keys count as -inf)
+    auto load_scores = [&](int t, float (&v)[KC]) -> bool {
+      const int sb = t & (NSB - 1);
+      const int tile0 = (split + t * a.nsplit) * kTileKeys;
+      const bool ok = mbar_wait(b_sready + 8 * sb, (uint32_t)(t / NSB) & 1u, s_abort, a.wait_ns);
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      // ---- this key's scores of this thread's columns (masked keys count as -inf)
-      const uint32_t s_addr = lane_base + (uint32_t)sp * cstride + (uint32_t)q0;
-      float v[kCols];
+      const uint32_t s_addr = lane_base + (uint32_t)sb * cstride + (uint32_t)q0;
 #pragma unroll
-      for (int c = 0; c < kCols / 8; ++c)
+      for (int c = 0; c < KC / 8; ++c)
         if (c < nch) tmem_ld8_nowait(s_addr + 8 * c, v + 8 * c);
       if (a.qstack) {                                    // the trailing query terms' share, NQ columns further
 #pragma unroll
-        for (int c = 0; c < kCols / 8; ++c)
+        for (int c = 0; c < KC / 8; ++c)
           if (c < nch) {
             float w[8];
             tmem_ld8_nowait(s_addr + (uint32_t)NQ + 8 * c, w);
@@ -470,34 +491,105 @@ k_attn_tcw(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUt
       } else {
         tmem_ld_wait();
 #pragma unroll
-        for (int c = 0; c < kCols / 8; ++c)
+        for (int c = 0; c < KC / 8; ++c)
           if (c < nch) tmem_landed8(v + 8 * c);
       }
-      if (!whole) {
+      if (tile0 + kTileKeys > limmin) {                  // some live query row masks a key of this tile
+        const int key = tile0 + row;                     // the key of this lane
 #pragma unroll
-        for (int c = 0; c < kCols / 8; ++c)
+        for (int c = 0; c < KC / 8; ++c)
           if (c < nch) {
 #pragma unroll
             for (int j = 0; j < 8; ++j)
               if (key >= s_lim[q0 + 8 * c + j]) v[8 * c + j] = -INFINITY;
           }
       }
-      // ---- does any score lie more than 2^8 above its column's reference point (or meet a column
-      // that has none)?  Softmax does not depend on the reference point, and weights up to 2^8 are
-      // as exact in two bf16 terms as weights up to 1, so the reference only has to follow the true
-      // maximum from afar: on most tiles nothing moves, no maximum is worked out and O^T is left alone.
+      return ok;
+    };
+    // Does any score lie more than 2^8 above its column's reference point (or meet a column that has
+    // none)?  Softmax does not depend on the reference point, and weights up to 2^8 are as exact in
+    // two bf16 terms as weights up to 1, so the reference only has to follow the true maximum from
+    // afar: on most tiles nothing moves, no maximum is worked out and O^T is left alone.
+    auto exceeds = [&](const float (&v)[KC]) -> bool {
       bool exceed = false;
 #pragma unroll
-      for (int c = 0; c < kCols / 8; ++c)
+      for (int c = 0; c < KC / 8; ++c)
         if (c < nch) {
           const float4 ta = *reinterpret_cast<const float4*>(w_thr + 8 * c), tb = *reinterpret_cast<const float4*>(w_thr + 8 * c + 4);
           exceed = exceed || v[8 * c] > ta.x || v[8 * c + 1] > ta.y || v[8 * c + 2] > ta.z || v[8 * c + 3] > ta.w ||
                    v[8 * c + 4] > tb.x || v[8 * c + 5] > tb.y || v[8 * c + 6] > tb.z || v[8 * c + 7] > tb.w;
         }
-      // this tile's P^T buffer was last read by the P V product of tile i - pbufs (long retired when
-      // there are two buffers: the softmax then runs a tile ahead of the tensor pipe)
-      if (i >= a.pbufs)
-        ok = mbar_wait(b_odone + 8 * ((i - a.pbufs) & 1), (uint32_t)((i - a.pbufs) >> 1) & 1u, s_abort, a.wait_ns) && ok;
+      return exceed;
+    };
+    // tile t's P^T buffer was last read by the P V product of tile t - pbufs
+    auto pbuf_free = [&](int t) -> bool {
+      return t < a.pbufs || mbar_wait(b_odone + 8 * ((t - a.pbufs) & 1), (uint32_t)((t - a.pbufs) >> 1) & 1u, s_abort, a.wait_ns);
+    };
+    // weights 2^(score * scale - m), this lane's share of the column sums, P^T, and the hand-over of tile t
+    auto emit = [&](int t, float (&v)[KC]) {
+      const int tile0 = (split + t * a.nsplit) * kTileKeys;
+      uint8_t* prow = sP + (size_t)(t % a.pbufs) * pbuf + (size_t)row * 128;
+#pragma unroll
+      for (int c = 0; c < KC / 8; ++c)
+        if (c < nch) {
+          const float4 na = *reinterpret_cast<const float4*>(w_nme + 8 * c), nb = *reinterpret_cast<const float4*>(w_nme + 8 * c + 4);
+          const float nm[8] = {na.x, na.y, na.z, na.w, nb.x, nb.y, nb.z, nb.w};
+          uint32_t hw[4], lw[4];                            // 8 columns = one 16-byte chunk of this key's row of the P^T operand
+#pragma unroll
+          for (int jj = 0; jj < 4; ++jj) {
+            const int j = 8 * c + 2 * jj;
+            float x0, x1;
+            unpack2(fma2(pack2(v[j], v[j + 1]), sc2, pack2(nm[2 * jj], nm[2 * jj + 1])), x0, x1);
+            const float w0 = ex2(x0), w1 = ex2(x1);         // masked scores are -inf: weight 0
+            const f32x2 w2 = pack2(w0, w1);
+            lsum[j >> 1] = add2(lsum[j >> 1], w2);
+            // leading bf16 terms and the bf16 terms of what that rounding lost
+            const __nv_bfloat162 h = __floats2bfloat162_rn(w0, w1);
+            hw[jj] = *reinterpret_cast<const uint32_t*>(&h);
+            float r0, r1;
+            unpack2(sub2(w2, pack2(__uint_as_float(hw[jj] << 16), __uint_as_float(hw[jj] & 0xffff0000u))), r0, r1);
+            const __nv_bfloat162 l = __floats2bfloat162_rn(r0, r1);
+            lw[jj] = *reinterpret_cast<const uint32_t*>(&l);
+          }
+          const int ch = (q0 >> 3) + c, cl = ch + (NQ >> 3);   // chunk index over all 2 NQ columns: leading terms, trailing terms
+          *reinterpret_cast<uint4*>(prow + (size_t)(ch >> 3) * kHalfBytes + ((((uint32_t)ch & 7u) ^ ((uint32_t)row & 7u)) << 4)) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+          *reinterpret_cast<uint4*>(prow + (size_t)(cl >> 3) * kHalfBytes + ((((uint32_t)cl & 7u) ^ ((uint32_t)row & 7u)) << 4)) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+        }
+      asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+      // keys past the longest row of this sequence hold whatever the cache held: zero their V rows
+      if (tile0 + kTileKeys > lmax) {
+        const int s = t % vstages;
+        if (!mbar_wait(b_vfull + 8 * s, (uint32_t)(t / vstages) & 1u, s_abort, a.wait_ns)) *s_abort = 1;
+        uint8_t* vs = sV + (size_t)s * 2 * kHalfBytes;
+        for (int rr = max(lmax - tile0, 0) + (warp * 32 + lane); rr < kTileKeys; rr += kSoftThreads) {
+#pragma unroll
+          for (int c = 0; c < 8; ++c) {
+            *reinterpret_cast<uint4*>(vs + (size_t)rr * 128 + c * 16) = make_uint4(0u, 0u, 0u, 0u);
+            *reinterpret_cast<uint4*>(vs + kHalfBytes + (size_t)rr * 128 + c * 16) = make_uint4(0u, 0u, 0u, 0u);
+          }
+        }
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      mbar_arrive(b_pready + 8 * (t & 1));
+    };
+    // With four S^T buffers the tiles are taken two at a time: one wait for both score products, one
+    // vote, then the two sets of weights back to back - half the hand-overs per key.  When the vote
+    // says that a reference point has to move, the tile is finished on its own and the next turn
+    // starts with its neighbour.
+    for (int i = 0; i < ntl;) {
+      const int sp = i & 1;
+      const bool pair = NSB == 4 && i + 1 < ntl;
+      float v[KC], v_next[NSB == 4 ? KC : 1];
+      bool ok = load_scores(i, v);
+      bool exceed = exceeds(v);
+      if constexpr (NSB == 4) {
+        if (pair) {
+          ok = load_scores(i + 1, v_next) && ok;
+          exceed = exceed || exceeds(v_next);
+        }
+      }
+      ok = pbuf_free(i) && ok;
       const bool bad = !ok || *s_abort != 0;
       const bool moved = group_any(1 + grp, exceed || bad);
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");   // (the waits above order the reads of O^T below)
@@ -508,7 +600,7 @@ k_attn_tcw(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUt
         {
           float x[32];
 #pragma unroll
-          for (int j = 0; j < 32; ++j) x[j] = (j < ncol) ? v[j] : -INFINITY;
+          for (int j = 0; j < 32; ++j) x[j] = (j < KC && j < ncol) ? v[j < KC ? j : 0] : -INFINITY;
           const float r = warp_max32(x, lane);
           if (lane < ncol) red_w[lane] = r;
         }
@@ -527,7 +619,7 @@ k_attn_tcw(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUt
         const unsigned grewA = __ballot_sync(0xffffffffu, mvA);
         bool prev_done = a.pbufs == 1;                   // is the P V product of tile i - 1 known to have retired?
 #pragma unroll
-        for (int c = 0; c < kCols / 8; ++c) {
+        for (int c = 0; c < KC / 8; ++c) {
           if (c < nch) {
             const bool grew = ((grewA >> (8 * c)) & 0xffu) != 0;   // the same in every thread of the group
             if (grew) {
@@ -535,7 +627,11 @@ k_attn_tcw(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUt
 #pragma unroll
               for (int j = 0; j < 8; ++j) {
                 cr[j] = __shfl_sync(0xffffffffu, crA, 8 * c + j);
-                lsum[8 * c + j] *= cr[j];
+                if (j & 1) {
+                  float s0, s1;
+                  unpack2(lsum[(8 * c + j) >> 1], s0, s1);
+                  lsum[(8 * c + j) >> 1] = pack2(s0 * cr[j - 1], s1 * cr[j]);
+                }
               }
               if (i > 0) {
                 if (!prev_done) {                        // O^T must hold all of tile i - 1 before it is rescaled
@@ -564,49 +660,18 @@ k_attn_tcw(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUt
           w_nme[lane] = (mnA == -INFINITY) ? -INFINITY : -mnA;
         }
         __syncwarp();
+              emit(i, v);
+        i += 1;
+        continue;
       }
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      // ---- weights 2^(score * scale - m), this lane's share of the column sums
-      uint8_t* prow = sP + (size_t)(i % a.pbufs) * pbuf + (size_t)row * 128;
-#pragma unroll
-      for (int c = 0; c < kCols / 8; ++c)
-        if (c < nch) {
-          const float4 na = *reinterpret_cast<const float4*>(w_nme + 8 * c), nb = *reinterpret_cast<const float4*>(w_nme + 8 * c + 4);
-          const float nm[8] = {na.x, na.y, na.z, na.w, nb.x, nb.y, nb.z, nb.w};
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            v[8 * c + j] = ex2(fmaf(v[8 * c + j], sc, nm[j]));      // masked scores are -inf: weight 0
-            lsum[8 * c + j] += v[8 * c + j];
-          }
-        }
-      // 8 columns = one 16-byte chunk of this key's row of the P^T operand
-#pragma unroll
-      for (int c = 0; c < kCols / 8; ++c) {
-        if (c < nch) {
-          uint4 hi, lo;
-          split8(v + 8 * c, hi, lo);
-          const int ch = (q0 >> 3) + c, cl = ch + (NQ >> 3);   // chunk index over all 2 NQ columns: leading terms, trailing terms
-          *reinterpret_cast<uint4*>(prow + (size_t)(ch >> 3) * kHalfBytes + ((((uint32_t)ch & 7u) ^ ((uint32_t)row & 7u)) << 4)) = hi;
-          *reinterpret_cast<uint4*>(prow + (size_t)(cl >> 3) * kHalfBytes + ((((uint32_t)cl & 7u) ^ ((uint32_t)row & 7u)) << 4)) = lo;
+      emit(i, v);
+      if constexpr (NSB == 4) {
+        if (pair) {
+          if (!pbuf_free(i + 1)) *s_abort = 1;
+          emit(i + 1, v_next);
         }
       }
-      asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-      // keys past the longest row of this sequence hold whatever the cache held: zero their V rows
-      if (tile0 + kTileKeys > lmax) {
-        const int s = i % vstages;
-        if (!mbar_wait(b_vfull + 8 * s, (uint32_t)(i / vstages) & 1u, s_abort, a.wait_ns)) *s_abort = 1;
-        uint8_t* vs = sV + (size_t)s * 2 * kHalfBytes;
-        for (int rr = max(lmax - tile0, 0) + (warp * 32 + lane); rr < kTileKeys; rr += kSoftThreads) {
-#pragma unroll
-          for (int c = 0; c < 8; ++c) {
-            *reinterpret_cast<uint4*>(vs + (size_t)rr * 128 + c * 16) = make_uint4(0u, 0u, 0u, 0u);
-            *reinterpret_cast<uint4*>(vs + kHalfBytes + (size_t)rr * 128 + c * 16) = make_uint4(0u, 0u, 0u, 0u);
-          }
-        }
-      }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      mbar_arrive(b_pready + 8 * sp);
+      i += pair ? 2 : 1;
     }
     // ---- un-normalised result of this key slice
     if (have) {
@@ -617,7 +682,7 @@ k_attn_tcw(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUt
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     // O^T: this thread holds head dim `row` of its columns; one 512-byte row of the partial output per column
 #pragma unroll
-    for (int c = 0; c < kCols / 8; ++c) {
+    for (int c = 0; c < KC / 8; ++c) {
       if (c < nch) {
         float o[8];
         if (have) {
@@ -646,11 +711,12 @@ k_attn_tcw(const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUt
     // the column sums: add the 128 key lanes' shares up (warp shuffle, then the four warps of the group)
     float* sum_w = s_red + warp * kCols;
 #pragma unroll
-    for (int c = 0; c < kCols / 8; ++c) {
+    for (int c = 0; c < KC / 8; ++c) {
       if (c < nch) {
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-          float t = lsum[8 * c + j];
+          float t, t_other;
+          if (j & 1) unpack2(lsum[(8 * c + j) >> 1], t_other, t); else unpack2(lsum[(8 * c + j) >> 1], t, t_other);
 #pragma unroll
           for (int off = 16; off > 0; off >>= 1) t += __shfl_xor_sync(0xffffffffu, t, off);
           if (lane == 0) sum_w[8 * c + j] = t;
@@ -728,8 +794,12 @@ int cs_launch_attention_tcw(cs_ctx* ctx, const void* kv_cache, int layer, int B,
   int nsplit = ctx->num_sms / (B * c.n_kv_heads * ngroups);
   if (nsplit > ctx->attn_splits) nsplit = ctx->attn_splits;
   if (nsplit < 1) nsplit = 1;
-  if (smem > ctx->attn_tcw_smem_set) {
-    if (cudaFuncSetAttribute(k_attn_tcw, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+  // up to 48 query rows (16 columns per softmax thread) with two P^T buffers: four S^T buffers, tiles in pairs
+  const bool dual = NQ <= 48 && pbufs == 2;
+  auto kernel = dual ? k_attn_tcw<16, 4> : k_attn_tcw<kCols, 2>;
+  if (smem > ctx->attn_tcw_smem_set) {                 // (both instantiations are raised together: one high-water mark)
+    if (cudaFuncSetAttribute(k_attn_tcw<16, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
+        cudaFuncSetAttribute(k_attn_tcw<kCols, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
       snprintf(ctx->err, sizeof(ctx->err), "attention needs %zu bytes of shared memory", smem);
       return -1;
     }
@@ -741,12 +811,13 @@ int cs_launch_attention_tcw(cs_ctx* ctx, const void* kv_cache, int layer, int B,
   a.layer = layer; a.R = R; a.Rg = Rg; a.G = G; a.H = c.n_heads; a.Hkv = c.n_kv_heads;
   a.max_batch = c.max_batch; a.max_seq = c.max_seq; a.nsplit = nsplit; a.NQ = NQ; a.rows = B * R; a.vstages = vstages; a.pbufs = pbufs;
   a.qstack = (3 * ((2 * NQ + 31) / 32 * 32) <= 512) ? 1 : 0;   // TMEM columns: two score buffers and the output, 2 NQ wide each
+  if (dual && 5 * ((2 * NQ + 31) / 32 * 32) > 512) return 0;   // (four score buffers and the output: 480 columns at 48 query rows)
   a.smem_bytes = (int)smem;
   a.scale_log2e = 1.4426950408889634f / sqrtf((float)kDh);
   a.out_o = ctx->attn_o; a.out_ml = ctx->attn_ml; a.status = ctx->d_status;
   a.wait_ns = ctx->wait_limit_ns;
   a.stamp = cs_next_stamp(ctx, CS_FAM_ATTENTION);
-  if (cs_launch_pdl(k_attn_tcw, dim3(B * c.n_kv_heads, nsplit, ngroups), dim3(kThreads), smem, st, ctx->tmKV, ctx->tmQ, a) != cudaSuccess) {
+  if (cs_launch_pdl(kernel, dim3(B * c.n_kv_heads, nsplit, ngroups), dim3(kThreads), smem, st, ctx->tmKV, ctx->tmQ, a) != cudaSuccess) {
     snprintf(ctx->err, sizeof(ctx->err), "attention launch failed");
     return -1;
   }
