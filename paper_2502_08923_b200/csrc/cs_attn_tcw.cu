@@ -32,8 +32,9 @@
 // columns into the row of the thread's key, which is exactly the MN-major operand layout, so
 // nothing is transposed.  S^T is double-buffered in TMEM: the score product of tile i+1 runs
 // during the softmax of tile i.  Blocks of up to 48 query rows have room for four S^T buffers:
-// their softmax takes the key tiles two at a time (one wait, one vote, two sets of weights).  K tiles move through a two-stage TMA ring and V tiles through a
-// one- or two-stage ring, each fed by its own producer thread, so K runs a tile ahead.  Each CTA
+// their softmax takes the key tiles two at a time (one wait, one vote, two sets of weights).
+// K tiles move through a two-stage TMA ring and V tiles through a one- or two-stage ring, each
+// fed by its own producer thread, so K runs a tile ahead.  Each CTA
 // writes its un-normalised (O, m, sum); k_attn_merge combines the key slices.  When the caller
 // vouches for the cached lengths (kv_len_early), tiles that lie wholly below the cached length
 // are requested before the wait for the preceding kernel: those rows were written by earlier
