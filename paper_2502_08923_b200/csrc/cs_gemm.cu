@@ -464,6 +464,11 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
           const int i = j % half, f1 = (j / half) * Q.Dh + i, f2 = f1 + half;
           const int head = (n0 + f1) / Q.Dh;
           const bool act = idx < total && head < Q.H + 2 * Q.Hkv;
+          // the rotation factors and the row's place in the cache do not depend on the sums: they are
+          // requested first, so that their latency runs under the remote reads
+          const float4* csp = reinterpret_cast<const float4*>(Q.rope_cs + 2 * ((size_t)tok * half + i));
+          const float4 cs01 = csp[0], cs23 = csp[1];      // (cos, sin) of dims i .. i + 3
+          const int row_w = Q.row_write[tok], row_p = Q.row_pos[tok];
           float4 av = make_float4(0.f, 0.f, 0.f, 0.f), bv = av;
           if (a.splits > 1) {
             if (act) {
@@ -479,9 +484,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
           const float a4[4] = {av.x, av.y, av.z, av.w}, b4[4] = {bv.x, bv.y, bv.z, bv.w};
           float r0[4], r1[4];
           const bool is_v = head >= Q.H + Q.Hkv;
+          const float2 csv[4] = {make_float2(cs01.x, cs01.y), make_float2(cs01.z, cs01.w), make_float2(cs23.x, cs23.y), make_float2(cs23.z, cs23.w)};
 #pragma unroll
           for (int t4 = 0; t4 < 4; ++t4) {
-            const float2 cs2 = *reinterpret_cast<const float2*>(Q.rope_cs + 2 * ((size_t)tok * half + i + t4));
+            const float2 cs2 = csv[t4];
             r0[t4] = is_v ? a4[t4] : a4[t4] * cs2.x - b4[t4] * cs2.y;
             r1[t4] = is_v ? b4[t4] : b4[t4] * cs2.x + a4[t4] * cs2.y;
           }
@@ -501,11 +507,11 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUten
             l1[0] = __floats2bfloat162_rn(r1[0] - f10.x, r1[1] - f10.y); l1[1] = __floats2bfloat162_rn(r1[2] - f11.x, r1[3] - f11.y);
             *reinterpret_cast<uint2*>(ql) = *reinterpret_cast<const uint2*>(l0);
             *reinterpret_cast<uint2*>(ql + half) = *reinterpret_cast<const uint2*>(l1);
-          } else if (Q.row_write[tok]) {
+          } else if (row_w) {
             // new K (rotated) / V row of the cache, stored in bf16
             const int kvh = is_v ? head - Q.H - Q.Hkv : head - Q.H;
             __nv_bfloat16* dst = Q.kv + ((((size_t)Q.layer * 2 + (is_v ? 1 : 0)) * Q.max_batch + tok / Q.R) * Q.Hkv + kvh) *
-                                            (size_t)Q.max_seq * Q.Dh + (size_t)Q.row_pos[tok] * Q.Dh + i;
+                                            (size_t)Q.max_seq * Q.Dh + (size_t)row_p * Q.Dh + i;
             *reinterpret_cast<uint2*>(dst) = *reinterpret_cast<const uint2*>(h0);
             *reinterpret_cast<uint2*>(dst + half) = *reinterpret_cast<const uint2*>(h1);
           }
